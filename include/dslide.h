@@ -1,0 +1,183 @@
+/*
+ * dslide.h -- C ABI of libdslide: the SLIDE adaptive-sparse training step of a
+ * two-layer fully connected network (sparse input -> dense ReLU hidden layer ->
+ * LSH-sampled softmax output layer) on one NVIDIA B200 (sm_100a).
+ *
+ * The operations follow "Distributed SLIDE" (arXiv 2201.12667): Section 2.1 (the
+ * three phases of SLIDE), Algorithm 1 (training procedure), Section 3.5 (Adam
+ * moments per weight and bias array), Section 3.6 (layer operations and the
+ * per-sample snapshot of active neurons), Section 4.1 (hash families, K, L, Adam
+ * constants).  Nothing is sharded or communicated between GPUs.
+ *
+ * Conventions
+ *  - Every function returns a dslide_status.  No exceptions, no abort, no output.
+ *  - "device" pointers are CUDA device pointers on the context's device, owned by
+ *    the caller, read-only unless stated, and must stay valid until the work
+ *    enqueued by the call has finished on the context's stream.
+ *  - Calls are asynchronous on the context's stream unless stated.  Errors the
+ *    host can see (bad arguments, wrong state) are returned at once and the call
+ *    has no effect.  Errors only the device can see (feature or label id out of
+ *    range, active set larger than configured) set a sticky status word; the
+ *    offending sample is skipped (it contributes no loss and no gradient), no
+ *    out-of-bounds access is made, and the status is returned, and cleared, by
+ *    the next dslide_sync.
+ *  - The context owns the model state, the hash tables and all work space.
+ *    One context must not be used from two host threads at once.
+ *  - Matrices are row-major fp32: W1[D][H], W2[N][H]; ids are int32.
+ */
+#ifndef DSLIDE_H
+#define DSLIDE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dslide_ctx dslide_ctx;
+
+typedef enum {
+  DSLIDE_OK = 0,
+  DSLIDE_ERR_INVALID_ARG = 1,
+  DSLIDE_ERR_OOM = 2,
+  DSLIDE_ERR_CUDA = 3,
+  DSLIDE_ERR_OVERFLOW = 4,   /* an active set, label list or batch exceeds the configured maximum */
+  DSLIDE_ERR_BAD_INDEX = 5,  /* feature id outside [0,D) or label id outside [0,N), seen on the device */
+  DSLIDE_ERR_STATE = 6,
+  DSLIDE_ERR_TIMEOUT = 7
+} dslide_status;
+
+enum { DSLIDE_SIMHASH = 0, DSLIDE_DWTA = 1 };
+
+typedef struct {
+  int32_t input_dim, hidden_dim, output_dim; /* D, H, N.  H must be a multiple of 4 and at most 1024.          */
+  int32_t hash_family;                       /* DSLIDE_SIMHASH (sparse +1/-1 projections) or DSLIDE_DWTA        */
+  int32_t K, L;                              /* K hash functions per table, L tables (Section 4.1)              */
+  int32_t dwta_bin_size;                     /* power of two, divides H; 0 means 8                              */
+  int32_t srp_nnz;                           /* nonzeros per SimHash projection; 0 means ceil(H/3)              */
+  int32_t bucket_cap;                        /* a query reads at most this many (lowest) ids of a bucket        */
+  int32_t rebuild_period0;                   /* first scheduled rebuild after this many steps; 0 = never        */
+  float rebuild_growth_lambda;               /* later gaps: max(1, floor(period0 * exp(lambda * rebuilds)))     */
+  int32_t redraw_hash_fns;                   /* 1: draw new hash functions at every rebuild (Algorithm 1)       */
+  int32_t force_dense;                       /* 1: every output neuron is active, no hashing (Section 3.6)      */
+  int32_t max_batch;                         /* largest batch a call may pass (at most 4096)                    */
+  int32_t max_labels;                        /* largest label list of one sample                                */
+  int32_t max_active_per_sample;             /* 0 means L * bucket_cap + max_labels (N when force_dense)        */
+  float lr, beta1, beta2, eps;               /* Adam (Section 4.1: 1e-4, 0.9, 0.999, 1e-8)                      */
+  float init_std;                            /* weights ~ N(0, init_std^2); biases and moments start at 0       */
+  uint64_t seed;
+  int32_t device;                            /* CUDA device ordinal                                             */
+  int32_t dedup_mode;                        /* 0 auto; 1 bitmap in shared memory; 2 sort in shared memory      */
+  void* stream;                              /* cudaStream_t the context enqueues on (NULL = default stream)    */
+} dslide_config;
+
+/* Tensors readable and writable through dslide_get_tensor / dslide_set_tensor. */
+enum {
+  DSLIDE_T_W1 = 0, DSLIDE_T_B1, DSLIDE_T_W2, DSLIDE_T_B2,          /* f32 [D*H], [H], [N*H], [N]                */
+  DSLIDE_T_M_W1, DSLIDE_T_V_W1, DSLIDE_T_M_B1, DSLIDE_T_V_B1,      /* Adam first / second moments (Section 3.5) */
+  DSLIDE_T_M_W2, DSLIDE_T_V_W2, DSLIDE_T_M_B2, DSLIDE_T_V_B2,
+  DSLIDE_T_HASH_IDX,    /* i32 [K*L][srp_nnz] (SimHash, ascending per projection) or [K*L][bin] (DWTA)          */
+  DSLIDE_T_HASH_SIGN,   /* i32 [K*L][srp_nnz], +1 / -1 (SimHash only; 0 bytes for DWTA)                         */
+  DSLIDE_T_BUCKET_OFF,  /* i32 [L][2^bits + 1], bits = K (SimHash) or K*log2(bin) (DWTA)                        */
+  DSLIDE_T_BUCKET_IDS,  /* i32 [L][N]: per table, neuron ids grouped by bucket, ascending inside a bucket       */
+  DSLIDE_T_COUNTERS,    /* i64 [3]: Adam step count t, rebuild count r, step of the next scheduled rebuild      */
+  DSLIDE_T_COUNT
+};
+
+/* Per-sample snapshot of the last dslide_train_step (Section 3.6), for dslide_get_last. */
+enum {
+  DSLIDE_LAST_HIDDEN = 0, /* f32 [B][H]                                                        */
+  DSLIDE_LAST_CODES,      /* u32 [B][L] bucket codes of the hidden activations                  */
+  DSLIDE_LAST_ACT_COUNT,  /* i32 [B] size of each active set                                    */
+  DSLIDE_LAST_ACT_IDS,    /* i32 [B][stride] ascending ids, first count[s] entries valid        */
+  DSLIDE_LAST_ACT_LOGIT,  /* f32 [B][stride]                                                    */
+  DSLIDE_LAST_ACT_PROB,   /* f32 [B][stride] softmax over the active set                        */
+  DSLIDE_LAST_ACT_ERR,    /* f32 [B][stride] (p - [label]/|labels|) / B                         */
+  DSLIDE_LAST_LOSS,       /* f32 [B]                                                            */
+  DSLIDE_LAST_DHIDDEN,    /* f32 [B][H] error back-propagated to the hidden layer               */
+  DSLIDE_LAST_COUNT
+};
+
+/* Algorithm 1, initialisation: allocates the model, draws the weights and the hash
+ * functions of rebuild count 0 and indexes every output neuron into the L tables
+ * (Section 2.1, phase 1).  Synchronous.  *out receives the context. */
+dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out);
+
+/* Frees everything the context owns after draining its stream.  Synchronous. */
+dslide_status dslide_destroy(dslide_ctx* ctx);
+
+/* Algorithm 1 "Rebuild hash tables and hash functions", outside the schedule: the
+ * rebuild count goes up by one, new functions are drawn when redraw_hash_fns is
+ * set, and every neuron's current weight row is hashed into the tables again. */
+dslide_status dslide_rebuild_tables(dslide_ctx* ctx);
+
+/* Hash the tables again with the hash functions currently loaded and the current
+ * weights; the rebuild count does not change.  For callers that load their own
+ * hash functions or weights with dslide_set_tensor. */
+dslide_status dslide_build_tables(dslide_ctx* ctx);
+
+/* One training step on one batch (Algorithm 1, inner loops and the Adam line; Section
+ * 2.1 feed-forward and back-propagation stages):
+ *   hidden layer from the CSR rows -> L bucket codes -> union of the retrieved buckets
+ *   plus the sample's labels -> logits and softmax over that set only -> errors ->
+ *   sparse back-propagation -> Adam on the touched rows of W2, b2, W1 and on b1 ->
+ *   the scheduled rebuild if this step is due.
+ * batch in [1, max_batch].  CSR: row_ptr[batch+1] (row_ptr[0] = 0, non-decreasing),
+ * col_idx / vals [row_ptr[batch]], column ids in [0, D), ascending inside a row.
+ * Labels: label_ptr[batch+1], labels[label_ptr[batch]], ids in [0, N), at least one and
+ * at most max_labels per sample; duplicates inside a sample count once.
+ * All five are device pointers.  loss_out: device float, may be NULL; receives the mean
+ * loss of the batch.  The loss of sample s is -(1/|Y_s|) sum_{y in Y_s} log p_y with p
+ * the softmax over the active set. */
+dslide_status dslide_train_step(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
+                                const int32_t* col_idx, const float* vals,
+                                const int32_t* label_ptr, const int32_t* labels, float* loss_out);
+
+/* The same step for callers whose batch lives in HOST memory: copies the five arrays to
+ * the device (nnz = row_ptr[batch] and label_ptr[batch] are read on the host), runs the
+ * step, copies the mean loss back to *loss_out (host, may be NULL) and waits for it.
+ * Returns the sticky device status like dslide_sync. */
+dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
+                                     const int32_t* col_idx, const float* vals,
+                                     const int32_t* label_ptr, const int32_t* labels,
+                                     float* loss_out);
+
+/* Inference: hidden layer -> codes -> retrieved set (dense = 0) or every neuron
+ * (dense = 1) -> logits -> the k largest by (logit descending, id ascending).
+ * out_ids [batch*k] (device, -1 where fewer than k candidates), out_scores [batch*k]
+ * (device, -inf there).  1 <= k <= 64.  The paper reports accuracy but not how it
+ * evaluates; this is the reading taken. */
+dslide_status dslide_predict_topk(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
+                                  const int32_t* col_idx, const float* vals, int32_t k,
+                                  int32_t dense, int32_t* out_ids, float* out_scores);
+
+/* Waits for the context's stream; returns and clears the sticky device status. */
+dslide_status dslide_sync(dslide_ctx* ctx);
+
+/* State I/O (check-pointing and the parity harness).  Synchronous.  host pointers.
+ * nbytes must equal the tensor's size exactly.  Setting weights or hash functions does
+ * not rebuild the tables; call dslide_build_tables. */
+dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes);
+dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, int64_t nbytes);
+dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host_src, int64_t nbytes);
+
+/* Snapshot of the last training step.  Synchronous.  host_dst receives min(nbytes,
+ * size) bytes; *stride (may be NULL) receives the row stride, in elements, of the
+ * per-sample active arrays. */
+dslide_status dslide_last_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes, int32_t* stride);
+dslide_status dslide_get_last(dslide_ctx* ctx, int32_t which, void* host_dst, int64_t nbytes);
+
+/* Per-step statistics of the last training step, read from the device.  Synchronous.
+ * out[0] = sum of active-set sizes, out[1] = distinct touched rows of W2, out[2] =
+ * distinct touched rows of W1, out[3] = nonzeros in the batch. */
+dslide_status dslide_last_stats(dslide_ctx* ctx, int64_t out[4]);
+
+/* Number of kernels the context has launched since dslide_init. */
+int64_t dslide_kernel_launches(const dslide_ctx* ctx);
+
+const char* dslide_status_str(dslide_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSLIDE_H */

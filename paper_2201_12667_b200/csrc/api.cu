@@ -1,0 +1,425 @@
+// The C ABI of libdslide (include/dslide.h): context life cycle, argument checks, the rebuild
+// schedule (Section 3.1; Algorithm 1 places the rebuild after the weight update), state I/O.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace dslide {
+int sort_tile_elems();
+int sort_max_width();
+}
+
+using namespace dslide;
+
+struct dslide_ctx { Ctx c; };
+
+namespace {
+
+#define CU(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return e_ == cudaErrorMemoryAllocation ? DSLIDE_ERR_OOM : DSLIDE_ERR_CUDA; } while (0)
+
+template <typename T>
+cudaError_t dalloc(T** p, size_t n, cudaStream_t st, bool zero) {
+  *p = nullptr;
+  if (n == 0) n = 1;
+  cudaError_t e = cudaMalloc((void**)p, n * sizeof(T));
+  if (e != cudaSuccess) return e;
+  if (zero) e = cudaMemsetAsync(*p, 0, n * sizeof(T), st);
+  return e;
+}
+
+void free_all(Ctx* c) {
+  void* ptrs[] = {c->W1, c->b1, c->W2, c->b2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2, c->mb2, c->vb2,
+                  c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
+                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->touched1, c->touched2, c->mask1,
+                  c->mask2, c->uniq1, c->uniq2, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
+                  c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
+  for (void* p : ptrs) if (p) cudaFree(p);
+  if (c->pinned_loss) cudaFreeHost(c->pinned_loss);
+}
+
+int ilog2_exact(int x) {
+  int l = 0;
+  while ((1 << l) < x) ++l;
+  return (1 << l) == x ? l : -1;
+}
+
+struct TensorRef { void* ptr; int64_t bytes; };
+
+TensorRef tensor_ref(Ctx* c, int which) {
+  const int64_t D = c->D, H = c->H, N = c->N, f = sizeof(float);
+  switch (which) {
+    case DSLIDE_T_W1: return {c->W1, D * H * f};
+    case DSLIDE_T_B1: return {c->b1, H * f};
+    case DSLIDE_T_W2: return {c->W2, N * H * f};
+    case DSLIDE_T_B2: return {c->b2, N * f};
+    case DSLIDE_T_M_W1: return {c->mW1, D * H * f};
+    case DSLIDE_T_V_W1: return {c->vW1, D * H * f};
+    case DSLIDE_T_M_B1: return {c->mb1, H * f};
+    case DSLIDE_T_V_B1: return {c->vb1, H * f};
+    case DSLIDE_T_M_W2: return {c->mW2, N * H * f};
+    case DSLIDE_T_V_W2: return {c->vW2, N * H * f};
+    case DSLIDE_T_M_B2: return {c->mb2, N * f};
+    case DSLIDE_T_V_B2: return {c->vb2, N * f};
+    case DSLIDE_T_HASH_IDX: return {c->hash_idx, (int64_t)c->KL * c->fn_len * 4};
+    case DSLIDE_T_HASH_SIGN: return {c->hash_sign, c->cfg.hash_family == DSLIDE_SIMHASH ? (int64_t)c->KL * c->fn_len * 4 : 0};
+    case DSLIDE_T_BUCKET_OFF: return {c->bucket_off, (int64_t)c->L * (c->nb + 1) * 4};
+    case DSLIDE_T_BUCKET_IDS: return {c->bucket_ids, (int64_t)c->L * N * 4};
+    case DSLIDE_T_COUNTERS: return {nullptr, 3 * 8};
+  }
+  return {nullptr, -1};
+}
+
+dslide_status drain(Ctx* c) {
+  CU(cudaStreamSynchronize(c->stream));
+  return DSLIDE_OK;
+}
+
+dslide_status rebuild(Ctx* c, bool bump) {
+  if (bump) {
+    c->r_host += 1;
+    if (c->cfg.redraw_hash_fns) CU(launch_draw_hash(c, c->r_host));
+  }
+  if (!c->dense) CU(launch_build_tables(c));
+  return DSLIDE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dslide_status_str(dslide_status s) {
+  switch (s) {
+    case DSLIDE_OK: return "ok";
+    case DSLIDE_ERR_INVALID_ARG: return "invalid argument";
+    case DSLIDE_ERR_OOM: return "out of device memory";
+    case DSLIDE_ERR_CUDA: return "CUDA error";
+    case DSLIDE_ERR_OVERFLOW: return "active set, label list or batch exceeds the configured maximum";
+    case DSLIDE_ERR_BAD_INDEX: return "feature or label id out of range, or columns not ascending";
+    case DSLIDE_ERR_STATE: return "call not valid in this state";
+    case DSLIDE_ERR_TIMEOUT: return "timeout";
+  }
+  return "unknown status";
+}
+
+dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
+  if (!cfg || !out) return DSLIDE_ERR_INVALID_ARG;
+  *out = nullptr;
+  dslide_config k = *cfg;
+  if (k.input_dim < 1 || k.hidden_dim < 4 || k.hidden_dim > 1024 || (k.hidden_dim & 3) || k.output_dim < 1)
+    return DSLIDE_ERR_INVALID_ARG;
+  if (k.hash_family != DSLIDE_SIMHASH && k.hash_family != DSLIDE_DWTA) return DSLIDE_ERR_INVALID_ARG;
+  if (k.K < 1 || k.L < 1 || k.L > 1024 || k.bucket_cap < 1) return DSLIDE_ERR_INVALID_ARG;
+  if (k.max_batch < 1 || k.max_batch > 4096 || k.max_labels < 1 || k.max_labels > 4096) return DSLIDE_ERR_INVALID_ARG;
+  if (!(k.lr > 0.f) || !(k.beta1 >= 0.f && k.beta1 < 1.f) || !(k.beta2 >= 0.f && k.beta2 < 1.f) || !(k.eps > 0.f))
+    return DSLIDE_ERR_INVALID_ARG;
+  if (k.rebuild_period0 < 0 || k.init_std < 0.f || k.dedup_mode < 0 || k.dedup_mode > 2) return DSLIDE_ERR_INVALID_ARG;
+  if (k.dwta_bin_size == 0) k.dwta_bin_size = 8;
+  if (k.srp_nnz == 0) k.srp_nnz = (k.hidden_dim + 2) / 3;
+  int lg_bin = 0, bits = 0, fn_len = 0;
+  if (k.hash_family == DSLIDE_DWTA) {
+    lg_bin = ilog2_exact(k.dwta_bin_size);
+    if (lg_bin < 1 || k.dwta_bin_size > 256 || k.hidden_dim % k.dwta_bin_size) return DSLIDE_ERR_INVALID_ARG;
+    bits = k.K * lg_bin;
+    fn_len = k.dwta_bin_size;
+  } else {
+    if (k.srp_nnz < 1 || k.srp_nnz > k.hidden_dim) return DSLIDE_ERR_INVALID_ARG;
+    bits = k.K;
+    fn_len = k.srp_nnz;
+  }
+  if (bits > 24 || (int64_t)k.K * k.L > 65536) return DSLIDE_ERR_INVALID_ARG;
+  if ((int64_t)k.L * k.output_dim >= (int64_t)1 << 31) return DSLIDE_ERR_INVALID_ARG;
+  int64_t act_stride = k.force_dense ? k.output_dim
+                       : (k.max_active_per_sample > 0 ? k.max_active_per_sample
+                                                      : (int64_t)k.L * k.bucket_cap + k.max_labels);
+  if (!k.force_dense && act_stride > (int64_t)k.L * k.bucket_cap + k.max_labels)
+    act_stride = (int64_t)k.L * k.bucket_cap + k.max_labels;
+  if (act_stride > k.output_dim) act_stride = k.output_dim;
+  if (act_stride < 1) return DSLIDE_ERR_INVALID_ARG;
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || k.device < 0 || k.device >= ndev) return DSLIDE_ERR_CUDA;
+  CU(cudaSetDevice(k.device));
+
+  dslide_ctx* h = new (std::nothrow) dslide_ctx;
+  if (!h) return DSLIDE_ERR_OOM;
+  memset(h, 0, sizeof(*h));
+  Ctx* c = &h->c;
+  c->cfg = k;
+  c->D = k.input_dim; c->H = k.hidden_dim; c->N = k.output_dim; c->K = k.K; c->L = k.L; c->KL = k.K * k.L;
+  c->bits = bits; c->lg_bin = lg_bin; c->fn_len = fn_len; c->cap = k.bucket_cap;
+  c->nb = (int64_t)1 << bits;
+  c->act_stride = (int)act_stride;
+  c->Wd = (k.max_batch + 31) / 32;
+  c->dense = k.force_dense ? 1 : 0;
+  c->stream = (cudaStream_t)k.stream;
+  c->next_rebuild = k.rebuild_period0;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, k.device) != cudaSuccess) { delete h; return DSLIDE_ERR_CUDA; }
+  c->num_sms = prop.multiProcessorCount;
+
+  // radix sort geometry
+  c->sort_passes = (bits + sort_max_width() - 1) / sort_max_width();
+  c->sort_width = (bits + c->sort_passes - 1) / c->sort_passes;
+  c->sort_tiles = (c->N + sort_tile_elems() - 1) / sort_tile_elems();
+
+  const size_t D = c->D, H = c->H, N = c->N, B = k.max_batch, S = c->act_stride;
+  cudaStream_t st = c->stream;
+  cudaError_t e = cudaSuccess;
+#define A(ptr, n, zero) if (e == cudaSuccess) e = dalloc(&c->ptr, (size_t)(n), st, zero)
+  A(W1, D * H, false); A(mW1, D * H, true); A(vW1, D * H, true);
+  A(b1, H, true); A(mb1, H, true); A(vb1, H, true);
+  A(W2, N * H, false); A(mW2, N * H, true); A(vW2, N * H, true);
+  A(b2, N, true); A(mb2, N, true); A(vb2, N, true);
+  A(hash_idx, (size_t)c->KL * fn_len, true); A(hash_sign, (size_t)c->KL * fn_len, true);
+  A(h, B * H, true); A(dh, B * H, true); A(loss, B, true); A(codes, B * c->L, true);
+  A(act_cnt, B, true); A(act_z, B * S, true); A(act_p, B * S, true); A(act_g, B * S, true);
+  A(touched1, (D + 31) / 32, true); A(mask1, D * c->Wd, true); A(uniq1, D, true);
+  A(dstate, 1, true);
+  if (!c->dense) {
+    A(act_ids, B * S, true);
+    A(touched2, (N + 31) / 32, true); A(mask2, N * c->Wd, true); A(uniq2, N, true);
+    A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
+    A(keysA, (size_t)c->L * N, false);
+    if (c->sort_passes > 1) { A(keysB, (size_t)c->L * N, false); A(valsA, (size_t)c->L * N, false); }
+    if (c->sort_passes > 2) { A(valsB, (size_t)c->L * N, false); }
+    A(tile_hist, (size_t)c->L * ((size_t)1 << c->sort_width) * c->sort_tiles, false);
+  }
+#undef A
+  if (e == cudaSuccess) e = cudaMallocHost((void**)&c->pinned_loss, sizeof(float));
+  if (e == cudaSuccess) e = dalloc(&c->st_loss, 1, st, true);
+  if (e == cudaSuccess) e = setup_forward(c);
+  if (e == cudaSuccess) e = launch_init_gauss(c, c->W1, (int64_t)(D * H), RNG_W1);
+  if (e == cudaSuccess) e = launch_init_gauss(c, c->W2, (int64_t)(N * H), RNG_W2);
+  if (e == cudaSuccess && !c->dense) e = launch_draw_hash(c, 0);
+  if (e == cudaSuccess && !c->dense) e = launch_build_tables(c);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    dslide_status s = e == cudaErrorMemoryAllocation ? DSLIDE_ERR_OOM
+                      : e == cudaErrorInvalidValue ? DSLIDE_ERR_INVALID_ARG : DSLIDE_ERR_CUDA;
+    cudaGetLastError();
+    free_all(c);
+    delete h;
+    return s;
+  }
+  *out = h;
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_destroy(dslide_ctx* ctx) {
+  if (!ctx) return DSLIDE_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->c.cfg.device);
+  cudaStreamSynchronize(ctx->c.stream);
+  free_all(&ctx->c);
+  delete ctx;
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_rebuild_tables(dslide_ctx* ctx) {
+  if (!ctx) return DSLIDE_ERR_INVALID_ARG;
+  return rebuild(&ctx->c, true);
+}
+
+dslide_status dslide_build_tables(dslide_ctx* ctx) {
+  if (!ctx) return DSLIDE_ERR_INVALID_ARG;
+  return rebuild(&ctx->c, false);
+}
+
+dslide_status dslide_train_step(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
+                                const float* vals, const int32_t* label_ptr, const int32_t* labels, float* loss_out) {
+  if (!ctx || !row_ptr || !col_idx || !vals || !label_ptr || !labels) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
+  if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
+  CU(launch_forward_train(c, batch, row_ptr, col_idx, vals, label_ptr, labels));
+  CU(launch_update(c, batch, row_ptr, col_idx, vals, loss_out));
+  c->t_host += 1;
+  if (c->cfg.rebuild_period0 > 0 && c->t_host == c->next_rebuild) {
+    dslide_status s = rebuild(c, true);
+    if (s != DSLIDE_OK) return s;
+    double gap = floor((double)c->cfg.rebuild_period0 * exp((double)c->cfg.rebuild_growth_lambda * (double)c->r_host));
+    if (gap < 1.0) gap = 1.0;
+    c->next_rebuild += (int64_t)gap;
+  }
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
+                                     const float* vals, const int32_t* label_ptr, const int32_t* labels,
+                                     float* loss_out) {
+  if (!ctx || !row_ptr || !col_idx || !vals || !label_ptr || !labels) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
+  if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
+  const int64_t nnz = row_ptr[batch], nlab = label_ptr[batch];
+  if (nnz < 0 || nlab < 0 || row_ptr[0] != 0 || label_ptr[0] != 0) return DSLIDE_ERR_INVALID_ARG;
+  if (!c->st_row_ptr) {
+    CU(dalloc(&c->st_row_ptr, (size_t)c->cfg.max_batch + 1, c->stream, false));
+    CU(dalloc(&c->st_label_ptr, (size_t)c->cfg.max_batch + 1, c->stream, false));
+  }
+  if (nnz > c->st_nnz_cap) {
+    CU(cudaStreamSynchronize(c->stream));
+    if (c->st_col) cudaFree(c->st_col);
+    if (c->st_vals) cudaFree(c->st_vals);
+    c->st_col = nullptr; c->st_vals = nullptr; c->st_nnz_cap = 0;
+    int64_t cap = nnz + nnz / 2 + 1024;
+    CU(dalloc(&c->st_col, (size_t)cap, c->stream, false));
+    CU(dalloc(&c->st_vals, (size_t)cap, c->stream, false));
+    c->st_nnz_cap = cap;
+  }
+  if (nlab > c->st_lab_cap) {
+    CU(cudaStreamSynchronize(c->stream));
+    if (c->st_labels) cudaFree(c->st_labels);
+    c->st_labels = nullptr; c->st_lab_cap = 0;
+    int64_t cap = nlab + nlab / 2 + 1024;
+    CU(dalloc(&c->st_labels, (size_t)cap, c->stream, false));
+    c->st_lab_cap = cap;
+  }
+  cudaStream_t st = c->stream;
+  CU(cudaMemcpyAsync(c->st_row_ptr, row_ptr, sizeof(int32_t) * ((size_t)batch + 1), cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(c->st_label_ptr, label_ptr, sizeof(int32_t) * ((size_t)batch + 1), cudaMemcpyHostToDevice, st));
+  if (nnz > 0) {
+    CU(cudaMemcpyAsync(c->st_col, col_idx, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(c->st_vals, vals, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+  }
+  if (nlab > 0) CU(cudaMemcpyAsync(c->st_labels, labels, sizeof(int32_t) * (size_t)nlab, cudaMemcpyHostToDevice, st));
+  dslide_status s = dslide_train_step(ctx, batch, c->st_row_ptr, c->st_col, c->st_vals, c->st_label_ptr,
+                                      c->st_labels, c->st_loss);
+  if (s != DSLIDE_OK) return s;
+  CU(cudaMemcpyAsync(c->pinned_loss, c->st_loss, sizeof(float), cudaMemcpyDeviceToHost, st));
+  s = dslide_sync(ctx);
+  if (loss_out) *loss_out = *c->pinned_loss;
+  return s;
+}
+
+dslide_status dslide_predict_topk(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
+                                  const float* vals, int32_t k, int32_t dense, int32_t* out_ids, float* out_scores) {
+  if (!ctx || !row_ptr || !col_idx || !vals || !out_ids || !out_scores) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (batch < 1 || k < 1 || k > 64) return DSLIDE_ERR_INVALID_ARG;
+  if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
+  CU(launch_predict(c, batch, row_ptr, col_idx, vals, k, (dense || c->dense) ? 1 : 0, out_ids, out_scores));
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_sync(dslide_ctx* ctx) {
+  if (!ctx) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  int status = 0;
+  CU(cudaMemcpyAsync(&status, &c->dstate->status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  if (status != 0) {
+    CU(cudaMemsetAsync(&c->dstate->status, 0, sizeof(int), c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+  }
+  return (dslide_status)status;
+}
+
+dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes) {
+  if (!ctx || !nbytes) return DSLIDE_ERR_INVALID_ARG;
+  TensorRef t = tensor_ref(&ctx->c, which);
+  if (t.bytes < 0) return DSLIDE_ERR_INVALID_ARG;
+  if (ctx->c.dense && (which == DSLIDE_T_BUCKET_OFF || which == DSLIDE_T_BUCKET_IDS)) t.bytes = 0;
+  *nbytes = t.bytes;
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, int64_t nbytes) {
+  if (!ctx || !host_dst) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  int64_t want = 0;
+  dslide_status s = dslide_tensor_info(ctx, which, &want);
+  if (s != DSLIDE_OK) return s;
+  if (nbytes != want) return DSLIDE_ERR_INVALID_ARG;
+  if (which == DSLIDE_T_COUNTERS) {
+    int64_t v[3] = {c->t_host, c->r_host, c->next_rebuild};
+    memcpy(host_dst, v, sizeof(v));
+    return DSLIDE_OK;
+  }
+  if (want == 0) return DSLIDE_OK;
+  CU(cudaMemcpyAsync(host_dst, tensor_ref(c, which).ptr, (size_t)want, cudaMemcpyDeviceToHost, c->stream));
+  return drain(c);
+}
+
+dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host_src, int64_t nbytes) {
+  if (!ctx || !host_src) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  int64_t want = 0;
+  dslide_status s = dslide_tensor_info(ctx, which, &want);
+  if (s != DSLIDE_OK) return s;
+  if (nbytes != want) return DSLIDE_ERR_INVALID_ARG;
+  if (which == DSLIDE_T_COUNTERS) {
+    int64_t v[3];
+    memcpy(v, host_src, sizeof(v));
+    if (v[0] < 0 || v[1] < 0) return DSLIDE_ERR_INVALID_ARG;
+    c->t_host = v[0]; c->r_host = v[1]; c->next_rebuild = v[2];
+    long long t = v[0];
+    CU(cudaMemcpyAsync(&c->dstate->t, &t, sizeof(t), cudaMemcpyHostToDevice, c->stream));
+    return drain(c);
+  }
+  if (which == DSLIDE_T_HASH_IDX) {
+    const int32_t* ix = (const int32_t*)host_src;
+    for (int64_t i = 0; i < want / 4; ++i)
+      if (ix[i] < 0 || ix[i] >= c->H) return DSLIDE_ERR_INVALID_ARG;
+  }
+  if (which == DSLIDE_T_BUCKET_OFF || which == DSLIDE_T_BUCKET_IDS) return DSLIDE_ERR_INVALID_ARG;  // derived state
+  if (want == 0) return DSLIDE_OK;
+  CU(cudaMemcpyAsync(tensor_ref(c, which).ptr, host_src, (size_t)want, cudaMemcpyHostToDevice, c->stream));
+  return drain(c);
+}
+
+dslide_status dslide_last_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes, int32_t* stride) {
+  if (!ctx || !nbytes) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int64_t B = c->cfg.max_batch, S = c->act_stride;
+  if (stride) *stride = c->act_stride;
+  switch (which) {
+    case DSLIDE_LAST_HIDDEN: case DSLIDE_LAST_DHIDDEN: *nbytes = B * c->H * 4; return DSLIDE_OK;
+    case DSLIDE_LAST_CODES: *nbytes = B * c->L * 4; return DSLIDE_OK;
+    case DSLIDE_LAST_ACT_COUNT: case DSLIDE_LAST_LOSS: *nbytes = B * 4; return DSLIDE_OK;
+    case DSLIDE_LAST_ACT_IDS: *nbytes = c->dense ? 0 : B * S * 4; return DSLIDE_OK;
+    case DSLIDE_LAST_ACT_LOGIT: case DSLIDE_LAST_ACT_PROB: case DSLIDE_LAST_ACT_ERR: *nbytes = B * S * 4; return DSLIDE_OK;
+  }
+  return DSLIDE_ERR_INVALID_ARG;
+}
+
+dslide_status dslide_get_last(dslide_ctx* ctx, int32_t which, void* host_dst, int64_t nbytes) {
+  if (!ctx || !host_dst || nbytes < 0) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  int64_t size = 0;
+  dslide_status s = dslide_last_info(ctx, which, &size, nullptr);
+  if (s != DSLIDE_OK) return s;
+  const void* src = nullptr;
+  switch (which) {
+    case DSLIDE_LAST_HIDDEN: src = c->h; break;
+    case DSLIDE_LAST_DHIDDEN: src = c->dh; break;
+    case DSLIDE_LAST_CODES: src = c->codes; break;
+    case DSLIDE_LAST_ACT_COUNT: src = c->act_cnt; break;
+    case DSLIDE_LAST_LOSS: src = c->loss; break;
+    case DSLIDE_LAST_ACT_IDS: src = c->act_ids; break;
+    case DSLIDE_LAST_ACT_LOGIT: src = c->act_z; break;
+    case DSLIDE_LAST_ACT_PROB: src = c->act_p; break;
+    case DSLIDE_LAST_ACT_ERR: src = c->act_g; break;
+  }
+  int64_t n = nbytes < size ? nbytes : size;
+  if (n == 0 || !src) return DSLIDE_OK;
+  CU(cudaMemcpyAsync(host_dst, src, (size_t)n, cudaMemcpyDeviceToHost, c->stream));
+  return drain(c);
+}
+
+dslide_status dslide_last_stats(dslide_ctx* ctx, int64_t out[4]) {
+  if (!ctx || !out) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  DevState s;
+  CU(cudaMemcpyAsync(&s, c->dstate, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  out[0] = (int64_t)s.last_sum_active; out[1] = s.U2; out[2] = s.U1; out[3] = (int64_t)s.last_nnz;
+  return DSLIDE_OK;
+}
+
+int64_t dslide_kernel_launches(const dslide_ctx* ctx) { return ctx ? ctx->c.launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,107 @@
+// Internal declarations of libdslide (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dslide.h"
+
+namespace dslide {
+
+// ---------------------------------------------------------------------------
+// Counter-based random numbers: three rounds of the splitmix64 output function
+// over (seed, stream, rebuild count, counter).  Used for the initial weights and
+// for the hash functions of every rebuild (Algorithm 1: "Rebuild hash tables and
+// hash functions").
+// ---------------------------------------------------------------------------
+__host__ __device__ inline uint64_t sm64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+__host__ __device__ inline uint64_t ctr_rng(uint64_t seed, uint64_t stream, uint64_t r, uint64_t ctr) {
+  const uint64_t g = 0x9E3779B97F4A7C15ull;
+  uint64_t a = sm64(seed + g * (stream + 1));
+  uint64_t b = sm64(a + g * (r + 1));
+  return sm64(b + g * (ctr + 1));
+}
+enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2 };
+
+// Device-resident step state (read and written by kernels only; the host reads it
+// in the synchronous statistics and status calls).
+struct DevState {
+  int status;              // sticky dslide_status seen on the device
+  int U1, U2;              // distinct touched rows of W1 / W2 in the current step
+  int pad;
+  unsigned long long sum_active;   // accumulated by the forward kernel of the step in flight
+  unsigned long long nnz;
+  unsigned long long last_sum_active;   // totals of the last finished step
+  unsigned long long last_nnz;
+  long long t;             // Adam step count
+  float bc1, bc2;          // 1 - beta1^t, 1 - beta2^t
+};
+
+struct Ctx;
+
+// launches (implemented in the .cu files)
+cudaError_t launch_init_gauss(Ctx* c, float* w, int64_t n, uint64_t stream_id);
+cudaError_t launch_draw_hash(Ctx* c, int64_t r);
+cudaError_t launch_build_tables(Ctx* c);
+cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
+                                 const float* vals, const int32_t* label_ptr, const int32_t* labels);
+cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
+                          float* loss_out);
+cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
+                           const float* vals, int k, int dense, int32_t* out_ids, float* out_scores);
+cudaError_t setup_forward(Ctx* c);   // chooses the dedup path and the shared-memory layout
+
+struct Ctx {
+  dslide_config cfg;
+  int D, H, N, K, L, KL;
+  int bits;            // bits of a bucket code
+  int lg_bin;          // log2(dwta bin)
+  int fn_len;          // indices per hash function: srp_nnz (SimHash) or bin (DWTA)
+  int cap;
+  int64_t nb;          // buckets per table = 2^bits
+  int act_stride;      // row stride of the per-sample active arrays
+  int Wd;              // 32-bit words of a per-row sample mask = ceil(max_batch / 32)
+  int dense;
+  cudaStream_t stream;
+
+  float *W1, *b1, *W2, *b2;
+  float *mW1, *vW1, *mb1, *vb1, *mW2, *vW2, *mb2, *vb2;
+  int32_t *hash_idx, *hash_sign;
+  int32_t *bucket_off, *bucket_ids;
+
+  // per-step work space
+  float *h, *dh, *loss;
+  uint32_t* codes;
+  int32_t *act_cnt, *act_ids;
+  float *act_z, *act_p, *act_g;
+  uint32_t *touched1, *touched2;   // one bit per row of W1 / W2
+  uint32_t *mask1, *mask2;         // per row: which samples of the batch touch it
+  int32_t *uniq1, *uniq2;          // ascending distinct touched rows
+  DevState* dstate;
+
+  // rebuild work space
+  uint32_t *keysA, *keysB;
+  int32_t *valsA, *valsB;
+  int32_t* tile_hist;
+  int sort_passes, sort_width, sort_tiles;
+
+  // forward kernel layout
+  int dedup_mode;      // 1 bitmap, 2 sort
+  int fwd_smem;        // dynamic shared memory of the forward kernel
+  int sort_cap;        // capacity (power of two) of the shared-memory sort buffer
+  int num_sms;
+
+  // staging for the host-buffer entry point
+  int32_t *st_row_ptr, *st_col, *st_label_ptr, *st_labels;
+  float *st_vals, *st_loss;
+  int64_t st_nnz_cap, st_lab_cap;
+  float* pinned_loss;
+
+  int64_t t_host, r_host, next_rebuild;
+  int64_t launches;
+};
+
+}  // namespace dslide

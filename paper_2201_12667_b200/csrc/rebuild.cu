@@ -1,0 +1,315 @@
+// Initialisation and table (re)build (Algorithm 1: "Initialize layers with randomly generated
+// weights", "Hash weights to hash tables", "Rebuild hash tables and hash functions"; Section 2.1
+// phase 1; Section 3.1 "locally updated with a frequency schedule").
+//
+//   k_init_gauss   : weights ~ N(0, std^2) from the counter-based generator (Box-Muller).
+//   k_draw_simhash / k_draw_dwta : the hash functions of rebuild count r.
+//   k_hash_neurons : the L bucket codes of every row of W2 (same functions as the queries) and
+//                    the size of every bucket.
+//   k_bucket_scan  : bucket sizes -> bucket offsets (one block per table).
+//   k_sort_hist / k_sort_scan / k_sort_scatter : a stable least-significant-digit radix sort of the
+//                    neuron ids of each table by bucket code, so that every bucket lists its
+//                    neurons in ascending id (the first `cap` of them are what a query reads).
+#include "common.cuh"
+
+namespace dslide {
+
+// ------------------------------------------------------------------ weights
+__global__ void k_init_gauss(float* w, long long n, uint64_t seed, uint64_t stream_id, double std) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long step = (long long)gridDim.x * blockDim.x;
+  for (; i < n; i += step) {
+    uint64_t a = ctr_rng(seed, stream_id, 0, 2ull * (uint64_t)i);
+    uint64_t b = ctr_rng(seed, stream_id, 0, 2ull * (uint64_t)i + 1ull);
+    double u1 = ((double)(a >> 11) + 0.5) * (1.0 / 9007199254740992.0);
+    double u2 = ((double)(b >> 11) + 0.5) * (1.0 / 9007199254740992.0);
+    w[i] = (float)(std * sqrt(-2.0 * log(u1)) * cos(6.283185307179586476925 * u2));
+  }
+}
+
+cudaError_t launch_init_gauss(Ctx* c, float* w, int64_t n, uint64_t stream_id) {
+  if (n <= 0) return cudaSuccess;
+  k_init_gauss<<<c->num_sms * 8, 256, 0, c->stream>>>(w, n, c->cfg.seed, stream_id, (double)c->cfg.init_std);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ hash functions
+// SimHash: projection f has fn_len distinct coordinates (partial Fisher-Yates over 0..H-1, then
+// sorted ascending) and a sign per coordinate.  One thread per projection; H <= 1024.
+__global__ void k_draw_simhash(int32_t* idx, int32_t* sign, int KL, int H, int m, uint64_t seed, uint64_t r) {
+  int f = blockIdx.x * blockDim.x + threadIdx.x;
+  if (f >= KL) return;
+  short perm[1024];
+  for (int i = 0; i < H; ++i) perm[i] = (short)i;
+  for (int i = 0; i < m; ++i) {
+    uint64_t u = ctr_rng(seed, RNG_HASH, r, (uint64_t)f * 2ull * (uint64_t)m + (uint64_t)i);
+    int j = i + (int)(u % (uint64_t)(H - i));
+    short tmp = perm[i]; perm[i] = perm[j]; perm[j] = tmp;
+  }
+  for (int i = 1; i < m; ++i) {      // insertion sort of the chosen coordinates
+    short v = perm[i];
+    int q = i;
+    while (q > 0 && perm[q - 1] > v) { perm[q] = perm[q - 1]; --q; }
+    perm[q] = v;
+  }
+  for (int i = 0; i < m; ++i) {
+    uint64_t u = ctr_rng(seed, RNG_HASH, r, (uint64_t)f * 2ull * (uint64_t)m + (uint64_t)m + (uint64_t)i);
+    idx[(size_t)f * m + i] = perm[i];
+    sign[(size_t)f * m + i] = (u & 1ull) ? 1 : -1;
+  }
+}
+
+// DWTA: ceil(K*L*bin / H) random permutations of the coordinates, concatenated; hash function f
+// reads entries [f*bin, (f+1)*bin).  One thread per permutation.
+__global__ void k_draw_dwta(int32_t* idx, long long total, int H, uint64_t seed, uint64_t r, int nperm) {
+  int q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= nperm) return;
+  short perm[1024];
+  for (int i = 0; i < H; ++i) perm[i] = (short)i;
+  for (int i = H - 1; i >= 1; --i) {
+    uint64_t u = ctr_rng(seed, RNG_HASH, r, (uint64_t)q * (uint64_t)H + (uint64_t)i);
+    int j = (int)(u % (uint64_t)(i + 1));
+    short tmp = perm[i]; perm[i] = perm[j]; perm[j] = tmp;
+  }
+  for (int i = 0; i < H; ++i) {
+    long long e = (long long)q * H + i;
+    if (e < total) idx[e] = perm[i];
+  }
+}
+
+cudaError_t launch_draw_hash(Ctx* c, int64_t r) {
+  if (c->cfg.hash_family == DSLIDE_SIMHASH) {
+    k_draw_simhash<<<(c->KL + 63) / 64, 64, 0, c->stream>>>(c->hash_idx, c->hash_sign, c->KL, c->H, c->fn_len,
+                                                           c->cfg.seed, (uint64_t)r);
+  } else {
+    long long total = (long long)c->KL * c->fn_len;
+    int nperm = (int)((total + c->H - 1) / c->H);
+    k_draw_dwta<<<(nperm + 63) / 64, 64, 0, c->stream>>>(c->hash_idx, total, c->H, c->cfg.seed, (uint64_t)r, nperm);
+  }
+  c->launches++;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ codes of all neurons
+constexpr int HN_ROWS = 32;
+constexpr int HN_THREADS = 256;
+
+// A block stages HN_ROWS rows of W2 in shared memory (padded, so that 32 threads reading the same
+// column of 32 different rows hit 32 banks) and evaluates the L codes of each row.
+// keys[t][j] = code of neuron j in table t; counts[t][code + 1] += 1.
+__global__ void __launch_bounds__(HN_THREADS)
+k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, const int32_t* __restrict__ hsign,
+               uint32_t* keys, int32_t* counts, int N, int H, int K, int L, int family, int lg_bin, int fn_len,
+               long long nb) {
+  extern __shared__ float tile[];              // [HN_ROWS][H + 1]
+  const int ld = H + 1;
+  const int ntiles = (N + HN_ROWS - 1) / HN_ROWS;
+  for (int tl = blockIdx.x; tl < ntiles; tl += gridDim.x) {
+    const int j0 = tl * HN_ROWS;
+    const int rows = min(HN_ROWS, N - j0);
+    __syncthreads();
+    for (int e = threadIdx.x; e < rows * H; e += HN_THREADS) {
+      int r = e / H, k = e - r * H;
+      tile[r * ld + k] = W2[(size_t)(j0 + r) * H + k];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < HN_ROWS * L; e += HN_THREADS) {
+      const int r = e & (HN_ROWS - 1), t = e / HN_ROWS;
+      if (r >= rows) continue;
+      const float* v = tile + r * ld;
+      uint32_t code = 0;
+      for (int k = 0; k < K; ++k) {
+        const int f = t * K + k;
+        const int32_t* ix = hidx + (size_t)f * fn_len;
+        if (family == DSLIDE_SIMHASH) {
+          const int32_t* sg = hsign + (size_t)f * fn_len;
+          float sum = 0.f;
+          for (int i = 0; i < fn_len; ++i) {
+            float x = v[__ldg(ix + i)];
+            sum = __fadd_rn(sum, __ldg(sg + i) > 0 ? x : -x);
+          }
+          code |= (sum >= 0.f ? 1u : 0u) << k;
+        } else {
+          int best = 0;
+          float bv = v[__ldg(ix)];
+          for (int i = 1; i < fn_len; ++i) {
+            float x = v[__ldg(ix + i)];
+            if (x > bv) { bv = x; best = i; }
+          }
+          code |= (uint32_t)best << (k * lg_bin);
+        }
+      }
+      keys[(size_t)t * N + j0 + r] = code;
+      atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code + 1, 1);
+    }
+  }
+}
+
+// counts[t][0] = 0, counts[t][c + 1] = size of bucket c  ->  inclusive running sum = bucket offsets.
+__global__ void __launch_bounds__(1024) k_bucket_scan(int32_t* off, long long nb) {
+  __shared__ int sh[33];
+  int32_t* o = off + (size_t)blockIdx.x * (size_t)(nb + 1);
+  const long long n = nb + 1;
+  const long long chunk = (n + 1023) / 1024;
+  const long long beg = min(n, (long long)threadIdx.x * chunk), end = min(n, beg + chunk);
+  int sum = 0;
+  for (long long i = beg; i < end; ++i) sum += o[i];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int v = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += v;
+  }
+  if (lane == 31) sh[warp] = incl;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    for (int w = 0; w < 32; ++w) { int c = sh[w]; sh[w] = run; run += c; }
+  }
+  __syncthreads();
+  int run = incl - sum + sh[warp];
+  for (long long i = beg; i < end; ++i) { run += o[i]; o[i] = run; }
+}
+
+// ------------------------------------------------------------------ stable LSD radix sort, per table
+constexpr int SORT_THREADS = 256;
+constexpr int SORT_WARPS = SORT_THREADS / 32;
+constexpr int SORT_TILE = 8192;                      // elements per block
+constexpr int SORT_SUB = SORT_TILE / SORT_WARPS;     // contiguous elements per warp
+constexpr int SORT_MAX_WIDTH = 9;                    // bits per pass
+
+// hist[t][digit][tile] = number of keys of that digit in the tile.
+__global__ void __launch_bounds__(SORT_THREADS)
+k_sort_hist(const uint32_t* keys, int32_t* hist, int N, int tiles, int shift, int width) {
+  __shared__ int cnt[1 << SORT_MAX_WIDTH];
+  const int radix = 1 << width, t = blockIdx.y, tl = blockIdx.x;
+  for (int d = threadIdx.x; d < radix; d += SORT_THREADS) cnt[d] = 0;
+  __syncthreads();
+  const uint32_t* k = keys + (size_t)t * N;
+  const int beg = tl * SORT_TILE, end = min(N, beg + SORT_TILE);
+  for (int i = beg + threadIdx.x; i < end; i += SORT_THREADS) atomicAdd(&cnt[(k[i] >> shift) & (radix - 1)], 1);
+  __syncthreads();
+  for (int d = threadIdx.x; d < radix; d += SORT_THREADS) hist[((size_t)t * radix + d) * tiles + tl] = cnt[d];
+}
+
+// Exclusive scan of hist[t][*][*] in (digit, tile) order: where each tile's run of each digit starts.
+__global__ void __launch_bounds__(1024) k_sort_scan(int32_t* hist, int n) {
+  __shared__ int sh[33];
+  int32_t* o = hist + (size_t)blockIdx.x * n;
+  const int chunk = (n + 1023) / 1024;
+  const int beg = min(n, (int)threadIdx.x * chunk), end = min(n, beg + chunk);
+  int sum = 0;
+  for (int i = beg; i < end; ++i) sum += o[i];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int v = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += v;
+  }
+  if (lane == 31) sh[warp] = incl;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    for (int w = 0; w < 32; ++w) { int c = sh[w]; sh[w] = run; run += c; }
+  }
+  __syncthreads();
+  int run = incl - sum + sh[warp];
+  for (int i = beg; i < end; ++i) { int c = o[i]; o[i] = run; run += c; }
+}
+
+// Each warp owns a contiguous part of the tile and walks it in order, 32 keys at a time; equal
+// digits inside a group of 32 are ranked by lane with a match mask, so the scatter is stable.
+// vals_in == nullptr means the value of element i is i (first pass).  keys_out may be nullptr
+// (last pass).
+__global__ void __launch_bounds__(SORT_THREADS)
+k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_out, int32_t* vals_out,
+               const int32_t* hist, int N, int tiles, int shift, int width) {
+  __shared__ int offs[SORT_WARPS][1 << SORT_MAX_WIDTH];
+  const int radix = 1 << width, t = blockIdx.y, tl = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t* kin = keys_in + (size_t)t * N;
+  const int32_t* vin = vals_in ? vals_in + (size_t)t * N : nullptr;
+  uint32_t* kout = keys_out ? keys_out + (size_t)t * N : nullptr;
+  int32_t* vout = vals_out + (size_t)t * N;
+  const int wbeg = min(N, tl * SORT_TILE + warp * SORT_SUB), wend = min(N, wbeg + SORT_SUB);
+
+  for (int d = lane; d < radix; d += 32) offs[warp][d] = 0;
+  __syncwarp();
+  for (int i = wbeg + lane; i < wend; i += 32) atomicAdd(&offs[warp][(kin[i] >> shift) & (radix - 1)], 1);
+  __syncthreads();
+  for (int d = threadIdx.x; d < radix; d += SORT_THREADS) {
+    int run = hist[((size_t)t * radix + d) * tiles + tl];
+    for (int w = 0; w < SORT_WARPS; ++w) { int c = offs[w][d]; offs[w][d] = run; run += c; }
+  }
+  __syncthreads();
+  for (int i0 = wbeg; i0 < wend; i0 += 32) {
+    const int i = i0 + lane;
+    const bool live = i < wend;
+    const uint32_t key = live ? kin[i] : 0u;
+    const int digit = live ? (int)((key >> shift) & (radix - 1)) : radix + lane;   // dead lanes match nobody
+    const unsigned peers = __match_any_sync(0xffffffffu, digit);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    int base = 0;
+    if (live) base = offs[warp][digit];
+    __syncwarp();
+    if (live && rank == 0) offs[warp][digit] = base + __popc(peers);
+    __syncwarp();
+    if (live) {
+      const int dst = base + rank;
+      if (kout) kout[dst] = key;
+      vout[dst] = vin ? vin[i] : i;
+    }
+  }
+}
+
+cudaError_t launch_build_tables(Ctx* c) {
+  const size_t off_bytes = (size_t)c->L * (size_t)(c->nb + 1) * sizeof(int32_t);
+  cudaError_t e = cudaMemsetAsync(c->bucket_off, 0, off_bytes, c->stream);
+  if (e != cudaSuccess) return e;
+  const int smem = HN_ROWS * (c->H + 1) * (int)sizeof(float);
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(k_hash_neurons, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+  }
+  k_hash_neurons<<<c->num_sms * 4, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
+                                                                 c->bucket_off, c->N, c->H, c->K, c->L,
+                                                                 c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
+  c->launches++;
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  k_bucket_scan<<<c->L, 1024, 0, c->stream>>>(c->bucket_off, c->nb);
+  c->launches++;
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+  const uint32_t* kin = c->keysA;
+  const int32_t* vin = nullptr;
+  for (int pass = 0; pass < c->sort_passes; ++pass) {
+    const bool last = pass == c->sort_passes - 1;
+    const int shift = pass * c->sort_width;
+    const int width = min(c->sort_width, c->bits - shift);
+    const int radix = 1 << width;
+    uint32_t* kout = last ? nullptr : (kin == c->keysA ? c->keysB : c->keysA);
+    int32_t* vout = last ? c->bucket_ids : (vin == c->valsA ? c->valsB : c->valsA);
+    dim3 grid(c->sort_tiles, c->L);
+    k_sort_hist<<<grid, SORT_THREADS, 0, c->stream>>>(kin, c->tile_hist, c->N, c->sort_tiles, shift, width);
+    c->launches++;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_sort_scan<<<c->L, 1024, 0, c->stream>>>(c->tile_hist, radix * c->sort_tiles);
+    c->launches++;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_sort_scatter<<<grid, SORT_THREADS, 0, c->stream>>>(kin, vin, kout, vout, c->tile_hist, c->N, c->sort_tiles,
+                                                        shift, width);
+    c->launches++;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    kin = kout;
+    vin = vout;
+  }
+  return cudaSuccess;
+}
+
+int sort_tile_elems() { return SORT_TILE; }
+int sort_max_width() { return SORT_MAX_WIDTH; }
+
+}  // namespace dslide

@@ -53,16 +53,17 @@ def small_batch(rng, B, D, N, nnz, max_labels=3, dtype=np.float64):
     return row_ptr, np.concatenate(cols), np.concatenate(vals), label_ptr, np.concatenate(labs)
 
 
-def max_rel_err(a, b):
-    """max_i |a_i - b_i| / max(|a_i|, |b_i|, floor), floor = 1e-3 of the tensor's largest magnitude.
+def max_rel_err(a, b, floor_frac=1e-3):
+    """max_i |a_i - b_i| / max(|a_i|, |b_i|, floor), floor = floor_frac * the tensor's largest magnitude.
 
-    The floor keeps elements that are (near) zero from turning a rounding-level
-    absolute difference into a huge relative one.
+    The floor keeps elements that are (near) zero through cancellation from turning a
+    rounding-level absolute difference into a huge relative one.
     """
     a = np.asarray(a, dtype=np.float64).ravel()
     b = np.asarray(b, dtype=np.float64).ravel()
+    assert a.shape == b.shape
     if a.size == 0:
         return 0.0
     scale = max(np.max(np.abs(a)), np.max(np.abs(b)), 1e-30)
-    den = np.maximum(np.maximum(np.abs(a), np.abs(b)), 1e-3 * scale)
+    den = np.maximum(np.maximum(np.abs(a), np.abs(b)), floor_frac * scale)
     return float(np.max(np.abs(a - b) / den))
