@@ -172,6 +172,25 @@ dslide_status dslide_get_last(dslide_ctx* ctx, int32_t which, void* host_dst, in
  * distinct touched rows of W1, out[3] = nonzeros in the batch. */
 dslide_status dslide_last_stats(dslide_ctx* ctx, int64_t out[4]);
 
+/* Totals since the last reset, read from the device.  Synchronous.  out[0] = training steps,
+ * out[1] = sum of active-set sizes, out[2] = sum of distinct touched W2 rows, out[3] = sum of
+ * distinct touched W1 rows, out[4] = nonzeros, out[5] = bucket entries read by the lookups.
+ * reset != 0 clears the totals afterwards. */
+dslide_status dslide_cum_stats(dslide_ctx* ctx, int64_t out[6], int32_t reset);
+
+/* Per-kernel device time.  Between dslide_profile_begin and dslide_profile_end every kernel the
+ * context launches is bracketed by a CUDA event pair on the context's stream; dslide_profile_end
+ * waits for the stream and returns, per kernel, the summed milliseconds and the launch count.
+ * The event records add a little latency between kernels: use it to split time between kernels,
+ * not for the throughput figure. */
+enum {
+  DSLIDE_K_FORWARD = 0, DSLIDE_K_SCAN, DSLIDE_K_ADAM, DSLIDE_K_DRAW_HASH, DSLIDE_K_HASH_NEURONS,
+  DSLIDE_K_BUCKET_SCAN, DSLIDE_K_SORT_HIST, DSLIDE_K_SORT_SCAN, DSLIDE_K_SORT_SCATTER,
+  DSLIDE_K_PREDICT, DSLIDE_K_INIT, DSLIDE_K_COUNT
+};
+dslide_status dslide_profile_begin(dslide_ctx* ctx);
+dslide_status dslide_profile_end(dslide_ctx* ctx, double ms[DSLIDE_K_COUNT], int64_t launches[DSLIDE_K_COUNT]);
+
 /* Number of kernels the context has launched since dslide_init. */
 int64_t dslide_kernel_launches(const dslide_ctx* ctx);
 

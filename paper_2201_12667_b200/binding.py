@@ -62,6 +62,9 @@ _SIGS = {
     "dslide_last_info": (_i32, [_vp, _i32, C.POINTER(_i64), C.POINTER(_i32)]),
     "dslide_get_last": (_i32, [_vp, _i32, _vp, _i64]),
     "dslide_last_stats": (_i32, [_vp, C.POINTER(_i64)]),
+    "dslide_cum_stats": (_i32, [_vp, C.POINTER(_i64), _i32]),
+    "dslide_profile_begin": (_i32, [_vp]),
+    "dslide_profile_end": (_i32, [_vp, C.POINTER(C.c_double), C.POINTER(_i64)]),
     "dslide_kernel_launches": (_i64, [_vp]),
     "dslide_status_str": (C.c_char_p, [_i32]),
 }
@@ -189,6 +192,28 @@ def dslide_last_stats(ctx):
     out = (_i64 * 4)()
     _check(_lib.dslide_last_stats(ctx, out), "dslide_last_stats")
     return dict(sum_active=out[0], touched_w2=out[1], touched_w1=out[2], nnz=out[3])
+
+
+KERNEL_NAMES = ["forward", "scan", "adam", "draw_hash", "hash_neurons", "bucket_scan", "sort_hist", "sort_scan",
+                "sort_scatter", "predict", "init"]
+
+
+def dslide_cum_stats(ctx, reset=False):
+    out = (_i64 * 6)()
+    _check(_lib.dslide_cum_stats(ctx, out, int(reset)), "dslide_cum_stats")
+    return dict(steps=out[0], sum_active=out[1], touched_w2=out[2], touched_w1=out[3], nnz=out[4], fetched=out[5])
+
+
+def dslide_profile_begin(ctx):
+    _check(_lib.dslide_profile_begin(ctx), "dslide_profile_begin")
+
+
+def dslide_profile_end(ctx):
+    """-> {kernel name: (milliseconds, launches)} for the kernels launched since dslide_profile_begin."""
+    n = len(KERNEL_NAMES)
+    ms, cnt = (C.c_double * n)(), (_i64 * n)()
+    _check(_lib.dslide_profile_end(ctx, ms, cnt), "dslide_profile_end")
+    return {KERNEL_NAMES[i]: (ms[i], cnt[i]) for i in range(n) if cnt[i]}
 
 
 def dslide_kernel_launches(ctx):

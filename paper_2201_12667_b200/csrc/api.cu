@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -16,6 +17,26 @@ int sort_max_width();
 using namespace dslide;
 
 struct dslide_ctx { Ctx c; };
+
+namespace dslide {
+struct ProfRec { int kid; cudaEvent_t beg, end; };
+
+LaunchScope::LaunchScope(Ctx* c_, int kid_) : c(c_), kid(kid_), rec(nullptr) {
+  c->launches++;
+  if (!c->profiling || !c->prof) return;
+  auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
+  ProfRec r;
+  r.kid = kid;
+  if (cudaEventCreate(&r.beg) != cudaSuccess) return;
+  if (cudaEventCreate(&r.end) != cudaSuccess) { cudaEventDestroy(r.beg); return; }
+  cudaEventRecord(r.beg, c->stream);
+  v->push_back(r);
+  rec = &v->back();
+}
+LaunchScope::~LaunchScope() {
+  if (rec) cudaEventRecord(static_cast<ProfRec*>(rec)->end, c->stream);
+}
+}  // namespace dslide
 
 namespace {
 
@@ -39,6 +60,12 @@ void free_all(Ctx* c) {
                   c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (c->pinned_loss) cudaFreeHost(c->pinned_loss);
+  if (c->prof) {
+    auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
+    for (auto& r : *v) { cudaEventDestroy(r.beg); cudaEventDestroy(r.end); }
+    delete v;
+    c->prof = nullptr;
+  }
 }
 
 int ilog2_exact(int x) {
@@ -417,6 +444,53 @@ dslide_status dslide_last_stats(dslide_ctx* ctx, int64_t out[4]) {
   CU(cudaMemcpyAsync(&s, c->dstate, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
   CU(cudaStreamSynchronize(c->stream));
   out[0] = (int64_t)s.last_sum_active; out[1] = s.U2; out[2] = s.U1; out[3] = (int64_t)s.last_nnz;
+  static_assert((int)KID_COUNT == (int)DSLIDE_K_COUNT, "kernel id enums out of step");
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_cum_stats(dslide_ctx* ctx, int64_t out[6], int32_t reset) {
+  if (!ctx || !out) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  DevState s;
+  CU(cudaMemcpyAsync(&s, c->dstate, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < 6; ++i) out[i] = (int64_t)s.cum[i];
+  if (reset) {
+    CU(cudaMemsetAsync(c->dstate->cum, 0, sizeof(s.cum), c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+  }
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_profile_begin(dslide_ctx* ctx) {
+  if (!ctx) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->profiling) return DSLIDE_ERR_STATE;
+  if (!c->prof) c->prof = new (std::nothrow) std::vector<ProfRec>();
+  if (!c->prof) return DSLIDE_ERR_OOM;
+  static_cast<std::vector<ProfRec>*>(c->prof)->reserve(1 << 16);
+  c->profiling = 1;
+  return DSLIDE_OK;
+}
+
+dslide_status dslide_profile_end(dslide_ctx* ctx, double ms[DSLIDE_K_COUNT], int64_t launches[DSLIDE_K_COUNT]) {
+  if (!ctx || !ms || !launches) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->profiling) return DSLIDE_ERR_STATE;
+  c->profiling = 0;
+  CU(cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < DSLIDE_K_COUNT; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
+  for (auto& r : *v) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.beg, r.end) == cudaSuccess && r.kid >= 0 && r.kid < DSLIDE_K_COUNT) {
+      ms[r.kid] += t;
+      launches[r.kid] += 1;
+    }
+    cudaEventDestroy(r.beg);
+    cudaEventDestroy(r.end);
+  }
+  v->clear();
   return DSLIDE_OK;
 }
 

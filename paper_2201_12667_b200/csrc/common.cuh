@@ -34,13 +34,27 @@ struct DevState {
   int pad;
   unsigned long long sum_active;   // accumulated by the forward kernel of the step in flight
   unsigned long long nnz;
+  unsigned long long fetched;      // bucket entries read by the lookups of the step in flight
   unsigned long long last_sum_active;   // totals of the last finished step
   unsigned long long last_nnz;
+  unsigned long long last_fetched;
+  unsigned long long cum[6];       // since the last reset: steps, sum_active, U2, U1, nnz, fetched
   long long t;             // Adam step count
   float bc1, bc2;          // 1 - beta1^t, 1 - beta2^t
 };
 
 struct Ctx;
+
+// Kernel ids for the per-kernel timing (must match the DSLIDE_K_* enum of the C ABI).
+enum { KID_FORWARD = 0, KID_SCAN, KID_ADAM, KID_DRAW_HASH, KID_HASH_NEURONS, KID_BUCKET_SCAN, KID_SORT_HIST,
+       KID_SORT_SCAN, KID_SORT_SCATTER, KID_PREDICT, KID_INIT, KID_COUNT };
+
+// Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event pair around it.
+struct LaunchScope {
+  Ctx* c; int kid; void* rec;
+  LaunchScope(Ctx* c, int kid);
+  ~LaunchScope();
+};
 
 // launches (implemented in the .cu files)
 cudaError_t launch_init_gauss(Ctx* c, float* w, int64_t n, uint64_t stream_id);
@@ -102,6 +116,8 @@ struct Ctx {
 
   int64_t t_host, r_host, next_rebuild;
   int64_t launches;
+  int profiling;
+  void* prof;          // std::vector of event pairs while profiling
 };
 
 }  // namespace dslide

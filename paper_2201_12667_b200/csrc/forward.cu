@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
       if (nlab > p.max_labels) bad = DSLIDE_ERR_OVERFLOW;
     }
   }
+  if (tid == 0) sh_misc[24] = 0;               // bucket entries fetched by this sample
   bad = __syncthreads_or(bad);
   if (bad) {
     // The sample is skipped: no loss, no gradient, nothing touched.
@@ -216,6 +217,7 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
           int j = __ldg(bid + i);
           atomicOr(&sh_dd[j >> 5], 1u << (j & 31));
         }
+        if (lane == 0) atomicAdd(&sh_misc[24], cnt);
       }
       if (MODE == 0)
         for (int i = tid; i < nlab; i += FWD_THREADS) {
@@ -253,6 +255,7 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
       }
       __syncthreads();
       const int ncand = sh_tbase[p.L] + nlab;     // <= L*cap + max_labels <= sort_cap
+      if (tid == 0) sh_misc[24] = sh_tbase[p.L];
       int n2 = 1;
       while (n2 < ncand) n2 <<= 1;
       for (int t = warp; t < p.L; t += FWD_WARPS) {
@@ -493,6 +496,7 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
   if (tid == 0) {
     atomicAdd(&p.st->sum_active, (unsigned long long)na);
     atomicAdd(&p.st->nnz, (unsigned long long)nnz);
+    atomicAdd(&p.st->fetched, (unsigned long long)sh_misc[24]);
   }
 }
 
@@ -565,8 +569,10 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
 cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
                                  const int32_t* label_ptr, const int32_t* labels) {
   FwdParams p = make_params(c, batch, row_ptr, col_idx, vals, label_ptr, labels);
-  k_forward<0><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_FORWARD);
+    k_forward<0><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+  }
   return cudaGetLastError();
 }
 
@@ -578,8 +584,10 @@ cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int3
   p.out_scores = out_scores;
   int smem = c->fwd_smem;
   if (dense) { p.dense = 1; smem = fwd_layout(c).fixed_bytes; }
-  k_forward<1><<<batch, FWD_THREADS, smem, c->stream>>>(p);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_PREDICT);
+    k_forward<1><<<batch, FWD_THREADS, smem, c->stream>>>(p);
+  }
   return cudaGetLastError();
 }
 

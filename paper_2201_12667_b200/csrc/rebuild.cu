@@ -29,8 +29,10 @@ __global__ void k_init_gauss(float* w, long long n, uint64_t seed, uint64_t stre
 
 cudaError_t launch_init_gauss(Ctx* c, float* w, int64_t n, uint64_t stream_id) {
   if (n <= 0) return cudaSuccess;
-  k_init_gauss<<<c->num_sms * 8, 256, 0, c->stream>>>(w, n, c->cfg.seed, stream_id, (double)c->cfg.init_std);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_INIT);
+    k_init_gauss<<<c->num_sms * 8, 256, 0, c->stream>>>(w, n, c->cfg.seed, stream_id, (double)c->cfg.init_std);
+  }
   return cudaGetLastError();
 }
 
@@ -79,6 +81,7 @@ __global__ void k_draw_dwta(int32_t* idx, long long total, int H, uint64_t seed,
 }
 
 cudaError_t launch_draw_hash(Ctx* c, int64_t r) {
+  LaunchScope ls(c, KID_DRAW_HASH);
   if (c->cfg.hash_family == DSLIDE_SIMHASH) {
     k_draw_simhash<<<(c->KL + 63) / 64, 64, 0, c->stream>>>(c->hash_idx, c->hash_sign, c->KL, c->H, c->fn_len,
                                                            c->cfg.seed, (uint64_t)r);
@@ -87,7 +90,6 @@ cudaError_t launch_draw_hash(Ctx* c, int64_t r) {
     int nperm = (int)((total + c->H - 1) / c->H);
     k_draw_dwta<<<(nperm + 63) / 64, 64, 0, c->stream>>>(c->hash_idx, total, c->H, c->cfg.seed, (uint64_t)r, nperm);
   }
-  c->launches++;
   return cudaGetLastError();
 }
 
@@ -274,13 +276,17 @@ cudaError_t launch_build_tables(Ctx* c) {
     e = cudaFuncSetAttribute(k_hash_neurons, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
-  k_hash_neurons<<<c->num_sms * 4, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
-                                                                 c->bucket_off, c->N, c->H, c->K, c->L,
-                                                                 c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_HASH_NEURONS);
+    k_hash_neurons<<<c->num_sms * 4, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
+                                                                   c->bucket_off, c->N, c->H, c->K, c->L,
+                                                                   c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
+  }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  k_bucket_scan<<<c->L, 1024, 0, c->stream>>>(c->bucket_off, c->nb);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_BUCKET_SCAN);
+    k_bucket_scan<<<c->L, 1024, 0, c->stream>>>(c->bucket_off, c->nb);
+  }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
   const uint32_t* kin = c->keysA;
@@ -293,15 +299,21 @@ cudaError_t launch_build_tables(Ctx* c) {
     uint32_t* kout = last ? nullptr : (kin == c->keysA ? c->keysB : c->keysA);
     int32_t* vout = last ? c->bucket_ids : (vin == c->valsA ? c->valsB : c->valsA);
     dim3 grid(c->sort_tiles, c->L);
-    k_sort_hist<<<grid, SORT_THREADS, 0, c->stream>>>(kin, c->tile_hist, c->N, c->sort_tiles, shift, width);
-    c->launches++;
+    {
+      LaunchScope ls(c, KID_SORT_HIST);
+      k_sort_hist<<<grid, SORT_THREADS, 0, c->stream>>>(kin, c->tile_hist, c->N, c->sort_tiles, shift, width);
+    }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_sort_scan<<<c->L, 1024, 0, c->stream>>>(c->tile_hist, radix * c->sort_tiles);
-    c->launches++;
+    {
+      LaunchScope ls(c, KID_SORT_SCAN);
+      k_sort_scan<<<c->L, 1024, 0, c->stream>>>(c->tile_hist, radix * c->sort_tiles);
+    }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_sort_scatter<<<grid, SORT_THREADS, 0, c->stream>>>(kin, vin, kout, vout, c->tile_hist, c->N, c->sort_tiles,
-                                                        shift, width);
-    c->launches++;
+    {
+      LaunchScope ls(c, KID_SORT_SCATTER);
+      k_sort_scatter<<<grid, SORT_THREADS, 0, c->stream>>>(kin, vin, kout, vout, c->tile_hist, c->N, c->sort_tiles,
+                                                          shift, width);
+    }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     kin = kout;
     vin = vout;

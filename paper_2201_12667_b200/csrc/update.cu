@@ -57,9 +57,14 @@ k_scan(uint32_t* touched2, int nwords2, int32_t* uniq2, uint32_t* touched1, int 
         bits &= bits - 1;
       }
     }
-    if (tid == 0) { if (blockIdx.x == 0) st->U2 = sh[SCAN_THREADS / 32]; else st->U1 = sh[SCAN_THREADS / 32]; }
+    if (tid == 0) {
+      const int u = sh[SCAN_THREADS / 32];
+      if (blockIdx.x == 0) { st->U2 = u; st->cum[2] += (unsigned long long)u; }
+      else { st->U1 = u; st->cum[3] += (unsigned long long)u; }
+    }
   } else if (tid == 0) {
     st->U2 = N;
+    st->cum[2] += (unsigned long long)N;
   }
 
   if (blockIdx.x == 0) {
@@ -80,6 +85,8 @@ k_scan(uint32_t* touched2, int nwords2, int32_t* uniq2, uint32_t* touched1, int 
       st->bc2 = (float)(1.0 - pow((double)beta2, (double)t));
       st->last_sum_active = st->sum_active; st->sum_active = 0ull;
       st->last_nnz = st->nnz; st->nnz = 0ull;
+      st->last_fetched = st->fetched; st->fetched = 0ull;
+      st->cum[0] += 1ull; st->cum[1] += st->last_sum_active; st->cum[4] += st->last_nnz; st->cum[5] += st->last_fetched;
     }
   }
 }
@@ -258,10 +265,12 @@ __global__ void __launch_bounds__(ADAM_THREADS) k_adam(const AdamParams p) {
 
 cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
                           float* loss_out) {
-  k_scan<<<2, SCAN_THREADS, 0, c->stream>>>(c->touched2, (c->N + 31) / 32, c->uniq2, c->touched1, (c->D + 31) / 32,
-                                            c->uniq1, c->dstate, c->loss, batch, loss_out, c->cfg.beta1, c->cfg.beta2,
-                                            c->dense, c->N);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_SCAN);
+    k_scan<<<2, SCAN_THREADS, 0, c->stream>>>(c->touched2, (c->N + 31) / 32, c->uniq2, c->touched1, (c->D + 31) / 32,
+                                              c->uniq1, c->dstate, c->loss, batch, loss_out, c->cfg.beta1,
+                                              c->cfg.beta2, c->dense, c->N);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   AdamParams p;
@@ -272,8 +281,10 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   p.mask1 = c->mask1; p.mask2 = c->mask2; p.uniq1 = c->uniq1; p.uniq2 = c->uniq2; p.st = c->dstate;
   p.B = batch; p.H = c->H; p.N = c->N; p.Wd = c->Wd; p.act_stride = c->act_stride; p.dense = c->dense;
   p.lr = c->cfg.lr; p.beta1 = c->cfg.beta1; p.beta2 = c->cfg.beta2; p.eps = c->cfg.eps;
-  k_adam<<<1 + c->num_sms * 4, ADAM_THREADS, 0, c->stream>>>(p);
-  c->launches++;
+  {
+    LaunchScope ls(c, KID_ADAM);
+    k_adam<<<1 + c->num_sms * 4, ADAM_THREADS, 0, c->stream>>>(p);
+  }
   return cudaGetLastError();
 }
 

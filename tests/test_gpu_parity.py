@@ -3,9 +3,11 @@
 Bars: hash functions, bucket codes, tables and active sets bit-exact; the hidden layer bit-exact on
 identical weights (its summation order is part of the definition); logits, probabilities, loss and
 back-propagated errors within 1e-4 relative; weights after 10 Adam steps within 1e-3 relative.
-Relative error is |a-b| / max(|a|,|b|,floor) with floor = 1e-2 (activations) or 1e-3 (weights) of the
-tensor's largest magnitude, so that entries that cancel to nearly zero are judged on an absolute
-scale.
+Relative error is |a-b| / max(|a|,|b|,floor) with floor = 1e-2 of the tensor's largest magnitude, so
+that entries that cancel to nearly zero are judged on an absolute scale.  (Adam divides by the
+gradient's magnitude, so fp32 rounding in a cancelling gradient sum moves a weight by a fraction of
+lr whatever the weight's size: the fp32 and fp64 builds of the oracle themselves differ by 2e-4 under
+this measure after 10 steps, and by more than 1e-3 with a floor ten times smaller.)
 """
 import numpy as np
 import pytest
@@ -69,7 +71,7 @@ def compare_forward(pr, batch, bit_exact_hidden=True, tol=ACT_TOL):
 
 def compare_weights(pr, tol=W_TOL, names=None):
     for n in names or (WEIGHTS + MOMENTS):
-        e = max_rel_err(ds.dslide_get_tensor(pr.ctx, n), pr.o.get(n), 1e-3)
+        e = max_rel_err(ds.dslide_get_tensor(pr.ctx, n), pr.o.get(n), 1e-2)
         assert e < tol, (n, e)
 
 
@@ -389,11 +391,11 @@ def test_full_size_670k_step_against_oracle():
         act = np.unique(pr.o.get("act_ids"))
         W2g = ds.dslide_get_tensor(pr.ctx, "W2").reshape(pr.N, pr.H)
         W2o = pr.o.view("W2").reshape(pr.N, pr.H)
-        assert max_rel_err(W2g[act], W2o[act], 1e-3) < W_TOL
+        assert max_rel_err(W2g[act], W2o[act], 1e-2) < W_TOL
         rest = np.setdiff1d(np.arange(0, pr.N, 97), act)
         assert np.array_equal(W2g[rest].view(np.uint32), W2o[rest].view(np.uint32))
         feats = np.unique(batch[1])
         W1g = ds.dslide_get_tensor(pr.ctx, "W1").reshape(pr.D, pr.H)
-        assert max_rel_err(W1g[feats], pr.o.view("W1").reshape(pr.D, pr.H)[feats], 1e-3) < W_TOL
+        assert max_rel_err(W1g[feats], pr.o.view("W1").reshape(pr.D, pr.H)[feats], 1e-2) < W_TOL
     finally:
         pr.close()
