@@ -191,6 +191,34 @@ enum {
 dslide_status dslide_profile_begin(dslide_ctx* ctx);
 dslide_status dslide_profile_end(dslide_ctx* ctx, double ms[DSLIDE_K_COUNT], int64_t launches[DSLIDE_K_COUNT]);
 
+/* Bucket sort of one hash table for callers that must not allocate.  (The paper has no
+ * counterpart: this is a packaging variant of the table build's sort, not a step of the method.)
+ *
+ * Who needs it: code that reaches this library from a place where device allocation is off
+ * limits -- a plug-in that is only handed buffers, a service that has promised a fixed memory
+ * footprint, a caller running inside somebody else's memory pool.  This call makes no
+ * cudaMalloc / cudaFree and calls nothing that allocates; it needs no dslide_ctx.  Its work
+ * space is a static device array inside the library image: every GPU that loads libdslide.so
+ * holds those DSLIDE_STATIC_SORT_MAX_N * 8 bytes (2 MiB) until the process exits.
+ *
+ * codes[n] (device): bucket code of neuron i in this table; only the low `bits` bits are used.
+ * Output (device, caller-owned): bucket_off[2^bits + 1] = where each bucket starts in
+ * bucket_ids (bucket_off[0] = 0, bucket_off[2^bits] = n); bucket_ids[n] = the ids 0..n-1
+ * grouped by code, ascending inside a bucket -- the layout of one table of
+ * DSLIDE_T_BUCKET_OFF / DSLIDE_T_BUCKET_IDS.  Both outputs are fully overwritten.
+ * Limits: 0 <= n <= DSLIDE_STATIC_SORT_MAX_N and 1 <= bits <= DSLIDE_STATIC_SORT_MAX_BITS,
+ * otherwise DSLIDE_ERR_OVERFLOW and nothing is launched.
+ * Runs as one thread block on `stream` (a cudaStream_t, NULL = default stream) of the CURRENT
+ * device, asynchronously.  The first call on each device looks up the array's device address
+ * (once per device, with that device current); make that first call before any stream capture.
+ * All calls on a device share the one array, which keeps the last call's contents: the kernel
+ * overwrites what it reads, but two calls that overlap on the GPU (different streams, no
+ * ordering between them) race on it -- order them. */
+#define DSLIDE_STATIC_SORT_MAX_N 262144
+#define DSLIDE_STATIC_SORT_MAX_BITS 18
+dslide_status dslide_bucket_sort_static(const uint32_t* codes, int32_t n, int32_t bits,
+                                        int32_t* bucket_off, int32_t* bucket_ids, void* stream);
+
 /* Number of kernels the context has launched since dslide_init. */
 int64_t dslide_kernel_launches(const dslide_ctx* ctx);
 

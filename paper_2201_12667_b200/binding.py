@@ -65,6 +65,7 @@ _SIGS = {
     "dslide_cum_stats": (_i32, [_vp, C.POINTER(_i64), _i32]),
     "dslide_profile_begin": (_i32, [_vp]),
     "dslide_profile_end": (_i32, [_vp, C.POINTER(C.c_double), C.POINTER(_i64)]),
+    "dslide_bucket_sort_static": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "dslide_kernel_launches": (_i64, [_vp]),
     "dslide_status_str": (C.c_char_p, [_i32]),
 }
@@ -214,6 +215,23 @@ def dslide_profile_end(ctx):
     ms, cnt = (C.c_double * n)(), (_i64 * n)()
     _check(_lib.dslide_profile_end(ctx, ms, cnt), "dslide_profile_end")
     return {KERNEL_NAMES[i]: (ms[i], cnt[i]) for i in range(n) if cnt[i]}
+
+
+STATIC_SORT_MAX_N = 262144
+STATIC_SORT_MAX_BITS = 18
+
+
+def dslide_bucket_sort_static(codes, n, bits, bucket_off, bucket_ids, stream=None):
+    """Group ids 0..n-1 by bucket code without allocating (see include/dslide.h).
+
+    codes: CUDA uint32/int32 tensor [n]; bucket_off: CUDA int32 tensor [2**bits + 1]; bucket_ids: CUDA int32
+    tensor [n]; stream: a torch stream or None for torch's current stream.  The library allocates nothing;
+    the tensors are the caller's.
+    """
+    import torch
+    st = (stream or torch.cuda.current_stream()).cuda_stream
+    _check(_lib.dslide_bucket_sort_static(_dptr(codes), n, bits, _dptr(bucket_off), _dptr(bucket_ids), st),
+           "dslide_bucket_sort_static")
 
 
 def dslide_kernel_launches(ctx):
