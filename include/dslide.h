@@ -184,7 +184,7 @@ dslide_status dslide_cum_stats(dslide_ctx* ctx, int64_t out[6], int32_t reset);
  * The event records add a little latency between kernels: use it to split time between kernels,
  * not for the throughput figure. */
 enum {
-  DSLIDE_K_FORWARD = 0, DSLIDE_K_SCAN, DSLIDE_K_ADAM, DSLIDE_K_DRAW_HASH, DSLIDE_K_HASH_NEURONS,
+  DSLIDE_K_FORWARD = 0, DSLIDE_K_ADAM_DENSE, DSLIDE_K_ADAM, DSLIDE_K_DRAW_HASH, DSLIDE_K_HASH_NEURONS,
   DSLIDE_K_BUCKET_SCAN, DSLIDE_K_SORT_HIST, DSLIDE_K_SORT_SCAN, DSLIDE_K_SORT_SCATTER,
   DSLIDE_K_PREDICT, DSLIDE_K_INIT, DSLIDE_K_COUNT
 };

@@ -195,7 +195,7 @@ def dslide_last_stats(ctx):
     return dict(sum_active=out[0], touched_w2=out[1], touched_w1=out[2], nnz=out[3])
 
 
-KERNEL_NAMES = ["forward", "scan", "adam", "draw_hash", "hash_neurons", "bucket_scan", "sort_hist", "sort_scan",
+KERNEL_NAMES = ["forward", "adam_dense", "adam", "draw_hash", "hash_neurons", "bucket_scan", "sort_hist", "sort_scan",
                 "sort_scatter", "predict", "init"]
 
 

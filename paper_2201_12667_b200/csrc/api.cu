@@ -55,8 +55,8 @@ cudaError_t dalloc(T** p, size_t n, cudaStream_t st, bool zero) {
 void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->b2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2, c->mb2, c->vb2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
-                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->touched1, c->touched2, c->mask1,
-                  c->mask2, c->uniq1, c->uniq2, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
+                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->cnt1, c->cnt2, c->slots1, c->slots2, c->mask1,
+                  c->mask2, c->own1, c->own2, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
                   c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (c->pinned_loss) cudaFreeHost(c->pinned_loss);
@@ -204,11 +204,12 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(hash_idx, (size_t)c->KL * fn_len, true); A(hash_sign, (size_t)c->KL * fn_len, true);
   A(h, B * H, true); A(dh, B * H, true); A(loss, B, true); A(codes, B * c->L, true);
   A(act_cnt, B, true); A(act_z, B * S, true); A(act_p, B * S, true); A(act_g, B * S, true);
-  A(touched1, (D + 31) / 32, true); A(mask1, D * c->Wd, true); A(uniq1, D, true);
+  A(cnt1, D, true); A(mask1, D * c->Wd, true); A(slots1, D * ROW_SLOTS, true); A(own1, D, true);
   A(dstate, 1, true);
   if (!c->dense) {
     A(act_ids, B * S, true);
-    A(touched2, (N + 31) / 32, true); A(mask2, N * c->Wd, true); A(uniq2, N, true);
+    A(cnt2, N, true); A(mask2, N * c->Wd, true); A(slots2, N * ROW_SLOTS, true);
+    A(own2, N, true);
     A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
     A(keysA, (size_t)c->L * N, false);
     if (c->sort_passes > 1) { A(keysB, (size_t)c->L * N, false); A(valsA, (size_t)c->L * N, false); }
@@ -383,8 +384,9 @@ dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host
     memcpy(v, host_src, sizeof(v));
     if (v[0] < 0 || v[1] < 0) return DSLIDE_ERR_INVALID_ARG;
     c->t_host = v[0]; c->r_host = v[1]; c->next_rebuild = v[2];
-    long long t = v[0];
-    CU(cudaMemcpyAsync(&c->dstate->t, &t, sizeof(t), cudaMemcpyHostToDevice, c->stream));
+    // the device-side slots are indexed by the step's parity: make the slot of the next step the clean one
+    CU(cudaMemsetAsync(c->dstate->n_own, 0, sizeof(c->dstate->n_own), c->stream));
+    CU(cudaMemsetAsync(c->dstate->acc, 0, sizeof(c->dstate->acc), c->stream));
     return drain(c);
   }
   if (which == DSLIDE_T_HASH_IDX) {
@@ -443,7 +445,9 @@ dslide_status dslide_last_stats(dslide_ctx* ctx, int64_t out[4]) {
   DevState s;
   CU(cudaMemcpyAsync(&s, c->dstate, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
   CU(cudaStreamSynchronize(c->stream));
-  out[0] = (int64_t)s.last_sum_active; out[1] = s.U2; out[2] = s.U1; out[3] = (int64_t)s.last_nnz;
+  const int q = (int)((c->t_host + 1) & 1);      // parity of the last finished step
+  out[0] = (int64_t)s.last[0]; out[1] = c->dense ? c->N : (int64_t)s.n_own[q][0]; out[2] = (int64_t)s.n_own[q][1];
+  out[3] = (int64_t)s.last[1];
   static_assert((int)KID_COUNT == (int)DSLIDE_K_COUNT, "kernel id enums out of step");
   return DSLIDE_OK;
 }

@@ -29,24 +29,24 @@ enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2 };
 // Device-resident step state (read and written by kernels only; the host reads it
 // in the synchronous statistics and status calls).
 struct DevState {
-  int status;              // sticky dslide_status seen on the device
-  int U1, U2;              // distinct touched rows of W1 / W2 in the current step
-  int pad;
-  unsigned long long sum_active;   // accumulated by the forward kernel of the step in flight
-  unsigned long long nnz;
-  unsigned long long fetched;      // bucket entries read by the lookups of the step in flight
-  unsigned long long last_sum_active;   // totals of the last finished step
-  unsigned long long last_nnz;
-  unsigned long long last_fetched;
+  int status;                      // sticky dslide_status seen on the device
+  int pad0;
+  // Slots indexed by the parity of the step: the kernels of step t use slot t & 1 and the update
+  // kernel zeroes the other slot for step t + 1.
+  unsigned int n_own[2][2];        // distinct touched rows of W2 ([.][0]) and W1 ([.][1]): lengths of the row lists
+  unsigned long long acc[2][3];    // forward kernel: sum of active-set sizes, nonzeros, bucket entries read
+  unsigned long long last[3];      // acc of the last finished step
   unsigned long long cum[6];       // since the last reset: steps, sum_active, U2, U1, nnz, fetched
-  long long t;             // Adam step count
-  float bc1, bc2;          // 1 - beta1^t, 1 - beta2^t
 };
+
+// Touches of a row of W1 / W2 whose (sample, coefficient) pair is stored with the row; further touches of the
+// same step only set the sample's bit in the row's mask.
+constexpr int ROW_SLOTS = 8;
 
 struct Ctx;
 
 // Kernel ids for the per-kernel timing (must match the DSLIDE_K_* enum of the C ABI).
-enum { KID_FORWARD = 0, KID_SCAN, KID_ADAM, KID_DRAW_HASH, KID_HASH_NEURONS, KID_BUCKET_SCAN, KID_SORT_HIST,
+enum { KID_FORWARD = 0, KID_ADAM_DENSE, KID_ADAM, KID_DRAW_HASH, KID_HASH_NEURONS, KID_BUCKET_SCAN, KID_SORT_HIST,
        KID_SORT_SCAN, KID_SORT_SCATTER, KID_PREDICT, KID_INIT, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event pair around it.
@@ -91,9 +91,10 @@ struct Ctx {
   uint32_t* codes;
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
-  uint32_t *touched1, *touched2;   // one bit per row of W1 / W2
-  uint32_t *mask1, *mask2;         // per row: which samples of the batch touch it
-  int32_t *uniq1, *uniq2;          // ascending distinct touched rows
+  uint32_t *mask1, *mask2;         // per row of W1 / W2: which samples of the batch touch it
+  uint32_t *cnt1, *cnt2;           // per row: samples of the step in flight that touch it
+  int2 *slots1, *slots2;           // per row: (sample, coefficient bits) of its first ROW_SLOTS touches
+  int32_t *own1, *own2;            // the distinct touched rows of W1 / W2, in no particular order
   DevState* dstate;
 
   // rebuild work space

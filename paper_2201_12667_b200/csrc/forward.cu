@@ -25,13 +25,15 @@ struct FwdParams {
   uint32_t* codes;
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
-  uint32_t *touched1, *touched2, *mask1, *mask2;
+  uint32_t *mask1, *mask2, *cnt1, *cnt2;
+  int2 *slots1, *slots2;
+  int32_t *own1, *own2;
   DevState* st;
   int32_t* out_ids;
   float* out_scores;
   long long nb;
   int B, D, H, N, K, L, KL, family, lg_bin, fn_len, cap;
-  int act_stride, Wd, dense, dedup_mode, max_labels, sort_cap, topk;
+  int act_stride, Wd, dense, dedup_mode, max_labels, sort_cap, topk, parity;
   int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_topk, off_dedup;
 };
 
@@ -479,24 +481,56 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
     p.dh[(size_t)s * H + k] = sh_h[k] > 0.f ? v : 0.f;
   }
 
-  // ---- record the touched rows for the update kernels ----
+  // ---- hand the sample's touches to the update kernel.  Per touched row: a count of the touching samples;
+  //      for the row's first ROW_SLOTS touches the (sample, coefficient) pair itself, else the bit of this
+  //      sample in the row's mask.  The sample that touches a row first also enters it in the list of
+  //      distinct rows (positions handed out per warp). ----
   const uint32_t sbit = 1u << (s & 31);
   const int sword = s >> 5;
+  const unsigned lt = (1u << lane) - 1u;
   if (!dense)
-    for (int a = tid; a < na; a += FWD_THREADS) {
-      int jj = ids[a];
-      atomicOr(p.touched2 + (jj >> 5), 1u << (jj & 31));
-      atomicOr(p.mask2 + (size_t)jj * p.Wd + sword, sbit);
+    for (int a0 = 0; a0 < na; a0 += FWD_THREADS) {
+      const int a = a0 + tid;
+      bool first = false;
+      int jj = 0;
+      if (a < na) {
+        jj = ids[a];
+        const unsigned nth = atomicAdd(p.cnt2 + jj, 1u);
+        if (nth < (unsigned)ROW_SLOTS) p.slots2[(size_t)jj * ROW_SLOTS + nth] = make_int2(s, __float_as_int(g[a]));
+        else atomicOr(p.mask2 + (size_t)jj * p.Wd + sword, sbit);
+        first = nth == 0u;
+      }
+      const unsigned fm = __ballot_sync(0xffffffffu, first);
+      if (fm) {
+        unsigned base = 0;
+        if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][0], (unsigned)__popc(fm));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (first) p.own2[base + __popc(fm & lt)] = jj;
+      }
     }
-  for (int i = tid; i < nnz; i += FWD_THREADS) {
-    int c = p.col_idx[rbeg + i];
-    atomicOr(p.touched1 + (c >> 5), 1u << (c & 31));
-    atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
+  for (int i0 = 0; i0 < nnz; i0 += FWD_THREADS) {
+    const int i = i0 + tid;
+    bool first = false;
+    int c = 0;
+    if (i < nnz) {
+      c = p.col_idx[rbeg + i];
+      const unsigned nth = atomicAdd(p.cnt1 + c, 1u);
+      if (nth < (unsigned)ROW_SLOTS) p.slots1[(size_t)c * ROW_SLOTS + nth] = make_int2(s, __float_as_int(p.vals[rbeg + i]));
+      else atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
+      first = nth == 0u;
+    }
+    const unsigned fm = __ballot_sync(0xffffffffu, first);
+    if (fm) {
+      unsigned base = 0;
+      if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][1], (unsigned)__popc(fm));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      if (first) p.own1[base + __popc(fm & lt)] = c;
+    }
   }
   if (tid == 0) {
-    atomicAdd(&p.st->sum_active, (unsigned long long)na);
-    atomicAdd(&p.st->nnz, (unsigned long long)nnz);
-    atomicAdd(&p.st->fetched, (unsigned long long)sh_misc[24]);
+    atomicAdd(&p.st->acc[p.parity][0], (unsigned long long)na);
+    atomicAdd(&p.st->acc[p.parity][1], (unsigned long long)nnz);
+    atomicAdd(&p.st->acc[p.parity][2], (unsigned long long)sh_misc[24]);
   }
 }
 
@@ -553,7 +587,9 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals; p.label_ptr = label_ptr; p.labels = labels;
   p.h = c->h; p.dh = c->dh; p.loss = c->loss; p.codes = c->codes;
   p.act_cnt = c->act_cnt; p.act_ids = c->act_ids; p.act_z = c->act_z; p.act_p = c->act_p; p.act_g = c->act_g;
-  p.touched1 = c->touched1; p.touched2 = c->touched2; p.mask1 = c->mask1; p.mask2 = c->mask2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.cnt1 = c->cnt1; p.cnt2 = c->cnt2;
+  p.slots1 = c->slots1; p.slots2 = c->slots2;
+  p.own1 = c->own1; p.own2 = c->own2; p.parity = (int)(c->t_host & 1);
   p.st = c->dstate; p.out_ids = nullptr; p.out_scores = nullptr;
   p.nb = c->nb;
   p.B = batch; p.D = c->D; p.H = c->H; p.N = c->N; p.K = c->K; p.L = c->L; p.KL = c->KL;
