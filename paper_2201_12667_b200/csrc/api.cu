@@ -56,7 +56,7 @@ void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->b2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2, c->mb2, c->vb2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->cnt1, c->cnt2, c->slots1, c->slots2, c->mask1,
-                  c->mask2, c->own1, c->own2, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
+                  c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
                   c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (c->pinned_loss) cudaFreeHost(c->pinned_loss);
@@ -205,6 +205,7 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(h, B * H, true); A(dh, B * H, true); A(loss, B, true); A(codes, B * c->L, true);
   A(act_cnt, B, true); A(act_z, B * S, true); A(act_p, B * S, true); A(act_g, B * S, true);
   A(cnt1, D, true); A(mask1, D * c->Wd, true); A(slots1, D * ROW_SLOTS, true); A(own1, D, true);
+  A(hot_rows, HOT_CAP, true); A(med_rows, MED_CAP, true); A(hot_done, HOT_CAP, true); A(hot_part, (size_t)HOT_CAP * HOT_SLICES * (H + 4), true);
   A(dstate, 1, true);
   if (!c->dense) {
     A(act_ids, B * S, true);
@@ -386,6 +387,9 @@ dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host
     c->t_host = v[0]; c->r_host = v[1]; c->next_rebuild = v[2];
     // the device-side slots are indexed by the step's parity: make the slot of the next step the clean one
     CU(cudaMemsetAsync(c->dstate->n_own, 0, sizeof(c->dstate->n_own), c->stream));
+    CU(cudaMemsetAsync(c->dstate->n_hot, 0, sizeof(c->dstate->n_hot), c->stream));
+    CU(cudaMemsetAsync(c->dstate->n_med, 0, sizeof(c->dstate->n_med), c->stream));
+    CU(cudaMemsetAsync(c->dstate->ticket, 0, sizeof(c->dstate->ticket), c->stream));
     CU(cudaMemsetAsync(c->dstate->acc, 0, sizeof(c->dstate->acc), c->stream));
     return drain(c);
   }

@@ -34,6 +34,9 @@ struct DevState {
   // Slots indexed by the parity of the step: the kernels of step t use slot t & 1 and the update
   // kernel zeroes the other slot for step t + 1.
   unsigned int n_own[2][2];        // distinct touched rows of W2 ([.][0]) and W1 ([.][1]): lengths of the row lists
+  unsigned int n_hot[2];           // rows touched by more than HOT_T samples (entries of the hot-row list)
+  unsigned int n_med[2];           // rows touched by more than ROW_SLOTS samples (entries of the medium-row list)
+  unsigned int ticket[2];          // work tickets handed out by the update kernel
   unsigned long long acc[2][3];    // forward kernel: sum of active-set sizes, nonzeros, bucket entries read
   unsigned long long last[3];      // acc of the last finished step
   unsigned long long cum[6];       // since the last reset: steps, sum_active, U2, U1, nnz, fetched
@@ -42,6 +45,17 @@ struct DevState {
 // Touches of a row of W1 / W2 whose (sample, coefficient) pair is stored with the row; further touches of the
 // same step only set the sample's bit in the row's mask.
 constexpr int ROW_SLOTS = 8;
+// A row touched by more than HOT_T samples of a step is listed by the forward kernel (top bit of its
+// count set) and summed in HOT_SLICES slices by different warps; at most HOT_CAP rows are listed, further
+// ones are summed by a single warp.
+constexpr int HOT_T = 32;
+constexpr int HOT_SLICES = 8;
+constexpr int HOT_CAP = 1024;
+// Rows touched by more than ROW_SLOTS samples are listed too (at most MED_CAP of them; further ones are found
+// by the warp that walks the ordinary row list).  A row's count word: low bits = touching samples, CNT_MED /
+// CNT_HOT = the row is on the medium / hot list.
+constexpr int MED_CAP = 65536;
+constexpr unsigned CNT_HOT = 0x80000000u, CNT_MED = 0x40000000u, CNT_MASK = 0x3fffffffu;
 
 struct Ctx;
 
@@ -95,6 +109,10 @@ struct Ctx {
   uint32_t *cnt1, *cnt2;           // per row: samples of the step in flight that touch it
   int2 *slots1, *slots2;           // per row: (sample, coefficient bits) of its first ROW_SLOTS touches
   int32_t *own1, *own2;            // the distinct touched rows of W1 / W2, in no particular order
+  int32_t* hot_rows;               // rows touched by many samples: row of W2, or ~row of W1
+  int32_t* med_rows;               // rows touched by more than ROW_SLOTS samples, same encoding
+  float* hot_part;                 // [HOT_CAP][HOT_SLICES][H + 4] slice sums of those rows
+  int* hot_done;                   // [HOT_CAP] finished slices per listed row (returns to 0)
   DevState* dstate;
 
   // rebuild work space

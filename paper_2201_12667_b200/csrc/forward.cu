@@ -27,7 +27,7 @@ struct FwdParams {
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2, *cnt1, *cnt2;
   int2 *slots1, *slots2;
-  int32_t *own1, *own2;
+  int32_t *own1, *own2, *hot_rows, *med_rows;
   DevState* st;
   int32_t* out_ids;
   float* out_scores;
@@ -38,6 +38,26 @@ struct FwdParams {
 };
 
 __device__ __forceinline__ void set_status(DevState* st, int code) { atomicCAS(&st->status, 0, code); }
+
+// The touch that takes a row past ROW_SLOTS touching samples enters the row in the list of rows that a warp of
+// the update kernel sums from slots and mask; the touch that takes it past HOT_T enters it in the list of rows
+// summed in slices.  The row's count word is marked so that the update kernel knows where the row is listed.
+__device__ __forceinline__ void list_row(const FwdParams& p, uint32_t* cnt, int code, unsigned nth) {
+  if (nth == (unsigned)ROW_SLOTS) {
+    const unsigned at = atomicAdd(&p.st->n_med[p.parity], 1u);
+    if (at < (unsigned)MED_CAP) {
+      p.med_rows[at] = code;
+      atomicOr(cnt, CNT_MED);
+    }
+  }
+  if (nth == (unsigned)HOT_T) {
+    const unsigned at = atomicAdd(&p.st->n_hot[p.parity], 1u);
+    if (at < (unsigned)HOT_CAP) {
+      p.hot_rows[at] = code;
+      atomicOr(cnt, CNT_HOT);
+    }
+  }
+}
 
 // Exclusive prefix sum of one int per thread over the block; *total gets the block sum.
 // sh needs FWD_WARPS + 1 ints.  Ends with a barrier, so sh may be reused afterwards.
@@ -495,10 +515,11 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
       int jj = 0;
       if (a < na) {
         jj = ids[a];
-        const unsigned nth = atomicAdd(p.cnt2 + jj, 1u);
+        const unsigned nth = atomicAdd(p.cnt2 + jj, 1u) & CNT_MASK;
         if (nth < (unsigned)ROW_SLOTS) p.slots2[(size_t)jj * ROW_SLOTS + nth] = make_int2(s, __float_as_int(g[a]));
         else atomicOr(p.mask2 + (size_t)jj * p.Wd + sword, sbit);
         first = nth == 0u;
+        list_row(p, p.cnt2 + jj, jj, nth);
       }
       const unsigned fm = __ballot_sync(0xffffffffu, first);
       if (fm) {
@@ -514,10 +535,11 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
     int c = 0;
     if (i < nnz) {
       c = p.col_idx[rbeg + i];
-      const unsigned nth = atomicAdd(p.cnt1 + c, 1u);
+      const unsigned nth = atomicAdd(p.cnt1 + c, 1u) & CNT_MASK;
       if (nth < (unsigned)ROW_SLOTS) p.slots1[(size_t)c * ROW_SLOTS + nth] = make_int2(s, __float_as_int(p.vals[rbeg + i]));
       else atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
       first = nth == 0u;
+      list_row(p, p.cnt1 + c, ~c, nth);
     }
     const unsigned fm = __ballot_sync(0xffffffffu, first);
     if (fm) {
@@ -589,7 +611,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.act_cnt = c->act_cnt; p.act_ids = c->act_ids; p.act_z = c->act_z; p.act_p = c->act_p; p.act_g = c->act_g;
   p.mask1 = c->mask1; p.mask2 = c->mask2; p.cnt1 = c->cnt1; p.cnt2 = c->cnt2;
   p.slots1 = c->slots1; p.slots2 = c->slots2;
-  p.own1 = c->own1; p.own2 = c->own2; p.parity = (int)(c->t_host & 1);
+  p.own1 = c->own1; p.own2 = c->own2; p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.parity = (int)(c->t_host & 1);
   p.st = c->dstate; p.out_ids = nullptr; p.out_scores = nullptr;
   p.nb = c->nb;
   p.B = batch; p.D = c->D; p.H = c->H; p.N = c->N; p.K = c->K; p.L = c->L; p.KL = c->KL;

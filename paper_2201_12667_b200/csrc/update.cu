@@ -7,17 +7,20 @@
 // samples of any further touches -- and two lists of the distinct touched rows (the sample that
 // touched a row first entered it).
 //
-//   k_update : every warp takes a contiguous share of the two row lists, a few rows at a time, so
-//              that the loads of a row's weights and moments, its touch count and its slots are
-//              all issued together.  A row touched by one sample takes its gradient from slot 0;
+//   k_update : a warp works on a few rows of the two row lists at a time, so that the loads of a
+//              row's weights and moments, its touch count and its slots are all issued together.  A row touched by one sample takes its gradient from slot 0;
 //              a row touched by up to ROW_SLOTS samples from its slots, put in ascending sample
 //              order; a row touched by more from slots and mask (the sample's coefficient for this
 //              row is found by binary search in the sample's ascending id list), again in ascending
 //              sample order.  So the sums do not depend on the order in which the forward kernel's
-//              blocks ran, and no floating-point atomics are used.  Rows touched by many samples are
-//              deferred to the end of the block and summed by all its warps.  Adam is then applied
-//              to that row only; untouched rows are neither read nor written.  The warp resets the
-//              row's count and mask for the next step.
+//              blocks ran, and no floating-point atomics are used.  Rows touched by more than
+//              ROW_SLOTS samples were listed by the forward kernel and are summed by a warp each; rows
+//              touched by more than HOT_T samples were listed a second time: each is cut into HOT_SLICES
+//              slices of its mask, summed by different warps, and the warp that finishes a row's last
+//              slice adds the slice sums in slice order.  Warps draw tickets from one counter: hot
+//              slices, then listed rows, then the ordinary rows eight at a time.  Adam is applied to the
+//              touched rows only; untouched rows are neither read nor written.  The warp that updates a
+//              row resets its count and mask for the next step.
 //              The last blocks of the grid update the hidden bias and reduce the batch loss.
 //   k_adam_dense : the output layer when every neuron is active (no lists, no masks).
 #include "common.cuh"
@@ -26,8 +29,6 @@ namespace dslide {
 
 constexpr int UPD_THREADS = 256;
 constexpr int UPD_WARPS = UPD_THREADS / 32;
-constexpr int HOT_T = 32;      // rows touched by more samples than this are summed by a whole block
-constexpr int HOT_MAX = 48;    // deferred rows a block can hold (more: summed by the owning warp)
 constexpr unsigned FULL = 0xffffffffu;
 // ROW_SLOTS (common.cuh): touches of a row whose (sample, coefficient) the forward kernel stores directly
 
@@ -40,19 +41,25 @@ struct UpdParams {
   const float* vals;
   uint32_t *mask1, *mask2, *cnt1, *cnt2;
   const int2 *slots1, *slots2;
-  const int32_t *own1, *own2;
+  const int32_t *own1, *own2, *hot_rows, *med_rows;
+  float* hot_part;
+  int* hot_done;
   DevState* st;
   float* loss_out;
   int B, H, N, D, Wd, act_stride, dense, parity;
-  float lr, beta1, beta2, eps, bc1, bc2;
+  float lr, beta1, beta2, eps, rb1, rb2;
 };
 
+// One element of Adam.  rb1 = 1 / (1 - beta1^t), rb2 = 1 / (1 - beta2^t).  The square root and the final
+// quotient use the hardware approximations (relative error below 2^-22): three orders of magnitude inside
+// the fp32 noise of the gradient sums, and free of the slow paths exact zeros take in the IEEE sequences.
 __device__ __forceinline__ void adam1(float& w, float& m, float& v, float g, float b1, float b2, float lr, float eps,
-                                      float bc1, float bc2) {
-  m = b1 * m + (1.f - b1) * g;
-  v = b2 * v + (1.f - b2) * g * g;
-  float mhat = m / bc1, vhat = v / bc2;
-  w = w - lr * mhat / (sqrtf(vhat) + eps);
+                                      float rb1, float rb2) {
+  m = fmaf(b1, m, (1.f - b1) * g);
+  v = fmaf(b2, v, (1.f - b2) * g * g);
+  float root;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(root) : "f"(v * rb2));
+  w = w - __fdividef(lr * (m * rb1), root + eps);
 }
 
 __device__ __forceinline__ void axpy4(float4& a, float g, const float4 x) {
@@ -247,10 +254,10 @@ __device__ __forceinline__ void adam_store(const UpdParams& p, const Side& sd, s
   for (int q = 0; q < NCH; ++q) {
     int c = lane + q * 32;
     if (c < H4) {
-      adam1(w[q].x, m[q].x, v[q].x, g[q].x, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
-      adam1(w[q].y, m[q].y, v[q].y, g[q].y, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
-      adam1(w[q].z, m[q].z, v[q].z, g[q].z, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
-      adam1(w[q].w, m[q].w, v[q].w, g[q].w, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
+      adam1(w[q].x, m[q].x, v[q].x, g[q].x, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      adam1(w[q].y, m[q].y, v[q].y, g[q].y, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      adam1(w[q].z, m[q].z, v[q].z, g[q].z, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      adam1(w[q].w, m[q].w, v[q].w, g[q].w, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
       w4[c] = w[q]; m4[c] = m[q]; v4[c] = v[q];
     }
   }
@@ -258,7 +265,7 @@ __device__ __forceinline__ void adam_store(const UpdParams& p, const Side& sd, s
 
 __device__ __forceinline__ void adam_bias(const UpdParams& p, const Side& sd, int row, float g) {
   float w = sd.bw[row], m = sd.bm[row], v = sd.bv[row];
-  adam1(w, m, v, g, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
+  adam1(w, m, v, g, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
   sd.bw[row] = w; sd.bm[row] = m; sd.bv[row] = v;
 }
 
@@ -288,7 +295,7 @@ __device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
     float tot = 0.f;
     for (int w = 0; w < UPD_WARPS; ++w) tot += sm_part[w * 32 + lane];
     float w = p.b1[k], m = p.mb1[k], v = p.vb1[k];
-    adam1(w, m, v, tot, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
+    adam1(w, m, v, tot, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
     p.b1[k] = w; p.mb1[k] = m; p.vb1[k] = v;
   }
   if (a != 0) return;
@@ -313,57 +320,163 @@ __device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
     st->acc[o][0] = 0ull; st->acc[o][1] = 0ull; st->acc[o][2] = 0ull;
     st->cum[3] += (unsigned long long)st->n_own[q][1];
     if (!p.dense) st->cum[2] += (unsigned long long)st->n_own[q][0];
-    st->n_own[o][0] = 0u; st->n_own[o][1] = 0u;
+    st->n_own[o][0] = 0u; st->n_own[o][1] = 0u; st->n_hot[o] = 0u; st->n_med[o] = 0u; st->ticket[o] = 0u;
   }
 }
 
+// One slice of a row touched by many samples: the samples of HOT_SLICES-th of the row's mask words.  The slice
+// sum goes to scratch memory; the warp that completes the row's last slice adds the slices in slice
+// order (so the result does not depend on which warp that is), applies Adam and resets the row's state.
+template <int NCH>
+__device__ __forceinline__ void hot_item(const UpdParams& p, const int* sm_rowptr, int item, int nwB, int* scr, int H,
+                                         int H4, int lane) {
+  const int hrow = item / HOT_SLICES, slice = item - hrow * HOT_SLICES;
+  const int code = p.hot_rows[hrow];
+  const bool w2 = code >= 0;
+  const int row = w2 ? code : ~code;
+  const Side sd = make_side(p, w2);
+  const int per_w = (nwB + HOT_SLICES - 1) / HOT_SLICES;
+  const int w0 = min(nwB, slice * per_w), w1 = min(nwB, w0 + per_w);
+  float4 acc[NCH];
+#pragma unroll
+  for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+  float csum = 0.f;
+  int slot_s = 0x7fffffff;
+  if (lane < ROW_SLOTS) slot_s = sd.slots[(size_t)row * ROW_SLOTS + lane].x;
+  sum_masked<NCH>(p, sd, sm_rowptr, row, slot_s, w0, w1, scr, acc, csum, H, H4, lane);
+  const int ld = H + 4;
+  float* part = p.hot_part + (size_t)hrow * HOT_SLICES * ld;
+  float4* mine = reinterpret_cast<float4*>(part + (size_t)slice * ld);
+#pragma unroll
+  for (int u = 0; u < NCH; ++u) {
+    const int c = lane + u * 32;
+    if (c < H4) __stcg(mine + c, acc[u]);
+  }
+  if (lane == 0) __stcg(part + (size_t)slice * ld + H, csum);
+  __threadfence();
+  __syncwarp();
+  int done = 0;
+  if (lane == 0) done = atomicAdd(p.hot_done + hrow, 1);
+  done = __shfl_sync(FULL, done, 0);
+  if (done != HOT_SLICES - 1) return;
+  __threadfence();
+  float4 w[NCH], m[NCH], v[NCH];
+  load_row<NCH>(sd.W, (size_t)row, H, H4, lane, w);
+  load_row<NCH>(sd.M, (size_t)row, H, H4, lane, m);
+  load_row<NCH>(sd.V, (size_t)row, H, H4, lane, v);
+#pragma unroll
+  for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+  csum = 0.f;
+  for (int sl = 0; sl < HOT_SLICES; ++sl) {
+    const float4* src4 = reinterpret_cast<const float4*>(part + (size_t)sl * ld);
+#pragma unroll
+    for (int u = 0; u < NCH; ++u) {
+      const int c = lane + u * 32;
+      if (c < H4) {
+        const float4 x = __ldcg(src4 + c);
+        acc[u].x += x.x; acc[u].y += x.y; acc[u].z += x.z; acc[u].w += x.w;
+      }
+    }
+    csum += __ldcg(part + (size_t)sl * ld + H);
+  }
+  adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
+  if (lane == 0) {
+    if (w2) adam_bias(p, sd, row, csum);
+    p.hot_done[hrow] = 0;
+    (w2 ? p.cnt2 : p.cnt1)[row] = 0u;
+  }
+}
+
+// A row touched by more than ROW_SLOTS samples that the forward kernel listed: one warp sums it from slots and
+// mask (ascending samples), applies Adam and resets the row's state.  Rows that went on to the hot list are
+// summed in slices instead and skipped here.
+template <int NCH>
+__device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_rowptr, int idx, int nwB, int* scr, int H,
+                                            int H4, int lane) {
+  const int code = p.med_rows[idx];
+  const bool w2 = code >= 0;
+  const int row = w2 ? code : ~code;
+  const Side sd = make_side(p, w2);
+  uint32_t* cnt = (w2 ? p.cnt2 : p.cnt1) + row;
+  unsigned cv = 0u;
+  if (lane == 0) cv = *cnt;
+  cv = __shfl_sync(FULL, cv, 0);
+  if ((cv & CNT_HOT) || (cv & CNT_MASK) == 0u) return;
+  int slot_s = 0x7fffffff;
+  if (lane < ROW_SLOTS) slot_s = sd.slots[(size_t)row * ROW_SLOTS + lane].x;
+  float4 w[NCH], m[NCH], v[NCH], acc[NCH];
+  load_row<NCH>(sd.W, (size_t)row, H, H4, lane, w);
+  load_row<NCH>(sd.M, (size_t)row, H, H4, lane, m);
+  load_row<NCH>(sd.V, (size_t)row, H, H4, lane, v);
+#pragma unroll
+  for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+  float csum = 0.f;
+  sum_masked<NCH>(p, sd, sm_rowptr, row, slot_s, 0, nwB, scr, acc, csum, H, H4, lane);
+  adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
+  if (lane == 0) {
+    if (w2) adam_bias(p, sd, row, csum);
+    *cnt = 0u;
+  }
+}
+
+// Work is handed out in tickets from one counter: first the slices of the hot rows (the longest items), then
+// the listed rows with more than ROW_SLOTS touches, then the ordinary rows, UPD_TROWS per ticket.
+constexpr int UPD_TROWS = 8;
+
 template <int NCH, int G>
-__global__ void __launch_bounds__(UPD_THREADS, (NCH <= 2 ? 2 : 1)) k_update(const UpdParams p) {
+__global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
   extern __shared__ __align__(16) unsigned char upd_smem[];
   int* sm_rowptr = reinterpret_cast<int*>(upd_smem);                               // [B + 1]
-  float* sm_part = reinterpret_cast<float*>(upd_smem + (((size_t)p.B + 1 + 3) & ~(size_t)3) * 4);   // [UPD_WARPS][H + 32]
-  __shared__ int hot_list[HOT_MAX];
-  __shared__ int hot_n;
+  float* sm_part = reinterpret_cast<float*>(upd_smem + (((size_t)p.B + 1 + 3) & ~(size_t)3) * 4);   // [UPD_WARPS * 32]
   __shared__ int scratch[UPD_WARPS][64];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = p.H, H4 = H >> 2, B = p.B;
   const int naux = (H + 31) >> 5;
-  const int nwork = (int)gridDim.x - naux;
-  if ((int)blockIdx.x >= nwork) { aux_block(p, (int)blockIdx.x - nwork, sm_part); return; }
+  if ((int)blockIdx.x < naux) { aux_block(p, (int)blockIdx.x, sm_part); return; }
 
   for (int i = tid; i <= B; i += UPD_THREADS) sm_rowptr[i] = p.row_ptr[i];
-  if (tid == 0) hot_n = 0;
   __syncthreads();
 
   const int n2 = p.dense ? 0 : (int)p.st->n_own[p.parity][0];
   const int n1 = (int)p.st->n_own[p.parity][1];
   const int nrows = n2 + n1;
   const int nwB = (B + 31) >> 5;
-  // The concatenated lists (rows of W2, then rows of W1) are dealt out row by row: consecutive rows go to
-  // different blocks, because rows touched by many samples tend to sit next to each other in the lists.
-  const int nwarps = nwork * UPD_WARPS;
-  const int gw = warp * nwork + blockIdx.x;
-  const int mine_n = gw < nrows ? (nrows - gw + nwarps - 1) / nwarps : 0;     // rows gw, gw + nwarps, ...
+  const unsigned nh_raw = p.st->n_hot[p.parity], nm_raw = p.st->n_med[p.parity];
+  const int n_hot_items = (int)(nh_raw < (unsigned)HOT_CAP ? nh_raw : (unsigned)HOT_CAP) * HOT_SLICES;
+  const int n_med = (int)(nm_raw < (unsigned)MED_CAP ? nm_raw : (unsigned)MED_CAP);
+  const int n_norm = (nrows + UPD_TROWS - 1) / UPD_TROWS;
+  const int n_tickets = n_hot_items + n_med + n_norm;
+  unsigned int* ticket = &p.st->ticket[p.parity];
 
-  for (int cb = 0; cb < mine_n; cb += 32) {
-    // ids of up to 32 rows of this warp's share, one per lane
-    int myrow = 0, myidx = 0;
-    if (cb + lane < mine_n) {
-      myidx = gw + (cb + lane) * nwarps;
-      myrow = myidx < n2 ? p.own2[myidx] : p.own1[myidx - n2];
+  int nxt = 0;
+  if (lane == 0) nxt = (int)atomicAdd(ticket, 1u);
+  for (;;) {
+    const int t = __shfl_sync(FULL, nxt, 0);
+    if (t >= n_tickets) break;
+    if (lane == 0) nxt = (int)atomicAdd(ticket, 1u);          // the next ticket is on its way while this one is worked on
+    if (t < n_hot_items) { hot_item<NCH>(p, sm_rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
+    if (t < n_hot_items + n_med) { medium_item<NCH>(p, sm_rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
+
+    // ---- ordinary rows: ticket k takes rows k, k + n_norm, k + 2 n_norm, ... of the concatenated lists (rows of
+    //      W2, then rows of W1), so that neighbours in a list (often alike in cost) go to different warps ----
+    const int k = t - n_hot_items - n_med;
+    int myrow = 0, myidx = nrows;
+    if (lane < UPD_TROWS) {
+      myidx = k + lane * n_norm;
+      if (myidx < nrows) myrow = myidx < n2 ? p.own2[myidx] : p.own1[myidx - n2];
     }
-    const int cend = min(32, mine_n - cb);
-    for (int b0 = 0; b0 < cend; b0 += G) {
+    for (int b0 = 0; b0 < UPD_TROWS; b0 += G) {
       int rr[G], tt[G];
-      bool live[G], w2[G];
+      bool live[G], w2[G], skip[G];
       int2 sl[G];
       float4 w[G][NCH], m[G][NCH], v[G][NCH], x[G][NCH];
 #pragma unroll
       for (int q = 0; q < G; ++q) {
-        live[q] = b0 + q < cend;
-        w2[q] = __shfl_sync(FULL, myidx, live[q] ? b0 + q : 0) < n2;
-        rr[q] = __shfl_sync(FULL, myrow, live[q] ? b0 + q : 0);
+        const int idx = __shfl_sync(FULL, myidx, b0 + q);
+        live[q] = idx < nrows;
+        w2[q] = idx < n2;
+        rr[q] = __shfl_sync(FULL, myrow, b0 + q);
         tt[q] = 0;
         sl[q] = make_int2(0x7fffffff, 0);
         if (live[q]) {
@@ -380,20 +493,22 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH <= 2 ? 2 : 1)) k_update(cons
       for (int q = 0; q < G; ++q)
         if (live[q]) {
           const Side sd = make_side(p, w2[q]);
-          if (lane == 0) (w2[q] ? p.cnt2 : p.cnt1)[rr[q]] = 0u;
-          tt[q] = __shfl_sync(FULL, tt[q], 0);
+          const unsigned cv = (unsigned)__shfl_sync(FULL, tt[q], 0);
+          // a listed row is summed by its own ticket (and its count may already be back at zero)
+          skip[q] = (cv & (CNT_HOT | CNT_MED)) != 0u || (cv & CNT_MASK) == 0u;
+          tt[q] = (int)(cv & CNT_MASK);
+          if (lane == 0 && !skip[q]) (w2[q] ? p.cnt2 : p.cnt1)[rr[q]] = 0u;
           const int s0 = __shfl_sync(FULL, sl[q].x, 0);
-          if (tt[q] == 1) load_row<NCH>(sd.src, (size_t)s0, H, H4, lane, x[q]);
+          if (tt[q] == 1 && !skip[q]) load_row<NCH>(sd.src, (size_t)s0, H, H4, lane, x[q]);
         }
 #pragma unroll
       for (int q = 0; q < G; ++q)
-        if (live[q]) {
+        if (live[q] && !skip[q]) {
           const Side sd = make_side(p, w2[q]);
           float4 acc[NCH];
 #pragma unroll
           for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
           float csum = 0.f;
-          bool defer = false;
           if (tt[q] == 1) {
             const float g0 = __int_as_float(__shfl_sync(FULL, sl[q].y, 0));
 #pragma unroll
@@ -401,66 +516,13 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH <= 2 ? 2 : 1)) k_update(cons
             csum = g0;
           } else if (tt[q] <= ROW_SLOTS) {
             sum_slots<NCH>(sd, sl[q], tt[q], scratch[warp], acc, csum, H, H4, lane);
-          } else {
-            if (tt[q] > HOT_T) {
-              int slot = 0;
-              if (lane == 0) slot = atomicAdd(&hot_n, 1);
-              slot = __shfl_sync(FULL, slot, 0);
-              if (slot < HOT_MAX) {
-                if (lane == 0) hot_list[slot] = w2[q] ? rr[q] : ~rr[q];
-                defer = true;
-              }
-            }
-            if (!defer) sum_masked<NCH>(p, sd, sm_rowptr, rr[q], sl[q].x, 0, nwB, scratch[warp], acc, csum, H, H4, lane);
+          } else {      // more touches than slots, yet not listed (the list was full)
+            sum_masked<NCH>(p, sd, sm_rowptr, rr[q], sl[q].x, 0, nwB, scratch[warp], acc, csum, H, H4, lane);
           }
-          if (!defer) {
-            adam_store<NCH>(p, sd, (size_t)rr[q], w[q], m[q], v[q], acc, H, H4, lane);
-            if (w2[q] && lane == 0) adam_bias(p, sd, rr[q], csum);
-          }
+          adam_store<NCH>(p, sd, (size_t)rr[q], w[q], m[q], v[q], acc, H, H4, lane);
+          if (w2[q] && lane == 0) adam_bias(p, sd, rr[q], csum);
         }
     }
-  }
-
-  // ---- rows touched by many samples: every warp sums a slice of the row's mask, slices added in order ----
-  __syncthreads();
-  const int nh = hot_n < HOT_MAX ? hot_n : HOT_MAX;
-  const int ld = H + 32;
-  for (int qh = 0; qh < nh; ++qh) {
-    const int code = hot_list[qh];
-    const bool w2 = code >= 0;
-    const int row = w2 ? code : ~code;
-    const Side sd = make_side(p, w2);
-    const int per_w = (nwB + UPD_WARPS - 1) / UPD_WARPS;
-    const int w0 = min(nwB, warp * per_w), w1 = min(nwB, w0 + per_w);
-    float4 acc[NCH];
-#pragma unroll
-    for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-    float csum = 0.f;
-    int slot_s = 0x7fffffff;
-    if (lane < ROW_SLOTS) slot_s = sd.slots[(size_t)row * ROW_SLOTS + lane].x;
-    sum_masked<NCH>(p, sd, sm_rowptr, row, slot_s, w0, w1, scratch[warp], acc, csum, H, H4, lane);
-    float4* mine = reinterpret_cast<float4*>(sm_part + (size_t)warp * ld);
-#pragma unroll
-    for (int u = 0; u < NCH; ++u) {
-      int cidx = lane + u * 32;
-      if (cidx < H4) mine[cidx] = acc[u];
-    }
-    if (lane == 0) sm_part[(size_t)warp * ld + H] = csum;
-    __syncthreads();
-    for (int k = tid; k < H; k += UPD_THREADS) {
-      float gsum = 0.f;
-      for (int w = 0; w < UPD_WARPS; ++w) gsum += sm_part[(size_t)w * ld + k];
-      const size_t e = (size_t)row * H + k;
-      float wv = sd.W[e], mv = sd.M[e], vv = sd.V[e];
-      adam1(wv, mv, vv, gsum, p.beta1, p.beta2, p.lr, p.eps, p.bc1, p.bc2);
-      sd.W[e] = wv; sd.M[e] = mv; sd.V[e] = vv;
-    }
-    if (w2 && tid == 0) {
-      float cs = 0.f;
-      for (int w = 0; w < UPD_WARPS; ++w) cs += sm_part[(size_t)w * ld + H];
-      adam_bias(p, sd, row, cs);
-    }
-    __syncthreads();
   }
 }
 
@@ -498,9 +560,15 @@ static cudaError_t launch_k_update(Ctx* c, const UpdParams& p, int smem) {
     e = cudaFuncSetAttribute(k_update<NCH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
+  // one wave: the blocks for the hidden bias come first, the rest fill the remaining block slots of the device
   const int naux = (c->H + 31) / 32;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_update<NCH, G>, UPD_THREADS, smem);
+  if (e != cudaSuccess) return e;
+  int nblocks = c->num_sms * (per_sm > 0 ? per_sm : 1);
+  if (nblocks < naux + 1) nblocks = naux + 1;
   LaunchScope ls(c, KID_ADAM);
-  k_update<NCH, G><<<c->num_sms * (NCH <= 2 ? 2 : 1) + naux, UPD_THREADS, smem, c->stream>>>(p);
+  k_update<NCH, G><<<nblocks, UPD_THREADS, smem, c->stream>>>(p);
   return cudaGetLastError();
 }
 
@@ -513,14 +581,15 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals;
   p.mask1 = c->mask1; p.mask2 = c->mask2; p.cnt1 = c->cnt1; p.cnt2 = c->cnt2;
   p.slots1 = c->slots1; p.slots2 = c->slots2; p.own1 = c->own1; p.own2 = c->own2;
+  p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.hot_part = c->hot_part; p.hot_done = c->hot_done;
   p.st = c->dstate; p.loss_out = loss_out;
   p.B = batch; p.H = c->H; p.N = c->N; p.D = c->D; p.Wd = c->Wd; p.act_stride = c->act_stride; p.dense = c->dense;
   p.parity = (int)(c->t_host & 1);
   p.lr = c->cfg.lr; p.beta1 = c->cfg.beta1; p.beta2 = c->cfg.beta2; p.eps = c->cfg.eps;
-  // bias corrections of Adam with the global step count (the step being taken is t + 1)
+  // reciprocal bias corrections of Adam with the global step count (the step being taken is t + 1)
   const double t = (double)(c->t_host + 1);
-  p.bc1 = (float)(1.0 - pow((double)c->cfg.beta1, t));
-  p.bc2 = (float)(1.0 - pow((double)c->cfg.beta2, t));
+  p.rb1 = (float)(1.0 / (1.0 - pow((double)c->cfg.beta1, t)));
+  p.rb2 = (float)(1.0 / (1.0 - pow((double)c->cfg.beta2, t)));
 
   if (c->dense) {
     LaunchScope ls(c, KID_ADAM_DENSE);
@@ -528,9 +597,9 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  const int smem = (((batch + 1 + 3) & ~3) + UPD_WARPS * (c->H + 32)) * 4;
+  const int smem = (((batch + 1 + 3) & ~3) + UPD_WARPS * 32) * 4;
   const int nch = (c->H / 4 + 31) / 32;
-  if (nch <= 1) return launch_k_update<1, 4>(c, p, smem);
+  if (nch <= 1) return launch_k_update<1, 2>(c, p, smem);
   if (nch <= 2) return launch_k_update<2, 2>(c, p, smem);
   if (nch <= 4) return launch_k_update<4, 1>(c, p, smem);
   return launch_k_update<8, 1>(c, p, smem);
