@@ -5,15 +5,27 @@
 //   -> logits over the active set only (feed forward of the second type)
 //   -> softmax, loss and errors over that ragged set (Algorithm 1 "Compute Errors")
 //   -> error back-propagated to the hidden layer (Section 2.1, back-propagation stage)
-// and records, for the update kernels, which rows of W2 and W1 the sample touches.
+// and hands the touched rows of W2 and W1 to the update kernel.
 // The same kernel in predict mode stops after the logits and selects the top k.
+//
+// Every phase is a short chain of memory rounds, so each round puts as much in flight as it can:
+// the rows of W1 of a chunk of nonzeros are fetched by all threads at once into shared memory and
+// then summed in the stored order; the L bucket offsets are fetched in one round and all bucket
+// entries in a second; the active rows of W2 are copied by the bulk-copy engine (cp.async.bulk,
+// completion on an mbarrier) into the shared memory the dedup work space no longer needs, and
+// serve both the logits and the back-propagated error.
 #include "common.cuh"
 
 namespace dslide {
 
 constexpr int FWD_THREADS = 256;
 constexpr int FWD_WARPS = FWD_THREADS / 32;
-constexpr int MAX_HCHUNK = 8;   // float4 chunks per lane: H <= 4 * 32 * 8 = 1024
+constexpr int MAX_HCHUNK = 8;     // float4 chunks per lane: H <= 4 * 32 * 8 = 1024
+constexpr int MAX_KPT = 4;        // hidden units per thread: H <= 4 * 256
+constexpr int ACT_SM = 1024;      // active ids and logits are mirrored in shared memory when the set is this small
+constexpr int HID_MIN_BYTES = 64 * 1024;   // staging space for the hidden layer's rows of W1
+constexpr int SORT_SMALL = 1024;  // candidate sets up to this size are sorted rather than run through the bitmap
+constexpr unsigned FULLM = 0xffffffffu;
 
 struct FwdParams {
   const float *W1, *b1, *W2, *b2;
@@ -34,10 +46,39 @@ struct FwdParams {
   long long nb;
   int B, D, H, N, K, L, KL, family, lg_bin, fn_len, cap;
   int act_stride, Wd, dense, dedup_mode, max_labels, sort_cap, topk, parity;
-  int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_topk, off_dedup;
+  int stage_bytes;     // bytes of the staging region (it starts at off_dedup and overlays the dedup work space)
+  int hid_rows;        // rows of W1 staged per chunk of the hidden layer
+  int sort_small;      // candidate sets up to this size are deduplicated by sorting even when a bitmap is available
+  int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_tbeg, off_topk, off_ids, off_z, off_col, off_val,
+      off_dedup;
 };
 
 __device__ __forceinline__ void set_status(DevState* st, int code) { atomicCAS(&st->status, 0, code); }
+
+// ---- bulk copy (global -> shared) with completion on an mbarrier ------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Waits for the phase with the given parity; gives up after a bounded number of polls (false).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t a = smem_u32(bar);
+  for (int it = 0; it < (1 << 22); ++it) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
 
 // The touch that takes a row past ROW_SLOTS touching samples enters the row in the list of rows that a warp of
 // the update kernel sums from slots and mask; the touch that takes it past HOT_T enters it in the list of rows
@@ -66,7 +107,7 @@ __device__ __forceinline__ int block_excl_scan(int v, int* sh, int* total) {
   int incl = v;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
-    int n = __shfl_up_sync(0xffffffffu, incl, d);
+    int n = __shfl_up_sync(FULLM, incl, d);
     if (lane >= d) incl += n;
   }
   if (lane == 31) sh[warp] = incl;
@@ -86,7 +127,7 @@ __device__ __forceinline__ int block_excl_scan(int v, int* sh, int* total) {
 // Block-wide max / sum in a fixed order (same value in every thread).  sh: FWD_WARPS floats.
 __device__ __forceinline__ float block_max(float v, float* sh) {
 #pragma unroll
-  for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, d));
+  for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(FULLM, v, d));
   if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
   __syncthreads();
   float r = sh[0];
@@ -96,7 +137,7 @@ __device__ __forceinline__ float block_max(float v, float* sh) {
 }
 __device__ __forceinline__ float block_sum(float v, float* sh) {
 #pragma unroll
-  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(FULLM, v, d);
   if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
   __syncthreads();
   float r = sh[0];
@@ -109,18 +150,41 @@ __device__ __forceinline__ bool topk_better(float za, int ia, float zb, int ib) 
   return za > zb || (za == zb && ia < ib);
 }
 
+// The sample is skipped: no loss, no gradient, nothing touched (predict: no candidates).
+template <int MODE>
+__device__ __forceinline__ void skip_sample(const FwdParams& p, int s, int code) {
+  const int tid = threadIdx.x;
+  if (MODE == 0) {
+    for (int k = tid; k < p.H; k += FWD_THREADS) { p.h[(size_t)s * p.H + k] = 0.f; p.dh[(size_t)s * p.H + k] = 0.f; }
+    if (tid == 0) { p.act_cnt[s] = 0; p.loss[s] = 0.f; }
+  } else {
+    for (int q = tid; q < p.topk; q += FWD_THREADS) {
+      p.out_ids[(size_t)s * p.topk + q] = -1;
+      p.out_scores[(size_t)s * p.topk + q] = -INFINITY;
+    }
+  }
+  if (tid == 0) set_status(p.st, code);
+}
+
 template <int MODE>   // 0 = training step, 1 = predict top-k
-__global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
-  extern __shared__ __align__(16) unsigned char smem[];
+__global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
   float* sh_h = reinterpret_cast<float*>(smem);
   float* sh_dh = reinterpret_cast<float*>(smem + p.off_dh);          // [FWD_WARPS][H]
   uint32_t* sh_code = reinterpret_cast<uint32_t*>(smem + p.off_code);
   unsigned char* sh_part = smem + p.off_part;
   int* sh_misc = reinterpret_cast<int*>(smem + p.off_misc);          // 32 ints
   float* sh_red = reinterpret_cast<float*>(sh_misc + 16);
+  uint64_t* sh_bar = reinterpret_cast<uint64_t*>(sh_misc + 26);      // 8-byte aligned: off_misc is 16-byte aligned
   int* sh_lab = reinterpret_cast<int*>(smem + p.off_lab);            // [max_labels]
   int* sh_tbase = reinterpret_cast<int*>(smem + p.off_tbase);        // [L + 1]
+  int* sh_tbeg = reinterpret_cast<int*>(smem + p.off_tbeg);          // [L]
+  int* sh_ids = reinterpret_cast<int*>(smem + p.off_ids);            // [ACT_SM]
+  float* sh_z = reinterpret_cast<float*>(smem + p.off_z);            // [ACT_SM]
+  int* sh_col = reinterpret_cast<int*>(smem + p.off_col);            // [hid_rows]
+  float* sh_val = reinterpret_cast<float*>(smem + p.off_val);        // [hid_rows]
   uint32_t* sh_dd = reinterpret_cast<uint32_t*>(smem + p.off_dedup);
+  float* stage = reinterpret_cast<float*>(smem + p.off_dedup);       // overlays the dedup work space
 
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = p.H, H4 = H >> 2, N = p.N;
@@ -129,61 +193,90 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
   int lbeg = 0, nlab = 0;
   if (MODE == 0) { lbeg = p.label_ptr[s]; nlab = p.label_ptr[s + 1] - lbeg; }
 
-  // ---- input checks: ids in range, columns ascending, label list within the maximum ----
-  int bad = 0;
-  if (nnz < 0 || nlab < 0) bad = DSLIDE_ERR_BAD_INDEX;
-  else {
-    for (int i = tid; i < nnz; i += FWD_THREADS) {
-      int c = p.col_idx[rbeg + i];
-      if (c < 0 || c >= p.D || (i > 0 && p.col_idx[rbeg + i - 1] >= c)) bad = DSLIDE_ERR_BAD_INDEX;
-    }
-    if (MODE == 0) {
-      for (int i = tid; i < nlab; i += FWD_THREADS) {
-        int y = p.labels[lbeg + i];
-        if (y < 0 || y >= N) bad = DSLIDE_ERR_BAD_INDEX;
-      }
-      if (nlab > p.max_labels) bad = DSLIDE_ERR_OVERFLOW;
-    }
-  }
-  if (tid == 0) sh_misc[24] = 0;               // bucket entries fetched by this sample
-  bad = __syncthreads_or(bad);
-  if (bad) {
-    // The sample is skipped: no loss, no gradient, nothing touched.
-    if (MODE == 0) {
-      for (int k = tid; k < H; k += FWD_THREADS) { p.h[(size_t)s * H + k] = 0.f; p.dh[(size_t)s * H + k] = 0.f; }
-      if (tid == 0) { p.act_cnt[s] = 0; p.loss[s] = 0.f; }
-    } else {
-      for (int q = tid; q < p.topk; q += FWD_THREADS) {
-        p.out_ids[(size_t)s * p.topk + q] = -1;
-        p.out_scores[(size_t)s * p.topk + q] = -INFINITY;
-      }
-    }
-    if (tid == 0) {
-      int code = DSLIDE_ERR_BAD_INDEX;
-      if (MODE == 0 && nnz >= 0 && nlab > p.max_labels) code = DSLIDE_ERR_OVERFLOW;
-      set_status(p.st, code);
-    }
-    return;
+  if (tid == 0) {
+    sh_misc[24] = 0;                 // bucket entries fetched by this sample
+    mbar_init(sh_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
 
-  // ---- hidden layer: bias, then one fused multiply-add per nonzero in stored order, ReLU ----
-  for (int k = tid; k < H; k += FWD_THREADS) {
-    float acc = p.b1[k];
-    int i = rbeg;
-    for (; i + 4 <= rend; i += 4) {
-      int c0 = __ldg(p.col_idx + i), c1 = __ldg(p.col_idx + i + 1), c2 = __ldg(p.col_idx + i + 2), c3 = __ldg(p.col_idx + i + 3);
-      float x0 = __ldg(p.vals + i), x1 = __ldg(p.vals + i + 1), x2 = __ldg(p.vals + i + 2), x3 = __ldg(p.vals + i + 3);
-      float w0 = __ldg(p.W1 + (size_t)c0 * H + k), w1 = __ldg(p.W1 + (size_t)c1 * H + k);
-      float w2 = __ldg(p.W1 + (size_t)c2 * H + k), w3 = __ldg(p.W1 + (size_t)c3 * H + k);
-      acc = __fmaf_rn(x0, w0, acc);
-      acc = __fmaf_rn(x1, w1, acc);
-      acc = __fmaf_rn(x2, w2, acc);
-      acc = __fmaf_rn(x3, w3, acc);
+  // ---- label checks: ids in range, list within the maximum ----
+  int bad = 0;
+  if (nnz < 0 || nlab < 0) bad = DSLIDE_ERR_BAD_INDEX;
+  else if (MODE == 0) {
+    for (int i = tid; i < nlab; i += FWD_THREADS) {
+      int y = p.labels[lbeg + i];
+      if (y < 0 || y >= N) bad = DSLIDE_ERR_BAD_INDEX;
     }
-    for (; i < rend; ++i) acc = __fmaf_rn(__ldg(p.vals + i), __ldg(p.W1 + (size_t)__ldg(p.col_idx + i) * H + k), acc);
-    float hv = acc > 0.f ? acc : 0.f;
-    sh_h[k] = hv;
-    if (MODE == 0) p.h[(size_t)s * H + k] = hv;
+  }
+  const bool too_many_labels = MODE == 0 && nnz >= 0 && nlab > p.max_labels;
+  bad = __syncthreads_or(bad);
+
+  // ---- hidden layer: bias, then one fused multiply-add per nonzero in stored order, ReLU.  The rows of W1 of a
+  //      chunk of nonzeros are fetched together into shared memory; the column ids are checked on the way
+  //      (in range, ascending) ----
+  float acc[MAX_KPT];
+#pragma unroll
+  for (int u = 0; u < MAX_KPT; ++u) {
+    const int k = tid + u * FWD_THREADS;
+    acc[u] = k < H ? p.b1[k] : 0.f;
+  }
+  const int R = p.hid_rows;
+  for (int c0 = 0; c0 < nnz && !bad; c0 += R) {       // `bad` is uniform over the block here
+    const int nr = min(R, nnz - c0);
+    for (int i = tid; i < nr; i += FWD_THREADS) {
+      const int c = __ldg(p.col_idx + rbeg + c0 + i);
+      const int prev = c0 + i > 0 ? __ldg(p.col_idx + rbeg + c0 + i - 1) : -1;
+      const bool okc = c >= 0 && c < p.D && prev < c;
+      if (!okc) bad = DSLIDE_ERR_BAD_INDEX;
+      sh_col[i] = okc ? c : 0;
+      sh_val[i] = __ldg(p.vals + rbeg + c0 + i);
+    }
+    bad = __syncthreads_or(bad);
+    if (bad) break;
+    {
+      float4* st4 = reinterpret_cast<float4*>(stage);
+      const int total4 = nr * H4;
+      for (int e0 = tid; e0 < total4; e0 += FWD_THREADS * 8) {
+        float4 x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int e = e0 + u * FWD_THREADS;
+          if (e < total4) {
+            const int r = e / H4, c4 = e - r * H4;
+            x[u] = __ldg(reinterpret_cast<const float4*>(p.W1 + (size_t)sh_col[r] * H) + c4);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int e = e0 + u * FWD_THREADS;
+          if (e < total4) st4[e] = x[u];
+        }
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < MAX_KPT; ++u) {
+      const int k = tid + u * FWD_THREADS;
+      if (k < H) {
+        float a = acc[u];
+        for (int i = 0; i < nr; ++i) a = __fmaf_rn(sh_val[i], stage[(size_t)i * H + k], a);
+        acc[u] = a;
+      }
+    }
+    __syncthreads();
+  }
+  if (bad || too_many_labels) {
+    skip_sample<MODE>(p, s, (!bad && too_many_labels) ? DSLIDE_ERR_OVERFLOW : DSLIDE_ERR_BAD_INDEX);
+    return;
+  }
+#pragma unroll
+  for (int u = 0; u < MAX_KPT; ++u) {
+    const int k = tid + u * FWD_THREADS;
+    if (k < H) {
+      const float hv = acc[u] > 0.f ? acc[u] : 0.f;
+      sh_h[k] = hv;
+      if (MODE == 0) p.h[(size_t)s * H + k] = hv;
+    }
   }
   __syncthreads();
 
@@ -214,82 +307,89 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
       }
     }
     __syncthreads();
+    // ---- codes, and the slice of every table's bucket the sample reads: all offsets in one round ----
     const int shift = p.family == DSLIDE_SIMHASH ? 1 : p.lg_bin;
     for (int t = tid; t < p.L; t += FWD_THREADS) {
       uint32_t code = 0;
       for (int k = 0; k < p.K; ++k) code |= (uint32_t)sh_part[t * p.K + k] << (k * shift);
       sh_code[t] = code;
       if (MODE == 0) p.codes[(size_t)s * p.L + t] = code;
+      const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1) + code;
+      const int beg = __ldg(off);
+      int cnt = __ldg(off + 1) - beg;
+      cnt = cnt < p.cap ? cnt : p.cap;
+      sh_tbeg[t] = beg;
+      sh_tbase[t + 1] = cnt;
+    }
+    __syncthreads();
+    if (warp == 0) {            // running sum of the slice lengths: where each table's candidates start
+      int run = 0;
+      for (int b = 0; b < p.L; b += 32) {
+        const int t = b + lane;
+        const int v = t < p.L ? sh_tbase[t + 1] : 0;
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          int n = __shfl_up_sync(FULLM, incl, d);
+          if (lane >= d) incl += n;
+        }
+        if (t < p.L) sh_tbase[t + 1] = run + incl;
+        run += __shfl_sync(FULLM, incl, 31);
+      }
+      if (lane == 0) { sh_tbase[0] = 0; sh_misc[24] = run; }
     }
     __syncthreads();
 
-    // ---- lookup, union over the tables, labels, duplicates removed, ascending ids ----
+    // ---- all bucket entries in one round; union over the tables, labels, duplicates removed, ascending ids.
+    //      A small candidate set is cheaper to sort than a bitmap over all N neurons is to clear and scan. ----
+    const int ncand = sh_tbase[p.L];
     int total = 0;
-    if (p.dedup_mode == 1) {
-      const int nwords = (N + 31) >> 5;
-      for (int w = tid; w < nwords; w += FWD_THREADS) sh_dd[w] = 0u;
+    const bool bitmap = p.dedup_mode == 1 && ncand + nlab > p.sort_small;
+    int n2 = 1;
+    if (!bitmap) while (n2 < ncand + nlab) n2 <<= 1;
+    if (bitmap) {
+      uint4* dd4 = reinterpret_cast<uint4*>(sh_dd);
+      const int n4 = (((N + 31) >> 5) + 3) >> 2;
+      for (int w = tid; w < n4; w += FWD_THREADS) dd4[w] = make_uint4(0u, 0u, 0u, 0u);
       __syncthreads();
-      for (int t = warp; t < p.L; t += FWD_WARPS) {
-        const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1);
-        const int beg = __ldg(off + sh_code[t]);
-        int cnt = __ldg(off + sh_code[t] + 1) - beg;
-        cnt = cnt < p.cap ? cnt : p.cap;
-        const int32_t* bid = p.bucket_ids + (size_t)t * N + beg;
-        for (int i = lane; i < cnt; i += 32) {
-          int j = __ldg(bid + i);
-          atomicOr(&sh_dd[j >> 5], 1u << (j & 31));
-        }
-        if (lane == 0) atomicAdd(&sh_misc[24], cnt);
+    }
+    for (int c = tid; c < ncand; c += FWD_THREADS) {
+      int lo = 0, hi = p.L - 1;          // last table whose candidates start at or before c
+      while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (sh_tbase[mid] <= c) lo = mid; else hi = mid - 1; }
+      const int j = __ldg(p.bucket_ids + (size_t)lo * N + sh_tbeg[lo] + (c - sh_tbase[lo]));
+      if (bitmap) atomicOr(&sh_dd[j >> 5], 1u << (j & 31));
+      else sh_dd[c] = (uint32_t)j;
+    }
+    if (MODE == 0)
+      for (int i = tid; i < nlab; i += FWD_THREADS) {
+        const int y = p.labels[lbeg + i];
+        if (bitmap) atomicOr(&sh_dd[y >> 5], 1u << (y & 31));
+        else sh_dd[ncand + i] = (uint32_t)y;
       }
-      if (MODE == 0)
-        for (int i = tid; i < nlab; i += FWD_THREADS) {
-          int y = p.labels[lbeg + i];
-          atomicOr(&sh_dd[y >> 5], 1u << (y & 31));
-        }
+    if (bitmap) {
       __syncthreads();
+      const int nwords = (N + 31) >> 5;
       const int chunk = (nwords + FWD_THREADS - 1) / FWD_THREADS;
       const int wbeg = tid * chunk, wend = min(nwords, wbeg + chunk);
       int cnt = 0;
       for (int w = wbeg; w < wend; ++w) cnt += __popc(sh_dd[w]);
       int pos = block_excl_scan(cnt, sh_misc, &total);
-      if (total <= p.act_stride) {
+      if (total <= p.act_stride && cnt > 0) {
         for (int w = wbeg; w < wend; ++w) {
           uint32_t bits = sh_dd[w];
           while (bits) {
-            int b = __ffs(bits) - 1;
-            ids[pos++] = (w << 5) + b;
+            const int b = __ffs(bits) - 1;
+            const int j = (w << 5) + b;
+            ids[pos] = j;
+            if (pos < ACT_SM) sh_ids[pos] = j;
+            ++pos;
             bits &= bits - 1;
           }
         }
       }
     } else {
-      // sort path: gather all candidates, bitonic sort, keep the first of each run
-      for (int t = tid; t < p.L; t += FWD_THREADS) {
-        const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1);
-        int cnt = __ldg(off + sh_code[t] + 1) - __ldg(off + sh_code[t]);
-        sh_tbase[t] = cnt < p.cap ? cnt : p.cap;
-      }
-      __syncthreads();
-      if (tid == 0) {
-        int run = 0;
-        for (int t = 0; t < p.L; ++t) { int c = sh_tbase[t]; sh_tbase[t] = run; run += c; }
-        sh_tbase[p.L] = run;
-      }
-      __syncthreads();
-      const int ncand = sh_tbase[p.L] + nlab;     // <= L*cap + max_labels <= sort_cap
-      if (tid == 0) sh_misc[24] = sh_tbase[p.L];
-      int n2 = 1;
-      while (n2 < ncand) n2 <<= 1;
-      for (int t = warp; t < p.L; t += FWD_WARPS) {
-        const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1);
-        const int beg = __ldg(off + sh_code[t]);
-        const int cnt = sh_tbase[t + 1] - sh_tbase[t];
-        const int32_t* bid = p.bucket_ids + (size_t)t * N + beg;
-        for (int i = lane; i < cnt; i += 32) sh_dd[sh_tbase[t] + i] = (uint32_t)__ldg(bid + i);
-      }
-      if (MODE == 0)
-        for (int i = tid; i < nlab; i += FWD_THREADS) sh_dd[sh_tbase[p.L] + i] = (uint32_t)p.labels[lbeg + i];
-      for (int i = ncand + tid; i < n2; i += FWD_THREADS) sh_dd[i] = 0x7fffffffu;
+      // sort path: bitonic sort of the candidates, keep the first of each run
+      for (int i = ncand + nlab + tid; i < n2; i += FWD_THREADS) sh_dd[i] = 0x7fffffffu;
       __syncthreads();
       for (int k = 2; k <= n2; k <<= 1)
         for (int j = k >> 1; j > 0; j >>= 1) {
@@ -314,81 +414,148 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
       if (total <= p.act_stride) {
         for (int i = ebeg; i < eend; ++i) {
           uint32_t a = sh_dd[i];
-          if (a != 0x7fffffffu && (i == 0 || sh_dd[i - 1] != a)) ids[pos++] = (int)a;
+          if (a != 0x7fffffffu && (i == 0 || sh_dd[i - 1] != a)) {
+            ids[pos] = (int)a;
+            if (pos < ACT_SM) sh_ids[pos] = (int)a;
+            ++pos;
+          }
         }
       }
     }
     if (total > p.act_stride) {      // uniform over the block
-      if (MODE == 0) {
-        for (int k = tid; k < H; k += FWD_THREADS) { p.h[(size_t)s * H + k] = 0.f; p.dh[(size_t)s * H + k] = 0.f; }
-        if (tid == 0) { p.act_cnt[s] = 0; p.loss[s] = 0.f; }
-      } else {
-        for (int q = tid; q < p.topk; q += FWD_THREADS) {
-          p.out_ids[(size_t)s * p.topk + q] = -1;
-          p.out_scores[(size_t)s * p.topk + q] = -INFINITY;
-        }
-      }
-      if (tid == 0) set_status(p.st, DSLIDE_ERR_OVERFLOW);
+      skip_sample<MODE>(p, s, DSLIDE_ERR_OVERFLOW);
       return;
     }
     na = total;
-    __syncthreads();
+    __syncthreads();                 // ids visible to the block; the dedup work space is free from here on
   }
   if (MODE == 0 && tid == 0) p.act_cnt[s] = na;
+  const bool small = !dense && na <= ACT_SM;      // ids and logits mirrored in shared memory
+  // one pointer per array, to shared or to global memory (a conditional expression over two loads would issue both)
+  const int* idp = small ? sh_ids : ids;
+  const float* zp = small ? sh_z : p.act_z + (size_t)s * p.act_stride;
+  const float* gp = small ? sh_z : p.act_g + (size_t)s * p.act_stride;
 
-  // ---- logits over the active set: one warp per neuron, four neurons in flight ----
+  // ---- the W1 side of the hand-off to the update kernel.  Per touched row a count of the touching samples; for
+  //      the row's first ROW_SLOTS touches the (sample, coefficient) pair itself, else the bit of this sample in
+  //      the row's mask.  The sample that touches a row first also enters it in the list of distinct rows
+  //      (positions handed out per warp). ----
+  const uint32_t sbit = 1u << (s & 31);
+  const int sword = s >> 5;
+  const unsigned ltm = (1u << lane) - 1u;
+  if (MODE == 0) {
+    for (int i0 = 0; i0 < nnz; i0 += FWD_THREADS) {
+      const int i = i0 + tid;
+      bool first = false;
+      int c = 0;
+      if (i < nnz) {
+        c = __ldg(p.col_idx + rbeg + i);
+        const unsigned nth = atomicAdd(p.cnt1 + c, 1u) & CNT_MASK;
+        if (nth < (unsigned)ROW_SLOTS) p.slots1[(size_t)c * ROW_SLOTS + nth] = make_int2(s, __float_as_int(__ldg(p.vals + rbeg + i)));
+        else atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
+        first = nth == 0u;
+        list_row(p, p.cnt1 + c, ~c, nth);
+      }
+      const unsigned fm = __ballot_sync(FULLM, first);
+      if (fm) {
+        unsigned base = 0;
+        if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][1], (unsigned)__popc(fm));
+        base = __shfl_sync(FULLM, base, 0);
+        if (first) p.own1[base + __popc(fm & ltm)] = c;
+      }
+    }
+  }
+
+  // ---- logits over the active set.  The active rows of W2 are copied into shared memory, as many as fit at a
+  //      time; when the whole set fits they stay there for the back-propagation below ----
   float* z = p.act_z + (size_t)s * p.act_stride;
   float* tk_z = reinterpret_cast<float*>(smem + p.off_topk);          // predict: [FWD_WARPS][topk]
   int* tk_id = reinterpret_cast<int*>(tk_z + FWD_WARPS * p.topk);
   int tk_cnt = 0;                                                     // used by lane 0
   const float4* sh_h4 = reinterpret_cast<const float4*>(sh_h);
-  for (int a0 = warp * 4; a0 < na; a0 += FWD_WARPS * 4) {
-    int j[4];
-    float acc[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      int a = a0 + r;
-      j[r] = a < na ? (dense ? a : ids[a]) : -1;
-      acc[r] = 0.f;
+  const int stage_rows = p.stage_bytes / (H * 4);
+  const uint32_t row_bytes = (uint32_t)H * 4u;
+  uint32_t phase = 0;
+  bool timed_out = false;
+  for (int c0 = 0; c0 < na; c0 += stage_rows) {
+    const int nr = min(stage_rows, na - c0);
+    __syncthreads();                               // earlier readers and writers of the staging space are done
+    if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * row_bytes);
+    fence_proxy_async();
+    __syncthreads();
+    for (int r = tid; r < nr; r += FWD_THREADS) {
+      const int j = dense ? c0 + r : idp[c0 + r];
+      bulk_g2s(stage + (size_t)r * H, p.W2 + (size_t)j * H, row_bytes, sh_bar);
     }
-    for (int c = lane; c < H4; c += 32) {
-      float4 x = sh_h4[c];
-      float4 w[4];
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
-        w[r] = j[r] >= 0 ? __ldg(reinterpret_cast<const float4*>(p.W2 + (size_t)j[r] * H) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    // the biases of a small active set are fetched in the same round, into the logits' place
+    if (small && c0 == 0)
+      for (int a = tid; a < na; a += FWD_THREADS) sh_z[a] = __ldg(p.b2 + sh_ids[a]);
+    if (!mbar_wait(sh_bar, phase)) timed_out = true;
+    phase ^= 1u;
+    if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
+    for (int a0 = warp * 4; a0 < nr; a0 += FWD_WARPS * 4) {
+      int j[4];
+      float dot[4];
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
-        acc[r] = fmaf(w[r].x, x.x, acc[r]);
-        acc[r] = fmaf(w[r].y, x.y, acc[r]);
-        acc[r] = fmaf(w[r].z, x.z, acc[r]);
-        acc[r] = fmaf(w[r].w, x.w, acc[r]);
+        const int a = a0 + r;
+        j[r] = a < nr ? (dense ? c0 + a : idp[c0 + a]) : -1;
+        dot[r] = 0.f;
       }
-    }
+      for (int c = lane; c < H4; c += 32) {
+        const float4 x = sh_h4[c];
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
+        for (int r = 0; r < 4; ++r)
+          if (j[r] >= 0) {
+            const float4 w = reinterpret_cast<const float4*>(stage + (size_t)(a0 + r) * H)[c];
+            dot[r] = fmaf(w.x, x.x, dot[r]);
+            dot[r] = fmaf(w.y, x.y, dot[r]);
+            dot[r] = fmaf(w.z, x.z, dot[r]);
+            dot[r] = fmaf(w.w, x.w, dot[r]);
+          }
+      }
 #pragma unroll
-      for (int r = 0; r < 4; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], d);
-    }
-    if (MODE == 0) {
+      for (int d = 16; d > 0; d >>= 1) {
 #pragma unroll
-      for (int r = 0; r < 4; ++r)
-        if (lane == r && j[r] >= 0) z[a0 + r] = __ldg(p.b2 + j[r]) + acc[r];
-    } else if (lane == 0) {
-      float* lz = tk_z + warp * p.topk;
-      int* li = tk_id + warp * p.topk;
+        for (int r = 0; r < 4; ++r) dot[r] += __shfl_xor_sync(FULLM, dot[r], d);
+      }
+      if (MODE == 0) {
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        if (j[r] < 0) continue;
-        float zv = __ldg(p.b2 + j[r]) + acc[r];
-        if (tk_cnt < p.topk || topk_better(zv, j[r], lz[tk_cnt - 1], li[tk_cnt - 1])) {
-          int q = tk_cnt < p.topk ? tk_cnt++ : p.topk - 1;
-          while (q > 0 && topk_better(zv, j[r], lz[q - 1], li[q - 1])) { lz[q] = lz[q - 1]; li[q] = li[q - 1]; --q; }
-          lz[q] = zv; li[q] = j[r];
+        for (int r = 0; r < 4; ++r)
+          if (lane == r && j[r] >= 0) {
+            if (small) {                       // the bias is already in the logit's place
+              const float zv = sh_z[c0 + a0 + r] + dot[r];
+              sh_z[c0 + a0 + r] = zv;
+              z[c0 + a0 + r] = zv;
+            } else {
+              z[c0 + a0 + r] = __ldg(p.b2 + j[r]) + dot[r];
+            }
+          }
+      } else if (lane == 0) {
+        float* lz = tk_z + warp * p.topk;
+        int* li = tk_id + warp * p.topk;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          if (j[r] < 0) continue;
+          float zv = __ldg(p.b2 + j[r]) + dot[r];
+          if (tk_cnt < p.topk || topk_better(zv, j[r], lz[tk_cnt - 1], li[tk_cnt - 1])) {
+            int q = tk_cnt < p.topk ? tk_cnt++ : p.topk - 1;
+            while (q > 0 && topk_better(zv, j[r], lz[q - 1], li[q - 1])) { lz[q] = lz[q - 1]; li[q] = li[q - 1]; --q; }
+            lz[q] = zv; li[q] = j[r];
+          }
         }
       }
     }
   }
+  if (timed_out) {
+    // a copy did not complete in time: give the copies still in flight one more bounded wait, then give the sample
+    // up (its rows of W1 are already handed over; with dh = 0 they receive a zero gradient)
+    mbar_wait(sh_bar, phase ^ 1u);
+    __syncthreads();
+    skip_sample<MODE>(p, s, DSLIDE_ERR_TIMEOUT);
+    return;
+  }
+  const bool staged_all = na <= stage_rows;      // every active row is still in shared memory
 
   if (MODE == 1) {
     // ---- merge the per-warp lists: k rounds over the list heads ----
@@ -416,6 +583,7 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
     }
     return;
   }
+  __syncthreads();           // logits visible to the block
 
   // ---- positions of the sample's distinct labels inside the active set ----
   for (int i = tid; i < nlab; i += FWD_THREADS) {
@@ -425,129 +593,122 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
     int pos = y;
     if (!dense) {
       int lo = 0, hi = na;
-      while (lo < hi) { int mid = (lo + hi) >> 1; if (ids[mid] < y) lo = mid + 1; else hi = mid; }
+      while (lo < hi) { int mid = (lo + hi) >> 1; if (idp[mid] < y) lo = mid + 1; else hi = mid; }
       pos = lo;
     }
     sh_lab[i] = first ? pos : -1;
   }
-  __syncthreads();
 
   // ---- softmax over the ragged active set, loss, errors ----
   float* pr = p.act_p + (size_t)s * p.act_stride;
   float* g = p.act_g + (size_t)s * p.act_stride;
   float m = -INFINITY;
-  for (int a = tid; a < na; a += FWD_THREADS) m = fmaxf(m, z[a]);
+  for (int a = tid; a < na; a += FWD_THREADS) m = fmaxf(m, zp[a]);
   const float M = block_max(m, sh_red);
   float e = 0.f;
-  for (int a = tid; a < na; a += FWD_THREADS) e += expf(z[a] - M);
-  const float E = block_sum(e, sh_red);
+  for (int a = tid; a < na; a += FWD_THREADS) e += expf(zp[a] - M);
+  const float E = block_sum(e, sh_red);            // its barriers also make sh_lab visible
   const float fB = (float)p.B;
-  for (int a = tid; a < na; a += FWD_THREADS) {
-    float pa = expf(z[a] - M) / E;
-    pr[a] = pa;
-    g[a] = pa / fB;
-  }
-  __syncthreads();
   if (tid == 0) {
     int ny = 0;
     for (int i = 0; i < nlab; ++i) ny += sh_lab[i] >= 0 ? 1 : 0;
     float sum = 0.f;
     const float logE = logf(E);
     for (int i = 0; i < nlab; ++i)
-      if (sh_lab[i] >= 0) sum += z[sh_lab[i]] - M - logE;
+      if (sh_lab[i] >= 0) sum += zp[sh_lab[i]] - M - logE;
     p.loss[s] = ny > 0 ? -sum / (float)ny : 0.f;
     sh_misc[0] = ny;
   }
   __syncthreads();
-  {
-    const int ny = sh_misc[0];
-    for (int i = tid; i < nlab; i += FWD_THREADS)
-      if (sh_lab[i] >= 0) g[sh_lab[i]] = (pr[sh_lab[i]] - 1.f / (float)ny) / fB;
+  const int ny = sh_misc[0];
+  // when the set is small the error takes the logit's place in shared memory, for the steps below
+  for (int a = tid; a < na; a += FWD_THREADS) {
+    const float pa = expf(zp[a] - M) / E;
+    pr[a] = pa;
+    float ga = pa / fB;
+    for (int i = 0; i < nlab; ++i)
+      if (sh_lab[i] == a) ga = (pa - 1.f / (float)ny) / fB;
+    g[a] = ga;
+    if (small) sh_z[a] = ga;
   }
   __syncthreads();
 
-  // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update) ----
-  {
-    float4 acc[MAX_HCHUNK];
-#pragma unroll
-    for (int q = 0; q < MAX_HCHUNK; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int a = warp; a < na; a += FWD_WARPS) {
-      const int jj = dense ? a : ids[a];
-      const float ga = g[a];
-      const float4* row = reinterpret_cast<const float4*>(p.W2 + (size_t)jj * H);
-#pragma unroll
-      for (int q = 0; q < MAX_HCHUNK; ++q) {
-        int c = lane + q * 32;
-        if (c < H4) {
-          float4 w = __ldg(row + c);
-          acc[q].x = fmaf(ga, w.x, acc[q].x);
-          acc[q].y = fmaf(ga, w.y, acc[q].y);
-          acc[q].z = fmaf(ga, w.z, acc[q].z);
-          acc[q].w = fmaf(ga, w.w, acc[q].w);
-        }
-      }
-    }
-    float4* mine = reinterpret_cast<float4*>(sh_dh + (size_t)warp * H);
-#pragma unroll
-    for (int q = 0; q < MAX_HCHUNK; ++q) {
-      int c = lane + q * 32;
-      if (c < H4) mine[c] = acc[q];
-    }
-  }
-  __syncthreads();
-  for (int k = tid; k < H; k += FWD_THREADS) {
-    float v = 0.f;
-    for (int w = 0; w < FWD_WARPS; ++w) v += sh_dh[(size_t)w * H + k];
-    p.dh[(size_t)s * H + k] = sh_h[k] > 0.f ? v : 0.f;
-  }
-
-  // ---- hand the sample's touches to the update kernel.  Per touched row: a count of the touching samples;
-  //      for the row's first ROW_SLOTS touches the (sample, coefficient) pair itself, else the bit of this
-  //      sample in the row's mask.  The sample that touches a row first also enters it in the list of
-  //      distinct rows (positions handed out per warp). ----
-  const uint32_t sbit = 1u << (s & 31);
-  const int sword = s >> 5;
-  const unsigned lt = (1u << lane) - 1u;
+  // ---- the W2 side of the hand-off, issued before the back-propagation so that its atomics overlap it ----
   if (!dense)
     for (int a0 = 0; a0 < na; a0 += FWD_THREADS) {
       const int a = a0 + tid;
       bool first = false;
       int jj = 0;
       if (a < na) {
-        jj = ids[a];
+        jj = idp[a];
+        const float ga = gp[a];
         const unsigned nth = atomicAdd(p.cnt2 + jj, 1u) & CNT_MASK;
-        if (nth < (unsigned)ROW_SLOTS) p.slots2[(size_t)jj * ROW_SLOTS + nth] = make_int2(s, __float_as_int(g[a]));
+        if (nth < (unsigned)ROW_SLOTS) p.slots2[(size_t)jj * ROW_SLOTS + nth] = make_int2(s, __float_as_int(ga));
         else atomicOr(p.mask2 + (size_t)jj * p.Wd + sword, sbit);
         first = nth == 0u;
         list_row(p, p.cnt2 + jj, jj, nth);
       }
-      const unsigned fm = __ballot_sync(0xffffffffu, first);
+      const unsigned fm = __ballot_sync(FULLM, first);
       if (fm) {
         unsigned base = 0;
         if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][0], (unsigned)__popc(fm));
-        base = __shfl_sync(0xffffffffu, base, 0);
-        if (first) p.own2[base + __popc(fm & lt)] = jj;
+        base = __shfl_sync(FULLM, base, 0);
+        if (first) p.own2[base + __popc(fm & ltm)] = jj;
       }
     }
-  for (int i0 = 0; i0 < nnz; i0 += FWD_THREADS) {
-    const int i = i0 + tid;
-    bool first = false;
-    int c = 0;
-    if (i < nnz) {
-      c = p.col_idx[rbeg + i];
-      const unsigned nth = atomicAdd(p.cnt1 + c, 1u) & CNT_MASK;
-      if (nth < (unsigned)ROW_SLOTS) p.slots1[(size_t)c * ROW_SLOTS + nth] = make_int2(s, __float_as_int(p.vals[rbeg + i]));
-      else atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
-      first = nth == 0u;
-      list_row(p, p.cnt1 + c, ~c, nth);
+
+  // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update) ----
+  {
+    float4 accd[MAX_HCHUNK];
+#pragma unroll
+    for (int q = 0; q < MAX_HCHUNK; ++q) accd[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = 0; c0 < na; c0 += stage_rows) {
+      const int nr = min(stage_rows, na - c0);
+      if (!staged_all) {
+        __syncthreads();
+        if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * row_bytes);
+        fence_proxy_async();
+        __syncthreads();
+        for (int r = tid; r < nr; r += FWD_THREADS) {
+          const int j = dense ? c0 + r : idp[c0 + r];
+          bulk_g2s(stage + (size_t)r * H, p.W2 + (size_t)j * H, row_bytes, sh_bar);
+        }
+        if (!mbar_wait(sh_bar, phase)) timed_out = true;
+        phase ^= 1u;
+        if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
+      }
+      for (int a = warp; a < nr; a += FWD_WARPS) {
+        const float ga = gp[c0 + a];
+        const float4* row = reinterpret_cast<const float4*>(stage + (size_t)a * H);
+#pragma unroll
+        for (int q = 0; q < MAX_HCHUNK; ++q) {
+          const int c = lane + q * 32;
+          if (c < H4) {
+            const float4 w = row[c];
+            accd[q].x = fmaf(ga, w.x, accd[q].x);
+            accd[q].y = fmaf(ga, w.y, accd[q].y);
+            accd[q].z = fmaf(ga, w.z, accd[q].z);
+            accd[q].w = fmaf(ga, w.w, accd[q].w);
+          }
+        }
+      }
     }
-    const unsigned fm = __ballot_sync(0xffffffffu, first);
-    if (fm) {
-      unsigned base = 0;
-      if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][1], (unsigned)__popc(fm));
-      base = __shfl_sync(0xffffffffu, base, 0);
-      if (first) p.own1[base + __popc(fm & lt)] = c;
+    float4* mine = reinterpret_cast<float4*>(sh_dh + (size_t)warp * H);
+#pragma unroll
+    for (int q = 0; q < MAX_HCHUNK; ++q) {
+      const int c = lane + q * 32;
+      if (c < H4) mine[c] = accd[q];
     }
+  }
+  __syncthreads();
+  if (timed_out) {
+    mbar_wait(sh_bar, phase ^ 1u);
+    if (tid == 0) set_status(p.st, DSLIDE_ERR_TIMEOUT);
+  }
+  for (int k = tid; k < H; k += FWD_THREADS) {
+    float v = 0.f;
+    for (int w = 0; w < FWD_WARPS; ++w) v += sh_dh[(size_t)w * H + k];
+    p.dh[(size_t)s * H + k] = (sh_h[k] > 0.f && !timed_out) ? v : 0.f;
   }
   if (tid == 0) {
     atomicAdd(&p.st->acc[p.parity][0], (unsigned long long)na);
@@ -560,11 +721,20 @@ __global__ void __launch_bounds__(FWD_THREADS) k_forward(const FwdParams p) {
 // Host side: shared-memory layout and launches
 // ---------------------------------------------------------------------------
 static int align16(int x) { return (x + 15) & ~15; }
+static int align128(int x) { return (x + 127) & ~127; }
 
-struct FwdLayout { int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_topk, off_dedup, fixed_bytes; };
+struct FwdLayout {
+  int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_tbeg, off_topk, off_ids, off_z, off_col, off_val,
+      off_dedup, fixed_bytes, hid_rows;
+};
 
 static FwdLayout fwd_layout(const Ctx* c) {
   FwdLayout l;
+  // rows of W1 staged per chunk of the hidden layer: HID_MIN_BYTES worth, between 8 and 128
+  int hid_rows = HID_MIN_BYTES / (c->H * 4);
+  if (hid_rows > 128) hid_rows = 128;
+  if (hid_rows < 8) hid_rows = 8;
+  l.hid_rows = hid_rows;
   int o = align16(c->H * 4);
   l.off_dh = o;      o = align16(o + FWD_WARPS * c->H * 4);
   l.off_code = o;    o = align16(o + c->L * 4);
@@ -572,7 +742,13 @@ static FwdLayout fwd_layout(const Ctx* c) {
   l.off_misc = o;    o = align16(o + 32 * 4);
   l.off_lab = o;     o = align16(o + (c->cfg.max_labels > 0 ? c->cfg.max_labels : 1) * 4);
   l.off_tbase = o;   o = align16(o + (c->L + 1) * 4);
+  l.off_tbeg = o;    o = align16(o + c->L * 4);
   l.off_topk = o;    o = align16(o + FWD_WARPS * 64 * 8);
+  l.off_ids = o;     o = align16(o + ACT_SM * 4);
+  l.off_z = o;       o = align16(o + ACT_SM * 4);
+  l.off_col = o;     o = align16(o + hid_rows * 4);
+  l.off_val = o;     o = align16(o + hid_rows * 4);
+  o = align128(o);
   l.off_dedup = o;
   l.fixed_bytes = o;
   return l;
@@ -581,21 +757,38 @@ static FwdLayout fwd_layout(const Ctx* c) {
 cudaError_t setup_forward(Ctx* c) {
   FwdLayout l = fwd_layout(c);
   const int budget = 227 * 1024 - l.fixed_bytes;
-  const int bitmap_bytes = ((c->N + 31) / 32) * 4;
+  const int bitmap_bytes = align16(((c->N + 31) / 32) * 4);
   int64_t worst = (int64_t)c->L * c->cap + c->cfg.max_labels;
   int64_t pow2 = 1;
   while (pow2 < worst) pow2 <<= 1;
   const int64_t sort_bytes = pow2 * 4;
+  // the staging space holds the hidden layer's chunk of W1 rows and, later, active rows of W2
+  const int stage_min = l.hid_rows * c->H * 4;
   int mode = c->cfg.dedup_mode;
-  if (c->dense) { mode = 1; c->fwd_smem = l.fixed_bytes; c->sort_cap = 0; c->dedup_mode = 1; }
+  int dd_bytes = 0;
+  if (c->dense) { mode = 1; c->sort_cap = 0; }
   else {
     if (mode == 0) mode = (bitmap_bytes <= 100 * 1024 || sort_bytes > budget) ? 1 : 2;
     if (mode == 1 && bitmap_bytes > budget) return cudaErrorInvalidValue;
     if (mode == 2 && sort_bytes > budget) return cudaErrorInvalidValue;
-    c->dedup_mode = mode;
     c->sort_cap = (int)pow2;
-    c->fwd_smem = l.fixed_bytes + (mode == 1 ? bitmap_bytes : (int)sort_bytes);
+    dd_bytes = mode == 1 ? bitmap_bytes : (int)sort_bytes;
   }
+  c->dedup_mode = mode;
+  int stage = dd_bytes > stage_min ? dd_bytes : stage_min;
+  // when the dedup work space leaves room for two blocks per multiprocessor, staging gets the rest of a half
+  const int two_per_sm = (227 * 1024) / 2 - 1024 - l.fixed_bytes;
+  if (stage < two_per_sm) stage = two_per_sm;
+  if (stage > budget) stage = budget;
+  if (stage < stage_min || stage < c->H * 4) return cudaErrorInvalidValue;
+  c->fwd_stage_bytes = stage & ~15;
+  // dedup by sorting for small candidate sets: mode 0 picks per sample, mode 1 always uses the bitmap, mode 2 always sorts
+  c->fwd_sort_small = 0;
+  if (mode == 1 && c->cfg.dedup_mode == 0 && !c->dense) {
+    int cap_small = c->fwd_stage_bytes / 8;      // the sort pads to a power of two
+    c->fwd_sort_small = cap_small < SORT_SMALL ? cap_small : SORT_SMALL;
+  }
+  c->fwd_smem = l.fixed_bytes + c->fwd_stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(k_forward<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(k_forward<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -619,8 +812,10 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.act_stride = c->act_stride; p.Wd = c->Wd; p.dense = c->dense; p.dedup_mode = c->dedup_mode;
   p.max_labels = c->cfg.max_labels; p.sort_cap = c->sort_cap; p.topk = 1;
   FwdLayout l = fwd_layout(c);
+  p.stage_bytes = c->fwd_stage_bytes; p.hid_rows = l.hid_rows; p.sort_small = c->fwd_sort_small;
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
-  p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_topk = l.off_topk; p.off_dedup = l.off_dedup;
+  p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;
+  p.off_ids = l.off_ids; p.off_z = l.off_z; p.off_col = l.off_col; p.off_val = l.off_val; p.off_dedup = l.off_dedup;
   return p;
 }
 
@@ -640,11 +835,10 @@ cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int3
   p.topk = k;
   p.out_ids = out_ids;
   p.out_scores = out_scores;
-  int smem = c->fwd_smem;
-  if (dense) { p.dense = 1; smem = fwd_layout(c).fixed_bytes; }
+  if (dense) p.dense = 1;
   {
     LaunchScope ls(c, KID_PREDICT);
-    k_forward<1><<<batch, FWD_THREADS, smem, c->stream>>>(p);
+    k_forward<1><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
   }
   return cudaGetLastError();
 }
