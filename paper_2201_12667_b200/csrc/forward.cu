@@ -473,7 +473,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   int* tk_id = reinterpret_cast<int*>(tk_z + FWD_WARPS * p.topk);
   int tk_cnt = 0;                                                     // used by lane 0
   const float4* sh_h4 = reinterpret_cast<const float4*>(sh_h);
-  const int stage_rows = p.stage_bytes / (H * 4);
+  const int ldr = H + 4;                           // staged rows are padded by 16 bytes: a thread per row reads without bank conflicts
+  const int stage_rows = p.stage_bytes / (ldr * 4);
   const uint32_t row_bytes = (uint32_t)H * 4u;
   uint32_t phase = 0;
   bool timed_out = false;
@@ -485,7 +486,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     __syncthreads();
     for (int r = tid; r < nr; r += FWD_THREADS) {
       const int j = dense ? c0 + r : idp[c0 + r];
-      bulk_g2s(stage + (size_t)r * H, p.W2 + (size_t)j * H, row_bytes, sh_bar);
+      bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)j * H, row_bytes, sh_bar);
     }
     // the biases of a small active set are fetched in the same round, into the logits' place
     if (small && c0 == 0)
@@ -493,55 +494,49 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     if (!mbar_wait(sh_bar, phase)) timed_out = true;
     phase ^= 1u;
     if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
-    for (int a0 = warp * 4; a0 < nr; a0 += FWD_WARPS * 4) {
-      int j[4];
-      float dot[4];
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const int a = a0 + r;
-        j[r] = a < nr ? (dense ? c0 + a : idp[c0 + a]) : -1;
-        dot[r] = 0.f;
-      }
-      for (int c = lane; c < H4; c += 32) {
-        const float4 x = sh_h4[c];
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-          if (j[r] >= 0) {
-            const float4 w = reinterpret_cast<const float4*>(stage + (size_t)(a0 + r) * H)[c];
-            dot[r] = fmaf(w.x, x.x, dot[r]);
-            dot[r] = fmaf(w.y, x.y, dot[r]);
-            dot[r] = fmaf(w.z, x.z, dot[r]);
-            dot[r] = fmaf(w.w, x.w, dot[r]);
-          }
-      }
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) {
-#pragma unroll
-        for (int r = 0; r < 4; ++r) dot[r] += __shfl_xor_sync(FULLM, dot[r], d);
+    // one thread per staged row
+    for (int ab = 0; ab < nr; ab += FWD_THREADS) {
+      const int a = ab + tid;
+      const bool live = a < nr;
+      float dot = 0.f;
+      if (live) {
+        const float4* row = reinterpret_cast<const float4*>(stage + (size_t)a * ldr);
+        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < H4; ++c) {
+          const float4 w = row[c], x = sh_h4[c];
+          d0 = fmaf(w.x, x.x, d0);
+          d1 = fmaf(w.y, x.y, d1);
+          d2 = fmaf(w.z, x.z, d2);
+          d3 = fmaf(w.w, x.w, d3);
+        }
+        dot = (d0 + d1) + (d2 + d3);
       }
       if (MODE == 0) {
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-          if (lane == r && j[r] >= 0) {
-            if (small) {                       // the bias is already in the logit's place
-              const float zv = sh_z[c0 + a0 + r] + dot[r];
-              sh_z[c0 + a0 + r] = zv;
-              z[c0 + a0 + r] = zv;
-            } else {
-              z[c0 + a0 + r] = __ldg(p.b2 + j[r]) + dot[r];
-            }
+        if (live) {
+          if (small) {                       // the bias is already in the logit's place
+            const float zv = sh_z[c0 + a] + dot;
+            sh_z[c0 + a] = zv;
+            z[c0 + a] = zv;
+          } else {
+            const int j = dense ? c0 + a : idp[c0 + a];
+            z[c0 + a] = __ldg(p.b2 + j) + dot;
           }
-      } else if (lane == 0) {
+        }
+      } else {
+        // predict: lane 0 of each warp keeps the warp's best k so far, fed one lane's logit at a time
+        int j = -1;
+        float zv = 0.f;
+        if (live) { j = dense ? c0 + a : idp[c0 + a]; zv = __ldg(p.b2 + j) + dot; }
         float* lz = tk_z + warp * p.topk;
         int* li = tk_id + warp * p.topk;
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          if (j[r] < 0) continue;
-          float zv = __ldg(p.b2 + j[r]) + dot[r];
-          if (tk_cnt < p.topk || topk_better(zv, j[r], lz[tk_cnt - 1], li[tk_cnt - 1])) {
+        for (int l = 0; l < 32; ++l) {
+          const int jl = __shfl_sync(FULLM, j, l);
+          const float zl = __shfl_sync(FULLM, zv, l);
+          if (lane == 0 && jl >= 0 && (tk_cnt < p.topk || topk_better(zl, jl, lz[tk_cnt - 1], li[tk_cnt - 1]))) {
             int q = tk_cnt < p.topk ? tk_cnt++ : p.topk - 1;
-            while (q > 0 && topk_better(zv, j[r], lz[q - 1], li[q - 1])) { lz[q] = lz[q - 1]; li[q] = li[q - 1]; --q; }
-            lz[q] = zv; li[q] = j[r];
+            while (q > 0 && topk_better(zl, jl, lz[q - 1], li[q - 1])) { lz[q] = lz[q - 1]; li[q] = li[q - 1]; --q; }
+            lz[q] = zl; li[q] = jl;
           }
         }
       }
@@ -657,11 +652,15 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
     }
 
-  // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update) ----
+  // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update).  A thread
+  //      per hidden unit walks the staged rows; with fewer hidden units than threads the rows are dealt to
+  //      several groups of threads whose sums are then added in group order ----
   {
-    float4 accd[MAX_HCHUNK];
+    const int ngrp = H >= FWD_THREADS ? 1 : min(FWD_WARPS, FWD_THREADS / H);   // groups of H threads (sh_dh holds FWD_WARPS)
+    const int grp = H >= FWD_THREADS ? 0 : tid / H;
+    float accd[MAX_KPT];
 #pragma unroll
-    for (int q = 0; q < MAX_HCHUNK; ++q) accd[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int u = 0; u < MAX_KPT; ++u) accd[u] = 0.f;
     for (int c0 = 0; c0 < na; c0 += stage_rows) {
       const int nr = min(stage_rows, na - c0);
       if (!staged_all) {
@@ -671,44 +670,41 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         __syncthreads();
         for (int r = tid; r < nr; r += FWD_THREADS) {
           const int j = dense ? c0 + r : idp[c0 + r];
-          bulk_g2s(stage + (size_t)r * H, p.W2 + (size_t)j * H, row_bytes, sh_bar);
+          bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)j * H, row_bytes, sh_bar);
         }
         if (!mbar_wait(sh_bar, phase)) timed_out = true;
         phase ^= 1u;
         if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
       }
-      for (int a = warp; a < nr; a += FWD_WARPS) {
-        const float ga = gp[c0 + a];
-        const float4* row = reinterpret_cast<const float4*>(stage + (size_t)a * H);
+      if (grp < ngrp) {
 #pragma unroll
-        for (int q = 0; q < MAX_HCHUNK; ++q) {
-          const int c = lane + q * 32;
-          if (c < H4) {
-            const float4 w = row[c];
-            accd[q].x = fmaf(ga, w.x, accd[q].x);
-            accd[q].y = fmaf(ga, w.y, accd[q].y);
-            accd[q].z = fmaf(ga, w.z, accd[q].z);
-            accd[q].w = fmaf(ga, w.w, accd[q].w);
+        for (int u = 0; u < MAX_KPT; ++u) {
+          const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
+          if (k < H && (u == 0 || H > FWD_THREADS)) {
+            float v = accd[u];
+            for (int a = grp; a < nr; a += ngrp) v = fmaf(gp[c0 + a], stage[(size_t)a * ldr + k], v);
+            accd[u] = v;
           }
         }
       }
     }
-    float4* mine = reinterpret_cast<float4*>(sh_dh + (size_t)warp * H);
+    if (grp < ngrp) {
 #pragma unroll
-    for (int q = 0; q < MAX_HCHUNK; ++q) {
-      const int c = lane + q * 32;
-      if (c < H4) mine[c] = accd[q];
+      for (int u = 0; u < MAX_KPT; ++u) {
+        const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
+        if (k < H && (u == 0 || H > FWD_THREADS)) sh_dh[(size_t)grp * H + k] = accd[u];
+      }
     }
-  }
-  __syncthreads();
-  if (timed_out) {
-    mbar_wait(sh_bar, phase ^ 1u);
-    if (tid == 0) set_status(p.st, DSLIDE_ERR_TIMEOUT);
-  }
-  for (int k = tid; k < H; k += FWD_THREADS) {
-    float v = 0.f;
-    for (int w = 0; w < FWD_WARPS; ++w) v += sh_dh[(size_t)w * H + k];
-    p.dh[(size_t)s * H + k] = (sh_h[k] > 0.f && !timed_out) ? v : 0.f;
+    __syncthreads();
+    if (timed_out) {
+      mbar_wait(sh_bar, phase ^ 1u);
+      if (tid == 0) set_status(p.st, DSLIDE_ERR_TIMEOUT);
+    }
+    for (int k = tid; k < H; k += FWD_THREADS) {
+      float v = 0.f;
+      for (int w = 0; w < ngrp; ++w) v += sh_dh[(size_t)w * H + k];
+      p.dh[(size_t)s * H + k] = (sh_h[k] > 0.f && !timed_out) ? v : 0.f;
+    }
   }
   if (tid == 0) {
     atomicAdd(&p.st->acc[p.parity][0], (unsigned long long)na);
