@@ -53,9 +53,9 @@ cudaError_t dalloc(T** p, size_t n, cudaStream_t st, bool zero) {
 }
 
 void free_all(Ctx* c) {
-  void* ptrs[] = {c->W1, c->b1, c->W2, c->b2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2, c->mb2, c->vb2,
+  void* ptrs[] = {c->W1, c->b1, c->W2, c->hdr1, c->hdr2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
-                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->cnt1, c->cnt2, c->slots1, c->slots2, c->mask1,
+                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1,
                   c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
                   c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -74,7 +74,7 @@ int ilog2_exact(int x) {
   return (1 << l) == x ? l : -1;
 }
 
-struct TensorRef { void* ptr; int64_t bytes; };
+struct TensorRef { void* ptr; int64_t bytes; int64_t pitch; };     // pitch != 0: one float every `pitch` bytes
 
 TensorRef tensor_ref(Ctx* c, int which) {
   const int64_t D = c->D, H = c->H, N = c->N, f = sizeof(float);
@@ -82,15 +82,15 @@ TensorRef tensor_ref(Ctx* c, int which) {
     case DSLIDE_T_W1: return {c->W1, D * H * f};
     case DSLIDE_T_B1: return {c->b1, H * f};
     case DSLIDE_T_W2: return {c->W2, N * H * f};
-    case DSLIDE_T_B2: return {c->b2, N * f};
+    case DSLIDE_T_B2: return {&c->hdr2->b, N * f, (int64_t)sizeof(RowHdr)};
     case DSLIDE_T_M_W1: return {c->mW1, D * H * f};
     case DSLIDE_T_V_W1: return {c->vW1, D * H * f};
     case DSLIDE_T_M_B1: return {c->mb1, H * f};
     case DSLIDE_T_V_B1: return {c->vb1, H * f};
     case DSLIDE_T_M_W2: return {c->mW2, N * H * f};
     case DSLIDE_T_V_W2: return {c->vW2, N * H * f};
-    case DSLIDE_T_M_B2: return {c->mb2, N * f};
-    case DSLIDE_T_V_B2: return {c->vb2, N * f};
+    case DSLIDE_T_M_B2: return {&c->hdr2->mb, N * f, (int64_t)sizeof(RowHdr)};
+    case DSLIDE_T_V_B2: return {&c->hdr2->vb, N * f, (int64_t)sizeof(RowHdr)};
     case DSLIDE_T_HASH_IDX: return {c->hash_idx, (int64_t)c->KL * c->fn_len * 4};
     case DSLIDE_T_HASH_SIGN: return {c->hash_sign, c->cfg.hash_family == DSLIDE_SIMHASH ? (int64_t)c->KL * c->fn_len * 4 : 0};
     case DSLIDE_T_BUCKET_OFF: return {c->bucket_off, (int64_t)c->L * (c->nb + 1) * 4};
@@ -200,16 +200,16 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(W1, D * H, false); A(mW1, D * H, true); A(vW1, D * H, true);
   A(b1, H, true); A(mb1, H, true); A(vb1, H, true);
   A(W2, N * H, false); A(mW2, N * H, true); A(vW2, N * H, true);
-  A(b2, N, true); A(mb2, N, true); A(vb2, N, true);
+  A(hdr2, N, true);
   A(hash_idx, (size_t)c->KL * fn_len, true); A(hash_sign, (size_t)c->KL * fn_len, true);
   A(h, B * H, true); A(dh, B * H, true); A(loss, B, true); A(codes, B * c->L, true);
   A(act_cnt, B, true); A(act_z, B * S, true); A(act_p, B * S, true); A(act_g, B * S, true);
-  A(cnt1, D, true); A(mask1, D * c->Wd, true); A(slots1, D * ROW_SLOTS, true); A(own1, D, true);
+  A(hdr1, D, true); A(mask1, D * c->Wd, true); A(own1, D, true);
   A(hot_rows, HOT_CAP, true); A(med_rows, MED_CAP, true); A(hot_done, HOT_CAP, true); A(hot_part, (size_t)HOT_CAP * HOT_SLICES * (H + 4), true);
   A(dstate, 1, true);
   if (!c->dense) {
     A(act_ids, B * S, true);
-    A(cnt2, N, true); A(mask2, N * c->Wd, true); A(slots2, N * ROW_SLOTS, true);
+    A(mask2, N * c->Wd, true);
     A(own2, N, true);
     A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
     A(keysA, (size_t)c->L * N, false);
@@ -369,7 +369,10 @@ dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, 
     return DSLIDE_OK;
   }
   if (want == 0) return DSLIDE_OK;
-  CU(cudaMemcpyAsync(host_dst, tensor_ref(c, which).ptr, (size_t)want, cudaMemcpyDeviceToHost, c->stream));
+  const TensorRef tr = tensor_ref(c, which);
+  if (tr.pitch) CU(cudaMemcpy2DAsync(host_dst, sizeof(float), tr.ptr, (size_t)tr.pitch, sizeof(float), (size_t)want / sizeof(float),
+                                     cudaMemcpyDeviceToHost, c->stream));
+  else CU(cudaMemcpyAsync(host_dst, tr.ptr, (size_t)want, cudaMemcpyDeviceToHost, c->stream));
   return drain(c);
 }
 
@@ -400,7 +403,10 @@ dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host
   }
   if (which == DSLIDE_T_BUCKET_OFF || which == DSLIDE_T_BUCKET_IDS) return DSLIDE_ERR_INVALID_ARG;  // derived state
   if (want == 0) return DSLIDE_OK;
-  CU(cudaMemcpyAsync(tensor_ref(c, which).ptr, host_src, (size_t)want, cudaMemcpyHostToDevice, c->stream));
+  const TensorRef tr = tensor_ref(c, which);
+  if (tr.pitch) CU(cudaMemcpy2DAsync(tr.ptr, (size_t)tr.pitch, host_src, sizeof(float), sizeof(float), (size_t)want / sizeof(float),
+                                     cudaMemcpyHostToDevice, c->stream));
+  else CU(cudaMemcpyAsync(tr.ptr, host_src, (size_t)want, cudaMemcpyHostToDevice, c->stream));
   return drain(c);
 }
 

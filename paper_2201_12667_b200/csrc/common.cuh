@@ -44,7 +44,7 @@ struct DevState {
 
 // Touches of a row of W1 / W2 whose (sample, coefficient) pair is stored with the row; further touches of the
 // same step only set the sample's bit in the row's mask.
-constexpr int ROW_SLOTS = 8;
+constexpr int ROW_SLOTS = 6;
 // A row touched by more than HOT_T samples of a step is listed by the forward kernel (top bit of its
 // count set) and summed in HOT_SLICES slices by different warps; at most HOT_CAP rows are listed, further
 // ones are summed by a single warp.
@@ -56,6 +56,17 @@ constexpr int HOT_CAP = 1024;
 // CNT_HOT = the row is on the medium / hot list.
 constexpr int MED_CAP = 65536;
 constexpr unsigned CNT_HOT = 0x80000000u, CNT_MED = 0x40000000u, CNT_MASK = 0x3fffffffu;
+
+// Per-row record next to a row of W1 / W2, one 64-byte line: the number of samples of the step in flight that
+// touch the row (plus the CNT_* list marks), the row's bias with its Adam moments (rows of W2 only) and the
+// (sample, coefficient bits) pairs of the row's first ROW_SLOTS touches.  The update kernel fetches it together
+// with the row.
+struct __align__(16) RowHdr {
+  uint32_t cnt;
+  float b, mb, vb;
+  int2 slot[ROW_SLOTS];
+};
+static_assert(sizeof(RowHdr) == 64, "the row record is one 64-byte line");
 
 struct Ctx;
 
@@ -95,8 +106,9 @@ struct Ctx {
   int dense;
   cudaStream_t stream;
 
-  float *W1, *b1, *W2, *b2;
-  float *mW1, *vW1, *mb1, *vb1, *mW2, *vW2, *mb2, *vb2;
+  float *W1, *b1, *W2;
+  float *mW1, *vW1, *mb1, *vb1, *mW2, *vW2;
+  RowHdr *hdr1, *hdr2;             // per row of W1 / W2: touch count, slots and (W2) the bias b2 with its moments
   int32_t *hash_idx, *hash_sign;
   int32_t *bucket_off, *bucket_ids;
 
@@ -106,8 +118,6 @@ struct Ctx {
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;         // per row of W1 / W2: which samples of the batch touch it
-  uint32_t *cnt1, *cnt2;           // per row: samples of the step in flight that touch it
-  int2 *slots1, *slots2;           // per row: (sample, coefficient bits) of its first ROW_SLOTS touches
   int32_t *own1, *own2;            // the distinct touched rows of W1 / W2, in no particular order
   int32_t* hot_rows;               // rows touched by many samples: row of W2, or ~row of W1
   int32_t* med_rows;               // rows touched by more than ROW_SLOTS samples, same encoding

@@ -28,7 +28,7 @@ constexpr int SORT_SMALL = 1024;  // candidate sets up to this size are sorted r
 constexpr unsigned FULLM = 0xffffffffu;
 
 struct FwdParams {
-  const float *W1, *b1, *W2, *b2;
+  const float *W1, *b1, *W2;
   const int32_t *hash_idx, *hash_sign, *bucket_off, *bucket_ids;
   const int32_t *row_ptr, *col_idx;
   const float* vals;
@@ -37,8 +37,8 @@ struct FwdParams {
   uint32_t* codes;
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
-  uint32_t *mask1, *mask2, *cnt1, *cnt2;
-  int2 *slots1, *slots2;
+  uint32_t *mask1, *mask2;
+  RowHdr *hdr1, *hdr2;
   int32_t *own1, *own2, *hot_rows, *med_rows;
   DevState* st;
   int32_t* out_ids;
@@ -450,11 +450,12 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       int c = 0;
       if (i < nnz) {
         c = __ldg(p.col_idx + rbeg + i);
-        const unsigned nth = atomicAdd(p.cnt1 + c, 1u) & CNT_MASK;
-        if (nth < (unsigned)ROW_SLOTS) p.slots1[(size_t)c * ROW_SLOTS + nth] = make_int2(s, __float_as_int(__ldg(p.vals + rbeg + i)));
+        RowHdr* hd = p.hdr1 + c;
+        const unsigned nth = atomicAdd(&hd->cnt, 1u) & CNT_MASK;
+        if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(__ldg(p.vals + rbeg + i)));
         else atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
         first = nth == 0u;
-        list_row(p, p.cnt1 + c, ~c, nth);
+        list_row(p, &hd->cnt, ~c, nth);
       }
       const unsigned fm = __ballot_sync(FULLM, first);
       if (fm) {
@@ -490,7 +491,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
     // the biases of a small active set are fetched in the same round, into the logits' place
     if (small && c0 == 0)
-      for (int a = tid; a < na; a += FWD_THREADS) sh_z[a] = __ldg(p.b2 + sh_ids[a]);
+      for (int a = tid; a < na; a += FWD_THREADS) sh_z[a] = __ldg(&p.hdr2[sh_ids[a]].b);
     if (!mbar_wait(sh_bar, phase)) timed_out = true;
     phase ^= 1u;
     if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
@@ -520,14 +521,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
             z[c0 + a] = zv;
           } else {
             const int j = dense ? c0 + a : idp[c0 + a];
-            z[c0 + a] = __ldg(p.b2 + j) + dot;
+            z[c0 + a] = __ldg(&p.hdr2[j].b) + dot;
           }
         }
       } else {
         // predict: lane 0 of each warp keeps the warp's best k so far, fed one lane's logit at a time
         int j = -1;
         float zv = 0.f;
-        if (live) { j = dense ? c0 + a : idp[c0 + a]; zv = __ldg(p.b2 + j) + dot; }
+        if (live) { j = dense ? c0 + a : idp[c0 + a]; zv = __ldg(&p.hdr2[j].b) + dot; }
         float* lz = tk_z + warp * p.topk;
         int* li = tk_id + warp * p.topk;
         for (int l = 0; l < 32; ++l) {
@@ -637,11 +638,12 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       if (a < na) {
         jj = idp[a];
         const float ga = gp[a];
-        const unsigned nth = atomicAdd(p.cnt2 + jj, 1u) & CNT_MASK;
-        if (nth < (unsigned)ROW_SLOTS) p.slots2[(size_t)jj * ROW_SLOTS + nth] = make_int2(s, __float_as_int(ga));
+        RowHdr* hd = p.hdr2 + jj;
+        const unsigned nth = atomicAdd(&hd->cnt, 1u) & CNT_MASK;
+        if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(ga));
         else atomicOr(p.mask2 + (size_t)jj * p.Wd + sword, sbit);
         first = nth == 0u;
-        list_row(p, p.cnt2 + jj, jj, nth);
+        list_row(p, &hd->cnt, jj, nth);
       }
       const unsigned fm = __ballot_sync(FULLM, first);
       if (fm) {
@@ -793,13 +795,12 @@ cudaError_t setup_forward(Ctx* c) {
 static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
                              const int32_t* label_ptr, const int32_t* labels) {
   FwdParams p;
-  p.W1 = c->W1; p.b1 = c->b1; p.W2 = c->W2; p.b2 = c->b2;
+  p.W1 = c->W1; p.b1 = c->b1; p.W2 = c->W2;
   p.hash_idx = c->hash_idx; p.hash_sign = c->hash_sign; p.bucket_off = c->bucket_off; p.bucket_ids = c->bucket_ids;
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals; p.label_ptr = label_ptr; p.labels = labels;
   p.h = c->h; p.dh = c->dh; p.loss = c->loss; p.codes = c->codes;
   p.act_cnt = c->act_cnt; p.act_ids = c->act_ids; p.act_z = c->act_z; p.act_p = c->act_p; p.act_g = c->act_g;
-  p.mask1 = c->mask1; p.mask2 = c->mask2; p.cnt1 = c->cnt1; p.cnt2 = c->cnt2;
-  p.slots1 = c->slots1; p.slots2 = c->slots2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
   p.own1 = c->own1; p.own2 = c->own2; p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.parity = (int)(c->t_host & 1);
   p.st = c->dstate; p.out_ids = nullptr; p.out_scores = nullptr;
   p.nb = c->nb;

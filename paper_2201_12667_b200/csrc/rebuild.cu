@@ -96,90 +96,154 @@ cudaError_t launch_draw_hash(Ctx* c, int64_t r) {
 // ------------------------------------------------------------------ codes of all neurons
 constexpr int HN_ROWS = 32;
 constexpr int HN_THREADS = 256;
+constexpr int HN_WARPS = HN_THREADS / 32;
+constexpr int HN_FN_SMEM_MAX = 96 * 1024;    // hash-function tables larger than this stay in global memory
 
 // A block stages HN_ROWS rows of W2 in shared memory (padded, so that 32 threads reading the same
-// column of 32 different rows hit 32 banks) and evaluates the L codes of each row.
+// column of 32 different rows hit 32 banks) and evaluates the L codes of each row: lane = row, the
+// warps share out the tables.  The hash functions sit in shared memory too, 16 bits per coordinate
+// (the top bit carries a negative SimHash sign), read as warp-wide broadcasts.
 // keys[t][j] = code of neuron j in table t; counts[t][code + 1] += 1.
+template <bool FN_SMEM>
 __global__ void __launch_bounds__(HN_THREADS)
 k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, const int32_t* __restrict__ hsign,
                uint32_t* keys, int32_t* counts, int N, int H, int K, int L, int family, int lg_bin, int fn_len,
                long long nb) {
-  extern __shared__ float tile[];              // [HN_ROWS][H + 1]
+  extern __shared__ __align__(16) unsigned char hn_smem[];
+  float* tile = reinterpret_cast<float*>(hn_smem);                    // [HN_ROWS][H + 1]
   const int ld = H + 1;
+  unsigned short* fn = reinterpret_cast<unsigned short*>(hn_smem + (((size_t)HN_ROWS * ld * 4 + 15) & ~(size_t)15));
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nfn = K * L * fn_len;
+  if (FN_SMEM) {
+    for (int e = threadIdx.x; e < nfn; e += HN_THREADS) {
+      unsigned v = (unsigned)hidx[e];
+      if (family == DSLIDE_SIMHASH && hsign[e] < 0) v |= 0x8000u;
+      fn[e] = (unsigned short)v;
+    }
+  }
   const int ntiles = (N + HN_ROWS - 1) / HN_ROWS;
   for (int tl = blockIdx.x; tl < ntiles; tl += gridDim.x) {
     const int j0 = tl * HN_ROWS;
     const int rows = min(HN_ROWS, N - j0);
     __syncthreads();
-    for (int e = threadIdx.x; e < rows * H; e += HN_THREADS) {
-      int r = e / H, k = e - r * H;
-      tile[r * ld + k] = W2[(size_t)(j0 + r) * H + k];
+    {
+      const int H4 = H >> 2, total4 = rows * H4;
+      const float4* src = reinterpret_cast<const float4*>(W2 + (size_t)j0 * H);
+      for (int e = threadIdx.x; e < total4; e += HN_THREADS) {
+        const float4 x = __ldg(src + e);
+        const int r = e / H4, k = (e - r * H4) << 2;
+        float* d = tile + r * ld + k;
+        d[0] = x.x; d[1] = x.y; d[2] = x.z; d[3] = x.w;
+      }
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < HN_ROWS * L; e += HN_THREADS) {
-      const int r = e & (HN_ROWS - 1), t = e / HN_ROWS;
-      if (r >= rows) continue;
-      const float* v = tile + r * ld;
-      uint32_t code = 0;
-      for (int k = 0; k < K; ++k) {
-        const int f = t * K + k;
-        const int32_t* ix = hidx + (size_t)f * fn_len;
-        if (family == DSLIDE_SIMHASH) {
-          const int32_t* sg = hsign + (size_t)f * fn_len;
-          float sum = 0.f;
-          for (int i = 0; i < fn_len; ++i) {
-            float x = v[__ldg(ix + i)];
-            sum = __fadd_rn(sum, __ldg(sg + i) > 0 ? x : -x);
+    if (lane < rows) {
+      const float* v = tile + lane * ld;
+      for (int t = warp; t < L; t += HN_WARPS) {
+        uint32_t code = 0;
+        for (int k = 0; k < K; ++k) {
+          const int f = t * K + k;
+          if (family == DSLIDE_SIMHASH) {
+            float sum = 0.f;
+            if (FN_SMEM) {
+              const unsigned short* ix = fn + (size_t)f * fn_len;
+              for (int i = 0; i < fn_len; ++i) {
+                const unsigned e = ix[i];
+                const float x = v[e & 0x7fffu];
+                sum = __fadd_rn(sum, (e & 0x8000u) ? -x : x);
+              }
+            } else {
+              const int32_t* ix = hidx + (size_t)f * fn_len;
+              const int32_t* sg = hsign + (size_t)f * fn_len;
+              for (int i = 0; i < fn_len; ++i) {
+                const float x = v[__ldg(ix + i)];
+                sum = __fadd_rn(sum, __ldg(sg + i) > 0 ? x : -x);
+              }
+            }
+            code |= (sum >= 0.f ? 1u : 0u) << k;
+          } else {
+            int best = 0;
+            float bv;
+            if (FN_SMEM) {
+              const unsigned short* ix = fn + (size_t)f * fn_len;
+              bv = v[ix[0]];
+              for (int i = 1; i < fn_len; ++i) {
+                const float x = v[ix[i]];
+                if (x > bv) { bv = x; best = i; }
+              }
+            } else {
+              const int32_t* ix = hidx + (size_t)f * fn_len;
+              bv = v[__ldg(ix)];
+              for (int i = 1; i < fn_len; ++i) {
+                const float x = v[__ldg(ix + i)];
+                if (x > bv) { bv = x; best = i; }
+              }
+            }
+            code |= (uint32_t)best << (k * lg_bin);
           }
-          code |= (sum >= 0.f ? 1u : 0u) << k;
-        } else {
-          int best = 0;
-          float bv = v[__ldg(ix)];
-          for (int i = 1; i < fn_len; ++i) {
-            float x = v[__ldg(ix + i)];
-            if (x > bv) { bv = x; best = i; }
-          }
-          code |= (uint32_t)best << (k * lg_bin);
         }
+        keys[(size_t)t * N + j0 + lane] = code;
+        atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code + 1, 1);
       }
-      keys[(size_t)t * N + j0 + r] = code;
-      atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code + 1, 1);
     }
   }
 }
 
 // counts[t][0] = 0, counts[t][c + 1] = size of bucket c  ->  inclusive running sum = bucket offsets.
+// One block per table walks the table's counters 4096 at a time (coalesced), carrying the running sum.
 __global__ void __launch_bounds__(1024) k_bucket_scan(int32_t* off, long long nb) {
   __shared__ int sh[33];
+  __shared__ int carry;
   int32_t* o = off + (size_t)blockIdx.x * (size_t)(nb + 1);
   const long long n = nb + 1;
-  const long long chunk = (n + 1023) / 1024;
-  const long long beg = min(n, (long long)threadIdx.x * chunk), end = min(n, beg + chunk);
-  int sum = 0;
-  for (long long i = beg; i < end; ++i) sum += o[i];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = sum;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (long long base = 0; base < n; base += 4096) {
+    const long long i0 = base + (long long)threadIdx.x * 4;
+    int v[4];
 #pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    int v = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += v;
+    for (int u = 0; u < 4; ++u) v[u] = i0 + u < n ? o[i0 + u] : 0;
+    const int sum = v[0] + v[1] + v[2] + v[3];
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int x = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += x;
+    }
+    if (lane == 31) sh[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = sh[lane];
+      int wi = w;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int x = __shfl_up_sync(0xffffffffu, wi, d);
+        if (lane >= d) wi += x;
+      }
+      sh[lane] = wi - w;                 // exclusive over the warps
+      if (lane == 31) sh[32] = wi;       // total of this round
+    }
+    __syncthreads();
+    int run = carry + sh[warp] + incl - sum;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      run += v[u];
+      if (i0 + u < n) o[i0 + u] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) carry += sh[32];
+    __syncthreads();
   }
-  if (lane == 31) sh[warp] = incl;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int run = 0;
-    for (int w = 0; w < 32; ++w) { int c = sh[w]; sh[w] = run; run += c; }
-  }
-  __syncthreads();
-  int run = incl - sum + sh[warp];
-  for (long long i = beg; i < end; ++i) { run += o[i]; o[i] = run; }
 }
 
 // ------------------------------------------------------------------ stable LSD radix sort, per table
-constexpr int SORT_THREADS = 256;
+constexpr int SORT_THREADS = 512;
 constexpr int SORT_WARPS = SORT_THREADS / 32;
 constexpr int SORT_TILE = 8192;                      // elements per block
 constexpr int SORT_SUB = SORT_TILE / SORT_WARPS;     // contiguous elements per warp
+constexpr int SORT_ITERS = SORT_SUB / 32;            // groups of 32 keys a warp walks, all fetched up front
 constexpr int SORT_MAX_WIDTH = 9;                    // bits per pass
 
 // hist[t][digit][tile] = number of keys of that digit in the tile.
@@ -224,9 +288,10 @@ __global__ void __launch_bounds__(1024) k_sort_scan(int32_t* hist, int n) {
 
 // Each warp owns a contiguous part of the tile and walks it in order, 32 keys at a time; equal
 // digits inside a group of 32 are ranked by lane with a match mask, so the scatter is stable.
+// All of a warp's keys (and values) are fetched before the walk, which then runs out of registers.
 // vals_in == nullptr means the value of element i is i (first pass).  keys_out may be nullptr
 // (last pass).
-__global__ void __launch_bounds__(SORT_THREADS)
+__global__ void __launch_bounds__(SORT_THREADS, 2)
 k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_out, int32_t* vals_out,
                const int32_t* hist, int N, int tiles, int shift, int width) {
   __shared__ int offs[SORT_WARPS][1 << SORT_MAX_WIDTH];
@@ -238,20 +303,29 @@ k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_o
   int32_t* vout = vals_out + (size_t)t * N;
   const int wbeg = min(N, tl * SORT_TILE + warp * SORT_SUB), wend = min(N, wbeg + SORT_SUB);
 
+  uint32_t key[SORT_ITERS];
+  int32_t val[SORT_ITERS];
+#pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it) {
+    const int i = wbeg + it * 32 + lane;
+    key[it] = i < wend ? kin[i] : 0u;
+    val[it] = i < wend ? (vin ? vin[i] : i) : 0;
+  }
   for (int d = lane; d < radix; d += 32) offs[warp][d] = 0;
   __syncwarp();
-  for (int i = wbeg + lane; i < wend; i += 32) atomicAdd(&offs[warp][(kin[i] >> shift) & (radix - 1)], 1);
+#pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it)
+    if (wbeg + it * 32 + lane < wend) atomicAdd(&offs[warp][(key[it] >> shift) & (radix - 1)], 1);
   __syncthreads();
   for (int d = threadIdx.x; d < radix; d += SORT_THREADS) {
     int run = hist[((size_t)t * radix + d) * tiles + tl];
     for (int w = 0; w < SORT_WARPS; ++w) { int c = offs[w][d]; offs[w][d] = run; run += c; }
   }
   __syncthreads();
-  for (int i0 = wbeg; i0 < wend; i0 += 32) {
-    const int i = i0 + lane;
-    const bool live = i < wend;
-    const uint32_t key = live ? kin[i] : 0u;
-    const int digit = live ? (int)((key >> shift) & (radix - 1)) : radix + lane;   // dead lanes match nobody
+#pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it) {
+    const bool live = wbeg + it * 32 + lane < wend;
+    const int digit = live ? (int)((key[it] >> shift) & (radix - 1)) : radix + lane;   // dead lanes match nobody
     const unsigned peers = __match_any_sync(0xffffffffu, digit);
     const int rank = __popc(peers & ((1u << lane) - 1u));
     int base = 0;
@@ -261,8 +335,8 @@ k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_o
     __syncwarp();
     if (live) {
       const int dst = base + rank;
-      if (kout) kout[dst] = key;
-      vout[dst] = vin ? vin[i] : i;
+      if (kout) kout[dst] = key[it];
+      vout[dst] = val[it];
     }
   }
 }
@@ -271,16 +345,24 @@ cudaError_t launch_build_tables(Ctx* c) {
   const size_t off_bytes = (size_t)c->L * (size_t)(c->nb + 1) * sizeof(int32_t);
   cudaError_t e = cudaMemsetAsync(c->bucket_off, 0, off_bytes, c->stream);
   if (e != cudaSuccess) return e;
-  const int smem = HN_ROWS * (c->H + 1) * (int)sizeof(float);
+  const int tile_bytes = (HN_ROWS * (c->H + 1) * (int)sizeof(float) + 15) & ~15;
+  const long long fn_bytes = (long long)c->KL * c->fn_len * 2;
+  const bool fn_smem = fn_bytes <= HN_FN_SMEM_MAX && c->H <= 0x7fff;
+  const int smem = tile_bytes + (fn_smem ? (int)fn_bytes : 0);
+  auto kern = fn_smem ? k_hash_neurons<true> : k_hash_neurons<false>;
   if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(k_hash_neurons, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
   {
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, HN_THREADS, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
     LaunchScope ls(c, KID_HASH_NEURONS);
-    k_hash_neurons<<<c->num_sms * 4, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
-                                                                   c->bucket_off, c->N, c->H, c->K, c->L,
-                                                                   c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
+    kern<<<c->num_sms * per_sm, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
+                                                             c->bucket_off, c->N, c->H, c->K, c->L,
+                                                             c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   {

@@ -2,10 +2,11 @@
 // momentum and a velocity array per weight and bias array; Section 2.1: gradients reach the
 // active neurons only).
 //
-// The forward kernel leaves, per step and per touched row of W2 / W1: the number of samples that
-// touch the row, the (sample, coefficient) pairs of its first ROW_SLOTS touches, a bit mask of the
-// samples of any further touches -- and two lists of the distinct touched rows (the sample that
-// touched a row first entered it).
+// The forward kernel leaves, per step and per touched row of W2 / W1: in the row's 64-byte record the
+// number of samples that touch the row and the (sample, coefficient) pairs of its first ROW_SLOTS
+// touches (the record also holds the bias of a row of W2 with its moments, so one line brings all of
+// it), a bit mask of the samples of any further touches -- and two lists of the distinct touched rows
+// (the sample that touched a row first entered it).
 //
 //   k_update : a warp works on a few rows of the two row lists at a time, so that the loads of a
 //              row's weights and moments, its touch count and its slots are all issued together.  A row touched by one sample takes its gradient from slot 0;
@@ -34,13 +35,13 @@ constexpr unsigned FULL = 0xffffffffu;
 
 struct UpdParams {
   float *W1, *mW1, *vW1, *b1, *mb1, *vb1;
-  float *W2, *mW2, *vW2, *b2, *mb2, *vb2;
+  float *W2, *mW2, *vW2;
   const float *h, *dh, *act_g, *loss;
   const int32_t *act_cnt, *act_ids;
   const int32_t *row_ptr, *col_idx;
   const float* vals;
-  uint32_t *mask1, *mask2, *cnt1, *cnt2;
-  const int2 *slots1, *slots2;
+  uint32_t *mask1, *mask2;
+  RowHdr *hdr1, *hdr2;
   const int32_t *own1, *own2, *hot_rows, *med_rows;
   float* hot_part;
   int* hot_done;
@@ -67,22 +68,22 @@ __device__ __forceinline__ void axpy4(float4& a, float g, const float4 x) {
 }
 
 // The pieces of one layer's update: the weight / moment arrays, the rows that multiply the
-// coefficients (h for W2, dh for W1), the per-row masks and the bias arrays (W2 only).
+// coefficients (h for W2, dh for W1), the per-row masks and the per-row records (touch count, slots and,
+// for W2, the bias with its moments).
 struct Side {
-  float *W, *M, *V, *bw, *bm, *bv;
+  float *W, *M, *V;
   const float* src;
   uint32_t* mask;
-  const int2* slots;
+  RowHdr* hdr;
   int is_w2;
 };
 
 __device__ __forceinline__ Side make_side(const UpdParams& p, bool w2) {
   Side sd;
   sd.W = w2 ? p.W2 : p.W1; sd.M = w2 ? p.mW2 : p.mW1; sd.V = w2 ? p.vW2 : p.vW1;
-  sd.bw = p.b2; sd.bm = p.mb2; sd.bv = p.vb2;
   sd.src = w2 ? p.h : p.dh;
   sd.mask = w2 ? p.mask2 : p.mask1;
-  sd.slots = w2 ? p.slots2 : p.slots1;
+  sd.hdr = w2 ? p.hdr2 : p.hdr1;
   sd.is_w2 = w2 ? 1 : 0;
   return sd;
 }
@@ -263,10 +264,30 @@ __device__ __forceinline__ void adam_store(const UpdParams& p, const Side& sd, s
   }
 }
 
-__device__ __forceinline__ void adam_bias(const UpdParams& p, const Side& sd, int row, float g) {
-  float w = sd.bw[row], m = sd.bm[row], v = sd.bv[row];
-  adam1(w, m, v, g, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
-  sd.bw[row] = w; sd.bm[row] = m; sd.bv[row] = v;
+// A row record as a warp holds it: lane l < 8 has the l-th 8-byte piece -- lane 0 (count, bias), lane 1 (the
+// bias moments), lanes 2.. the slots.
+__device__ __forceinline__ int2 load_hdr(const RowHdr* hd, int lane) {
+  int2 v = make_int2(0, 0);
+  if (lane < 8) v = reinterpret_cast<const int2*>(hd)[lane];
+  return v;
+}
+// Slot k of the record in lane k (k < ROW_SLOTS).
+__device__ __forceinline__ int2 hdr_slots(int2 hv) {
+  return make_int2(__shfl_down_sync(FULL, hv.x, 2), __shfl_down_sync(FULL, hv.y, 2));
+}
+// Closes a row: Adam on the bias of a row of W2 with the gradient g, and the touch count back to zero for the
+// next step.  Called by the whole warp.
+__device__ __forceinline__ void finish_hdr(const UpdParams& p, RowHdr* hd, bool w2, int2 hv, float g, int lane) {
+  if (w2) {
+    float b = __int_as_float(__shfl_sync(FULL, hv.y, 0));
+    float mb = __int_as_float(__shfl_sync(FULL, hv.x, 1));
+    float vb = __int_as_float(__shfl_sync(FULL, hv.y, 1));
+    adam1(b, mb, vb, g, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+    if (lane == 0) reinterpret_cast<int2*>(hd)[0] = make_int2(0, __float_as_int(b));
+    if (lane == 1) reinterpret_cast<int2*>(hd)[1] = make_int2(__float_as_int(mb), __float_as_int(vb));
+  } else if (lane == 0) {
+    hd->cnt = 0u;
+  }
 }
 
 // The hidden bias (dense gradient, summed over the samples in eight fixed slices) and, in the first
@@ -341,9 +362,8 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* sm_rowpt
 #pragma unroll
   for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   float csum = 0.f;
-  int slot_s = 0x7fffffff;
-  if (lane < ROW_SLOTS) slot_s = sd.slots[(size_t)row * ROW_SLOTS + lane].x;
-  sum_masked<NCH>(p, sd, sm_rowptr, row, slot_s, w0, w1, scr, acc, csum, H, H4, lane);
+  const int2 hv = load_hdr(sd.hdr + row, lane);
+  sum_masked<NCH>(p, sd, sm_rowptr, row, hdr_slots(hv).x, w0, w1, scr, acc, csum, H, H4, lane);
   const int ld = H + 4;
   float* part = p.hot_part + (size_t)hrow * HOT_SLICES * ld;
   float4* mine = reinterpret_cast<float4*>(part + (size_t)slice * ld);
@@ -380,11 +400,8 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* sm_rowpt
     csum += __ldcg(part + (size_t)sl * ld + H);
   }
   adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
-  if (lane == 0) {
-    if (w2) adam_bias(p, sd, row, csum);
-    p.hot_done[hrow] = 0;
-    (w2 ? p.cnt2 : p.cnt1)[row] = 0u;
-  }
+  finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
+  if (lane == 0) p.hot_done[hrow] = 0;
 }
 
 // A row touched by more than ROW_SLOTS samples that the forward kernel listed: one warp sums it from slots and
@@ -397,13 +414,10 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_ro
   const bool w2 = code >= 0;
   const int row = w2 ? code : ~code;
   const Side sd = make_side(p, w2);
-  uint32_t* cnt = (w2 ? p.cnt2 : p.cnt1) + row;
-  unsigned cv = 0u;
-  if (lane == 0) cv = *cnt;
-  cv = __shfl_sync(FULL, cv, 0);
+  const int2 hv = load_hdr(sd.hdr + row, lane);
+  const unsigned cv = (unsigned)__shfl_sync(FULL, hv.x, 0);
   if ((cv & CNT_HOT) || (cv & CNT_MASK) == 0u) return;
-  int slot_s = 0x7fffffff;
-  if (lane < ROW_SLOTS) slot_s = sd.slots[(size_t)row * ROW_SLOTS + lane].x;
+  const int slot_s = hdr_slots(hv).x;
   float4 w[NCH], m[NCH], v[NCH], acc[NCH];
   load_row<NCH>(sd.W, (size_t)row, H, H4, lane, w);
   load_row<NCH>(sd.M, (size_t)row, H, H4, lane, m);
@@ -413,10 +427,7 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_ro
   float csum = 0.f;
   sum_masked<NCH>(p, sd, sm_rowptr, row, slot_s, 0, nwB, scr, acc, csum, H, H4, lane);
   adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
-  if (lane == 0) {
-    if (w2) adam_bias(p, sd, row, csum);
-    *cnt = 0u;
-  }
+  finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
 }
 
 // Work is handed out in tickets from one counter: first the slices of the hot rows (the longest items), then
@@ -424,7 +435,7 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_ro
 constexpr int UPD_TROWS = 8;
 
 template <int NCH, int G>
-__global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
+__global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 3 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
   extern __shared__ __align__(16) unsigned char upd_smem[];
   int* sm_rowptr = reinterpret_cast<int*>(upd_smem);                               // [B + 1]
   float* sm_part = reinterpret_cast<float*>(upd_smem + (((size_t)p.B + 1 + 3) & ~(size_t)3) * 4);   // [UPD_WARPS * 32]
@@ -449,12 +460,18 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1
   const int n_tickets = n_hot_items + n_med + n_norm;
   unsigned int* ticket = &p.st->ticket[p.parity];
 
+  // every warp's first ticket is its own number; further tickets come from the counter (one is always on its way
+  // while the current one is worked on)
+  const int nwork = (int)gridDim.x - naux;
+  const int nwarps = nwork * UPD_WARPS;
+  int cur = warp * nwork + ((int)blockIdx.x - naux);
   int nxt = 0;
-  if (lane == 0) nxt = (int)atomicAdd(ticket, 1u);
-  for (;;) {
-    const int t = __shfl_sync(FULL, nxt, 0);
+  if (lane == 0) nxt = nwarps + (int)atomicAdd(ticket, 1u);
+  for (;; ) {
+    const int t = cur;
     if (t >= n_tickets) break;
-    if (lane == 0) nxt = (int)atomicAdd(ticket, 1u);          // the next ticket is on its way while this one is worked on
+    cur = __shfl_sync(FULL, nxt, 0);
+    if (lane == 0 && cur < n_tickets) nxt = nwarps + (int)atomicAdd(ticket, 1u);
     if (t < n_hot_items) { hot_item<NCH>(p, sm_rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
     if (t < n_hot_items + n_med) { medium_item<NCH>(p, sm_rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
 
@@ -469,7 +486,7 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1
     for (int b0 = 0; b0 < UPD_TROWS; b0 += G) {
       int rr[G], tt[G];
       bool live[G], w2[G], skip[G];
-      int2 sl[G];
+      int2 hv[G], sl[G];
       float4 w[G][NCH], m[G][NCH], v[G][NCH], x[G][NCH];
 #pragma unroll
       for (int q = 0; q < G; ++q) {
@@ -478,26 +495,25 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1
         w2[q] = idx < n2;
         rr[q] = __shfl_sync(FULL, myrow, b0 + q);
         tt[q] = 0;
-        sl[q] = make_int2(0x7fffffff, 0);
+        hv[q] = make_int2(0, 0);
         if (live[q]) {
           const Side sd = make_side(p, w2[q]);
-          if (lane == 0) tt[q] = (int)(w2[q] ? p.cnt2 : p.cnt1)[rr[q]];     // read and reset by lane 0 only
-          if (lane < ROW_SLOTS) sl[q] = sd.slots[(size_t)rr[q] * ROW_SLOTS + lane];
+          hv[q] = load_hdr(sd.hdr + rr[q], lane);
           load_row<NCH>(sd.W, (size_t)rr[q], H, H4, lane, w[q]);
           load_row<NCH>(sd.M, (size_t)rr[q], H, H4, lane, m[q]);
           load_row<NCH>(sd.V, (size_t)rr[q], H, H4, lane, v[q]);
         }
       }
-      // second level: the one sample's row for rows touched once; counts are reset for the next step
+      // second level: the one sample's row for rows touched once
 #pragma unroll
       for (int q = 0; q < G; ++q)
         if (live[q]) {
           const Side sd = make_side(p, w2[q]);
-          const unsigned cv = (unsigned)__shfl_sync(FULL, tt[q], 0);
+          const unsigned cv = (unsigned)__shfl_sync(FULL, hv[q].x, 0);
+          sl[q] = hdr_slots(hv[q]);
           // a listed row is summed by its own ticket (and its count may already be back at zero)
           skip[q] = (cv & (CNT_HOT | CNT_MED)) != 0u || (cv & CNT_MASK) == 0u;
           tt[q] = (int)(cv & CNT_MASK);
-          if (lane == 0 && !skip[q]) (w2[q] ? p.cnt2 : p.cnt1)[rr[q]] = 0u;
           const int s0 = __shfl_sync(FULL, sl[q].x, 0);
           if (tt[q] == 1 && !skip[q]) load_row<NCH>(sd.src, (size_t)s0, H, H4, lane, x[q]);
         }
@@ -520,7 +536,7 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 4 : (NCH == 2 ? 2 : 1
             sum_masked<NCH>(p, sd, sm_rowptr, rr[q], sl[q].x, 0, nwB, scratch[warp], acc, csum, H, H4, lane);
           }
           adam_store<NCH>(p, sd, (size_t)rr[q], w[q], m[q], v[q], acc, H, H4, lane);
-          if (w2[q] && lane == 0) adam_bias(p, sd, rr[q], csum);
+          finish_hdr(p, sd.hdr + rr[q], w2[q], hv[q], csum, lane);
         }
     }
   }
@@ -549,7 +565,7 @@ __global__ void __launch_bounds__(UPD_THREADS) k_adam_dense(const UpdParams p) {
     load_row<DENSE_CH>(sd.M, (size_t)j, H, H4, lane, m);
     load_row<DENSE_CH>(sd.V, (size_t)j, H, H4, lane, v);
     adam_store<DENSE_CH>(p, sd, (size_t)j, w, m, v, acc, H, H4, lane);
-    if (lane == 0) adam_bias(p, sd, j, csum);
+    finish_hdr(p, sd.hdr + j, true, load_hdr(sd.hdr + j, lane), csum, lane);
   }
 }
 
@@ -576,11 +592,11 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
                           float* loss_out) {
   UpdParams p;
   p.W1 = c->W1; p.mW1 = c->mW1; p.vW1 = c->vW1; p.b1 = c->b1; p.mb1 = c->mb1; p.vb1 = c->vb1;
-  p.W2 = c->W2; p.mW2 = c->mW2; p.vW2 = c->vW2; p.b2 = c->b2; p.mb2 = c->mb2; p.vb2 = c->vb2;
+  p.W2 = c->W2; p.mW2 = c->mW2; p.vW2 = c->vW2;
   p.h = c->h; p.dh = c->dh; p.act_g = c->act_g; p.loss = c->loss; p.act_cnt = c->act_cnt; p.act_ids = c->act_ids;
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals;
-  p.mask1 = c->mask1; p.mask2 = c->mask2; p.cnt1 = c->cnt1; p.cnt2 = c->cnt2;
-  p.slots1 = c->slots1; p.slots2 = c->slots2; p.own1 = c->own1; p.own2 = c->own2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
+  p.own1 = c->own1; p.own2 = c->own2;
   p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.hot_part = c->hot_part; p.hot_done = c->hot_done;
   p.st = c->dstate; p.loss_out = loss_out;
   p.B = batch; p.H = c->H; p.N = c->N; p.D = c->D; p.Wd = c->Wd; p.act_stride = c->act_stride; p.dense = c->dense;
