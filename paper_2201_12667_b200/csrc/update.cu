@@ -435,7 +435,7 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_ro
 constexpr int UPD_TROWS = 8;
 
 template <int NCH, int G>
-__global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 3 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
+__global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
   extern __shared__ __align__(16) unsigned char upd_smem[];
   int* sm_rowptr = reinterpret_cast<int*>(upd_smem);                               // [B + 1]
   float* sm_part = reinterpret_cast<float*>(upd_smem + (((size_t)p.B + 1 + 3) & ~(size_t)3) * 4);   // [UPD_WARPS * 32]
