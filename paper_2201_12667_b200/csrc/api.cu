@@ -12,6 +12,7 @@
 namespace dslide {
 int sort_tile_elems();
 int sort_max_width();
+int bucket_scan_chunk();
 }
 
 using namespace dslide;
@@ -56,7 +57,7 @@ void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->hdr1, c->hdr2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1,
-                  c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist,
+                  c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part,
                   c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (c->pinned_loss) cudaFreeHost(c->pinned_loss);
@@ -216,6 +217,7 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     if (c->sort_passes > 1) { A(keysB, (size_t)c->L * N, false); A(valsA, (size_t)c->L * N, false); }
     if (c->sort_passes > 2) { A(valsB, (size_t)c->L * N, false); }
     A(tile_hist, (size_t)c->L * ((size_t)1 << c->sort_width) * c->sort_tiles, false);
+    A(bucket_part, (size_t)c->L * (size_t)((c->nb + 1 + bucket_scan_chunk() - 1) / bucket_scan_chunk()), false);
   }
 #undef A
   if (e == cudaSuccess) e = cudaMallocHost((void**)&c->pinned_loss, sizeof(float));

@@ -129,6 +129,7 @@ struct Ctx {
   uint32_t *keysA, *keysB;
   int32_t *valsA, *valsB;
   int32_t* tile_hist;
+  int32_t* bucket_part;   // per table: sums of chunks of bucket counters (bucket offset scan)
   int sort_passes, sort_width, sort_tiles;
 
   // forward kernel layout

@@ -20,7 +20,6 @@ namespace dslide {
 
 constexpr int FWD_THREADS = 256;
 constexpr int FWD_WARPS = FWD_THREADS / 32;
-constexpr int MAX_HCHUNK = 8;     // float4 chunks per lane: H <= 4 * 32 * 8 = 1024
 constexpr int MAX_KPT = 4;        // hidden units per thread: H <= 4 * 256
 constexpr int ACT_SM = 1024;      // active ids and logits are mirrored in shared memory when the set is this small
 constexpr int HID_MIN_BYTES = 64 * 1024;   // staging space for the hidden layer's rows of W1

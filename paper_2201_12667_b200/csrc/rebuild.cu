@@ -142,6 +142,7 @@ k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, c
       const float* v = tile + lane * ld;
       for (int t = warp; t < L; t += HN_WARPS) {
         uint32_t code = 0;
+#pragma unroll 2
         for (int k = 0; k < K; ++k) {
           const int f = t * K + k;
           if (family == DSLIDE_SIMHASH) {
@@ -165,7 +166,20 @@ k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, c
           } else {
             int best = 0;
             float bv;
-            if (FN_SMEM) {
+            if (FN_SMEM && fn_len == 8) {
+              // bin of eight: the eight coordinates come in one 16-byte broadcast load
+              const uint4 q = *reinterpret_cast<const uint4*>(fn + (size_t)f * 8);
+              const float x0 = v[q.x & 0xffffu], x1 = v[q.x >> 16], x2 = v[q.y & 0xffffu], x3 = v[q.y >> 16];
+              const float x4 = v[q.z & 0xffffu], x5 = v[q.z >> 16], x6 = v[q.w & 0xffffu], x7 = v[q.w >> 16];
+              bv = x0;
+              if (x1 > bv) { bv = x1; best = 1; }
+              if (x2 > bv) { bv = x2; best = 2; }
+              if (x3 > bv) { bv = x3; best = 3; }
+              if (x4 > bv) { bv = x4; best = 4; }
+              if (x5 > bv) { bv = x5; best = 5; }
+              if (x6 > bv) { bv = x6; best = 6; }
+              if (x7 > bv) { bv = x7; best = 7; }
+            } else if (FN_SMEM) {
               const unsigned short* ix = fn + (size_t)f * fn_len;
               bv = v[ix[0]];
               for (int i = 1; i < fn_len; ++i) {
@@ -191,50 +205,75 @@ k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, c
 }
 
 // counts[t][0] = 0, counts[t][c + 1] = size of bucket c  ->  inclusive running sum = bucket offsets.
-// One block per table walks the table's counters 4096 at a time (coalesced), carrying the running sum.
-__global__ void __launch_bounds__(1024) k_bucket_scan(int32_t* off, long long nb) {
-  __shared__ int sh[33];
-  __shared__ int carry;
-  int32_t* o = off + (size_t)blockIdx.x * (size_t)(nb + 1);
-  const long long n = nb + 1;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) carry = 0;
-  __syncthreads();
-  for (long long base = 0; base < n; base += 4096) {
-    const long long i0 = base + (long long)threadIdx.x * 4;
-    int v[4];
+// Two kernels over chunks of BS_CHUNK counters: the sum of every chunk, then per chunk the sum of the
+// table's earlier chunks plus a scan inside the chunk.
+constexpr int BS_THREADS = 256;
+constexpr int BS_PER = 16;
+constexpr int BS_CHUNK = BS_THREADS * BS_PER;
+
+__global__ void __launch_bounds__(BS_THREADS) k_bucket_sums(const int32_t* off, long long nb, int32_t* part, int nchunks) {
+  __shared__ int sh[BS_THREADS / 32];
+  const int32_t* o = off + (size_t)blockIdx.y * (size_t)(nb + 1);
+  const long long n = nb + 1, base = (long long)blockIdx.x * BS_CHUNK;
+  int sum = 0;
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = i0 + u < n ? o[i0 + u] : 0;
-    const int sum = v[0] + v[1] + v[2] + v[3];
-    int incl = sum;
+  for (int u = 0; u < BS_PER; ++u) {
+    const long long i = base + threadIdx.x + (long long)u * BS_THREADS;
+    sum += i < n ? o[i] : 0;
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int tot = 0;
+    for (int w = 0; w < BS_THREADS / 32; ++w) tot += sh[w];
+    part[(size_t)blockIdx.y * nchunks + blockIdx.x] = tot;
+  }
+}
+
+__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks) {
+  __shared__ int sh[BS_THREADS / 32 + 1];
+  int32_t* o = off + (size_t)blockIdx.y * (size_t)(nb + 1);
+  const long long n = nb + 1, base = (long long)blockIdx.x * BS_CHUNK;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // everything before this chunk
+  int before = 0;
+  for (int c = threadIdx.x; c < (int)blockIdx.x; c += BS_THREADS) before += part[(size_t)blockIdx.y * nchunks + c];
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) before += __shfl_xor_sync(0xffffffffu, before, d);
+  if (lane == 0) sh[warp] = before;
+  __syncthreads();
+  before = 0;
+  for (int w = 0; w < BS_THREADS / 32; ++w) before += sh[w];
+  __syncthreads();
+  // the chunk itself: every warp owns BS_PER * 32 consecutive counters and walks them 32 at a time
+  const long long wbase = base + (long long)warp * (BS_PER * 32);
+  int v[BS_PER];
+  int wsum = 0;
+#pragma unroll
+  for (int u = 0; u < BS_PER; ++u) {
+    const long long i = wbase + u * 32 + lane;
+    v[u] = i < n ? o[i] : 0;
+    wsum += v[u];
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, d);
+  if (lane == 0) sh[warp] = wsum;
+  __syncthreads();
+  int run = before;
+  for (int w = 0; w < warp; ++w) run += sh[w];
+#pragma unroll
+  for (int u = 0; u < BS_PER; ++u) {
+    int incl = v[u];
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       int x = __shfl_up_sync(0xffffffffu, incl, d);
       if (lane >= d) incl += x;
     }
-    if (lane == 31) sh[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      int w = sh[lane];
-      int wi = w;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        int x = __shfl_up_sync(0xffffffffu, wi, d);
-        if (lane >= d) wi += x;
-      }
-      sh[lane] = wi - w;                 // exclusive over the warps
-      if (lane == 31) sh[32] = wi;       // total of this round
-    }
-    __syncthreads();
-    int run = carry + sh[warp] + incl - sum;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      run += v[u];
-      if (i0 + u < n) o[i0 + u] = run;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) carry += sh[32];
-    __syncthreads();
+    const long long i = wbase + u * 32 + lane;
+    if (i < n) o[i] = run + incl;
+    run += __shfl_sync(0xffffffffu, incl, 31);
   }
 }
 
@@ -287,41 +326,45 @@ __global__ void __launch_bounds__(1024) k_sort_scan(int32_t* hist, int n) {
 }
 
 // Each warp owns a contiguous part of the tile and walks it in order, 32 keys at a time; equal
-// digits inside a group of 32 are ranked by lane with a match mask, so the scatter is stable.
-// All of a warp's keys (and values) are fetched before the walk, which then runs out of registers.
+// digits inside a group of 32 are ranked by lane with a match mask, so the order of equal digits is
+// kept.  All of a warp's keys (and values) are fetched before the walk.  The walk places the elements
+// in shared memory in digit order; they are then written out in that order, so that a warp's stores
+// cover a few contiguous runs instead of 32 scattered words.
 // vals_in == nullptr means the value of element i is i (first pass).  keys_out may be nullptr
 // (last pass).
+constexpr int SORT_RADIX_MAX = 1 << SORT_MAX_WIDTH;
+constexpr int SORT_SMEM = (2 * SORT_TILE + SORT_WARPS * SORT_RADIX_MAX + 2 * SORT_RADIX_MAX + 64) * 4;
+
 __global__ void __launch_bounds__(SORT_THREADS, 2)
 k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_out, int32_t* vals_out,
                const int32_t* hist, int N, int tiles, int shift, int width) {
-  __shared__ int offs[SORT_WARPS][1 << SORT_MAX_WIDTH];
+  extern __shared__ __align__(16) int ss_smem[];
+  uint32_t* skey = reinterpret_cast<uint32_t*>(ss_smem);                 // [SORT_TILE] the tile in digit order
+  int* sval = ss_smem + SORT_TILE;                                       // [SORT_TILE]
+  int* offs = ss_smem + 2 * SORT_TILE;                                   // [SORT_WARPS][radix] cursor of (warp, digit) in the tile
+  int* gbase = offs + SORT_WARPS * SORT_RADIX_MAX;                       // [radix] where the tile's run of a digit starts globally
+  int* tbase = gbase + SORT_RADIX_MAX;                                   // [radix] where it starts inside the tile
+  int* sh = tbase + SORT_RADIX_MAX;                                      // [33] scan scratch
   const int radix = 1 << width, t = blockIdx.y, tl = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t* kin = keys_in + (size_t)t * N;
   const int32_t* vin = vals_in ? vals_in + (size_t)t * N : nullptr;
   uint32_t* kout = keys_out ? keys_out + (size_t)t * N : nullptr;
   int32_t* vout = vals_out + (size_t)t * N;
-  const int wbeg = min(N, tl * SORT_TILE + warp * SORT_SUB), wend = min(N, wbeg + SORT_SUB);
+  const int tbeg = tl * SORT_TILE, tn = min(SORT_TILE, N - tbeg);
+  const int wbeg = min(N, tbeg + warp * SORT_SUB), wend = min(N, wbeg + SORT_SUB);
 
   uint32_t key[SORT_ITERS];
-  int32_t val[SORT_ITERS];
 #pragma unroll
   for (int it = 0; it < SORT_ITERS; ++it) {
     const int i = wbeg + it * 32 + lane;
     key[it] = i < wend ? kin[i] : 0u;
-    val[it] = i < wend ? (vin ? vin[i] : i) : 0;
   }
-  for (int d = lane; d < radix; d += 32) offs[warp][d] = 0;
+  int* myoffs = offs + warp * SORT_RADIX_MAX;
+  for (int d = lane; d < radix; d += 32) myoffs[d] = 0;
   __syncwarp();
-#pragma unroll
-  for (int it = 0; it < SORT_ITERS; ++it)
-    if (wbeg + it * 32 + lane < wend) atomicAdd(&offs[warp][(key[it] >> shift) & (radix - 1)], 1);
-  __syncthreads();
-  for (int d = threadIdx.x; d < radix; d += SORT_THREADS) {
-    int run = hist[((size_t)t * radix + d) * tiles + tl];
-    for (int w = 0; w < SORT_WARPS; ++w) { int c = offs[w][d]; offs[w][d] = run; run += c; }
-  }
-  __syncthreads();
+  // walk 1: rank of every element among the warp's elements of the same digit (counts fall out at the end)
+  unsigned short lrank[SORT_ITERS];
 #pragma unroll
   for (int it = 0; it < SORT_ITERS; ++it) {
     const bool live = wbeg + it * 32 + lane < wend;
@@ -329,15 +372,73 @@ k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_o
     const unsigned peers = __match_any_sync(0xffffffffu, digit);
     const int rank = __popc(peers & ((1u << lane) - 1u));
     int base = 0;
-    if (live) base = offs[warp][digit];
+    if (live) base = myoffs[digit];
     __syncwarp();
-    if (live && rank == 0) offs[warp][digit] = base + __popc(peers);
+    if (live && rank == 0) myoffs[digit] = base + __popc(peers);
     __syncwarp();
-    if (live) {
-      const int dst = base + rank;
-      if (kout) kout[dst] = key[it];
-      vout[dst] = val[it];
+    lrank[it] = (unsigned short)(base + rank);
+  }
+  __syncthreads();
+  // per digit: the tile's count, the warps' starts relative to the digit's run, the global start of the run
+  int cnt[(SORT_RADIX_MAX + SORT_THREADS - 1) / SORT_THREADS];
+#pragma unroll
+  for (int u = 0; u < (SORT_RADIX_MAX + SORT_THREADS - 1) / SORT_THREADS; ++u) {
+    const int d = threadIdx.x + u * SORT_THREADS;
+    cnt[u] = 0;
+    if (d < radix) {
+      int run = 0;
+      for (int w = 0; w < SORT_WARPS; ++w) { int c = offs[w * SORT_RADIX_MAX + d]; offs[w * SORT_RADIX_MAX + d] = run; run += c; }
+      cnt[u] = run;
+      gbase[d] = hist[((size_t)t * radix + d) * tiles + tl];
     }
+  }
+  // exclusive scan of the counts over the digits (digit d lives in thread d % SORT_THREADS, round d / SORT_THREADS)
+  int carry = 0;
+#pragma unroll
+  for (int u = 0; u < (SORT_RADIX_MAX + SORT_THREADS - 1) / SORT_THREADS; ++u) {
+    int incl = cnt[u];
+#pragma unroll
+    for (int dd = 1; dd < 32; dd <<= 1) {
+      int x = __shfl_up_sync(0xffffffffu, incl, dd);
+      if (lane >= dd) incl += x;
+    }
+    __syncthreads();
+    if (lane == 31) sh[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = lane < SORT_WARPS ? sh[lane] : 0, wi = w;
+#pragma unroll
+      for (int dd = 1; dd < 32; dd <<= 1) {
+        int x = __shfl_up_sync(0xffffffffu, wi, dd);
+        if (lane >= dd) wi += x;
+      }
+      if (lane < SORT_WARPS) sh[lane] = wi - w;
+      if (lane == 31) sh[32] = wi;
+    }
+    __syncthreads();
+    const int d = threadIdx.x + u * SORT_THREADS;
+    if (d < radix) tbase[d] = carry + sh[warp] + incl - cnt[u];
+    carry += sh[32];
+  }
+  __syncthreads();
+  // walk 2: place the elements in digit order in shared memory
+#pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it) {
+    const int i = wbeg + it * 32 + lane;
+    if (i < wend) {
+      const int digit = (int)((key[it] >> shift) & (radix - 1));
+      const int lpos = tbase[digit] + myoffs[digit] + (int)lrank[it];
+      skey[lpos] = key[it];
+      sval[lpos] = vin ? vin[i] : i;
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < tn; i += SORT_THREADS) {
+    const uint32_t k = skey[i];
+    const int d = (int)((k >> shift) & (radix - 1));
+    const int g = gbase[d] + (i - tbase[d]);
+    if (kout) kout[g] = k;
+    vout[g] = sval[i];
   }
 }
 
@@ -366,11 +467,15 @@ cudaError_t launch_build_tables(Ctx* c) {
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   {
+    const int nchunks = (int)((c->nb + 1 + BS_CHUNK - 1) / BS_CHUNK);
+    dim3 grid(nchunks, c->L);
     LaunchScope ls(c, KID_BUCKET_SCAN);
-    k_bucket_scan<<<c->L, 1024, 0, c->stream>>>(c->bucket_off, c->nb);
+    k_bucket_sums<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
+    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
+  if ((e = cudaFuncSetAttribute(k_sort_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, SORT_SMEM)) != cudaSuccess) return e;
   const uint32_t* kin = c->keysA;
   const int32_t* vin = nullptr;
   for (int pass = 0; pass < c->sort_passes; ++pass) {
@@ -393,7 +498,7 @@ cudaError_t launch_build_tables(Ctx* c) {
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     {
       LaunchScope ls(c, KID_SORT_SCATTER);
-      k_sort_scatter<<<grid, SORT_THREADS, 0, c->stream>>>(kin, vin, kout, vout, c->tile_hist, c->N, c->sort_tiles,
+      k_sort_scatter<<<grid, SORT_THREADS, SORT_SMEM, c->stream>>>(kin, vin, kout, vout, c->tile_hist, c->N, c->sort_tiles,
                                                           shift, width);
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -404,6 +509,7 @@ cudaError_t launch_build_tables(Ctx* c) {
 }
 
 int sort_tile_elems() { return SORT_TILE; }
+int bucket_scan_chunk() { return BS_CHUNK; }
 int sort_max_width() { return SORT_MAX_WIDTH; }
 
 }  // namespace dslide
