@@ -23,6 +23,7 @@ constexpr int FWD_WARPS = FWD_THREADS / 32;
 constexpr int MAX_KPT = 4;        // hidden units per thread: H <= 4 * 256
 constexpr int ACT_SM = 1024;      // active ids and logits are mirrored in shared memory when the set is this small
 constexpr int HID_MIN_BYTES = 64 * 1024;   // staging space for the hidden layer's rows of W1
+constexpr int RANK_MAX = 1024;    // candidate sets up to this size are put in order by counting, larger ones by a bitonic sort
 constexpr int SORT_SMALL = 1024;  // candidate sets up to this size are sorted rather than run through the bitmap
 constexpr unsigned FULLM = 0xffffffffu;
 
@@ -99,6 +100,29 @@ __device__ __forceinline__ void list_row(const FwdParams& p, uint32_t* cnt, int 
   }
 }
 
+// Second half of handing a touched row to the update kernel, once the row's touch counter has answered
+// (nth = touches before this one): the (sample, coefficient) pair goes into the row's slot nth, or, past the
+// slots, the sample's bit into the row's mask; the first toucher enters the row in the list of distinct rows
+// (positions handed out per warp).  Called by whole warps; `live` tells whether this thread has a touch.
+__device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int32_t* own,
+                                             unsigned int* n_own, int row, int code, unsigned nth, int s, float coef) {
+  const int lane = threadIdx.x & 31;
+  bool first = false;
+  if (live) {
+    if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(coef));
+    else atomicOr(maskrow + (s >> 5), 1u << (s & 31));
+    first = nth == 0u;
+    list_row(p, &hd->cnt, code, nth);
+  }
+  const unsigned fm = __ballot_sync(FULLM, first);
+  if (fm) {
+    unsigned base = 0;
+    if (lane == 0) base = atomicAdd(n_own, (unsigned)__popc(fm));
+    base = __shfl_sync(FULLM, base, 0);
+    if (first) own[base + __popc(fm & ((1u << lane) - 1u))] = row;
+  }
+}
+
 // Exclusive prefix sum of one int per thread over the block; *total gets the block sum.
 // sh needs FWD_WARPS + 1 ints.  Ends with a barrier, so sh may be reused afterwards.
 __device__ __forceinline__ int block_excl_scan(int v, int* sh, int* total) {
@@ -147,6 +171,32 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
 
 __device__ __forceinline__ bool topk_better(float za, int ia, float zb, int ib) {
   return za > zb || (za == zb && ia < ib);
+}
+
+// Puts n <= PER * FWD_THREADS values in ascending order by counting: the place of a value is the number of values
+// before it (by value, then by position).  src and dst are in shared memory; thread t owns the values t, t +
+// FWD_THREADS, ...; threads without a value skip the counting loop.
+template <int PER>
+__device__ __forceinline__ void rank_sort(const uint32_t* src, uint32_t* dst, int n) {
+  const int tid = threadIdx.x;
+  if (tid >= n) return;
+  uint32_t v[PER];
+  int pos[PER];
+#pragma unroll
+  for (int u = 0; u < PER; ++u) {
+    const int i = tid + u * FWD_THREADS;
+    v[u] = i < n ? src[i] : 0xffffffffu;
+    pos[u] = 0;
+  }
+#pragma unroll 4
+  for (int k = 0; k < n; ++k) {
+    const uint32_t a = src[k];
+#pragma unroll
+    for (int u = 0; u < PER; ++u) pos[u] += (a < v[u] || (a == v[u] && k < tid + u * FWD_THREADS)) ? 1 : 0;
+  }
+#pragma unroll
+  for (int u = 0; u < PER; ++u)
+    if (tid + u * FWD_THREADS < n) dst[pos[u]] = v[u];
 }
 
 // The sample is skipped: no loss, no gradient, nothing touched (predict: no candidates).
@@ -386,6 +436,35 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
           }
         }
       }
+    } else if (ncand + nlab <= RANK_MAX) {
+      const int n = ncand + nlab;
+      __syncthreads();
+      uint32_t* srt = sh_dd + RANK_MAX;
+      const int per = (n + FWD_THREADS - 1) / FWD_THREADS;
+      if (per <= 1) rank_sort<1>(sh_dd, srt, n);
+      else if (per == 2) rank_sort<2>(sh_dd, srt, n);
+      else rank_sort<RANK_MAX / FWD_THREADS>(sh_dd, srt, n);
+      __syncthreads();
+      // thread t looks at the sorted elements PER * t ... PER * t + PER - 1 and keeps the first of each run
+      constexpr int PER = RANK_MAX / FWD_THREADS;
+      int cnt = 0;
+#pragma unroll
+      for (int u = 0; u < PER; ++u) {
+        const int i = tid * PER + u;
+        cnt += (i < n && (i == 0 || srt[i - 1] != srt[i])) ? 1 : 0;
+      }
+      int at = block_excl_scan(cnt, sh_misc, &total);
+      if (total <= p.act_stride && cnt > 0) {
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+          const int i = tid * PER + u;
+          if (i < n && (i == 0 || srt[i - 1] != srt[i])) {
+            ids[at] = (int)srt[i];
+            if (at < ACT_SM) sh_ids[at] = (int)srt[i];
+            ++at;
+          }
+        }
+      }
     } else {
       // sort path: bitonic sort of the candidates, keep the first of each run
       for (int i = ncand + nlab + tid; i < n2; i += FWD_THREADS) sh_dd[i] = 0x7fffffffu;
@@ -435,37 +514,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   const float* zp = small ? sh_z : p.act_z + (size_t)s * p.act_stride;
   const float* gp = small ? sh_z : p.act_g + (size_t)s * p.act_stride;
 
-  // ---- the W1 side of the hand-off to the update kernel.  Per touched row a count of the touching samples; for
-  //      the row's first ROW_SLOTS touches the (sample, coefficient) pair itself, else the bit of this sample in
-  //      the row's mask.  The sample that touches a row first also enters it in the list of distinct rows
-  //      (positions handed out per warp). ----
-  const uint32_t sbit = 1u << (s & 31);
-  const int sword = s >> 5;
-  const unsigned ltm = (1u << lane) - 1u;
-  if (MODE == 0) {
-    for (int i0 = 0; i0 < nnz; i0 += FWD_THREADS) {
-      const int i = i0 + tid;
-      bool first = false;
-      int c = 0;
-      if (i < nnz) {
-        c = __ldg(p.col_idx + rbeg + i);
-        RowHdr* hd = p.hdr1 + c;
-        const unsigned nth = atomicAdd(&hd->cnt, 1u) & CNT_MASK;
-        if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(__ldg(p.vals + rbeg + i)));
-        else atomicOr(p.mask1 + (size_t)c * p.Wd + sword, sbit);
-        first = nth == 0u;
-        list_row(p, &hd->cnt, ~c, nth);
-      }
-      const unsigned fm = __ballot_sync(FULLM, first);
-      if (fm) {
-        unsigned base = 0;
-        if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][1], (unsigned)__popc(fm));
-        base = __shfl_sync(FULLM, base, 0);
-        if (first) p.own1[base + __popc(fm & ltm)] = c;
-      }
-    }
-  }
-
   // ---- logits over the active set.  The active rows of W2 are copied into shared memory, as many as fit at a
   //      time; when the whole set fits they stay there for the back-propagation below ----
   float* z = p.act_z + (size_t)s * p.act_stride;
@@ -488,9 +536,27 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       const int j = dense ? c0 + r : idp[c0 + r];
       bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)j * H, row_bytes, sh_bar);
     }
-    // the biases of a small active set are fetched in the same round, into the logits' place
-    if (small && c0 == 0)
-      for (int a = tid; a < na; a += FWD_THREADS) sh_z[a] = __ldg(&p.hdr2[sh_ids[a]].b);
+    if (c0 == 0) {
+      // the biases of a small active set are fetched in the same round, into the logits' place
+      if (small)
+        for (int a = tid; a < na; a += FWD_THREADS) sh_z[a] = __ldg(&p.hdr2[sh_ids[a]].b);
+      // ---- the W1 side of the hand-off to the update kernel runs while the copies are in flight: per touched row
+      //      a count of the touching samples, then (finish_touch) the slot or mask entry and the row list ----
+      if (MODE == 0)
+        for (int i0 = 0; i0 < nnz; i0 += FWD_THREADS) {
+          const int i = i0 + tid;
+          const bool live = i < nnz;
+          int c = 0;
+          unsigned nth = 0u;
+          float x = 0.f;
+          if (live) {
+            c = __ldg(p.col_idx + rbeg + i);
+            x = __ldg(p.vals + rbeg + i);
+            nth = atomicAdd(&p.hdr1[c].cnt, 1u) & CNT_MASK;
+          }
+          finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
+        }
+    }
     if (!mbar_wait(sh_bar, phase)) timed_out = true;
     phase ^= 1u;
     if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
@@ -628,30 +694,17 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   }
   __syncthreads();
 
-  // ---- the W2 side of the hand-off, issued before the back-propagation so that its atomics overlap it ----
-  if (!dense)
-    for (int a0 = 0; a0 < na; a0 += FWD_THREADS) {
-      const int a = a0 + tid;
-      bool first = false;
-      int jj = 0;
-      if (a < na) {
-        jj = idp[a];
-        const float ga = gp[a];
-        RowHdr* hd = p.hdr2 + jj;
-        const unsigned nth = atomicAdd(&hd->cnt, 1u) & CNT_MASK;
-        if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(ga));
-        else atomicOr(p.mask2 + (size_t)jj * p.Wd + sword, sbit);
-        first = nth == 0u;
-        list_row(p, &hd->cnt, jj, nth);
-      }
-      const unsigned fm = __ballot_sync(FULLM, first);
-      if (fm) {
-        unsigned base = 0;
-        if (lane == 0) base = atomicAdd(&p.st->n_own[p.parity][0], (unsigned)__popc(fm));
-        base = __shfl_sync(FULLM, base, 0);
-        if (first) p.own2[base + __popc(fm & ltm)] = jj;
-      }
-    }
+  // ---- the W2 side of the hand-off: the touch counters of the first FWD_THREADS active rows are asked now and
+  //      answered while the back-propagation below runs ----
+  int jj0 = 0;
+  unsigned nth0 = 0u;
+  float ga0 = 0.f;
+  const bool live0 = !dense && tid < na;
+  if (live0) {
+    jj0 = idp[tid];
+    ga0 = gp[tid];
+    nth0 = atomicAdd(&p.hdr2[jj0].cnt, 1u) & CNT_MASK;
+  }
 
   // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update).  A thread
   //      per hidden unit walks the staged rows; with fewer hidden units than threads the rows are dealt to
@@ -682,9 +735,16 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         for (int u = 0; u < MAX_KPT; ++u) {
           const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
           if (k < H && (u == 0 || H > FWD_THREADS)) {
-            float v = accd[u];
-            for (int a = grp; a < nr; a += ngrp) v = fmaf(gp[c0 + a], stage[(size_t)a * ldr + k], v);
-            accd[u] = v;
+            float v0 = accd[u], v1 = 0.f, v2 = 0.f, v3 = 0.f;
+            int a = grp;
+            for (; a + 3 * ngrp < nr; a += 4 * ngrp) {
+              v0 = fmaf(gp[c0 + a], stage[(size_t)a * ldr + k], v0);
+              v1 = fmaf(gp[c0 + a + ngrp], stage[(size_t)(a + ngrp) * ldr + k], v1);
+              v2 = fmaf(gp[c0 + a + 2 * ngrp], stage[(size_t)(a + 2 * ngrp) * ldr + k], v2);
+              v3 = fmaf(gp[c0 + a + 3 * ngrp], stage[(size_t)(a + 3 * ngrp) * ldr + k], v3);
+            }
+            for (; a < nr; a += ngrp) v0 = fmaf(gp[c0 + a], stage[(size_t)a * ldr + k], v0);
+            accd[u] = (v0 + v1) + (v2 + v3);
           }
         }
       }
@@ -705,6 +765,22 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       float v = 0.f;
       for (int w = 0; w < ngrp; ++w) v += sh_dh[(size_t)w * H + k];
       p.dh[(size_t)s * H + k] = (sh_h[k] > 0.f && !timed_out) ? v : 0.f;
+    }
+  }
+  if (!dense) {
+    finish_touch(p, live0, p.hdr2 + jj0, p.mask2 + (size_t)jj0 * p.Wd, p.own2, &p.st->n_own[p.parity][0], jj0, jj0, nth0, s, ga0);
+    for (int a0 = FWD_THREADS; a0 < na; a0 += FWD_THREADS) {
+      const int a = a0 + tid;
+      const bool live = a < na;
+      int jj = 0;
+      unsigned nth = 0u;
+      float ga = 0.f;
+      if (live) {
+        jj = idp[a];
+        ga = gp[a];
+        nth = atomicAdd(&p.hdr2[jj].cnt, 1u) & CNT_MASK;
+      }
+      finish_touch(p, live, p.hdr2 + jj, p.mask2 + (size_t)jj * p.Wd, p.own2, &p.st->n_own[p.parity][0], jj, jj, nth, s, ga);
     }
   }
   if (tid == 0) {
