@@ -150,6 +150,17 @@ def dist_setup(ngpus):
     return world, rank, local
 
 
+def max_over_ranks(ms, world, device):
+    """The slowest rank's time: every multi-GPU number is the maximum over the ranks."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def shard_seed(rank):
     """Every rank draws its own batches: replicas share no data and exchange nothing."""
     return 1000 * rank
@@ -281,10 +292,7 @@ def run_dslide(args):
     clocks = sampler.stop() if rank == 0 else None
     status = ds.dslide_sync(ctx, check=False)
     cum = ds.dslide_cum_stats(ctx, reset=True)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, "cuda")
     value = world * B * K / (ms * 1e-3)
 
     # ---- second pass of the same K steps with a CUDA event pair around every kernel launch ----
@@ -306,10 +314,7 @@ def run_dslide(args):
         e1.record()
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = max_over_ranks(ms_e2e, world, "cuda")
         h2d = float(np.mean([sum(a.numel() * a.element_size() for a in b) for b in pinned]))
         e2e = {"value": world * B * K / (ms_e2e * 1e-3), "unit": "samples/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / K}

@@ -1,0 +1,145 @@
+"""GPU-vs-oracle parity on shapes chosen to reach every path of the two step kernels (run with -m gpu).
+
+The forward kernel switches between three ways of removing duplicate candidates (counting ranks, bitonic
+sort, bitmap) by the size of the candidate set, stages the active rows of W2 in shared memory in one or
+several chunks, and hands rows to the update kernel through slots, masks and two lists whose capacity is
+bounded; the update kernel has code paths per touch count (1, up to the slots, listed, listed hot and cut
+in slices) and per hidden width.  Each case below states which of these it drives.  Bars as in
+test_gpu_parity.py.
+"""
+import numpy as np
+import pytest
+import torch
+
+from tests.helpers import max_rel_err
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2201_12667_b200 import binding as ds
+    from paper_2201_12667_b200 import workloads
+    from tests.gpu_harness import Pair
+    from tests.test_gpu_parity import ACT_TOL, W_TOL, compare_forward, compare_weights
+
+SIMHASH, DWTA = 0, 1
+
+
+def dense_features_batch(rng, B, D, N, nnz, nlab):
+    """Every sample draws nnz of only D features, so every feature row is touched by about B*nnz/D samples."""
+    cols, vals, labs = [], [], []
+    row_ptr = np.zeros(B + 1, dtype=np.int32)
+    label_ptr = np.zeros(B + 1, dtype=np.int32)
+    for s in range(B):
+        ids = np.sort(rng.choice(D, size=nnz, replace=False)).astype(np.int32)
+        cols.append(ids)
+        v = rng.standard_normal(nnz).astype(np.float32)
+        vals.append(v / np.sqrt(np.sum(v * v)))
+        labs.append(rng.choice(N, size=nlab, replace=False).astype(np.int32))
+        row_ptr[s + 1] = row_ptr[s] + nnz
+        label_ptr[s + 1] = label_ptr[s] + nlab
+    return row_ptr, np.concatenate(cols), np.concatenate(vals), label_ptr, np.concatenate(labs)
+
+
+def one_and_two_steps(pr, batches):
+    for i, batch in enumerate(batches):
+        lo = pr.o.train_step(*batch)
+        lg = pr.gpu_step(batch)
+        tol = ACT_TOL if i == 0 else W_TOL
+        assert abs(lo - lg) <= tol * abs(lo), (i, lo, lg)
+        compare_forward(pr, batch, bit_exact_hidden=(i == 0), tol=tol)
+    compare_weights(pr)
+
+
+@pytest.mark.parametrize("H", [64, 256, 512, 1024])
+def test_hidden_widths(H):
+    """H = 64: two groups of threads per hidden unit in the back-propagation; 256 / 512 / 1024: the wider
+    register layouts of the update kernel and several hidden units per thread in the forward kernel."""
+    c = workloads.config("mid")
+    pr = Pair(D=c["D"], H=H, N=8009, family=DWTA, K=3, L=6, bucket_cap=16, max_batch=24, max_labels=16, lr=1e-3, seed=2)
+    try:
+        wl = workloads.Workload(workloads.config("mid", N=8009), seed=11)
+        one_and_two_steps(pr, [wl.batch(i, batch_size=24) for i in range(2)])
+    finally:
+        pr.close()
+
+
+@pytest.mark.parametrize("family,K,L,cap,dedup_mode", [
+    (SIMHASH, 3, 12, 40, 0),     # 300-480 candidates per sample: ranks counted with two or more values per thread
+    (SIMHASH, 2, 30, 64, 0),     # up to 1,920 candidates: past the counting limit, bitmap (N bits fit in shared memory)
+    (SIMHASH, 2, 30, 64, 2),     # the same through the bitonic sort
+    (DWTA, 1, 16, 48, 0),        # 8 buckets per table: about 770 candidates, chunked staging of the active rows
+])
+def test_large_candidate_sets(family, K, L, cap, dedup_mode):
+    """Active sets of several hundred to a thousand neurons: every dedup path, active rows staged in more than one
+    chunk (the staging space holds about 190 rows of 128 floats), logits and errors beyond the shared-memory mirror."""
+    pr = Pair(D=3001, H=128, N=12007, family=family, K=K, L=L, bucket_cap=cap, max_batch=16, max_labels=16, lr=1e-3,
+              seed=3, dedup_mode=dedup_mode)
+    try:
+        wl = workloads.Workload(workloads.config("mid", D=3001, N=12007), seed=12)
+        batches = [wl.batch(i, batch_size=16) for i in range(2)]
+        one_and_two_steps(pr, batches)
+        cnt = ds.dslide_get_last(pr.ctx, "act_count", 16)
+        assert cnt.max() > 256
+    finally:
+        pr.close()
+
+
+def test_batch_beyond_256_and_rows_touched_by_most_samples():
+    """Batch 300 (ten mask words per row, so a slice of a hot row covers two words and some slices are empty) with
+    only 400 features, 60 per sample: every row of W1 is touched by about 45 samples -> the hot list and its slices."""
+    rng = np.random.default_rng(5)
+    pr = Pair(D=400, H=128, N=6007, family=DWTA, K=3, L=8, bucket_cap=16, max_batch=300, max_labels=4, lr=1e-3, seed=4)
+    try:
+        batches = [dense_features_batch(rng, 300, 400, 6007, 60, 2) for _ in range(2)]
+        one_and_two_steps(pr, batches)
+        st = ds.dslide_last_stats(pr.ctx)
+        assert st["touched_w1"] == 400
+    finally:
+        pr.close()
+
+
+def test_more_hot_rows_than_the_hot_list_holds():
+    """2,000 features, 200 per sample, batch 512: each of the 2,000 rows of W1 is touched by about 51 samples, more
+    rows than the hot list holds (1,024): the rest must be summed through the list of rows past the slots."""
+    rng = np.random.default_rng(6)
+    pr = Pair(D=2000, H=32, N=3001, family=DWTA, K=2, L=4, bucket_cap=8, max_batch=512, max_labels=4, lr=1e-3, seed=5)
+    try:
+        batch = dense_features_batch(rng, 512, 2000, 3001, 200, 1)
+        lo = pr.o.train_step(*batch)
+        lg = pr.gpu_step(batch)
+        assert abs(lo - lg) <= ACT_TOL * abs(lo)
+        compare_weights(pr, names=["W1", "mW1", "vW1", "W2", "b2", "b1"])
+        # a second step proves that counters, masks and lists were left clean
+        batch = dense_features_batch(rng, 512, 2000, 3001, 200, 1)
+        lo = pr.o.train_step(*batch)
+        lg = pr.gpu_step(batch)
+        assert abs(lo - lg) <= W_TOL * abs(lo)
+        compare_weights(pr, names=["W1", "W2", "b2", "b1"])
+    finally:
+        pr.close()
+
+
+def test_more_listed_rows_than_the_list_holds():
+    """One table with two buckets and no cap: every sample retrieves about half of 140,000 neurons, so with 16
+    samples some 70,000 rows of W2 are touched by more samples than a row has slots -- more than the list of such
+    rows holds (65,536); the rest are found and summed by the walk over the ordinary row list."""
+    N = 140000
+    pr = Pair(D=200, H=32, N=N, family=SIMHASH, K=1, L=1, bucket_cap=N, max_batch=16, max_labels=2, lr=1e-3, seed=6,
+              init_std=0.05)
+    try:
+        wl = workloads.Workload(workloads.config("tiny", D=200, N=N, max_labels=2), seed=13)
+        for i in range(2):
+            batch = wl.batch(i, batch_size=16)
+            lo = pr.o.train_step(*batch)
+            lg = pr.gpu_step(batch)
+            assert abs(lo - lg) <= (ACT_TOL if i == 0 else W_TOL) * abs(lo)
+            sets, cnt = pr.gpu_active_sets(16)
+            for s, a in enumerate(pr.o.active_sets()):
+                assert np.array_equal(sets[s], a)
+            if i == 0:
+                touches = np.bincount(np.concatenate(sets), minlength=N)
+                assert (touches > 6).sum() > 65536
+        for n in ("W2", "b2", "mW2", "vW2", "W1"):
+            assert max_rel_err(ds.dslide_get_tensor(pr.ctx, n), pr.o.get(n), 1e-2) < W_TOL, n
+    finally:
+        pr.close()
