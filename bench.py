@@ -40,7 +40,7 @@ REBUILD_PERIOD = 50
 REF_BATCH = 32            # samples per step of the CPU-oracle arm (a bounded sample of the 256-sample batch)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists)
-NCU_TRAFFIC_BYTES = {"adam": None, "forward": None}
+NCU_TRAFFIC_BYTES = {"adam": 106.5e6, "forward": 34.3e6}
 
 
 def parse_args():
