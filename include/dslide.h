@@ -44,7 +44,7 @@ typedef enum {
   DSLIDE_ERR_OVERFLOW = 4,   /* an active set, label list or batch exceeds the configured maximum */
   DSLIDE_ERR_BAD_INDEX = 5,  /* feature id outside [0,D) or label id outside [0,N), seen on the device */
   DSLIDE_ERR_STATE = 6,
-  DSLIDE_ERR_TIMEOUT = 7
+  DSLIDE_ERR_TIMEOUT = 7     /* a bounded wait inside a kernel ran out (the sample concerned is skipped)               */
 } dslide_status;
 
 enum { DSLIDE_SIMHASH = 0, DSLIDE_DWTA = 1 };
