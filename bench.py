@@ -8,8 +8,8 @@ union, active logits and softmax, sparse back-propagation, row-wise Adam, and th
 whenever the schedule (every 50 steps) places one inside the window.  Prints ONE JSON line.
 
   value      train samples/s with the batches already resident in HBM (CUDA events, max over ranks)
-  e2e        the same through dslide_train_step_host: HOST (pinned) buffers, the host->device copies
-             and the device->host read of the loss inside the timed region
+  e2e        the same through dslide_train_step_host_async: HOST (pinned) buffers, every step's host->device copy
+             and the device->host read of its loss and status inside the timed region
   roofline   the dominant kernel: algorithmic bytes per launch / its mean launch duration (CUDA
              events around every launch of a second, separately timed pass) against the measured
              HBM copy bandwidth
@@ -305,19 +305,27 @@ def run_dslide(args):
     # ---- end to end: host buffers in, loss out, every step ----
     e2e = None
     if not args.no_e2e:
+        # the pipelined host-buffer entry point: every step copies its inputs from pinned host memory to the device
+        # and its {status, loss} back; the loss of step i is handed out by call i + 1 (the last one by
+        # dslide_host_result), so the device always has one step queued while the host packs the next
         for i in range(3):
-            ds.dslide_train_step_host(ctx, B, *pinned[i % nb])
+            ds.dslide_train_step_host_async(ctx, B, *pinned[i % nb])
+        ds.dslide_host_result(ctx)
         barrier()
         e0.record()
+        losses = 0
         for i in range(K):
-            ds.dslide_train_step_host(ctx, B, *pinned[(W + i) % nb])
+            losses += ds.dslide_train_step_host_async(ctx, B, *pinned[(W + i) % nb]) is not None
+        losses += ds.dslide_host_result(ctx) is not None
         e1.record()
         barrier()
+        assert losses == K
         ms_e2e = e0.elapsed_time(e1)
         ms_e2e = max_over_ranks(ms_e2e, world, "cuda")
         h2d = float(np.mean([sum(a.numel() * a.element_size() for a in b) for b in pinned]))
         e2e = {"value": world * B * K / (ms_e2e * 1e-3), "unit": "samples/s", "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / K}
+               "d2h_bytes_per_step": 8, "ms_per_step": ms_e2e / K,
+               "api": "dslide_train_step_host_async + dslide_host_result (loss and status of every step read back)"}
 
     if rank == 0:
         per_step = {k: cum[k] / max(1, cum["steps"]) for k in ("nnz", "sum_active", "touched_w1", "touched_w2", "fetched")}

@@ -142,6 +142,20 @@ dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32
                                      const int32_t* label_ptr, const int32_t* labels,
                                      float* loss_out);
 
+/* The same step, pipelined: the call packs and enqueues this batch and returns as soon as the PREVIOUS
+ * host-buffer step has finished, handing out that step's mean loss (*prev_loss_out, may be NULL) and sticky
+ * status (the return value); *have_prev (may be NULL) tells whether there was a previous step to report.
+ * The device therefore always has one step queued while the host prepares the next.  The arrays are copied
+ * into the library's pinned buffer before the call returns, so the caller may reuse them at once.
+ * dslide_host_result waits for the newest pipelined step and hands out its loss and status (*have = 0 and
+ * DSLIDE_OK when none is outstanding) and, like dslide_sync, clears the sticky status; between those calls a
+ * status seen by one step is reported by the following steps as well.  dslide_train_step_host may be mixed in
+ * (it drops uncollected results). */
+dslide_status dslide_train_step_host_async(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
+                                           const int32_t* col_idx, const float* vals, const int32_t* label_ptr,
+                                           const int32_t* labels, float* prev_loss_out, int32_t* have_prev);
+dslide_status dslide_host_result(dslide_ctx* ctx, float* loss_out, int32_t* have);
+
 /* Inference: hidden layer -> codes -> retrieved set (dense = 0) or every neuron
  * (dense = 1) -> logits -> the k largest by (logit descending, id ascending).
  * out_ids [batch*k] (device, -1 where fewer than k candidates), out_scores [batch*k]

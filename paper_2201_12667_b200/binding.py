@@ -54,6 +54,8 @@ _SIGS = {
     "dslide_build_tables": (_i32, [_vp]),
     "dslide_train_step": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dslide_train_step_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, C.POINTER(C.c_float)]),
+    "dslide_train_step_host_async": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, C.POINTER(C.c_float), C.POINTER(_i32)]),
+    "dslide_host_result": (_i32, [_vp, C.POINTER(C.c_float), C.POINTER(_i32)]),
     "dslide_predict_topk": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _vp]),
     "dslide_sync": (_i32, [_vp]),
     "dslide_tensor_info": (_i32, [_vp, _i32, C.POINTER(_i64)]),
@@ -138,6 +140,21 @@ def dslide_train_step_host(ctx, batch, row_ptr, col_idx, vals, label_ptr, labels
     ptr = [a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data for a in (row_ptr, col_idx, vals, label_ptr, labels)]
     _check(_lib.dslide_train_step_host(ctx, batch, *ptr, C.byref(loss)), "dslide_train_step_host")
     return loss.value
+
+
+def dslide_train_step_host_async(ctx, batch, row_ptr, col_idx, vals, label_ptr, labels):
+    """Pipelined host-buffer step: enqueues this batch, returns the mean loss of the PREVIOUS such step (None if none)."""
+    loss, have = C.c_float(0.0), _i32(0)
+    ptr = [a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data for a in (row_ptr, col_idx, vals, label_ptr, labels)]
+    _check(_lib.dslide_train_step_host_async(ctx, batch, *ptr, C.byref(loss), C.byref(have)), "dslide_train_step_host_async")
+    return loss.value if have.value else None
+
+
+def dslide_host_result(ctx):
+    """Waits for the newest pipelined host-buffer step; returns its mean loss (None if none is outstanding)."""
+    loss, have = C.c_float(0.0), _i32(0)
+    _check(_lib.dslide_host_result(ctx, C.byref(loss), C.byref(have)), "dslide_host_result")
+    return loss.value if have.value else None
 
 
 def dslide_predict_topk(ctx, batch, row_ptr, col_idx, vals, k, dense, out_ids, out_scores):

@@ -1,6 +1,7 @@
 // The C ABI of libdslide (include/dslide.h): context life cycle, argument checks, the rebuild
 // schedule (Section 3.1; Algorithm 1 places the rebuild after the weight update), state I/O.
 #include <math.h>
+#include <stddef.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -58,9 +59,17 @@ void free_all(Ctx* c) {
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1,
                   c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part,
-                  c->st_row_ptr, c->st_col, c->st_label_ptr, c->st_labels, c->st_vals, c->st_loss};
+                  c->st_dev[0], c->st_dev[1]};
   for (void* p : ptrs) if (p) cudaFree(p);
-  if (c->pinned_loss) cudaFreeHost(c->pinned_loss);
+  for (int b = 0; b < 2; ++b) {
+    if (c->st_host[b]) cudaFreeHost(c->st_host[b]);
+    if (c->st_result[b]) cudaFreeHost(c->st_result[b]);
+    if (c->st_event[b]) cudaEventDestroy(c->st_event[b]);
+    if (c->st_in[b]) cudaEventDestroy(c->st_in[b]);
+    if (c->st_done[b]) cudaEventDestroy(c->st_done[b]);
+  }
+  if (c->st_copy_in) cudaStreamDestroy(c->st_copy_in);
+  if (c->st_copy_out) cudaStreamDestroy(c->st_copy_out);
   if (c->prof) {
     auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
     for (auto& r : *v) { cudaEventDestroy(r.beg); cudaEventDestroy(r.end); }
@@ -220,8 +229,14 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     A(bucket_part, (size_t)c->L * (size_t)((c->nb + 1 + bucket_scan_chunk() - 1) / bucket_scan_chunk()), false);
   }
 #undef A
-  if (e == cudaSuccess) e = cudaMallocHost((void**)&c->pinned_loss, sizeof(float));
-  if (e == cudaSuccess) e = dalloc(&c->st_loss, 1, st, true);
+  for (int b = 0; b < 2; ++b) {
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&c->st_result[b], 4 * sizeof(float));
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->st_event[b], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->st_in[b], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->st_done[b], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_copy_in, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_copy_out, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = setup_forward(c);
   if (e == cudaSuccess) e = launch_init_gauss(c, c->W1, (int64_t)(D * H), RNG_W1);
   if (e == cudaSuccess) e = launch_init_gauss(c, c->W2, (int64_t)(N * H), RNG_W2);
@@ -278,6 +293,83 @@ dslide_status dslide_train_step(dslide_ctx* ctx, int32_t batch, const int32_t* r
   return DSLIDE_OK;
 }
 
+namespace {
+
+// Hands out the result of the step that used staging set b: waits for it, returns the sticky status as it stood
+// at the end of that step, stores its mean loss.
+dslide_status take_result(Ctx* c, int b, float* loss_out) {
+  if (!c->st_pending[b]) return DSLIDE_OK;
+  CU(cudaEventSynchronize(c->st_event[b]));
+  c->st_pending[b] = 0;
+  int status = 0;
+  memcpy(&status, c->st_result[b], sizeof(int));
+  if (loss_out) *loss_out = c->st_result[b][1 + b];
+  return (dslide_status)status;
+}
+
+// With the stream drained, a reported status is cleared on the device (as dslide_sync does).
+dslide_status drain_and_clear(Ctx* c, dslide_status s) {
+  CU(cudaStreamSynchronize(c->stream));
+  if (s != DSLIDE_OK) {
+    CU(cudaMemsetAsync(&c->dstate->status, 0, sizeof(int), c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+  }
+  return s;
+}
+
+// Packs a host batch into staging set b (one pinned buffer, 16-byte aligned pieces), sends it in a single copy,
+// enqueues the step and the copy of {status, loss} back, and records the set's event.
+dslide_status enqueue_host_step(dslide_ctx* ctx, int b, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
+                                const float* vals, const int32_t* label_ptr, const int32_t* labels) {
+  Ctx* c = &ctx->c;
+  const int64_t nnz = row_ptr[batch], nlab = label_ptr[batch];
+  if (nnz < 0 || nlab < 0 || row_ptr[0] != 0 || label_ptr[0] != 0) return DSLIDE_ERR_INVALID_ARG;
+  auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
+  const size_t o_rp = 0;
+  const size_t o_lp = o_rp + up16(sizeof(int32_t) * ((size_t)batch + 1));
+  const size_t o_col = o_lp + up16(sizeof(int32_t) * ((size_t)batch + 1));
+  const size_t o_val = o_col + up16(sizeof(int32_t) * (size_t)nnz);
+  const size_t o_lab = o_val + up16(sizeof(float) * (size_t)nnz);
+  const size_t total = o_lab + up16(sizeof(int32_t) * (size_t)nlab);
+  if ((int64_t)total > c->st_cap[b]) {
+    CU(cudaStreamSynchronize(c->stream));
+    if (c->st_dev[b]) cudaFree(c->st_dev[b]);
+    if (c->st_host[b]) cudaFreeHost(c->st_host[b]);
+    c->st_dev[b] = nullptr; c->st_host[b] = nullptr; c->st_cap[b] = 0;
+    const size_t cap = total + total / 2 + 4096;
+    CU(cudaMalloc((void**)&c->st_dev[b], cap));
+    CU(cudaMallocHost((void**)&c->st_host[b], cap));
+    c->st_cap[b] = (int64_t)cap;
+  }
+  cudaStream_t st = c->stream;
+  unsigned char *hb = c->st_host[b], *db = c->st_dev[b];
+  memcpy(hb + o_rp, row_ptr, sizeof(int32_t) * ((size_t)batch + 1));
+  memcpy(hb + o_lp, label_ptr, sizeof(int32_t) * ((size_t)batch + 1));
+  memcpy(hb + o_col, col_idx, sizeof(int32_t) * (size_t)nnz);
+  memcpy(hb + o_val, vals, sizeof(float) * (size_t)nnz);
+  memcpy(hb + o_lab, labels, sizeof(int32_t) * (size_t)nlab);
+  // The input copy and the result copy run on streams of their own, tied to the step by events, so that they
+  // overlap the kernels of the neighbouring steps.  (The device buffer of this set was last read two steps ago;
+  // the caller waited for that step when it collected its result.)
+  CU(cudaMemcpyAsync(db, hb, total, cudaMemcpyHostToDevice, c->st_copy_in));
+  CU(cudaEventRecord(c->st_in[b], c->st_copy_in));
+  CU(cudaStreamWaitEvent(st, c->st_in[b], 0));
+  dslide_status s = dslide_train_step(ctx, batch, (const int32_t*)(db + o_rp), (const int32_t*)(db + o_col),
+                                      (const float*)(db + o_val), (const int32_t*)(db + o_lp),
+                                      (const int32_t*)(db + o_lab), &c->dstate->host_loss[b]);
+  if (s != DSLIDE_OK) { cudaStreamSynchronize(st); return s; }
+  // the sticky status and the two sets' losses sit side by side: one copy brings them back
+  static_assert(offsetof(DevState, host_loss) == sizeof(int), "status and losses are copied together");
+  CU(cudaEventRecord(c->st_done[b], st));
+  CU(cudaStreamWaitEvent(c->st_copy_out, c->st_done[b], 0));
+  CU(cudaMemcpyAsync(c->st_result[b], c->dstate, 3 * sizeof(float), cudaMemcpyDeviceToHost, c->st_copy_out));
+  CU(cudaEventRecord(c->st_event[b], c->st_copy_out));
+  c->st_pending[b] = 1;
+  return DSLIDE_OK;
+}
+
+}  // namespace
+
 dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
                                      const float* vals, const int32_t* label_ptr, const int32_t* labels,
                                      float* loss_out) {
@@ -285,45 +377,45 @@ dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32
   Ctx* c = &ctx->c;
   if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
   if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
-  const int64_t nnz = row_ptr[batch], nlab = label_ptr[batch];
-  if (nnz < 0 || nlab < 0 || row_ptr[0] != 0 || label_ptr[0] != 0) return DSLIDE_ERR_INVALID_ARG;
-  if (!c->st_row_ptr) {
-    CU(dalloc(&c->st_row_ptr, (size_t)c->cfg.max_batch + 1, c->stream, false));
-    CU(dalloc(&c->st_label_ptr, (size_t)c->cfg.max_batch + 1, c->stream, false));
-  }
-  if (nnz > c->st_nnz_cap) {
-    CU(cudaStreamSynchronize(c->stream));
-    if (c->st_col) cudaFree(c->st_col);
-    if (c->st_vals) cudaFree(c->st_vals);
-    c->st_col = nullptr; c->st_vals = nullptr; c->st_nnz_cap = 0;
-    int64_t cap = nnz + nnz / 2 + 1024;
-    CU(dalloc(&c->st_col, (size_t)cap, c->stream, false));
-    CU(dalloc(&c->st_vals, (size_t)cap, c->stream, false));
-    c->st_nnz_cap = cap;
-  }
-  if (nlab > c->st_lab_cap) {
-    CU(cudaStreamSynchronize(c->stream));
-    if (c->st_labels) cudaFree(c->st_labels);
-    c->st_labels = nullptr; c->st_lab_cap = 0;
-    int64_t cap = nlab + nlab / 2 + 1024;
-    CU(dalloc(&c->st_labels, (size_t)cap, c->stream, false));
-    c->st_lab_cap = cap;
-  }
-  cudaStream_t st = c->stream;
-  CU(cudaMemcpyAsync(c->st_row_ptr, row_ptr, sizeof(int32_t) * ((size_t)batch + 1), cudaMemcpyHostToDevice, st));
-  CU(cudaMemcpyAsync(c->st_label_ptr, label_ptr, sizeof(int32_t) * ((size_t)batch + 1), cudaMemcpyHostToDevice, st));
-  if (nnz > 0) {
-    CU(cudaMemcpyAsync(c->st_col, col_idx, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, st));
-    CU(cudaMemcpyAsync(c->st_vals, vals, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
-  }
-  if (nlab > 0) CU(cudaMemcpyAsync(c->st_labels, labels, sizeof(int32_t) * (size_t)nlab, cudaMemcpyHostToDevice, st));
-  dslide_status s = dslide_train_step(ctx, batch, c->st_row_ptr, c->st_col, c->st_vals, c->st_label_ptr,
-                                      c->st_labels, c->st_loss);
+  // results of earlier pipelined steps that nobody collected are dropped (their status stays sticky on the device)
+  for (int b = 0; b < 2; ++b)
+    if (c->st_pending[b]) { CU(cudaEventSynchronize(c->st_event[b])); c->st_pending[b] = 0; }
+  const int b = c->st_next;
+  dslide_status s = enqueue_host_step(ctx, b, batch, row_ptr, col_idx, vals, label_ptr, labels);
   if (s != DSLIDE_OK) return s;
-  CU(cudaMemcpyAsync(c->pinned_loss, c->st_loss, sizeof(float), cudaMemcpyDeviceToHost, st));
-  s = dslide_sync(ctx);
-  if (loss_out) *loss_out = *c->pinned_loss;
-  return s;
+  c->st_next ^= 1;
+  s = take_result(c, b, loss_out);
+  return drain_and_clear(c, s);
+}
+
+dslide_status dslide_train_step_host_async(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
+                                           const int32_t* col_idx, const float* vals, const int32_t* label_ptr,
+                                           const int32_t* labels, float* prev_loss_out, int32_t* have_prev) {
+  if (!ctx || !row_ptr || !col_idx || !vals || !label_ptr || !labels) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
+  if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
+  const int b = c->st_next;
+  // the set about to be reused belongs to the step before the previous one: its result was handed out one call
+  // ago, or is dropped here if that call failed
+  if (c->st_pending[b]) { CU(cudaEventSynchronize(c->st_event[b])); c->st_pending[b] = 0; }
+  dslide_status s = enqueue_host_step(ctx, b, batch, row_ptr, col_idx, vals, label_ptr, labels);
+  if (s != DSLIDE_OK) return s;
+  c->st_next ^= 1;
+  // while the device works on this step, collect the previous one
+  const int had = c->st_pending[b ^ 1];
+  if (have_prev) *have_prev = had;
+  return take_result(c, b ^ 1, prev_loss_out);
+}
+
+dslide_status dslide_host_result(dslide_ctx* ctx, float* loss_out, int32_t* have) {
+  if (!ctx) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int newest = c->st_next ^ 1, older = c->st_next;
+  dslide_status s_old = take_result(c, older, nullptr);     // only pending if its collection was skipped
+  if (have) *have = c->st_pending[newest];
+  dslide_status s = take_result(c, newest, loss_out);
+  return drain_and_clear(c, s != DSLIDE_OK ? s : s_old);
 }
 
 dslide_status dslide_predict_topk(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,

@@ -30,6 +30,7 @@ enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2 };
 // in the synchronous statistics and status calls).
 struct DevState {
   int status;                      // sticky dslide_status seen on the device
+  float host_loss[2];              // mean loss of the last host-buffer step that used staging set 0 / 1
   int pad0;
   // Slots indexed by the parity of the step: the kernels of step t use slot t & 1 and the update
   // kernel zeroes the other slot for step t + 1.
@@ -141,10 +142,15 @@ struct Ctx {
   int num_sms;
 
   // staging for the host-buffer entry point
-  int32_t *st_row_ptr, *st_col, *st_label_ptr, *st_labels;
-  float *st_vals, *st_loss;
-  int64_t st_nnz_cap, st_lab_cap;
-  float* pinned_loss;
+  // host-buffer entry points: two sets of (device buffer, pinned host buffer, pinned result, event), used in turn
+  unsigned char *st_dev[2], *st_host[2];
+  int64_t st_cap[2];
+  float* st_result[2];        // pinned: {sticky status (int bits), mean loss} of the step that used the set
+  cudaEvent_t st_event[2];    // recorded after that step's result copy
+  cudaEvent_t st_in[2], st_done[2];   // input copy finished / kernels of the step finished
+  cudaStream_t st_copy_in, st_copy_out;   // the copies run beside the kernels of the neighbouring steps
+  int st_pending[2];          // a step was enqueued on the set and its result has not been handed out yet
+  int st_next;                // set the next host-buffer step uses
 
   int64_t t_host, r_host, next_rebuild;
   int64_t launches;

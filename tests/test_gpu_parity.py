@@ -245,6 +245,39 @@ def test_ten_steps_mid_through_host_entry_point():
         pr.close()
 
 
+def test_pipelined_host_steps_match_synchronous_ones():
+    """dslide_train_step_host_async hands out each step's loss one call late; losses and weights must be the very
+    bits the synchronous entry point produces (the kernels and their order are the same)."""
+    wl = workloads.Workload(workloads.config("mid"), seed=8)
+    batches = [wl.batch(i) for i in range(7)]
+    B = len(batches[0][0]) - 1
+    a, b = mid_pair(rebuild_period0=3), mid_pair(rebuild_period0=3)
+    try:
+        sync_losses = [ds.dslide_train_step_host(a.ctx, B, *bt) for bt in batches]
+        got = []
+        for bt in batches:
+            prev = ds.dslide_train_step_host_async(b.ctx, B, *[x.copy() for x in bt])   # the arrays may be reused at once
+            if prev is not None:
+                got.append(prev)
+        got.append(ds.dslide_host_result(b.ctx))
+        assert ds.dslide_host_result(b.ctx) is None
+        assert np.array_equal(np.array(got, dtype=np.float32), np.array(sync_losses, dtype=np.float32))
+        for n in WEIGHTS + MOMENTS:
+            x, y = ds.dslide_get_tensor(a.ctx, n), ds.dslide_get_tensor(b.ctx, n)
+            assert np.array_equal(x.view(np.uint32), y.view(np.uint32)), n
+        # an out-of-range feature id is reported with the step it belongs to (one call late) and cleared by the collect
+        bad = [x.copy() for x in batches[0]]
+        bad[1][3] = a.D + 7
+        assert ds.dslide_train_step_host_async(b.ctx, B, *bad) is None
+        with pytest.raises(ds.DslideError) as e:
+            ds.dslide_host_result(b.ctx)
+        assert e.value.status == ds.ERR_BAD_INDEX
+        assert ds.dslide_sync(b.ctx, check=False) == ds.OK
+    finally:
+        a.close()
+        b.close()
+
+
 # ------------------------------------------------------------------ dense limit
 def test_force_dense_matches_oracle_and_dense_softmax():
     pr = tiny_pair(force_dense=1)
