@@ -204,6 +204,74 @@ k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, c
   }
 }
 
+// DWTA with bins of eight, hash functions in shared memory: the same tiles, but two rows per lane.  A tile holds
+// 64 rows as 32 pairs (row r and row r + 32 interleaved per coordinate), so that one 8-byte load fetches a
+// coordinate of both rows and the index arithmetic is shared; the two rows' winners are found side by side.
+constexpr int HN2_ROWS = 64;
+
+__device__ __forceinline__ void wta_step(float x, int i, float& bv, int& best) {
+  if (x > bv) { bv = x; best = i; }          // strict: the lowest position wins ties
+}
+
+__global__ void __launch_bounds__(HN_THREADS)
+k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ hidx, uint32_t* keys, int32_t* counts,
+                     int N, int H, int K, int L, int lg_bin, long long nb) {
+  extern __shared__ __align__(16) unsigned char hn_smem[];
+  float2* tile = reinterpret_cast<float2*>(hn_smem);                  // [32 pairs][H + 1]
+  const int ld = H + 1;
+  unsigned short* fn = reinterpret_cast<unsigned short*>(hn_smem + (((size_t)32 * ld * 8 + 15) & ~(size_t)15));
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nfn = K * L * 8;
+  for (int e = threadIdx.x; e < nfn; e += HN_THREADS) fn[e] = (unsigned short)hidx[e];
+  const int ntiles = (N + HN2_ROWS - 1) / HN2_ROWS;
+  for (int tl = blockIdx.x; tl < ntiles; tl += gridDim.x) {
+    const int j0 = tl * HN2_ROWS;
+    const int rows = min(HN2_ROWS, N - j0);
+    __syncthreads();
+    {
+      const int H4 = H >> 2, total4 = rows * H4;
+      const float4* src = reinterpret_cast<const float4*>(W2 + (size_t)j0 * H);
+      float* tile1 = reinterpret_cast<float*>(tile);
+      for (int e = threadIdx.x; e < total4; e += HN_THREADS) {
+        const float4 x = __ldg(src + e);
+        const int r = e / H4, k = (e - r * H4) << 2;
+        float* d = tile1 + ((size_t)(r & 31) * ld + k) * 2 + (r >> 5);
+        d[0] = x.x; d[2] = x.y; d[4] = x.z; d[6] = x.w;
+      }
+    }
+    __syncthreads();
+    const bool live0 = lane < rows, live1 = lane + 32 < rows;
+    if (live0) {
+      const float2* v = tile + (size_t)lane * ld;
+      for (int t = warp; t < L; t += HN_WARPS) {
+        uint32_t code0 = 0, code1 = 0;
+        for (int k = 0; k < K; ++k) {
+          const uint4 q = *reinterpret_cast<const uint4*>(fn + (size_t)(t * K + k) * 8);
+          const float2 x0 = v[q.x & 0xffffu], x1 = v[q.x >> 16], x2 = v[q.y & 0xffffu], x3 = v[q.y >> 16];
+          const float2 x4 = v[q.z & 0xffffu], x5 = v[q.z >> 16], x6 = v[q.w & 0xffffu], x7 = v[q.w >> 16];
+          float a = x0.x, b = x0.y;
+          int ia = 0, ib = 0;
+          wta_step(x1.x, 1, a, ia); wta_step(x1.y, 1, b, ib);
+          wta_step(x2.x, 2, a, ia); wta_step(x2.y, 2, b, ib);
+          wta_step(x3.x, 3, a, ia); wta_step(x3.y, 3, b, ib);
+          wta_step(x4.x, 4, a, ia); wta_step(x4.y, 4, b, ib);
+          wta_step(x5.x, 5, a, ia); wta_step(x5.y, 5, b, ib);
+          wta_step(x6.x, 6, a, ia); wta_step(x6.y, 6, b, ib);
+          wta_step(x7.x, 7, a, ia); wta_step(x7.y, 7, b, ib);
+          code0 |= (uint32_t)ia << (k * lg_bin);
+          code1 |= (uint32_t)ib << (k * lg_bin);
+        }
+        keys[(size_t)t * N + j0 + lane] = code0;
+        atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code0 + 1, 1);
+        if (live1) {
+          keys[(size_t)t * N + j0 + 32 + lane] = code1;
+          atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code1 + 1, 1);
+        }
+      }
+    }
+  }
+}
+
 // counts[t][0] = 0, counts[t][c + 1] = size of bucket c  ->  inclusive running sum = bucket offsets.
 // Two kernels over chunks of BS_CHUNK counters: the sum of every chunk, then per chunk the sum of the
 // table's earlier chunks plus a scan inside the chunk.
@@ -450,12 +518,26 @@ cudaError_t launch_build_tables(Ctx* c) {
   const long long fn_bytes = (long long)c->KL * c->fn_len * 2;
   const bool fn_smem = fn_bytes <= HN_FN_SMEM_MAX && c->H <= 0x7fff;
   const int smem = tile_bytes + (fn_smem ? (int)fn_bytes : 0);
-  auto kern = fn_smem ? k_hash_neurons<true> : k_hash_neurons<false>;
-  if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const long long smem2_ll = ((32LL * (c->H + 1) * 8 + 15) & ~15LL) + fn_bytes;
+  if (fn_smem && c->cfg.hash_family == DSLIDE_DWTA && c->fn_len == 8 && smem2_ll <= 100 * 1024) {
+    const int smem2 = (int)smem2_ll;
+    if (smem2 > 48 * 1024) {
+      e = cudaFuncSetAttribute(k_hash_neurons_dwta8, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2);
+      if (e != cudaSuccess) return e;
+    }
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_hash_neurons_dwta8, HN_THREADS, smem2);
     if (e != cudaSuccess) return e;
-  }
-  {
+    if (per_sm < 1) per_sm = 1;
+    LaunchScope ls(c, KID_HASH_NEURONS);
+    k_hash_neurons_dwta8<<<c->num_sms * per_sm, HN_THREADS, smem2, c->stream>>>(c->W2, c->hash_idx, c->keysA, c->bucket_off,
+                                                                              c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
+  } else {
+    auto kern = fn_smem ? k_hash_neurons<true> : k_hash_neurons<false>;
+    if (smem > 48 * 1024) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      if (e != cudaSuccess) return e;
+    }
     int per_sm = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, HN_THREADS, smem);
     if (e != cudaSuccess) return e;
