@@ -200,7 +200,7 @@ dslide_status dslide_cum_stats(dslide_ctx* ctx, int64_t out[6], int32_t reset);
 enum {
   DSLIDE_K_FORWARD = 0, DSLIDE_K_ADAM_DENSE, DSLIDE_K_ADAM, DSLIDE_K_DRAW_HASH, DSLIDE_K_HASH_NEURONS,
   DSLIDE_K_BUCKET_SCAN, DSLIDE_K_SORT_HIST, DSLIDE_K_SORT_SCAN, DSLIDE_K_SORT_SCATTER,
-  DSLIDE_K_PREDICT, DSLIDE_K_INIT, DSLIDE_K_COUNT
+  DSLIDE_K_PREDICT, DSLIDE_K_INIT, DSLIDE_K_PLACE_IDS, DSLIDE_K_ORDER_BUCKETS, DSLIDE_K_COUNT
 };
 dslide_status dslide_profile_begin(dslide_ctx* ctx);
 dslide_status dslide_profile_end(dslide_ctx* ctx, double ms[DSLIDE_K_COUNT], int64_t launches[DSLIDE_K_COUNT]);

@@ -213,7 +213,7 @@ def dslide_last_stats(ctx):
 
 
 KERNEL_NAMES = ["forward", "adam_dense", "adam", "draw_hash", "hash_neurons", "bucket_scan", "sort_hist", "sort_scan",
-                "sort_scatter", "predict", "init"]
+                "sort_scatter", "predict", "init", "place_ids", "order_buckets"]
 
 
 def dslide_cum_stats(ctx, reset=False):

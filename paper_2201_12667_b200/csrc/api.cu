@@ -14,6 +14,8 @@ namespace dslide {
 int sort_tile_elems();
 int sort_max_width();
 int bucket_scan_chunk();
+int order_small_max();
+int order_block_max();
 }
 
 using namespace dslide;
@@ -58,7 +60,7 @@ void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->hdr1, c->hdr2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1,
-                  c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part,
+                  c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
                   c->st_dev[0], c->st_dev[1]};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (int b = 0; b < 2; ++b) {
@@ -223,9 +225,17 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     A(own2, N, true);
     A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
     A(keysA, (size_t)c->L * N, false);
-    if (c->sort_passes > 1) { A(keysB, (size_t)c->L * N, false); A(valsA, (size_t)c->L * N, false); }
-    if (c->sort_passes > 2) { A(valsB, (size_t)c->L * N, false); }
-    A(tile_hist, (size_t)c->L * ((size_t)1 << c->sort_width) * c->sort_tiles, false);
+    // codes wider than one radix digit: ids are placed by atomics and ordered inside their buckets, no radix passes
+    c->place_path = c->bits > sort_max_width() ? 1 : 0;
+    if (c->place_path) {
+      A(ord_mid, (size_t)c->L * (N / (order_small_max() + 1) + 1), false);
+      A(ord_big, (size_t)c->L * (N / (order_block_max() + 1) + 1), false);
+      A(ord_cnt, 2, true);
+    } else {
+      if (c->sort_passes > 1) { A(keysB, (size_t)c->L * N, false); A(valsA, (size_t)c->L * N, false); }
+      if (c->sort_passes > 2) { A(valsB, (size_t)c->L * N, false); }
+      A(tile_hist, (size_t)c->L * ((size_t)1 << c->sort_width) * c->sort_tiles, false);
+    }
     A(bucket_part, (size_t)c->L * (size_t)((c->nb + 1 + bucket_scan_chunk() - 1) / bucket_scan_chunk()), false);
   }
 #undef A
@@ -463,6 +473,11 @@ dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, 
     return DSLIDE_OK;
   }
   if (want == 0) return DSLIDE_OK;
+  if (which == DSLIDE_T_BUCKET_IDS && c->place_path && c->ids_ordered_above > 1) {
+    // the step only needs buckets beyond the cap in order; a reader gets every bucket ascending
+    CU(launch_order_buckets(c, 1));
+    c->ids_ordered_above = 1;
+  }
   const TensorRef tr = tensor_ref(c, which);
   if (tr.pitch) CU(cudaMemcpy2DAsync(host_dst, sizeof(float), tr.ptr, (size_t)tr.pitch, sizeof(float), (size_t)want / sizeof(float),
                                      cudaMemcpyDeviceToHost, c->stream));

@@ -73,7 +73,7 @@ struct Ctx;
 
 // Kernel ids for the per-kernel timing (must match the DSLIDE_K_* enum of the C ABI).
 enum { KID_FORWARD = 0, KID_ADAM_DENSE, KID_ADAM, KID_DRAW_HASH, KID_HASH_NEURONS, KID_BUCKET_SCAN, KID_SORT_HIST,
-       KID_SORT_SCAN, KID_SORT_SCATTER, KID_PREDICT, KID_INIT, KID_COUNT };
+       KID_SORT_SCAN, KID_SORT_SCATTER, KID_PREDICT, KID_INIT, KID_PLACE_IDS, KID_ORDER_BUCKETS, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event pair around it.
 struct LaunchScope {
@@ -86,6 +86,7 @@ struct LaunchScope {
 cudaError_t launch_init_gauss(Ctx* c, float* w, int64_t n, uint64_t stream_id);
 cudaError_t launch_draw_hash(Ctx* c, int64_t r);
 cudaError_t launch_build_tables(Ctx* c);
+cudaError_t launch_order_buckets(Ctx* c, int min_n);
 cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
                                  const float* vals, const int32_t* label_ptr, const int32_t* labels);
 cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
@@ -119,7 +120,7 @@ struct Ctx {
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;         // per row of W1 / W2: which samples of the batch touch it
-  int32_t *own1, *own2;            // the distinct touched rows of W1 / W2, in no particular order
+  int2 *own1, *own2;               // the distinct touched rows of W1 / W2 with their first-touching sample, in no particular order
   int32_t* hot_rows;               // rows touched by many samples: row of W2, or ~row of W1
   int32_t* med_rows;               // rows touched by more than ROW_SLOTS samples, same encoding
   float* hot_part;                 // [HOT_CAP][HOT_SLICES][H + 4] slice sums of those rows
@@ -131,6 +132,10 @@ struct Ctx {
   int32_t *valsA, *valsB;
   int32_t* tile_hist;
   int32_t* bucket_part;   // per table: sums of chunks of bucket counters (bucket offset scan)
+  int place_path;         // 1: codes wider than a radix digit: ids placed by atomics, then ordered inside buckets
+  int2 *ord_mid, *ord_big; // (table, bucket) of the buckets too large to order in registers / in shared memory
+  int* ord_cnt;           // lengths of those two lists
+  int ids_ordered_above;  // place path: buckets with more ids than this are in ascending order (1 = every bucket)
   int sort_passes, sort_width, sort_tiles;
 
   // forward kernel layout

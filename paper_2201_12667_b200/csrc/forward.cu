@@ -39,7 +39,8 @@ struct FwdParams {
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;
   RowHdr *hdr1, *hdr2;
-  int32_t *own1, *own2, *hot_rows, *med_rows;
+  int2 *own1, *own2;
+  int32_t *hot_rows, *med_rows;
   DevState* st;
   int32_t* out_ids;
   float* out_scores;
@@ -102,9 +103,9 @@ __device__ __forceinline__ void list_row(const FwdParams& p, uint32_t* cnt, int 
 
 // Second half of handing a touched row to the update kernel, once the row's touch counter has answered
 // (nth = touches before this one): the (sample, coefficient) pair goes into the row's slot nth, or, past the
-// slots, the sample's bit into the row's mask; the first toucher enters the row in the list of distinct rows
-// (positions handed out per warp).  Called by whole warps; `live` tells whether this thread has a touch.
-__device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int32_t* own,
+// slots, the sample's bit into the row's mask; the first toucher enters (row, its own sample) in the list of
+// distinct rows (positions handed out per warp), so that the update kernel can fetch that sample's row at once.  Called by whole warps; `live` tells whether this thread has a touch.
+__device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int2* own,
                                              unsigned int* n_own, int row, int code, unsigned nth, int s, float coef) {
   const int lane = threadIdx.x & 31;
   bool first = false;
@@ -119,7 +120,7 @@ __device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowH
     unsigned base = 0;
     if (lane == 0) base = atomicAdd(n_own, (unsigned)__popc(fm));
     base = __shfl_sync(FULLM, base, 0);
-    if (first) own[base + __popc(fm & ((1u << lane) - 1u))] = row;
+    if (first) own[base + __popc(fm & ((1u << lane) - 1u))] = make_int2(row, s);
   }
 }
 

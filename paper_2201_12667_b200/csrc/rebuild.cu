@@ -300,7 +300,9 @@ __global__ void __launch_bounds__(BS_THREADS) k_bucket_sums(const int32_t* off, 
   }
 }
 
-__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks) {
+// exclusive != 0: every counter is replaced by the sum of the counters before it instead of the sum up to and including it.
+__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks,
+                                                            int exclusive) {
   __shared__ int sh[BS_THREADS / 32 + 1];
   int32_t* o = off + (size_t)blockIdx.y * (size_t)(nb + 1);
   const long long n = nb + 1, base = (long long)blockIdx.x * BS_CHUNK;
@@ -340,7 +342,7 @@ __global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long l
       if (lane >= d) incl += x;
     }
     const long long i = wbase + u * 32 + lane;
-    if (i < n) o[i] = run + incl;
+    if (i < n) o[i] = run + incl - (exclusive ? v[u] : 0);
     run += __shfl_sync(0xffffffffu, incl, 31);
   }
 }
@@ -510,6 +512,140 @@ k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_o
   }
 }
 
+// ------------------------------------------------------------------ wide codes: place, then order inside buckets
+// With codes wider than one radix digit the buckets are small (a few ids on average), and sorting the whole table
+// twice is a detour.  Instead every id reserves its slot with an atomic add on its bucket's offset word -- stored
+// one place up and started at the bucket's start, the word ends as the next bucket's start, i.e. exactly the final
+// offset array -- and the ids of each bucket are then put in ascending order where they stand: in registers for
+// buckets of up to ORD_SMALL ids, by a block-wide sort in shared memory up to ORD_BLOCK, and for a larger bucket by
+// one ordered pass over the table's codes that writes the matching ids out again.
+constexpr int ORD_SMALL = 16;
+constexpr int ORD_BLOCK = 4096;
+constexpr int ORD_THREADS = 256;
+
+__global__ void __launch_bounds__(256) k_place_ids(const uint32_t* keys, int32_t* off, int32_t* ids, int N, long long nb) {
+  const int t = blockIdx.y;
+  const uint32_t* k = keys + (size_t)t * N;
+  int32_t* o = off + (size_t)t * (size_t)(nb + 1);
+  int32_t* out = ids + (size_t)t * N;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < N; j += gridDim.x * blockDim.x) {
+    const int slot = atomicAdd(o + k[j] + 1, 1);
+    out[slot] = j;
+  }
+}
+
+// Sorts n <= M ids in place with an odd-even transposition network (fully unrolled: the ids stay in registers).
+template <int M>
+__device__ __forceinline__ void order_in_registers(int32_t* p, int n) {
+  int a[M];
+#pragma unroll
+  for (int i = 0; i < M; ++i) a[i] = i < n ? p[i] : 0x7fffffff;
+#pragma unroll
+  for (int round = 0; round < M; ++round) {
+#pragma unroll
+    for (int i = round & 1; i + 1 < M; i += 2) {
+      const int lo = min(a[i], a[i + 1]), hi = max(a[i], a[i + 1]);
+      a[i] = lo; a[i + 1] = hi;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < M; ++i)
+    if (i < n) p[i] = a[i];
+}
+
+// One thread per bucket.  cnt[0] / cnt[1]: lengths of the lists of buckets left to the block-wide and to the ordered-
+// pass kernels.
+// Only buckets of more than min_n ids are touched.
+__global__ void __launch_bounds__(256) k_order_small(const int32_t* off, int32_t* ids, int N, long long nb, int2* mid,
+                                                     int2* big, int* cnt, int min_n) {
+  const int t = blockIdx.y;
+  const int32_t* o = off + (size_t)t * (size_t)(nb + 1);
+  int32_t* out = ids + (size_t)t * N;
+  for (long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x; c < nb; c += (long long)gridDim.x * blockDim.x) {
+    const int beg = o[c], n = o[c + 1] - beg;
+    if (n <= min_n) continue;
+    if (n <= 4) order_in_registers<4>(out + beg, n);
+    else if (n <= 8) order_in_registers<8>(out + beg, n);
+    else if (n <= ORD_SMALL) order_in_registers<ORD_SMALL>(out + beg, n);
+    else if (n <= ORD_BLOCK) {
+      mid[atomicAdd(cnt, 1)] = make_int2(t, (int)c);
+    } else {
+      big[atomicAdd(cnt + 1, 1)] = make_int2(t, (int)c);
+    }
+  }
+}
+
+// Buckets of ORD_SMALL + 1 .. ORD_BLOCK ids: a block loads one, sorts it in shared memory (bitonic) and writes it back.
+__global__ void __launch_bounds__(ORD_THREADS) k_order_mid(const int32_t* off, int32_t* ids, int N, long long nb, const int2* mid,
+                                                           const int* cnt) {
+  __shared__ int sm[ORD_BLOCK];
+  const int nmid = cnt[0];
+  for (int q = blockIdx.x; q < nmid; q += gridDim.x) {
+    const int2 tc = mid[q];
+    const int32_t* o = off + (size_t)tc.x * (size_t)(nb + 1);
+    int32_t* out = ids + (size_t)tc.x * N;
+    const int beg = o[tc.y], n = o[tc.y + 1] - beg;
+    int n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n2; i += ORD_THREADS) sm[i] = i < n ? out[beg + i] : 0x7fffffff;
+    __syncthreads();
+    for (int k = 2; k <= n2; k <<= 1)
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int i = threadIdx.x; i < n2; i += ORD_THREADS) {
+          const int x = i ^ j;
+          if (x > i) {
+            const int a = sm[i], b = sm[x];
+            const bool asc = (i & k) == 0;
+            if ((a > b) == asc) { sm[i] = b; sm[x] = a; }
+          }
+        }
+        __syncthreads();
+      }
+    for (int i = threadIdx.x; i < n; i += ORD_THREADS) out[beg + i] = sm[i];
+  }
+}
+
+// Larger buckets: the ids of bucket c in ascending order are the j, ascending, whose code is c.
+__global__ void __launch_bounds__(ORD_THREADS) k_order_big(const uint32_t* keys, const int32_t* off, int32_t* ids, int N,
+                                                           long long nb, const int2* big, const int* cnt) {
+  __shared__ int sh[ORD_THREADS / 32 + 1];
+  const int nbig = cnt[1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int q = blockIdx.x; q < nbig; q += gridDim.x) {
+    const int2 tc = big[q];
+    const uint32_t* k = keys + (size_t)tc.x * N;
+    int32_t* out = ids + (size_t)tc.x * N + off[(size_t)tc.x * (size_t)(nb + 1) + tc.y];
+    int run = 0;
+    for (int base = 0; base < N; base += ORD_THREADS) {
+      const int j = base + threadIdx.x;
+      const bool hit = j < N && k[j] == (uint32_t)tc.y;
+      const unsigned m = __ballot_sync(0xffffffffu, hit);
+      __syncthreads();
+      if (lane == 0) sh[warp] = __popc(m);
+      __syncthreads();
+      int before = 0, total = 0;
+      for (int w = 0; w < ORD_THREADS / 32; ++w) { const int x = sh[w]; if (w < warp) before += x; total += x; }
+      if (hit) out[run + before + __popc(m & ((1u << lane) - 1u))] = j;
+      run += total;
+    }
+  }
+}
+
+// Puts the ids of every bucket with more than min_n ids in ascending order (place path only).
+cudaError_t launch_order_buckets(Ctx* c, int min_n) {
+  if (min_n < 1) min_n = 1;
+  cudaError_t e = cudaMemsetAsync(c->ord_cnt, 0, 2 * sizeof(int), c->stream);
+  if (e != cudaSuccess) return e;
+  LaunchScope ls(c, KID_ORDER_BUCKETS);
+  dim3 grid((unsigned)min((long long)((c->nb + 255) / 256), 2048LL), c->L);
+  k_order_small<<<grid, 256, 0, c->stream>>>(c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_mid, c->ord_big, c->ord_cnt, min_n);
+  k_order_mid<<<c->num_sms * 4, ORD_THREADS, 0, c->stream>>>(c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_mid, c->ord_cnt);
+  k_order_big<<<c->num_sms, ORD_THREADS, 0, c->stream>>>(c->keysA, c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_big,
+                                                          c->ord_cnt);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_build_tables(Ctx* c) {
   const size_t off_bytes = (size_t)c->L * (size_t)(c->nb + 1) * sizeof(int32_t);
   cudaError_t e = cudaMemsetAsync(c->bucket_off, 0, off_bytes, c->stream);
@@ -553,9 +689,23 @@ cudaError_t launch_build_tables(Ctx* c) {
     dim3 grid(nchunks, c->L);
     LaunchScope ls(c, KID_BUCKET_SCAN);
     k_bucket_sums<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
-    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
+    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks, c->place_path);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+  if (c->place_path) {
+    {
+      LaunchScope ls(c, KID_PLACE_IDS);
+      dim3 grid((unsigned)min((long long)(c->N + 255) / 256, 1024LL), c->L);
+      k_place_ids<<<grid, 256, 0, c->stream>>>(c->keysA, c->bucket_off, c->bucket_ids, c->N, c->nb);
+    }
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    // A query reads a whole bucket unless it holds more than `cap` ids, and the union of the buckets is put in
+    // order afterwards anyway: only buckets larger than the cap must be in ascending order for the step.  The
+    // smaller ones are ordered when the table is read back (launch_order_buckets(c, 1)).
+    c->ids_ordered_above = c->cap;
+    return launch_order_buckets(c, c->cap);
+  }
 
   if ((e = cudaFuncSetAttribute(k_sort_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, SORT_SMEM)) != cudaSuccess) return e;
   const uint32_t* kin = c->keysA;
@@ -591,6 +741,8 @@ cudaError_t launch_build_tables(Ctx* c) {
 }
 
 int sort_tile_elems() { return SORT_TILE; }
+int order_small_max() { return ORD_SMALL; }
+int order_block_max() { return ORD_BLOCK; }
 int bucket_scan_chunk() { return BS_CHUNK; }
 int sort_max_width() { return SORT_MAX_WIDTH; }
 

@@ -42,7 +42,8 @@ struct UpdParams {
   const float* vals;
   uint32_t *mask1, *mask2;
   RowHdr *hdr1, *hdr2;
-  const int32_t *own1, *own2, *hot_rows, *med_rows;
+  const int2 *own1, *own2;
+  const int32_t *hot_rows, *med_rows;
   float* hot_part;
   int* hot_done;
   DevState* st;
@@ -478,7 +479,8 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
     // ---- ordinary rows: ticket k takes rows k, k + n_norm, k + 2 n_norm, ... of the concatenated lists (rows of
     //      W2, then rows of W1), so that neighbours in a list (often alike in cost) go to different warps ----
     const int k = t - n_hot_items - n_med;
-    int myrow = 0, myidx = nrows;
+    int2 myrow = make_int2(0, 0);        // (row, the sample that touched it first = the sample of slot 0)
+    int myidx = nrows;
     if (lane < UPD_TROWS) {
       myidx = k + lane * n_norm;
       if (myidx < nrows) myrow = myidx < n2 ? p.own2[myidx] : p.own1[myidx - n2];
@@ -493,29 +495,27 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
         const int idx = __shfl_sync(FULL, myidx, b0 + q);
         live[q] = idx < nrows;
         w2[q] = idx < n2;
-        rr[q] = __shfl_sync(FULL, myrow, b0 + q);
+        rr[q] = __shfl_sync(FULL, myrow.x, b0 + q);
+        const int s0 = __shfl_sync(FULL, myrow.y, b0 + q);
         tt[q] = 0;
         hv[q] = make_int2(0, 0);
         if (live[q]) {
           const Side sd = make_side(p, w2[q]);
           hv[q] = load_hdr(sd.hdr + rr[q], lane);
+          load_row<NCH>(sd.src, (size_t)s0, H, H4, lane, x[q]);      // the row of slot 0's sample: all a once-touched row needs
           load_row<NCH>(sd.W, (size_t)rr[q], H, H4, lane, w[q]);
           load_row<NCH>(sd.M, (size_t)rr[q], H, H4, lane, m[q]);
           load_row<NCH>(sd.V, (size_t)rr[q], H, H4, lane, v[q]);
         }
       }
-      // second level: the one sample's row for rows touched once
 #pragma unroll
       for (int q = 0; q < G; ++q)
         if (live[q]) {
-          const Side sd = make_side(p, w2[q]);
           const unsigned cv = (unsigned)__shfl_sync(FULL, hv[q].x, 0);
           sl[q] = hdr_slots(hv[q]);
           // a listed row is summed by its own ticket (and its count may already be back at zero)
           skip[q] = (cv & (CNT_HOT | CNT_MED)) != 0u || (cv & CNT_MASK) == 0u;
           tt[q] = (int)(cv & CNT_MASK);
-          const int s0 = __shfl_sync(FULL, sl[q].x, 0);
-          if (tt[q] == 1 && !skip[q]) load_row<NCH>(sd.src, (size_t)s0, H, H4, lane, x[q]);
         }
 #pragma unroll
       for (int q = 0; q < G; ++q)

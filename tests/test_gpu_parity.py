@@ -111,6 +111,34 @@ def test_tables_bit_exact(family, K, L, N, H):
         pr.close()
 
 
+@pytest.mark.parametrize("K", [4, 6])
+def test_tables_with_crowded_buckets(K):
+    """Codes wider than one radix digit take the place-then-order table build.  5,000 all-zero rows land in one
+    bucket per table (larger than a block sorts: the ordered pass over the codes), 600 copies of one random row in
+    another (the block-wide sort), the other rows in buckets of a few ids (ordered in registers)."""
+    N, H = 9000, 64
+    pr = Pair(D=50, H=H, N=N, family=DWTA, K=K, L=3, bucket_cap=16, max_batch=8)
+    try:
+        rng = np.random.default_rng(9)
+        W2 = pr.o.get("W2").reshape(N, H)
+        perm = rng.permutation(N)
+        W2[perm[:5000]] = 0.0
+        W2[perm[5000:5600]] = rng.standard_normal(H).astype(np.float32)
+        pr.o.set("W2", W2)
+        pr.o.build_tables()
+        pr.push_state()
+        for trial in range(2):
+            off_o = pr.o.get("bucket_off").reshape(3, -1)
+            assert np.diff(off_o, axis=1).max() >= 5000
+            assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_off"), pr.o.get("bucket_off"))
+            assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_ids"), pr.o.get("bucket_ids"))
+            ds.dslide_rebuild_tables(pr.ctx)
+            ds.dslide_sync(pr.ctx)
+            pr.o.rebuild_tables()
+    finally:
+        pr.close()
+
+
 def test_initial_weights_have_the_stated_distribution():
     pr = Pair(D=300, H=64, N=4000, family=DWTA, K=2, L=3, bucket_cap=8, max_batch=8, init_std=0.02,
               sync_weights=False)
