@@ -91,7 +91,7 @@ __device__ __forceinline__ Side make_side(const UpdParams& p, bool w2) {
 
 // Coefficient of (row, sample s): the error of neuron `row` in sample s, or the value of feature
 // `row` in sample s.  Both lists are ascending, so a binary search finds it.
-__device__ __forceinline__ float find_coef(const UpdParams& p, const Side& sd, const int* sm_rowptr, int row, int s) {
+__device__ __forceinline__ float find_coef(const UpdParams& p, const Side& sd, const int* rowptr, int row, int s) {
   if (sd.is_w2) {
     const int32_t* ids = p.act_ids + (size_t)s * p.act_stride;
     const int n = p.act_cnt[s];
@@ -99,8 +99,8 @@ __device__ __forceinline__ float find_coef(const UpdParams& p, const Side& sd, c
     while (lo < hi) { int mid = (lo + hi) >> 1; if (__ldg(ids + mid) < row) lo = mid + 1; else hi = mid; }
     return (lo < n && __ldg(ids + lo) == row) ? __ldg(p.act_g + (size_t)s * p.act_stride + lo) : 0.f;
   }
-  int lo = sm_rowptr[s];
-  const int end = sm_rowptr[s + 1];
+  int lo = __ldg(rowptr + s);
+  const int end = __ldg(rowptr + s + 1);
   int hi = end;
   while (lo < hi) { int mid = (lo + hi) >> 1; if (__ldg(p.col_idx + mid) < row) lo = mid + 1; else hi = mid; }
   return (lo < end && __ldg(p.col_idx + lo) == row) ? __ldg(p.vals + lo) : 0.f;
@@ -193,7 +193,7 @@ __device__ __forceinline__ void sum_slots(const Side& sd, int2 sl, int total, in
 // [w0, w1): the samples of the slots and of the mask, ascending.  Up to 32 samples at a time are listed
 // in the warp's scratch, their coefficients looked up in parallel, then added in order.  Clears the mask.
 template <int NCH>
-__device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, const int* sm_rowptr, int row,
+__device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, const int* rowptr, int row,
                                            int slot_s, int w0, int w1, int* scr, float4 (&acc)[NCH], float& csum,
                                            int H, int H4, int lane) {
   uint32_t* mrow = sd.mask + (size_t)row * p.Wd;
@@ -217,7 +217,7 @@ __device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, c
       if (fill + nb > 32) {
         __syncwarp();
         const int s_mine = lane < fill ? scr[lane] : 0;
-        const float g_mine = lane < fill ? find_coef(p, sd, sm_rowptr, row, s_mine) : 0.f;
+        const float g_mine = lane < fill ? find_coef(p, sd, rowptr, row, s_mine) : 0.f;
         accumulate_list<NCH>(acc, csum, fill, s_mine, g_mine, sd.src, H, H4, lane);
         fill = 0;
         __syncwarp();
@@ -229,7 +229,7 @@ __device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, c
   __syncwarp();
   if (fill > 0) {
     const int s_mine = lane < fill ? scr[lane] : 0;
-    const float g_mine = lane < fill ? find_coef(p, sd, sm_rowptr, row, s_mine) : 0.f;
+    const float g_mine = lane < fill ? find_coef(p, sd, rowptr, row, s_mine) : 0.f;
     accumulate_list<NCH>(acc, csum, fill, s_mine, g_mine, sd.src, H, H4, lane);
   }
   __syncwarp();
@@ -350,7 +350,7 @@ __device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
 // sum goes to scratch memory; the warp that completes the row's last slice adds the slices in slice
 // order (so the result does not depend on which warp that is), applies Adam and resets the row's state.
 template <int NCH>
-__device__ __forceinline__ void hot_item(const UpdParams& p, const int* sm_rowptr, int item, int nwB, int* scr, int H,
+__device__ __forceinline__ void hot_item(const UpdParams& p, const int* rowptr, int item, int nwB, int* scr, int H,
                                          int H4, int lane) {
   const int hrow = item / HOT_SLICES, slice = item - hrow * HOT_SLICES;
   const int code = p.hot_rows[hrow];
@@ -364,7 +364,7 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* sm_rowpt
   for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   float csum = 0.f;
   const int2 hv = load_hdr(sd.hdr + row, lane);
-  sum_masked<NCH>(p, sd, sm_rowptr, row, hdr_slots(hv).x, w0, w1, scr, acc, csum, H, H4, lane);
+  sum_masked<NCH>(p, sd, rowptr, row, hdr_slots(hv).x, w0, w1, scr, acc, csum, H, H4, lane);
   const int ld = H + 4;
   float* part = p.hot_part + (size_t)hrow * HOT_SLICES * ld;
   float4* mine = reinterpret_cast<float4*>(part + (size_t)slice * ld);
@@ -409,7 +409,7 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* sm_rowpt
 // mask (ascending samples), applies Adam and resets the row's state.  Rows that went on to the hot list are
 // summed in slices instead and skipped here.
 template <int NCH>
-__device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_rowptr, int idx, int nwB, int* scr, int H,
+__device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowptr, int idx, int nwB, int* scr, int H,
                                             int H4, int lane) {
   const int code = p.med_rows[idx];
   const bool w2 = code >= 0;
@@ -426,20 +426,20 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* sm_ro
 #pragma unroll
   for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   float csum = 0.f;
-  sum_masked<NCH>(p, sd, sm_rowptr, row, slot_s, 0, nwB, scr, acc, csum, H, H4, lane);
+  sum_masked<NCH>(p, sd, rowptr, row, slot_s, 0, nwB, scr, acc, csum, H, H4, lane);
   adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
   finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
 }
 
 // Work is handed out in tickets from one counter: first the slices of the hot rows (the longest items), then
-// the listed rows with more than ROW_SLOTS touches, then the ordinary rows, UPD_TROWS per ticket.
-constexpr int UPD_TROWS = 8;
+// the listed rows with more than ROW_SLOTS touches, then the ordinary rows, UPD_TROWS per ticket (small tickets keep the tail of the kernel short).
+constexpr int UPD_TROWS = 4;
 
 template <int NCH, int G>
 __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
   extern __shared__ __align__(16) unsigned char upd_smem[];
-  int* sm_rowptr = reinterpret_cast<int*>(upd_smem);                               // [B + 1]
-  float* sm_part = reinterpret_cast<float*>(upd_smem + (((size_t)p.B + 1 + 3) & ~(size_t)3) * 4);   // [UPD_WARPS * 32]
+  const int* rowptr = p.row_ptr;      // the batch's row offsets (read through the read-only path where needed)
+  float* sm_part = reinterpret_cast<float*>(upd_smem);   // [UPD_WARPS * 32]
   __shared__ int scratch[UPD_WARPS][64];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -447,8 +447,6 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
   const int naux = (H + 31) >> 5;
   if ((int)blockIdx.x < naux) { aux_block(p, (int)blockIdx.x, sm_part); return; }
 
-  for (int i = tid; i <= B; i += UPD_THREADS) sm_rowptr[i] = p.row_ptr[i];
-  __syncthreads();
 
   const int n2 = p.dense ? 0 : (int)p.st->n_own[p.parity][0];
   const int n1 = (int)p.st->n_own[p.parity][1];
@@ -473,8 +471,8 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
     if (t >= n_tickets) break;
     cur = __shfl_sync(FULL, nxt, 0);
     if (lane == 0 && cur < n_tickets) nxt = nwarps + (int)atomicAdd(ticket, 1u);
-    if (t < n_hot_items) { hot_item<NCH>(p, sm_rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
-    if (t < n_hot_items + n_med) { medium_item<NCH>(p, sm_rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
+    if (t < n_hot_items) { hot_item<NCH>(p, rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
+    if (t < n_hot_items + n_med) { medium_item<NCH>(p, rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
 
     // ---- ordinary rows: ticket k takes rows k, k + n_norm, k + 2 n_norm, ... of the concatenated lists (rows of
     //      W2, then rows of W1), so that neighbours in a list (often alike in cost) go to different warps ----
@@ -533,7 +531,7 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
           } else if (tt[q] <= ROW_SLOTS) {
             sum_slots<NCH>(sd, sl[q], tt[q], scratch[warp], acc, csum, H, H4, lane);
           } else {      // more touches than slots, yet not listed (the list was full)
-            sum_masked<NCH>(p, sd, sm_rowptr, rr[q], sl[q].x, 0, nwB, scratch[warp], acc, csum, H, H4, lane);
+            sum_masked<NCH>(p, sd, rowptr, rr[q], sl[q].x, 0, nwB, scratch[warp], acc, csum, H, H4, lane);
           }
           adam_store<NCH>(p, sd, (size_t)rr[q], w[q], m[q], v[q], acc, H, H4, lane);
           finish_hdr(p, sd.hdr + rr[q], w2[q], hv[q], csum, lane);
@@ -613,7 +611,7 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  const int smem = (((batch + 1 + 3) & ~3) + UPD_WARPS * 32) * 4;
+  const int smem = UPD_WARPS * 32 * 4;
   const int nch = (c->H / 4 + 31) / 32;
   if (nch <= 1) return launch_k_update<1, 2>(c, p, smem);
   if (nch <= 2) return launch_k_update<2, 2>(c, p, smem);
