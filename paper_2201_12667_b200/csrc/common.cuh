@@ -69,6 +69,25 @@ struct __align__(16) RowHdr {
 };
 static_assert(sizeof(RowHdr) == 64, "the row record is one 64-byte line");
 
+// Programmatic dependent launch: a kernel launched with launch_dependent() may become resident while the kernel
+// before it in the stream is still running; it must not touch anything that kernel reads or writes before
+// griddep_wait(), which returns once that kernel has completed and its writes are visible.
+// griddep_launch_dependents() tells the runtime that the next kernel may start to be placed.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 struct Ctx;
 
 // Kernel ids for the per-kernel timing (must match the DSLIDE_K_* enum of the C ABI).

@@ -243,6 +243,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   int lbeg = 0, nlab = 0;
   if (MODE == 0) { lbeg = p.label_ptr[s]; nlab = p.label_ptr[s + 1] - lbeg; }
 
+  griddep_launch_dependents();       // the update kernel may be placed as blocks of this one leave
   if (tid == 0) {
     sh_misc[24] = 0;                 // bucket entries fetched by this sample
     mbar_init(sh_bar, 1);
@@ -264,12 +265,10 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   // ---- hidden layer: bias, then one fused multiply-add per nonzero in stored order, ReLU.  The rows of W1 of a
   //      chunk of nonzeros are fetched together into shared memory; the column ids are checked on the way
   //      (in range, ascending) ----
+  //      Up to here, and through the first chunk's column ids and values, only the caller's batch is read: the
+  //      kernel may run that far while the previous step's update kernel is still finishing (griddep_wait).
   float acc[MAX_KPT];
-#pragma unroll
-  for (int u = 0; u < MAX_KPT; ++u) {
-    const int k = tid + u * FWD_THREADS;
-    acc[u] = k < H ? p.b1[k] : 0.f;
-  }
+  bool waited = false;
   const int R = p.hid_rows;
   for (int c0 = 0; c0 < nnz && !bad; c0 += R) {       // `bad` is uniform over the block here
     const int nr = min(R, nnz - c0);
@@ -283,6 +282,15 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
     bad = __syncthreads_or(bad);
     if (bad) break;
+    if (!waited) {
+      griddep_wait();
+      waited = true;
+#pragma unroll
+      for (int u = 0; u < MAX_KPT; ++u) {
+        const int k = tid + u * FWD_THREADS;
+        acc[u] = k < H ? p.b1[k] : 0.f;
+      }
+    }
     {
       float4* st4 = reinterpret_cast<float4*>(stage);
       const int total4 = nr * H4;
@@ -314,6 +322,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
     }
     __syncthreads();
+  }
+  if (!waited) {                     // no nonzeros, or a bad column id: nothing of the model has been read yet
+    griddep_wait();
+#pragma unroll
+    for (int u = 0; u < MAX_KPT; ++u) {
+      const int k = tid + u * FWD_THREADS;
+      acc[u] = k < H ? p.b1[k] : 0.f;
+    }
   }
   if (bad || too_many_labels) {
     skip_sample<MODE>(p, s, (!bad && too_many_labels) ? DSLIDE_ERR_OVERFLOW : DSLIDE_ERR_BAD_INDEX);
@@ -897,7 +913,8 @@ cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, cons
   FwdParams p = make_params(c, batch, row_ptr, col_idx, vals, label_ptr, labels);
   {
     LaunchScope ls(c, KID_FORWARD);
-    k_forward<0><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+    cudaError_t e = launch_dependent(k_forward<0>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p);
+    if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }

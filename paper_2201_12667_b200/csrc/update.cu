@@ -445,6 +445,10 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = p.H, H4 = H >> 2, B = p.B;
   const int naux = (H + 31) >> 5;
+  // the next step's forward kernel may be placed as blocks of this one leave; everything this kernel reads was
+  // written by the forward kernel before it
+  griddep_launch_dependents();
+  griddep_wait();
   if ((int)blockIdx.x < naux) { aux_block(p, (int)blockIdx.x, sm_part); return; }
 
 
@@ -582,7 +586,8 @@ static cudaError_t launch_k_update(Ctx* c, const UpdParams& p, int smem) {
   int nblocks = c->num_sms * (per_sm > 0 ? per_sm : 1);
   if (nblocks < naux + 1) nblocks = naux + 1;
   LaunchScope ls(c, KID_ADAM);
-  k_update<NCH, G><<<nblocks, UPD_THREADS, smem, c->stream>>>(p);
+  e = launch_dependent(k_update<NCH, G>, dim3(nblocks), dim3(UPD_THREADS), (size_t)smem, c->stream, p);
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 
