@@ -711,16 +711,21 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   }
   __syncthreads();
 
-  // ---- the W2 side of the hand-off: the touch counters of the first FWD_THREADS active rows are asked now and
-  //      answered while the back-propagation below runs ----
-  int jj0 = 0;
-  unsigned nth0 = 0u;
-  float ga0 = 0.f;
-  const bool live0 = !dense && tid < na;
-  if (live0) {
-    jj0 = idp[tid];
-    ga0 = gp[tid];
-    nth0 = atomicAdd(&p.hdr2[jj0].cnt, 1u) & CNT_MASK;
+  // ---- the W2 side of the hand-off: the touch counters of the first HO_PER * FWD_THREADS active rows are asked now
+  //      and answered while the back-propagation below runs ----
+  constexpr int HO_PER = 4;
+  int jj0[HO_PER];
+  unsigned nth0[HO_PER];
+  float ga0[HO_PER];
+#pragma unroll
+  for (int u = 0; u < HO_PER; ++u) {
+    const int a = tid + u * FWD_THREADS;
+    jj0[u] = 0; nth0[u] = 0u; ga0[u] = 0.f;
+    if (!dense && a < na) {
+      jj0[u] = idp[a];
+      ga0[u] = gp[a];
+      nth0[u] = atomicAdd(&p.hdr2[jj0[u]].cnt, 1u) & CNT_MASK;
+    }
   }
 
   // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update).  A thread
@@ -785,8 +790,12 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
   }
   if (!dense) {
-    finish_touch(p, live0, p.hdr2 + jj0, p.mask2 + (size_t)jj0 * p.Wd, p.own2, &p.st->n_own[p.parity][0], jj0, jj0, nth0, s, ga0);
-    for (int a0 = FWD_THREADS; a0 < na; a0 += FWD_THREADS) {
+#pragma unroll
+    for (int u = 0; u < HO_PER; ++u)
+      if (u * FWD_THREADS < na)            // uniform over the block
+        finish_touch(p, tid + u * FWD_THREADS < na, p.hdr2 + jj0[u], p.mask2 + (size_t)jj0[u] * p.Wd, p.own2,
+                     &p.st->n_own[p.parity][0], jj0[u], jj0[u], nth0[u], s, ga0[u]);
+    for (int a0 = HO_PER * FWD_THREADS; a0 < na; a0 += FWD_THREADS) {
       const int a = a0 + tid;
       const bool live = a < na;
       int jj = 0;

@@ -260,7 +260,9 @@ __device__ __forceinline__ void adam_store(const UpdParams& p, const Side& sd, s
       adam1(w[q].y, m[q].y, v[q].y, g[q].y, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
       adam1(w[q].z, m[q].z, v[q].z, g[q].z, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
       adam1(w[q].w, m[q].w, v[q].w, g[q].w, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
-      w4[c] = w[q]; m4[c] = m[q]; v4[c] = v[q];
+      w4[c] = w[q];
+      __stcs(m4 + c, m[q]);      // the moments are not read again before the next update of this row
+      __stcs(v4 + c, v[q]);
     }
   }
 }
