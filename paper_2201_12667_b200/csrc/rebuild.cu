@@ -222,7 +222,13 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
   unsigned short* fn = reinterpret_cast<unsigned short*>(hn_smem + (((size_t)32 * ld * 8 + 15) & ~(size_t)15));
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nfn = K * L * 8;
-  for (int e = threadIdx.x; e < nfn; e += HN_THREADS) fn[e] = (unsigned short)hidx[e];
+  // Inside a tile coordinate k sits at place (k / 4) + (H / 4) * (k % 4): the four components of a 16-byte global
+  // load then go to four distant places and a warp's stores spread over the banks.  The function table holds places.
+  const int Hq = H >> 2;
+  for (int e = threadIdx.x; e < nfn; e += HN_THREADS) {
+    const int k = hidx[e];
+    fn[e] = (unsigned short)((k >> 2) + Hq * (k & 3));
+  }
   const int ntiles = (N + HN2_ROWS - 1) / HN2_ROWS;
   for (int tl = blockIdx.x; tl < ntiles; tl += gridDim.x) {
     const int j0 = tl * HN2_ROWS;
@@ -234,9 +240,9 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
       float* tile1 = reinterpret_cast<float*>(tile);
       for (int e = threadIdx.x; e < total4; e += HN_THREADS) {
         const float4 x = __ldg(src + e);
-        const int r = e / H4, k = (e - r * H4) << 2;
-        float* d = tile1 + ((size_t)(r & 31) * ld + k) * 2 + (r >> 5);
-        d[0] = x.x; d[2] = x.y; d[4] = x.z; d[6] = x.w;
+        const int r = e / H4, c4 = e - r * H4;
+        float* d = tile1 + ((size_t)(r & 31) * ld + c4) * 2 + (r >> 5);
+        d[0] = x.x; d[2 * H4] = x.y; d[4 * H4] = x.z; d[6 * H4] = x.w;
       }
     }
     __syncthreads();
