@@ -531,15 +531,48 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   const float* zp = small ? sh_z : p.act_z + (size_t)s * p.act_stride;
   const float* gp = small ? sh_z : p.act_g + (size_t)s * p.act_stride;
 
+  // ---- positions of the sample's distinct labels inside the active set (needed while the rows are staged) ----
+  if (MODE == 0) {
+    for (int i = tid; i < nlab; i += FWD_THREADS) {
+      int y = p.labels[lbeg + i];
+      bool first = true;
+      for (int q = 0; q < i; ++q) first = first && (p.labels[lbeg + q] != y);
+      int pos = y;
+      if (!dense) {
+        int lo = 0, hi = na;
+        while (lo < hi) { int mid = (lo + hi) >> 1; if (idp[mid] < y) lo = mid + 1; else hi = mid; }
+        pos = lo;
+      }
+      sh_lab[i] = first ? pos : -1;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int ny = 0;
+      for (int i = 0; i < nlab; ++i) ny += sh_lab[i] >= 0 ? 1 : 0;
+      sh_misc[0] = ny;
+    }
+  }
+
   // ---- logits over the active set.  The active rows of W2 are copied into shared memory, as many as fit at a
-  //      time; when the whole set fits they stay there for the back-propagation below ----
+  //      time.  When the whole set fits, the rows stay there for the back-propagation below.  When it does not, the
+  //      back-propagated error is accumulated in the same pass, chunk by chunk, with a running maximum M and sums
+  //      rescaled whenever M grows: S = sum_a exp(z_a - M) W2[j_a,:], E = sum_a exp(z_a - M), and T = the sum of the
+  //      label rows; then dh = (S / E - T / |Y|) / B, and every row is fetched once. ----
   float* z = p.act_z + (size_t)s * p.act_stride;
   float* tk_z = reinterpret_cast<float*>(smem + p.off_topk);          // predict: [FWD_WARPS][topk]
   int* tk_id = reinterpret_cast<int*>(tk_z + FWD_WARPS * p.topk);
   int tk_cnt = 0;                                                     // used by lane 0
   const float4* sh_h4 = reinterpret_cast<const float4*>(sh_h);
   const int ldr = H + 4;                           // staged rows are padded by 16 bytes: a thread per row reads without bank conflicts
-  const int stage_rows = p.stage_bytes / (ldr * 4);
+  const int stage_rows = p.stage_bytes / (ldr * 4 + 4);      // a row and one float of the chunk's exp(z - M)
+  float* sh_ce = stage + (size_t)stage_rows * ldr;           // [stage_rows]
+  const bool streaming = MODE == 0 && na > stage_rows;
+  float Mrun = -INFINITY, Erun = 0.f;
+  float accS[MAX_KPT], accT[MAX_KPT];
+#pragma unroll
+  for (int u = 0; u < MAX_KPT; ++u) { accS[u] = 0.f; accT[u] = 0.f; }
+  const int ngrp = H >= FWD_THREADS ? 1 : min(FWD_WARPS, FWD_THREADS / H);   // groups of H threads (sh_dh holds FWD_WARPS)
+  const int grp = H >= FWD_THREADS ? 0 : tid / H;
   const uint32_t row_bytes = (uint32_t)H * 4u;
   uint32_t phase = 0;
   bool timed_out = false;
@@ -597,14 +630,16 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
       if (MODE == 0) {
         if (live) {
+          float zv;
           if (small) {                       // the bias is already in the logit's place
-            const float zv = sh_z[c0 + a] + dot;
+            zv = sh_z[c0 + a] + dot;
             sh_z[c0 + a] = zv;
-            z[c0 + a] = zv;
           } else {
             const int j = dense ? c0 + a : idp[c0 + a];
-            z[c0 + a] = __ldg(&p.hdr2[j].b) + dot;
+            zv = __ldg(&p.hdr2[j].b) + dot;
           }
+          z[c0 + a] = zv;
+          if (streaming) sh_ce[a] = zv;
         }
       } else {
         // predict: lane 0 of each warp keeps the warp's best k so far, fed one lane's logit at a time
@@ -624,6 +659,44 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         }
       }
     }
+    if (streaming) {
+      __syncthreads();
+      float cm = -INFINITY;
+      for (int a = tid; a < nr; a += FWD_THREADS) cm = fmaxf(cm, sh_ce[a]);
+      const float Mnew = fmaxf(Mrun, block_max(cm, sh_red));
+      const float scale = expf(Mrun - Mnew);            // 0 for the first chunk
+      float es = 0.f;
+      for (int a = tid; a < nr; a += FWD_THREADS) {
+        const float ea = expf(sh_ce[a] - Mnew);
+        sh_ce[a] = ea;
+        es += ea;
+      }
+      Erun = Erun * scale + block_sum(es, sh_red);      // its barriers make the chunk's exp values visible
+      Mrun = Mnew;
+      if (grp < ngrp) {
+#pragma unroll
+        for (int u = 0; u < MAX_KPT; ++u) {
+          const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
+          if (k < H && (u == 0 || H > FWD_THREADS)) {
+            float v0 = accS[u] * scale, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+            int a = grp;
+            for (; a + 3 * ngrp < nr; a += 4 * ngrp) {
+              v0 = fmaf(sh_ce[a], stage[(size_t)a * ldr + k], v0);
+              v1 = fmaf(sh_ce[a + ngrp], stage[(size_t)(a + ngrp) * ldr + k], v1);
+              v2 = fmaf(sh_ce[a + 2 * ngrp], stage[(size_t)(a + 2 * ngrp) * ldr + k], v2);
+              v3 = fmaf(sh_ce[a + 3 * ngrp], stage[(size_t)(a + 3 * ngrp) * ldr + k], v3);
+            }
+            for (; a < nr; a += ngrp) v0 = fmaf(sh_ce[a], stage[(size_t)a * ldr + k], v0);
+            accS[u] = (v0 + v1) + (v2 + v3);
+            if (grp == 0)                               // the label rows of this chunk, once
+              for (int i = 0; i < nlab; ++i) {
+                const int pos = sh_lab[i] - c0;
+                if (sh_lab[i] >= 0 && pos >= 0 && pos < nr) accT[u] += stage[(size_t)pos * ldr + k];
+              }
+          }
+        }
+      }
+    }
   }
   if (timed_out) {
     // a copy did not complete in time: give the copies still in flight one more bounded wait, then give the sample
@@ -633,7 +706,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     skip_sample<MODE>(p, s, DSLIDE_ERR_TIMEOUT);
     return;
   }
-  const bool staged_all = na <= stage_rows;      // every active row is still in shared memory
 
   if (MODE == 1) {
     // ---- merge the per-warp lists: k rounds over the list heads ----
@@ -663,41 +735,27 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   }
   __syncthreads();           // logits visible to the block
 
-  // ---- positions of the sample's distinct labels inside the active set ----
-  for (int i = tid; i < nlab; i += FWD_THREADS) {
-    int y = p.labels[lbeg + i];
-    bool first = true;
-    for (int q = 0; q < i; ++q) first = first && (p.labels[lbeg + q] != y);
-    int pos = y;
-    if (!dense) {
-      int lo = 0, hi = na;
-      while (lo < hi) { int mid = (lo + hi) >> 1; if (idp[mid] < y) lo = mid + 1; else hi = mid; }
-      pos = lo;
-    }
-    sh_lab[i] = first ? pos : -1;
-  }
-
   // ---- softmax over the ragged active set, loss, errors ----
   float* pr = p.act_p + (size_t)s * p.act_stride;
   float* g = p.act_g + (size_t)s * p.act_stride;
-  float m = -INFINITY;
-  for (int a = tid; a < na; a += FWD_THREADS) m = fmaxf(m, zp[a]);
-  const float M = block_max(m, sh_red);
-  float e = 0.f;
-  for (int a = tid; a < na; a += FWD_THREADS) e += expf(zp[a] - M);
-  const float E = block_sum(e, sh_red);            // its barriers also make sh_lab visible
+  float M = Mrun, E = Erun;                        // known already when the rows were streamed
+  if (!streaming) {
+    float m = -INFINITY;
+    for (int a = tid; a < na; a += FWD_THREADS) m = fmaxf(m, zp[a]);
+    M = block_max(m, sh_red);
+    float e = 0.f;
+    for (int a = tid; a < na; a += FWD_THREADS) e += expf(zp[a] - M);
+    E = block_sum(e, sh_red);
+  }
   const float fB = (float)p.B;
   if (tid == 0) {
-    int ny = 0;
-    for (int i = 0; i < nlab; ++i) ny += sh_lab[i] >= 0 ? 1 : 0;
+    const int ny = sh_misc[0];
     float sum = 0.f;
     const float logE = logf(E);
     for (int i = 0; i < nlab; ++i)
       if (sh_lab[i] >= 0) sum += zp[sh_lab[i]] - M - logE;
     p.loss[s] = ny > 0 ? -sum / (float)ny : 0.f;
-    sh_misc[0] = ny;
   }
-  __syncthreads();
   const int ny = sh_misc[0];
   // when the set is small the error takes the logit's place in shared memory, for the steps below
   for (int a = tid; a < na; a += FWD_THREADS) {
@@ -730,44 +788,29 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
 
   // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update).  A thread
   //      per hidden unit walks the staged rows; with fewer hidden units than threads the rows are dealt to
-  //      several groups of threads whose sums are then added in group order ----
+  //      several groups of threads whose sums are then added in group order.  When the rows were streamed the
+  //      sums exist already. ----
   {
-    const int ngrp = H >= FWD_THREADS ? 1 : min(FWD_WARPS, FWD_THREADS / H);   // groups of H threads (sh_dh holds FWD_WARPS)
-    const int grp = H >= FWD_THREADS ? 0 : tid / H;
     float accd[MAX_KPT];
 #pragma unroll
-    for (int u = 0; u < MAX_KPT; ++u) accd[u] = 0.f;
-    for (int c0 = 0; c0 < na; c0 += stage_rows) {
-      const int nr = min(stage_rows, na - c0);
-      if (!staged_all) {
-        __syncthreads();
-        if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * row_bytes);
-        fence_proxy_async();
-        __syncthreads();
-        for (int r = tid; r < nr; r += FWD_THREADS) {
-          const int j = dense ? c0 + r : idp[c0 + r];
-          bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)j * H, row_bytes, sh_bar);
-        }
-        if (!mbar_wait(sh_bar, phase)) timed_out = true;
-        phase ^= 1u;
-        if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
-      }
-      if (grp < ngrp) {
+    for (int u = 0; u < MAX_KPT; ++u)
+      accd[u] = streaming ? (accS[u] / E - (ny > 0 ? accT[u] / (float)ny : 0.f)) / fB : 0.f;
+    if (!streaming && grp < ngrp) {
+      const int nr = na;                           // all rows are still staged
 #pragma unroll
-        for (int u = 0; u < MAX_KPT; ++u) {
-          const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
-          if (k < H && (u == 0 || H > FWD_THREADS)) {
-            float v0 = accd[u], v1 = 0.f, v2 = 0.f, v3 = 0.f;
-            int a = grp;
-            for (; a + 3 * ngrp < nr; a += 4 * ngrp) {
-              v0 = fmaf(gp[c0 + a], stage[(size_t)a * ldr + k], v0);
-              v1 = fmaf(gp[c0 + a + ngrp], stage[(size_t)(a + ngrp) * ldr + k], v1);
-              v2 = fmaf(gp[c0 + a + 2 * ngrp], stage[(size_t)(a + 2 * ngrp) * ldr + k], v2);
-              v3 = fmaf(gp[c0 + a + 3 * ngrp], stage[(size_t)(a + 3 * ngrp) * ldr + k], v3);
-            }
-            for (; a < nr; a += ngrp) v0 = fmaf(gp[c0 + a], stage[(size_t)a * ldr + k], v0);
-            accd[u] = (v0 + v1) + (v2 + v3);
+      for (int u = 0; u < MAX_KPT; ++u) {
+        const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
+        if (k < H && (u == 0 || H > FWD_THREADS)) {
+          float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+          int a = grp;
+          for (; a + 3 * ngrp < nr; a += 4 * ngrp) {
+            v0 = fmaf(gp[a], stage[(size_t)a * ldr + k], v0);
+            v1 = fmaf(gp[a + ngrp], stage[(size_t)(a + ngrp) * ldr + k], v1);
+            v2 = fmaf(gp[a + 2 * ngrp], stage[(size_t)(a + 2 * ngrp) * ldr + k], v2);
+            v3 = fmaf(gp[a + 3 * ngrp], stage[(size_t)(a + 3 * ngrp) * ldr + k], v3);
           }
+          for (; a < nr; a += ngrp) v0 = fmaf(gp[a], stage[(size_t)a * ldr + k], v0);
+          accd[u] = (v0 + v1) + (v2 + v3);
         }
       }
     }
@@ -779,14 +822,10 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
     }
     __syncthreads();
-    if (timed_out) {
-      mbar_wait(sh_bar, phase ^ 1u);
-      if (tid == 0) set_status(p.st, DSLIDE_ERR_TIMEOUT);
-    }
     for (int k = tid; k < H; k += FWD_THREADS) {
       float v = 0.f;
       for (int w = 0; w < ngrp; ++w) v += sh_dh[(size_t)w * H + k];
-      p.dh[(size_t)s * H + k] = (sh_h[k] > 0.f && !timed_out) ? v : 0.f;
+      p.dh[(size_t)s * H + k] = sh_h[k] > 0.f ? v : 0.f;
     }
   }
   if (!dense) {
