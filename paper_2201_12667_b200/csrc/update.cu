@@ -462,35 +462,41 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
   const unsigned nh_raw = p.st->n_hot[p.parity], nm_raw = p.st->n_med[p.parity];
   const int n_hot_items = (int)(nh_raw < (unsigned)HOT_CAP ? nh_raw : (unsigned)HOT_CAP) * HOT_SLICES;
   const int n_med = (int)(nm_raw < (unsigned)MED_CAP ? nm_raw : (unsigned)MED_CAP);
-  const int n_norm = (nrows + UPD_TROWS - 1) / UPD_TROWS;
+  // ordinary rows go out UPD_TROWS per ticket, except the last few thousand, which go out G per ticket so that the
+  // warps finish close together
+  const int nwork = (int)gridDim.x - naux;
+  const int nwarps = nwork * UPD_WARPS;
+  const int rows_small = min(nrows, UPD_TROWS * nwarps);
+  const int rows_big = (nrows - rows_small) / UPD_TROWS * UPD_TROWS;
+  const int n_big = rows_big / UPD_TROWS;
+  const int n_norm = n_big + (nrows - rows_big + G - 1) / G;
   const int n_tickets = n_hot_items + n_med + n_norm;
   unsigned int* ticket = &p.st->ticket[p.parity];
 
-  // every warp's first ticket is its own number; further tickets come from the counter (one is always on its way
-  // while the current one is worked on)
-  const int nwork = (int)gridDim.x - naux;
-  const int nwarps = nwork * UPD_WARPS;
+  // a warp's first two tickets are fixed by its number; further tickets come from the counter, each asked for a
+  // whole ticket before it is needed
   int cur = warp * nwork + ((int)blockIdx.x - naux);
-  int nxt = 0;
-  if (lane == 0) nxt = nwarps + (int)atomicAdd(ticket, 1u);
-  for (;; ) {
+  int nxt = nwarps + cur;
+  int fut = 0;
+  if (lane == 0) fut = 2 * nwarps + (int)atomicAdd(ticket, 1u);
+  for (;; cur = nxt, nxt = __shfl_sync(FULL, fut, 0), fut = (lane == 0 && nxt < n_tickets) ? 2 * nwarps + (int)atomicAdd(ticket, 1u) : fut) {
     const int t = cur;
     if (t >= n_tickets) break;
-    cur = __shfl_sync(FULL, nxt, 0);
-    if (lane == 0 && cur < n_tickets) nxt = nwarps + (int)atomicAdd(ticket, 1u);
     if (t < n_hot_items) { hot_item<NCH>(p, rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
     if (t < n_hot_items + n_med) { medium_item<NCH>(p, rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
 
-    // ---- ordinary rows: ticket k takes rows k, k + n_norm, k + 2 n_norm, ... of the concatenated lists (rows of
-    //      W2, then rows of W1), so that neighbours in a list (often alike in cost) go to different warps ----
+    // ---- ordinary rows: consecutive entries of the concatenated lists (rows of W2, then rows of W1) ----
     const int k = t - n_hot_items - n_med;
+    const int first = k < n_big ? k * UPD_TROWS : rows_big + (k - n_big) * G;
+    const int trows = k < n_big ? UPD_TROWS : G;
     int2 myrow = make_int2(0, 0);        // (row, the sample that touched it first = the sample of slot 0)
     int myidx = nrows;
-    if (lane < UPD_TROWS) {
-      myidx = k + lane * n_norm;
+    if (lane < trows) {
+      myidx = first + lane;
       if (myidx < nrows) myrow = myidx < n2 ? p.own2[myidx] : p.own1[myidx - n2];
+      else myidx = nrows;
     }
-    for (int b0 = 0; b0 < UPD_TROWS; b0 += G) {
+    for (int b0 = 0; b0 < trows; b0 += G) {
       int rr[G], tt[G];
       bool live[G], w2[G], skip[G];
       int2 hv[G], sl[G];
