@@ -161,6 +161,7 @@ struct Ctx {
   int dedup_mode;      // 1 bitmap, 2 sort
   int fwd_smem;        // dynamic shared memory of the forward kernel
   int fwd_stage_bytes; // of which: staging space for rows of W1 / W2 (overlays the dedup work space)
+  int fwd_hash_sm_off, fwd_hash_sm_bytes;  // the hash functions' mirror inside the forward kernel's staging region (-1: none)
   int fwd_sort_small;  // candidate sets up to this size are deduplicated by sorting
   int sort_cap;        // capacity (power of two) of the shared-memory sort buffer
   int num_sms;

@@ -49,6 +49,8 @@ struct FwdParams {
   int act_stride, Wd, dense, dedup_mode, max_labels, sort_cap, topk, parity;
   int stage_bytes;     // bytes of the staging region (it starts at off_dedup and overlays the dedup work space)
   int hid_rows;        // rows of W1 staged per chunk of the hidden layer
+  int hash_sm_off;     // where in the staging region the hash functions' index tables are mirrored (-1: read from global memory)
+  int hash_sm_bytes;
   int sort_small;      // candidate sets up to this size are deduplicated by sorting even when a bitmap is available
   int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_tbeg, off_topk, off_ids, off_z, off_col, off_val,
       off_dedup;
@@ -177,7 +179,10 @@ __device__ __forceinline__ bool topk_better(float za, int ia, float zb, int ib) 
 // Puts n <= PER * FWD_THREADS values in ascending order by counting: the place of a value is the number of values
 // before it (by value, then by position).  src and dst are in shared memory; thread t owns the values t, t +
 // FWD_THREADS, ...; threads without a value skip the counting loop.
-template <int PER>
+// PACKED: src holds (value << RANK_BITS | position), padded with 0xffffffff to a multiple of four -- all distinct,
+// so one comparison per pair decides; dst receives the values alone.
+constexpr int RANK_BITS = 10;
+template <int PER, bool PACKED>
 __device__ __forceinline__ void rank_sort(const uint32_t* src, uint32_t* dst, int n) {
   const int tid = threadIdx.x;
   if (tid >= n) return;
@@ -189,15 +194,30 @@ __device__ __forceinline__ void rank_sort(const uint32_t* src, uint32_t* dst, in
     v[u] = i < n ? src[i] : 0xffffffffu;
     pos[u] = 0;
   }
+  if (PACKED) {
+    const uint4* src4 = reinterpret_cast<const uint4*>(src);
+    const int n4 = (n + 3) >> 2;
+#pragma unroll 2
+    for (int k = 0; k < n4; ++k) {
+      const uint4 a = src4[k];
+#pragma unroll
+      for (int u = 0; u < PER; ++u)
+        pos[u] += (a.x < v[u] ? 1 : 0) + (a.y < v[u] ? 1 : 0) + (a.z < v[u] ? 1 : 0) + (a.w < v[u] ? 1 : 0);
+    }
+#pragma unroll
+    for (int u = 0; u < PER; ++u)
+      if (tid + u * FWD_THREADS < n) dst[pos[u]] = v[u] >> RANK_BITS;
+  } else {
 #pragma unroll 4
-  for (int k = 0; k < n; ++k) {
-    const uint32_t a = src[k];
+    for (int k = 0; k < n; ++k) {
+      const uint32_t a = src[k];
 #pragma unroll
-    for (int u = 0; u < PER; ++u) pos[u] += (a < v[u] || (a == v[u] && k < tid + u * FWD_THREADS)) ? 1 : 0;
+      for (int u = 0; u < PER; ++u) pos[u] += (a < v[u] || (a == v[u] && k < tid + u * FWD_THREADS)) ? 1 : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < PER; ++u)
+      if (tid + u * FWD_THREADS < n) dst[pos[u]] = v[u];
   }
-#pragma unroll
-  for (int u = 0; u < PER; ++u)
-    if (tid + u * FWD_THREADS < n) dst[pos[u]] = v[u];
 }
 
 // The sample is skipped: no loss, no gradient, nothing touched (predict: no candidates).
@@ -226,6 +246,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   int* sh_misc = reinterpret_cast<int*>(smem + p.off_misc);          // 32 ints
   float* sh_red = reinterpret_cast<float*>(sh_misc + 16);
   uint64_t* sh_bar = reinterpret_cast<uint64_t*>(sh_misc + 26);      // 8-byte aligned: off_misc is 16-byte aligned
+  uint64_t* sh_bar2 = reinterpret_cast<uint64_t*>(sh_misc + 28);     // completion of the hash functions' mirror
   int* sh_lab = reinterpret_cast<int*>(smem + p.off_lab);            // [max_labels]
   int* sh_tbase = reinterpret_cast<int*>(smem + p.off_tbase);        // [L + 1]
   int* sh_tbeg = reinterpret_cast<int*>(smem + p.off_tbeg);          // [L]
@@ -247,7 +268,16 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   if (tid == 0) {
     sh_misc[24] = 0;                 // bucket entries fetched by this sample
     mbar_init(sh_bar, 1);
+    mbar_init(sh_bar2, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // the hash functions' tables (constant between rebuilds) come into the upper part of the staging region, which
+    // is free until the candidates are collected
+    if (p.hash_sm_off >= 0 && !p.dense) {
+      mbar_expect_tx(sh_bar2, (uint32_t)p.hash_sm_bytes);
+      const int half = p.family == DSLIDE_SIMHASH ? p.hash_sm_bytes / 2 : p.hash_sm_bytes;
+      bulk_g2s(smem + p.off_dedup + p.hash_sm_off, p.hash_idx, (uint32_t)half, sh_bar2);
+      if (p.family == DSLIDE_SIMHASH) bulk_g2s(smem + p.off_dedup + p.hash_sm_off + half, p.hash_sign, (uint32_t)half, sh_bar2);
+    }
   }
 
   // ---- label checks: ids in range, list within the maximum ----
@@ -332,6 +362,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
   }
   if (bad || too_many_labels) {
+    if (p.hash_sm_off >= 0 && !p.dense) mbar_wait(sh_bar2, 0u);     // no copy into this block may be left in flight
     skip_sample<MODE>(p, s, (!bad && too_many_labels) ? DSLIDE_ERR_OVERFLOW : DSLIDE_ERR_BAD_INDEX);
     return;
   }
@@ -352,21 +383,34 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
 
   if (!dense) {
     // ---- bucket codes of the hidden activation ----
+    const int32_t* hidx = p.hash_idx;
+    const int32_t* hsgn = p.hash_sign;
+    if (p.hash_sm_off >= 0) {
+      const bool ok = mbar_wait(sh_bar2, 0u);
+      if (__syncthreads_or(ok ? 0 : 1)) {          // the mirror did not arrive in time: the sample is given up
+        mbar_wait(sh_bar2, 0u);
+        __syncthreads();
+        skip_sample<MODE>(p, s, DSLIDE_ERR_TIMEOUT);
+        return;
+      }
+      hidx = reinterpret_cast<const int32_t*>(smem + p.off_dedup + p.hash_sm_off);
+      hsgn = reinterpret_cast<const int32_t*>(smem + p.off_dedup + p.hash_sm_off + p.hash_sm_bytes / 2);
+    }
     for (int f = tid; f < p.KL; f += FWD_THREADS) {
-      const int32_t* ix = p.hash_idx + (size_t)f * p.fn_len;
+      const int32_t* ix = hidx + (size_t)f * p.fn_len;
       if (p.family == DSLIDE_SIMHASH) {
-        const int32_t* sg = p.hash_sign + (size_t)f * p.fn_len;
+        const int32_t* sg = hsgn + (size_t)f * p.fn_len;
         float sum = 0.f;
         for (int i = 0; i < p.fn_len; ++i) {
-          float x = sh_h[__ldg(ix + i)];
-          sum = __fadd_rn(sum, __ldg(sg + i) > 0 ? x : -x);
+          float x = sh_h[ix[i]];
+          sum = __fadd_rn(sum, sg[i] > 0 ? x : -x);
         }
         sh_part[f] = sum >= 0.f ? 1 : 0;
       } else {
         int best = 0;
-        float bv = sh_h[__ldg(ix)];
+        float bv = sh_h[ix[0]];
         for (int i = 1; i < p.fn_len; ++i) {
-          float v = sh_h[__ldg(ix + i)];
+          float v = sh_h[ix[i]];
           if (v > bv) { bv = v; best = i; }       // strict: the lowest position wins ties
         }
         sh_part[f] = (unsigned char)best;
@@ -413,6 +457,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     const bool bitmap = p.dedup_mode == 1 && ncand + nlab > p.sort_small;
     int n2 = 1;
     if (!bitmap) while (n2 < ncand + nlab) n2 <<= 1;
+    // ids short enough to share a word with their position are sorted as such words
+    const bool packed = !bitmap && ncand + nlab <= RANK_MAX && N <= (1 << (32 - RANK_BITS));
     if (bitmap) {
       uint4* dd4 = reinterpret_cast<uint4*>(sh_dd);
       const int n4 = (((N + 31) >> 5) + 3) >> 2;
@@ -424,13 +470,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (sh_tbase[mid] <= c) lo = mid; else hi = mid - 1; }
       const int j = __ldg(p.bucket_ids + (size_t)lo * N + sh_tbeg[lo] + (c - sh_tbase[lo]));
       if (bitmap) atomicOr(&sh_dd[j >> 5], 1u << (j & 31));
-      else sh_dd[c] = (uint32_t)j;
+      else sh_dd[c] = packed ? ((uint32_t)j << RANK_BITS) | (uint32_t)c : (uint32_t)j;
     }
     if (MODE == 0)
       for (int i = tid; i < nlab; i += FWD_THREADS) {
         const int y = p.labels[lbeg + i];
         if (bitmap) atomicOr(&sh_dd[y >> 5], 1u << (y & 31));
-        else sh_dd[ncand + i] = (uint32_t)y;
+        else sh_dd[ncand + i] = packed ? ((uint32_t)y << RANK_BITS) | (uint32_t)(ncand + i) : (uint32_t)y;
       }
     if (bitmap) {
       __syncthreads();
@@ -455,12 +501,19 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
     } else if (ncand + nlab <= RANK_MAX) {
       const int n = ncand + nlab;
+      if (packed && tid < 4 && n + tid < ((n + 3) & ~3)) sh_dd[n + tid] = 0xffffffffu;
       __syncthreads();
       uint32_t* srt = sh_dd + RANK_MAX;
       const int per = (n + FWD_THREADS - 1) / FWD_THREADS;
-      if (per <= 1) rank_sort<1>(sh_dd, srt, n);
-      else if (per == 2) rank_sort<2>(sh_dd, srt, n);
-      else rank_sort<RANK_MAX / FWD_THREADS>(sh_dd, srt, n);
+      if (packed) {
+        if (per <= 1) rank_sort<1, true>(sh_dd, srt, n);
+        else if (per == 2) rank_sort<2, true>(sh_dd, srt, n);
+        else rank_sort<RANK_MAX / FWD_THREADS, true>(sh_dd, srt, n);
+      } else {
+        if (per <= 1) rank_sort<1, false>(sh_dd, srt, n);
+        else if (per == 2) rank_sort<2, false>(sh_dd, srt, n);
+        else rank_sort<RANK_MAX / FWD_THREADS, false>(sh_dd, srt, n);
+      }
       __syncthreads();
       // thread t looks at the sorted elements PER * t ... PER * t + PER - 1 and keeps the first of each run
       constexpr int PER = RANK_MAX / FWD_THREADS;
@@ -926,6 +979,17 @@ cudaError_t setup_forward(Ctx* c) {
     int cap_small = c->fwd_stage_bytes / 8;      // the sort pads to a power of two
     c->fwd_sort_small = cap_small < SORT_SMALL ? cap_small : SORT_SMALL;
   }
+  // the hash functions' tables are mirrored above the hidden layer's chunk when they fit there
+  {
+    const long long one = (long long)c->KL * c->fn_len * 4;
+    const long long hb = c->cfg.hash_family == DSLIDE_SIMHASH ? 2 * one : one;
+    c->fwd_hash_sm_off = -1;
+    c->fwd_hash_sm_bytes = 0;
+    if (!c->dense && one % 16 == 0 && hb <= 32 * 1024 && stage_min + hb <= (long long)c->fwd_stage_bytes) {
+      c->fwd_hash_sm_bytes = (int)hb;
+      c->fwd_hash_sm_off = (c->fwd_stage_bytes - (int)hb) & ~15;
+    }
+  }
   c->fwd_smem = l.fixed_bytes + c->fwd_stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(k_forward<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
@@ -950,6 +1014,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.max_labels = c->cfg.max_labels; p.sort_cap = c->sort_cap; p.topk = 1;
   FwdLayout l = fwd_layout(c);
   p.stage_bytes = c->fwd_stage_bytes; p.hid_rows = l.hid_rows; p.sort_small = c->fwd_sort_small;
+  p.hash_sm_off = c->fwd_hash_sm_off; p.hash_sm_bytes = c->fwd_hash_sm_bytes;
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
   p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;
   p.off_ids = l.off_ids; p.off_z = l.off_z; p.off_col = l.off_col; p.off_val = l.off_val; p.off_dedup = l.off_dedup;
