@@ -299,6 +299,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   //      kernel may run that far while the previous step's update kernel is still finishing (griddep_wait).
   float acc[MAX_KPT];
   bool waited = false;
+  uint32_t phase = 0;                // of sh_bar, which serves the staging of W1 rows here and of W2 rows below
+  bool timed_out = false;
   const int R = p.hid_rows;
   for (int c0 = 0; c0 < nnz && !bad; c0 += R) {       // `bad` is uniform over the block here
     const int nr = min(R, nnz - c0);
@@ -310,38 +312,27 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       sh_col[i] = okc ? c : 0;
       sh_val[i] = __ldg(p.vals + rbeg + c0 + i);
     }
+    if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * (uint32_t)H * 4u);
+    fence_proxy_async();             // the staging space was read through ordinary loads (the previous chunk)
     bad = __syncthreads_or(bad);
-    if (bad) break;
+    if (bad) break;                  // nothing was copied; the barrier is not used again
     if (!waited) {
       griddep_wait();
       waited = true;
+    }
+    // one bulk copy per row of W1: every row of the chunk is in flight at once
+    for (int i = tid; i < nr; i += FWD_THREADS)
+      bulk_g2s(stage + (size_t)i * H, p.W1 + (size_t)sh_col[i] * H, (uint32_t)H * 4u, sh_bar);
+    if (c0 == 0) {
 #pragma unroll
       for (int u = 0; u < MAX_KPT; ++u) {
         const int k = tid + u * FWD_THREADS;
         acc[u] = k < H ? p.b1[k] : 0.f;
       }
     }
-    {
-      float4* st4 = reinterpret_cast<float4*>(stage);
-      const int total4 = nr * H4;
-      for (int e0 = tid; e0 < total4; e0 += FWD_THREADS * 8) {
-        float4 x[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int e = e0 + u * FWD_THREADS;
-          if (e < total4) {
-            const int r = e / H4, c4 = e - r * H4;
-            x[u] = __ldg(reinterpret_cast<const float4*>(p.W1 + (size_t)sh_col[r] * H) + c4);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int e = e0 + u * FWD_THREADS;
-          if (e < total4) st4[e] = x[u];
-        }
-      }
-    }
-    __syncthreads();
+    if (!mbar_wait(sh_bar, phase)) timed_out = true;
+    phase ^= 1u;
+    if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
 #pragma unroll
     for (int u = 0; u < MAX_KPT; ++u) {
       const int k = tid + u * FWD_THREADS;
@@ -360,6 +351,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       const int k = tid + u * FWD_THREADS;
       acc[u] = k < H ? p.b1[k] : 0.f;
     }
+  }
+  if (timed_out) {                   // a row of W1 did not arrive in time: one more bounded wait, then the sample is given up
+    mbar_wait(sh_bar, phase ^ 1u);
+    if (p.hash_sm_off >= 0 && !p.dense) mbar_wait(sh_bar2, 0u);
+    __syncthreads();
+    skip_sample<MODE>(p, s, DSLIDE_ERR_TIMEOUT);
+    return;
   }
   if (bad || too_many_labels) {
     if (p.hash_sm_off >= 0 && !p.dense) mbar_wait(sh_bar2, 0u);     // no copy into this block may be left in flight
@@ -627,8 +625,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   const int ngrp = H >= FWD_THREADS ? 1 : min(FWD_WARPS, FWD_THREADS / H);   // groups of H threads (sh_dh holds FWD_WARPS)
   const int grp = H >= FWD_THREADS ? 0 : tid / H;
   const uint32_t row_bytes = (uint32_t)H * 4u;
-  uint32_t phase = 0;
-  bool timed_out = false;
   for (int c0 = 0; c0 < na; c0 += stage_rows) {
     const int nr = min(stage_rows, na - c0);
     __syncthreads();                               // earlier readers and writers of the staging space are done
@@ -809,6 +805,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       if (sh_lab[i] >= 0) sum += zp[sh_lab[i]] - M - logE;
     p.loss[s] = ny > 0 ? -sum / (float)ny : 0.f;
   }
+  __syncthreads();           // the logits at the label positions have been read: their places may now take the errors
   const int ny = sh_misc[0];
   // when the set is small the error takes the logit's place in shared memory, for the steps below
   for (int a = tid; a < na; a += FWD_THREADS) {

@@ -143,3 +143,49 @@ def test_more_listed_rows_than_the_list_holds():
             assert max_rel_err(ds.dslide_get_tensor(pr.ctx, n), pr.o.get(n), 1e-2) < W_TOL, n
     finally:
         pr.close()
+
+
+def test_neuron_ids_too_long_to_sort_packed():
+    """More than 2^22 neurons: an id and its position among the candidates no longer share a 32-bit word, so the
+    candidates are ranked by comparing ids and positions separately."""
+    N = (1 << 22) + 5003
+    pr = Pair(D=300, H=8, N=N, family=SIMHASH, K=12, L=4, bucket_cap=32, max_batch=8, max_labels=2, lr=1e-3, seed=7,
+              init_std=0.05)
+    try:
+        wl = workloads.Workload(workloads.config("tiny", D=300, N=N, max_labels=2), seed=14)
+        for i in range(2):
+            batch = wl.batch(i, batch_size=8)
+            lo = pr.o.train_step(*batch)
+            lg = pr.gpu_step(batch)
+            assert abs(lo - lg) <= (ACT_TOL if i == 0 else W_TOL) * abs(lo)
+            sets, cnt = pr.gpu_active_sets(8)
+            for s, a in enumerate(pr.o.active_sets()):
+                assert np.array_equal(sets[s], a)
+        for n in ("W2", "b2", "W1"):
+            assert max_rel_err(ds.dslide_get_tensor(pr.ctx, n), pr.o.get(n), 1e-2) < W_TOL, n
+    finally:
+        pr.close()
+
+
+@pytest.mark.parametrize("H", [128, 1024])
+def test_same_step_repeated_gives_the_same_outputs(H):
+    """With a vanishing learning rate the weights do not move, so repeating a batch must reproduce every per-sample
+    output of the forward kernel bit for bit (H = 1024: the active rows are streamed in several chunks).  A barrier
+    missing between two uses of a shared array shows up here as an occasional difference."""
+    pr = Pair(D=workloads.config("mid")["D"], H=H, N=8009, family=DWTA, K=3, L=6, bucket_cap=16, max_batch=24,
+              max_labels=16, lr=1e-30, seed=2)
+    try:
+        wl = workloads.Workload(workloads.config("mid", N=8009), seed=11)
+        batch = wl.batch(0, batch_size=24)
+        names = ("hidden", "codes", "act_count", "act_logit", "act_err", "loss", "dhidden")
+        ref = None
+        for it in range(150):
+            pr.gpu_step(batch)
+            cur = {n: ds.dslide_get_last(pr.ctx, n, 24).copy() for n in names}
+            if ref is None:
+                ref = cur
+                continue
+            for n in names:
+                assert np.array_equal(cur[n], ref[n]), (it, n)
+    finally:
+        pr.close()
