@@ -404,6 +404,21 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
           sum = __fadd_rn(sum, sg[i] > 0 ? x : -x);
         }
         sh_part[f] = sum >= 0.f ? 1 : 0;
+      } else if (p.fn_len == 8 && (reinterpret_cast<uintptr_t>(hidx) & 15) == 0) {
+        // bins of eight: both halves of the index list in one load each, the eight values fetched side by side
+        const int4 ia = reinterpret_cast<const int4*>(ix)[0], ib = reinterpret_cast<const int4*>(ix)[1];
+        const float v0 = sh_h[ia.x], v1 = sh_h[ia.y], v2 = sh_h[ia.z], v3 = sh_h[ia.w];
+        const float v4 = sh_h[ib.x], v5 = sh_h[ib.y], v6 = sh_h[ib.z], v7 = sh_h[ib.w];
+        int best = 0;
+        float bv = v0;
+        if (v1 > bv) { bv = v1; best = 1; }       // strict: the lowest position wins ties
+        if (v2 > bv) { bv = v2; best = 2; }
+        if (v3 > bv) { bv = v3; best = 3; }
+        if (v4 > bv) { bv = v4; best = 4; }
+        if (v5 > bv) { bv = v5; best = 5; }
+        if (v6 > bv) { bv = v6; best = 6; }
+        if (v7 > bv) { bv = v7; best = 7; }
+        sh_part[f] = (unsigned char)best;
       } else {
         int best = 0;
         float bv = sh_h[ix[0]];
