@@ -225,9 +225,11 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     A(own2, N, true);
     A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
     A(keysA, (size_t)c->L * N, false);
-    // codes wider than one radix digit: ids are placed by atomics and ordered inside their buckets, no radix passes
+    // codes wider than one radix digit: every id is placed at its bucket's start plus its rank of arrival there and the
+    // large buckets are ordered afterwards, no radix passes
     c->place_path = c->bits > sort_max_width() ? 1 : 0;
     if (c->place_path) {
+      A(keysB, (size_t)c->L * N, false);      // here: the rank of every id inside its bucket
       A(ord_mid, (size_t)c->L * (N / (order_small_max() + 1) + 1), false);
       A(ord_big, (size_t)c->L * (N / (order_block_max() + 1) + 1), false);
       A(ord_cnt, 2, true);

@@ -103,12 +103,13 @@ constexpr int HN_FN_SMEM_MAX = 96 * 1024;    // hash-function tables larger than
 // column of 32 different rows hit 32 banks) and evaluates the L codes of each row: lane = row, the
 // warps share out the tables.  The hash functions sit in shared memory too, 16 bits per coordinate
 // (the top bit carries a negative SimHash sign), read as warp-wide broadcasts.
-// keys[t][j] = code of neuron j in table t; counts[t][code + 1] += 1.
+// keys[t][j] = code of neuron j in table t; counts[t][code + 1] += 1; with `ranks`, ranks[t][j] = the count before
+// (the neuron's place inside its bucket, in order of arrival).
 template <bool FN_SMEM>
 __global__ void __launch_bounds__(HN_THREADS)
 k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, const int32_t* __restrict__ hsign,
-               uint32_t* keys, int32_t* counts, int N, int H, int K, int L, int family, int lg_bin, int fn_len,
-               long long nb) {
+               uint32_t* keys, uint32_t* ranks, int32_t* counts, int N, int H, int K, int L, int family, int lg_bin,
+               int fn_len, long long nb) {
   extern __shared__ __align__(16) unsigned char hn_smem[];
   float* tile = reinterpret_cast<float*>(hn_smem);                    // [HN_ROWS][H + 1]
   const int ld = H + 1;
@@ -198,7 +199,9 @@ k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, c
           }
         }
         keys[(size_t)t * N + j0 + lane] = code;
-        atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code + 1, 1);
+        int32_t* cnt = counts + (size_t)t * (size_t)(nb + 1) + code + 1;
+        if (ranks) ranks[(size_t)t * N + j0 + lane] = (uint32_t)atomicAdd(cnt, 1);
+        else atomicAdd(cnt, 1);
       }
     }
   }
@@ -214,8 +217,8 @@ __device__ __forceinline__ void wta_step(float x, int i, float& bv, int& best) {
 }
 
 __global__ void __launch_bounds__(HN_THREADS)
-k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ hidx, uint32_t* keys, int32_t* counts,
-                     int N, int H, int K, int L, int lg_bin, long long nb) {
+k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ hidx, uint32_t* keys, uint32_t* ranks,
+                     int32_t* counts, int N, int H, int K, int L, int lg_bin, long long nb) {
   extern __shared__ __align__(16) unsigned char hn_smem[];
   float2* tile = reinterpret_cast<float2*>(hn_smem);                  // [32 pairs][H + 1]
   const int ld = H + 1;
@@ -249,6 +252,9 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
     const bool live0 = lane < rows, live1 = lane + 32 < rows;
     if (live0) {
       const float2* v = tile + (size_t)lane * ld;
+      uint32_t pr0 = 0, pr1 = 0;
+      size_t pidx = 0;
+      bool pend = false, pend1 = false;
       for (int t = warp; t < L; t += HN_WARPS) {
         uint32_t code0 = 0, code1 = 0;
         for (int k = 0; k < K; ++k) {
@@ -267,12 +273,31 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
           code0 |= (uint32_t)ia << (k * lg_bin);
           code1 |= (uint32_t)ib << (k * lg_bin);
         }
+        // the ranks asked for in the previous round have arrived by now: they are stored a round late so that
+        // no warp waits on its atomics
+        if (pend) {
+          ranks[pidx] = pr0;
+          if (pend1) ranks[pidx + 32] = pr1;
+        }
         keys[(size_t)t * N + j0 + lane] = code0;
-        atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code0 + 1, 1);
+        int32_t* cnt = counts + (size_t)t * (size_t)(nb + 1) + 1;
+        if (ranks) {
+          pr0 = (uint32_t)atomicAdd(cnt + code0, 1);
+          pidx = (size_t)t * N + j0 + lane;
+          pend = true;
+          pend1 = live1;
+        } else {
+          atomicAdd(cnt + code0, 1);
+        }
         if (live1) {
           keys[(size_t)t * N + j0 + 32 + lane] = code1;
-          atomicAdd(counts + (size_t)t * (size_t)(nb + 1) + code1 + 1, 1);
+          if (ranks) pr1 = (uint32_t)atomicAdd(cnt + code1, 1);
+          else atomicAdd(cnt + code1, 1);
         }
+      }
+      if (pend) {
+        ranks[pidx] = pr0;
+        if (pend1) ranks[pidx + 32] = pr1;
       }
     }
   }
@@ -306,9 +331,7 @@ __global__ void __launch_bounds__(BS_THREADS) k_bucket_sums(const int32_t* off, 
   }
 }
 
-// exclusive != 0: every counter is replaced by the sum of the counters before it instead of the sum up to and including it.
-__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks,
-                                                            int exclusive) {
+__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks) {
   __shared__ int sh[BS_THREADS / 32 + 1];
   int32_t* o = off + (size_t)blockIdx.y * (size_t)(nb + 1);
   const long long n = nb + 1, base = (long long)blockIdx.x * BS_CHUNK;
@@ -348,7 +371,7 @@ __global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long l
       if (lane >= d) incl += x;
     }
     const long long i = wbase + u * 32 + lane;
-    if (i < n) o[i] = run + incl - (exclusive ? v[u] : 0);
+    if (i < n) o[i] = run + incl;
     run += __shfl_sync(0xffffffffu, incl, 31);
   }
 }
@@ -520,24 +543,24 @@ k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_o
 
 // ------------------------------------------------------------------ wide codes: place, then order inside buckets
 // With codes wider than one radix digit the buckets are small (a few ids on average), and sorting the whole table
-// twice is a detour.  Instead every id reserves its slot with an atomic add on its bucket's offset word -- stored
-// one place up and started at the bucket's start, the word ends as the next bucket's start, i.e. exactly the final
-// offset array -- and the ids of each bucket are then put in ascending order where they stand: in registers for
+// twice is a detour.  Instead the hashing kernel's counting atomics hand every id its rank of arrival inside its
+// bucket, the id goes to the bucket's start plus that rank, and the ids of each bucket are then put in ascending
+// order where they stand: in registers for
 // buckets of up to ORD_SMALL ids, by a block-wide sort in shared memory up to ORD_BLOCK, and for a larger bucket by
 // one ordered pass over the table's codes that writes the matching ids out again.
 constexpr int ORD_SMALL = 16;
 constexpr int ORD_BLOCK = 4096;
 constexpr int ORD_THREADS = 256;
 
-__global__ void __launch_bounds__(256) k_place_ids(const uint32_t* keys, int32_t* off, int32_t* ids, int N, long long nb) {
+__global__ void __launch_bounds__(256) k_place_ids(const uint32_t* keys, const uint32_t* ranks, const int32_t* off, int32_t* ids,
+                                                   int N, long long nb) {
   const int t = blockIdx.y;
   const uint32_t* k = keys + (size_t)t * N;
-  int32_t* o = off + (size_t)t * (size_t)(nb + 1);
+  const uint32_t* r = ranks + (size_t)t * N;
+  const int32_t* o = off + (size_t)t * (size_t)(nb + 1);
   int32_t* out = ids + (size_t)t * N;
-  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < N; j += gridDim.x * blockDim.x) {
-    const int slot = atomicAdd(o + k[j] + 1, 1);
-    out[slot] = j;
-  }
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < N; j += gridDim.x * blockDim.x)
+    out[__ldg(o + k[j]) + (int)r[j]] = j;
 }
 
 // Sorts n <= M ids in place with an odd-even transposition network (fully unrolled: the ids stay in registers).
@@ -672,8 +695,8 @@ cudaError_t launch_build_tables(Ctx* c) {
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     LaunchScope ls(c, KID_HASH_NEURONS);
-    k_hash_neurons_dwta8<<<c->num_sms * per_sm, HN_THREADS, smem2, c->stream>>>(c->W2, c->hash_idx, c->keysA, c->bucket_off,
-                                                                              c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
+    k_hash_neurons_dwta8<<<c->num_sms * per_sm, HN_THREADS, smem2, c->stream>>>(c->W2, c->hash_idx, c->keysA, c->place_path ? c->keysB : nullptr,
+                                                                              c->bucket_off, c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
   } else {
     auto kern = fn_smem ? k_hash_neurons<true> : k_hash_neurons<false>;
     if (smem > 48 * 1024) {
@@ -686,7 +709,7 @@ cudaError_t launch_build_tables(Ctx* c) {
     if (per_sm < 1) per_sm = 1;
     LaunchScope ls(c, KID_HASH_NEURONS);
     kern<<<c->num_sms * per_sm, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
-                                                             c->bucket_off, c->N, c->H, c->K, c->L,
+                                                             c->place_path ? c->keysB : nullptr, c->bucket_off, c->N, c->H, c->K, c->L,
                                                              c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -695,7 +718,7 @@ cudaError_t launch_build_tables(Ctx* c) {
     dim3 grid(nchunks, c->L);
     LaunchScope ls(c, KID_BUCKET_SCAN);
     k_bucket_sums<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
-    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks, c->place_path);
+    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
@@ -703,7 +726,7 @@ cudaError_t launch_build_tables(Ctx* c) {
     {
       LaunchScope ls(c, KID_PLACE_IDS);
       dim3 grid((unsigned)min((long long)(c->N + 255) / 256, 1024LL), c->L);
-      k_place_ids<<<grid, 256, 0, c->stream>>>(c->keysA, c->bucket_off, c->bucket_ids, c->N, c->nb);
+      k_place_ids<<<grid, 256, 0, c->stream>>>(c->keysA, c->keysB, c->bucket_off, c->bucket_ids, c->N, c->nb);
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     // A query reads a whole bucket unless it holds more than `cap` ids, and the union of the buckets is put in
