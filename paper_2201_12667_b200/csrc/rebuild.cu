@@ -63,19 +63,28 @@ __global__ void k_draw_simhash(int32_t* idx, int32_t* sign, int KL, int H, int m
 }
 
 // DWTA: ceil(K*L*bin / H) random permutations of the coordinates, concatenated; hash function f
-// reads entries [f*bin, (f+1)*bin).  One thread per permutation.
-__global__ void k_draw_dwta(int32_t* idx, long long total, int H, uint64_t seed, uint64_t r, int nperm) {
-  int q = blockIdx.x * blockDim.x + threadIdx.x;
-  if (q >= nperm) return;
-  short perm[1024];
-  for (int i = 0; i < H; ++i) perm[i] = (short)i;
-  for (int i = H - 1; i >= 1; --i) {
-    uint64_t u = ctr_rng(seed, RNG_HASH, r, (uint64_t)q * (uint64_t)H + (uint64_t)i);
-    int j = (int)(u % (uint64_t)(i + 1));
-    short tmp = perm[i]; perm[i] = perm[j]; perm[j] = tmp;
+// reads entries [f*bin, (f+1)*bin).  One block per permutation: the swap partner of every position is drawn by
+// its own thread (the generator is counter-based), then one thread applies the swaps from the last position down.
+constexpr int DRAW_THREADS = 128;
+__global__ void __launch_bounds__(DRAW_THREADS) k_draw_dwta(int32_t* idx, long long total, int H, uint64_t seed, uint64_t r) {
+  extern __shared__ int draw_sm[];          // [H] permutation, [H] swap partners
+  int* perm = draw_sm;
+  int* partner = draw_sm + H;
+  const int q = blockIdx.x;
+  for (int i = threadIdx.x; i < H; i += DRAW_THREADS) {
+    perm[i] = i;
+    const uint64_t u = ctr_rng(seed, RNG_HASH, r, (uint64_t)q * (uint64_t)H + (uint64_t)i);
+    partner[i] = i >= 1 ? (int)(u % (uint64_t)(i + 1)) : 0;
   }
-  for (int i = 0; i < H; ++i) {
-    long long e = (long long)q * H + i;
+  __syncthreads();
+  if (threadIdx.x == 0)
+    for (int i = H - 1; i >= 1; --i) {
+      const int j = partner[i];
+      const int tmp = perm[i]; perm[i] = perm[j]; perm[j] = tmp;
+    }
+  __syncthreads();
+  for (int i = threadIdx.x; i < H; i += DRAW_THREADS) {
+    const long long e = (long long)q * H + i;
     if (e < total) idx[e] = perm[i];
   }
 }
@@ -88,7 +97,7 @@ cudaError_t launch_draw_hash(Ctx* c, int64_t r) {
   } else {
     long long total = (long long)c->KL * c->fn_len;
     int nperm = (int)((total + c->H - 1) / c->H);
-    k_draw_dwta<<<(nperm + 63) / 64, 64, 0, c->stream>>>(c->hash_idx, total, c->H, c->cfg.seed, (uint64_t)r, nperm);
+    k_draw_dwta<<<nperm, DRAW_THREADS, 2 * c->H * sizeof(int), c->stream>>>(c->hash_idx, total, c->H, c->cfg.seed, (uint64_t)r);
   }
   return cudaGetLastError();
 }
