@@ -236,7 +236,7 @@ __device__ __forceinline__ void skip_sample(const FwdParams& p, int s, int code)
   if (tid == 0) set_status(p.st, code);
 }
 
-template <int MODE>   // 0 = training step, 1 = predict top-k
+template <int MODE, int KPT>   // MODE 0 = training step, 1 = predict top-k; KPT = hidden units per thread (H <= KPT * FWD_THREADS)
 __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   float* sh_h = reinterpret_cast<float*>(smem);
@@ -297,7 +297,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   //      (in range, ascending) ----
   //      Up to here, and through the first chunk's column ids and values, only the caller's batch is read: the
   //      kernel may run that far while the previous step's update kernel is still finishing (griddep_wait).
-  float acc[MAX_KPT];
+  float acc[KPT];
   bool waited = false;
   uint32_t phase = 0;                // of sh_bar, which serves the staging of W1 rows here and of W2 rows below
   bool timed_out = false;
@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       bulk_g2s(stage + (size_t)i * H, p.W1 + (size_t)sh_col[i] * H, (uint32_t)H * 4u, sh_bar);
     if (c0 == 0) {
 #pragma unroll
-      for (int u = 0; u < MAX_KPT; ++u) {
+      for (int u = 0; u < KPT; ++u) {
         const int k = tid + u * FWD_THREADS;
         acc[u] = k < H ? p.b1[k] : 0.f;
       }
@@ -334,7 +334,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     phase ^= 1u;
     if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
 #pragma unroll
-    for (int u = 0; u < MAX_KPT; ++u) {
+    for (int u = 0; u < KPT; ++u) {
       const int k = tid + u * FWD_THREADS;
       if (k < H) {
         float a = acc[u];
@@ -347,7 +347,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   if (!waited) {                     // no nonzeros, or a bad column id: nothing of the model has been read yet
     griddep_wait();
 #pragma unroll
-    for (int u = 0; u < MAX_KPT; ++u) {
+    for (int u = 0; u < KPT; ++u) {
       const int k = tid + u * FWD_THREADS;
       acc[u] = k < H ? p.b1[k] : 0.f;
     }
@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     return;
   }
 #pragma unroll
-  for (int u = 0; u < MAX_KPT; ++u) {
+  for (int u = 0; u < KPT; ++u) {
     const int k = tid + u * FWD_THREADS;
     if (k < H) {
       const float hv = acc[u] > 0.f ? acc[u] : 0.f;
@@ -634,9 +634,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   float* sh_ce = stage + (size_t)stage_rows * ldr;           // [stage_rows]
   const bool streaming = MODE == 0 && na > stage_rows;
   float Mrun = -INFINITY, Erun = 0.f;
-  float accS[MAX_KPT], accT[MAX_KPT];
+  float accS[KPT], accT[KPT];
 #pragma unroll
-  for (int u = 0; u < MAX_KPT; ++u) { accS[u] = 0.f; accT[u] = 0.f; }
+  for (int u = 0; u < KPT; ++u) { accS[u] = 0.f; accT[u] = 0.f; }
   const int ngrp = H >= FWD_THREADS ? 1 : min(FWD_WARPS, FWD_THREADS / H);   // groups of H threads (sh_dh holds FWD_WARPS)
   const int grp = H >= FWD_THREADS ? 0 : tid / H;
   const uint32_t row_bytes = (uint32_t)H * 4u;
@@ -739,7 +739,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       Mrun = Mnew;
       if (grp < ngrp) {
 #pragma unroll
-        for (int u = 0; u < MAX_KPT; ++u) {
+        for (int u = 0; u < KPT; ++u) {
           const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
           if (k < H && (u == 0 || H > FWD_THREADS)) {
             float v0 = accS[u] * scale, v1 = 0.f, v2 = 0.f, v3 = 0.f;
@@ -856,14 +856,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   //      several groups of threads whose sums are then added in group order.  When the rows were streamed the
   //      sums exist already. ----
   {
-    float accd[MAX_KPT];
+    float accd[KPT];
 #pragma unroll
-    for (int u = 0; u < MAX_KPT; ++u)
+    for (int u = 0; u < KPT; ++u)
       accd[u] = streaming ? (accS[u] / E - (ny > 0 ? accT[u] / (float)ny : 0.f)) / fB : 0.f;
     if (!streaming && grp < ngrp) {
       const int nr = na;                           // all rows are still staged
 #pragma unroll
-      for (int u = 0; u < MAX_KPT; ++u) {
+      for (int u = 0; u < KPT; ++u) {
         const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
         if (k < H && (u == 0 || H > FWD_THREADS)) {
           float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
@@ -881,7 +881,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
     if (grp < ngrp) {
 #pragma unroll
-      for (int u = 0; u < MAX_KPT; ++u) {
+      for (int u = 0; u < KPT; ++u) {
         const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
         if (k < H && (u == 0 || H > FWD_THREADS)) sh_dh[(size_t)grp * H + k] = accd[u];
       }
@@ -1003,9 +1003,11 @@ cudaError_t setup_forward(Ctx* c) {
     }
   }
   c->fwd_smem = l.fixed_bytes + c->fwd_stage_bytes;
-  cudaError_t e = cudaFuncSetAttribute(k_forward<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_forward<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(k_forward<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<0, MAX_KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<1, MAX_KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  return e;
 }
 
 static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
@@ -1038,7 +1040,10 @@ cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, cons
   FwdParams p = make_params(c, batch, row_ptr, col_idx, vals, label_ptr, labels);
   {
     LaunchScope ls(c, KID_FORWARD);
-    cudaError_t e = launch_dependent(k_forward<0>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p);
+    // hidden layers of up to FWD_THREADS units take the variant with one unit per thread (less code, fewer registers)
+    cudaError_t e = c->H <= FWD_THREADS
+                        ? launch_dependent(k_forward<0, 1>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p)
+                        : launch_dependent(k_forward<0, MAX_KPT>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p);
     if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
@@ -1053,7 +1058,8 @@ cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int3
   if (dense) p.dense = 1;
   {
     LaunchScope ls(c, KID_PREDICT);
-    k_forward<1><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+    if (c->H <= FWD_THREADS) k_forward<1, 1><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+    else k_forward<1, MAX_KPT><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
   }
   return cudaGetLastError();
 }
