@@ -295,12 +295,20 @@ def run_dslide(args):
     ms = max_over_ranks(ms, world, "cuda")
     value = world * B * K / (ms * 1e-3)
 
-    # ---- second pass of the same K steps with a CUDA event pair around every kernel launch ----
+    # ---- second pass of the same K steps with a CUDA event pair around every kernel launch: on a fresh model taken
+    #      through the same warm-up, because the active sets grow as the model trains and a later window of steps
+    #      touches more rows ----
+    ds.dslide_destroy(ctx)
+    ctx = ds.dslide_init(cfg)
+    for i in range(W):
+        step(i)
+    ds.dslide_sync(ctx)
+    ds.dslide_cum_stats(ctx, reset=True)
     ds.dslide_profile_begin(ctx)
     for i in range(K):
-        step(W + K + i)
+        step(W + i)
     prof = ds.dslide_profile_end(ctx)
-    ds.dslide_cum_stats(ctx, reset=True)
+    cum_prof = ds.dslide_cum_stats(ctx, reset=True)      # the per-kernel times go with the rows these steps touched
 
     # ---- end to end: host buffers in, loss out, every step ----
     e2e = None
@@ -308,7 +316,11 @@ def run_dslide(args):
         # the pipelined host-buffer entry point: every step copies its inputs from pinned host memory to the device
         # and its {status, loss} back; the loss of step i is handed out by call i + 1 (the last one by
         # dslide_host_result), so the device always has one step queued while the host packs the next
-        for i in range(3):
+        # on a fresh model taken through the same warm-up, so that the timed steps are the same training steps as in
+        # the device-resident pass (the active sets grow as the model trains, and later windows run slower)
+        ds.dslide_destroy(ctx)
+        ctx = ds.dslide_init(cfg)
+        for i in range(W):
             ds.dslide_train_step_host_async(ctx, B, *pinned[i % nb])
         ds.dslide_host_result(ctx)
         barrier()
@@ -338,10 +350,12 @@ def run_dslide(args):
                              "share": kms / total_prof}
         dominant = max((n for n in prof if n in ("adam", "forward")), key=lambda n: prof[n][0])
         dur = prof[dominant][0] * 1e-3 / prof[dominant][1]
-        achieved = model[dominant] / dur / 1e9
+        per_step_prof = {k: cum_prof[k] / max(1, cum_prof["steps"]) for k in per_step}
+        model_prof = byte_model(c, B, per_step_prof, labels_per_step, args.rebuild_period)
+        achieved = model_prof[dominant] / dur / 1e9
         roofline = {"bound": "hbm", "kernel": "k_" + dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(dominant),
-                    "algorithmic_bytes_per_launch": model[dominant], "us_per_launch": dur * 1e6,
+                    "algorithmic_bytes_per_launch": model_prof[dominant], "us_per_launch": dur * 1e6,
                     "peak_source": "MEASURED_PEAKS.json hbm_gbs (of %s)" % peak_kind}
         step_gbs = model["total"] / (ms * 1e-3 / K) / 1e9
         out = {

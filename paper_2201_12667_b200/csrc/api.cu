@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <new>
+#include <atomic>
 #include <vector>
 
 #include "common.cuh"
@@ -61,17 +62,14 @@ void free_all(Ctx* c) {
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1,
                   c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
-                  c->st_dev[0], c->st_dev[1]};
+                  c->st_dev[0], c->st_dev[1], c->st_dev[2]};
   for (void* p : ptrs) if (p) cudaFree(p);
-  for (int b = 0; b < 2; ++b) {
+  for (int b = 0; b < ST_SETS; ++b) {
     if (c->st_host[b]) cudaFreeHost(c->st_host[b]);
-    if (c->st_result[b]) cudaFreeHost(c->st_result[b]);
-    if (c->st_event[b]) cudaEventDestroy(c->st_event[b]);
+    if (c->st_res[b]) cudaFreeHost(c->st_res[b]);
     if (c->st_in[b]) cudaEventDestroy(c->st_in[b]);
-    if (c->st_done[b]) cudaEventDestroy(c->st_done[b]);
   }
   if (c->st_copy_in) cudaStreamDestroy(c->st_copy_in);
-  if (c->st_copy_out) cudaStreamDestroy(c->st_copy_out);
   if (c->prof) {
     auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
     for (auto& r : *v) { cudaEventDestroy(r.beg); cudaEventDestroy(r.end); }
@@ -241,14 +239,15 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     A(bucket_part, (size_t)c->L * (size_t)((c->nb + 1 + bucket_scan_chunk() - 1) / bucket_scan_chunk()), false);
   }
 #undef A
-  for (int b = 0; b < 2; ++b) {
-    if (e == cudaSuccess) e = cudaMallocHost((void**)&c->st_result[b], 4 * sizeof(float));
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->st_event[b], cudaEventDisableTiming);
+  for (int b = 0; b < ST_SETS; ++b) {
+    if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->st_res[b], sizeof(HostResult), cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+      memset(c->st_res[b], 0, sizeof(HostResult));
+      e = cudaHostGetDevicePointer((void**)&c->st_res_dev[b], c->st_res[b], 0);
+    }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->st_in[b], cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->st_done[b], cudaEventDisableTiming);
   }
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_copy_in, cudaStreamNonBlocking);
-  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->st_copy_out, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = setup_forward(c);
   if (e == cudaSuccess) e = launch_init_gauss(c, c->W1, (int64_t)(D * H), RNG_W1);
   if (e == cudaSuccess) e = launch_init_gauss(c, c->W2, (int64_t)(N * H), RNG_W2);
@@ -286,14 +285,15 @@ dslide_status dslide_build_tables(dslide_ctx* ctx) {
   return rebuild(&ctx->c, false);
 }
 
-dslide_status dslide_train_step(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
-                                const float* vals, const int32_t* label_ptr, const int32_t* labels, float* loss_out) {
-  if (!ctx || !row_ptr || !col_idx || !vals || !label_ptr || !labels) return DSLIDE_ERR_INVALID_ARG;
+namespace {
+
+// One step.  With host_res, the update kernel also reports {status, loss, host_seq} into mapped host memory.
+dslide_status train_step_impl(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
+                              const float* vals, const int32_t* label_ptr, const int32_t* labels, float* loss_out,
+                              HostResult* host_res, unsigned int host_seq) {
   Ctx* c = &ctx->c;
-  if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
-  if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
   CU(launch_forward_train(c, batch, row_ptr, col_idx, vals, label_ptr, labels));
-  CU(launch_update(c, batch, row_ptr, col_idx, vals, loss_out));
+  CU(launch_update(c, batch, row_ptr, col_idx, vals, loss_out, host_res, host_seq));
   c->t_host += 1;
   if (c->cfg.rebuild_period0 > 0 && c->t_host == c->next_rebuild) {
     dslide_status s = rebuild(c, true);
@@ -305,18 +305,39 @@ dslide_status dslide_train_step(dslide_ctx* ctx, int32_t batch, const int32_t* r
   return DSLIDE_OK;
 }
 
+}  // namespace
+
+dslide_status dslide_train_step(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
+                                const float* vals, const int32_t* label_ptr, const int32_t* labels, float* loss_out) {
+  if (!ctx || !row_ptr || !col_idx || !vals || !label_ptr || !labels) return DSLIDE_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
+  if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
+  return train_step_impl(ctx, batch, row_ptr, col_idx, vals, label_ptr, labels, loss_out, nullptr, 0u);
+}
+
 namespace {
 
-// Hands out the result of the step that used staging set b: waits for it, returns the sticky status as it stood
-// at the end of that step, stores its mean loss.
+// Hands out the result of the step that used staging set b: waits until the update kernel of that step has
+// written its sequence number into the set's mapped result record, returns the sticky status as it stood at the
+// end of that step, stores its mean loss.  The wait polls host memory; every so often it also asks whether the
+// stream has gone idle or failed, so that a step that never reports ends the wait with an error.
 dslide_status take_result(Ctx* c, int b, float* loss_out) {
   if (!c->st_pending[b]) return DSLIDE_OK;
-  CU(cudaEventSynchronize(c->st_event[b]));
   c->st_pending[b] = 0;
-  int status = 0;
-  memcpy(&status, c->st_result[b], sizeof(int));
-  if (loss_out) *loss_out = c->st_result[b][1 + b];
-  return (dslide_status)status;
+  volatile HostResult* r = c->st_res[b];
+  const unsigned int want = c->st_seq[b];
+  for (unsigned long long spins = 1; r->seq != want; ++spins) {
+    if ((spins & 0x3ffu) == 0) {
+      cudaError_t q = cudaStreamQuery(c->stream);
+      if (q == cudaErrorNotReady) continue;
+      if (q != cudaSuccess) return DSLIDE_ERR_CUDA;
+      if (r->seq != want) return DSLIDE_ERR_CUDA;      // the stream is idle and the step has not reported
+    }
+  }
+  std::atomic_thread_fence(std::memory_order_acquire);
+  if (loss_out) *loss_out = r->loss;
+  return (dslide_status)r->status;
 }
 
 // With the stream drained, a reported status is cleared on the device (as dslide_sync does).
@@ -329,8 +350,8 @@ dslide_status drain_and_clear(Ctx* c, dslide_status s) {
   return s;
 }
 
-// Packs a host batch into staging set b (one pinned buffer, 16-byte aligned pieces), sends it in a single copy,
-// enqueues the step and the copy of {status, loss} back, and records the set's event.
+// Packs a host batch into staging set b (one pinned buffer, 16-byte aligned pieces), sends it in a single copy
+// and enqueues the step.
 dslide_status enqueue_host_step(dslide_ctx* ctx, int b, int32_t batch, const int32_t* row_ptr, const int32_t* col_idx,
                                 const float* vals, const int32_t* label_ptr, const int32_t* labels) {
   Ctx* c = &ctx->c;
@@ -360,22 +381,19 @@ dslide_status enqueue_host_step(dslide_ctx* ctx, int b, int32_t batch, const int
   memcpy(hb + o_col, col_idx, sizeof(int32_t) * (size_t)nnz);
   memcpy(hb + o_val, vals, sizeof(float) * (size_t)nnz);
   memcpy(hb + o_lab, labels, sizeof(int32_t) * (size_t)nlab);
-  // The input copy and the result copy run on streams of their own, tied to the step by events, so that they
-  // overlap the kernels of the neighbouring steps.  (The device buffer of this set was last read two steps ago;
-  // the caller waited for that step when it collected its result.)
+  // The input copy runs on a stream of its own, beside the kernels of the previous step, and the host waits for
+  // it here (the device is busy with that step meanwhile).  Nothing but the step's kernels then goes into the
+  // compute stream, so consecutive steps keep their kernel-to-kernel overlap; the result comes back through the
+  // set's mapped record, written by the update kernel.  (The device buffer of this set was last read three steps
+  // ago, by kernels that had finished before the result collected last could be written.)
   CU(cudaMemcpyAsync(db, hb, total, cudaMemcpyHostToDevice, c->st_copy_in));
   CU(cudaEventRecord(c->st_in[b], c->st_copy_in));
-  CU(cudaStreamWaitEvent(st, c->st_in[b], 0));
-  dslide_status s = dslide_train_step(ctx, batch, (const int32_t*)(db + o_rp), (const int32_t*)(db + o_col),
-                                      (const float*)(db + o_val), (const int32_t*)(db + o_lp),
-                                      (const int32_t*)(db + o_lab), &c->dstate->host_loss[b]);
+  CU(cudaEventSynchronize(c->st_in[b]));
+  c->st_seq[b] = ++c->st_counter;
+  dslide_status s = train_step_impl(ctx, batch, (const int32_t*)(db + o_rp), (const int32_t*)(db + o_col),
+                                    (const float*)(db + o_val), (const int32_t*)(db + o_lp),
+                                    (const int32_t*)(db + o_lab), nullptr, c->st_res_dev[b], c->st_seq[b]);
   if (s != DSLIDE_OK) { cudaStreamSynchronize(st); return s; }
-  // the sticky status and the two sets' losses sit side by side: one copy brings them back
-  static_assert(offsetof(DevState, host_loss) == sizeof(int), "status and losses are copied together");
-  CU(cudaEventRecord(c->st_done[b], st));
-  CU(cudaStreamWaitEvent(c->st_copy_out, c->st_done[b], 0));
-  CU(cudaMemcpyAsync(c->st_result[b], c->dstate, 3 * sizeof(float), cudaMemcpyDeviceToHost, c->st_copy_out));
-  CU(cudaEventRecord(c->st_event[b], c->st_copy_out));
   c->st_pending[b] = 1;
   return DSLIDE_OK;
 }
@@ -390,12 +408,12 @@ dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32
   if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
   if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
   // results of earlier pipelined steps that nobody collected are dropped (their status stays sticky on the device)
-  for (int b = 0; b < 2; ++b)
-    if (c->st_pending[b]) { CU(cudaEventSynchronize(c->st_event[b])); c->st_pending[b] = 0; }
+  for (int b = 0; b < ST_SETS; ++b)
+    if (c->st_pending[b]) { dslide_status w = take_result(c, b, nullptr); if (w == DSLIDE_ERR_CUDA) return w; }
   const int b = c->st_next;
   dslide_status s = enqueue_host_step(ctx, b, batch, row_ptr, col_idx, vals, label_ptr, labels);
   if (s != DSLIDE_OK) return s;
-  c->st_next ^= 1;
+  c->st_next = (b + 1) % ST_SETS;
   s = take_result(c, b, loss_out);
   return drain_and_clear(c, s);
 }
@@ -408,22 +426,27 @@ dslide_status dslide_train_step_host_async(dslide_ctx* ctx, int32_t batch, const
   if (batch < 1) return DSLIDE_ERR_INVALID_ARG;
   if (batch > c->cfg.max_batch) return DSLIDE_ERR_OVERFLOW;
   const int b = c->st_next;
-  // the set about to be reused belongs to the step before the previous one: its result was handed out one call
-  // ago, or is dropped here if that call failed
-  if (c->st_pending[b]) { CU(cudaEventSynchronize(c->st_event[b])); c->st_pending[b] = 0; }
+  // the set about to be reused belongs to the step three calls back, whose result was handed out long ago -- unless a
+  // call in between failed: then it is dropped here and the stream is drained, so that no kernel still reads the set
+  if (c->st_pending[b]) {
+    dslide_status w = take_result(c, b, nullptr);
+    if (w == DSLIDE_ERR_CUDA) return w;
+    CU(cudaStreamSynchronize(c->stream));
+  }
   dslide_status s = enqueue_host_step(ctx, b, batch, row_ptr, col_idx, vals, label_ptr, labels);
   if (s != DSLIDE_OK) return s;
-  c->st_next ^= 1;
+  c->st_next = (b + 1) % ST_SETS;
   // while the device works on this step, collect the previous one
-  const int had = c->st_pending[b ^ 1];
+  const int prev = (b + ST_SETS - 1) % ST_SETS;
+  const int had = c->st_pending[prev];
   if (have_prev) *have_prev = had;
-  return take_result(c, b ^ 1, prev_loss_out);
+  return take_result(c, prev, prev_loss_out);
 }
 
 dslide_status dslide_host_result(dslide_ctx* ctx, float* loss_out, int32_t* have) {
   if (!ctx) return DSLIDE_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
-  const int newest = c->st_next ^ 1, older = c->st_next;
+  const int newest = (c->st_next + ST_SETS - 1) % ST_SETS, older = (c->st_next + ST_SETS - 2) % ST_SETS;
   dslide_status s_old = take_result(c, older, nullptr);     // only pending if its collection was skipped
   if (have) *have = c->st_pending[newest];
   dslide_status s = take_result(c, newest, loss_out);

@@ -30,8 +30,7 @@ enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2 };
 // in the synchronous statistics and status calls).
 struct DevState {
   int status;                      // sticky dslide_status seen on the device
-  float host_loss[2];              // mean loss of the last host-buffer step that used staging set 0 / 1
-  int pad0;
+  int pad0[3];
   // Slots indexed by the parity of the step: the kernels of step t use slot t & 1 and the update
   // kernel zeroes the other slot for step t + 1.
   unsigned int n_own[2][2];        // distinct touched rows of W2 ([.][0]) and W1 ([.][1]): lengths of the row lists
@@ -41,6 +40,16 @@ struct DevState {
   unsigned long long acc[2][3];    // forward kernel: sum of active-set sizes, nonzeros, bucket entries read
   unsigned long long last[3];      // acc of the last finished step
   unsigned long long cum[6];       // since the last reset: steps, sum_active, U2, U1, nnz, fetched
+};
+
+// What a host-buffer step reports straight into pinned host memory: the update kernel writes status and loss,
+// then (after a system-wide fence) the step's sequence number, which the host polls.
+constexpr int ST_SETS = 3;      // staging sets of the host-buffer steps
+struct HostResult {
+  unsigned int seq;
+  int status;
+  float loss;
+  int pad;
 };
 
 // Touches of a row of W1 / W2 whose (sample, coefficient) pair is stored with the row; further touches of the
@@ -109,7 +118,7 @@ cudaError_t launch_order_buckets(Ctx* c, int min_n);
 cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
                                  const float* vals, const int32_t* label_ptr, const int32_t* labels);
 cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
-                          float* loss_out);
+                          float* loss_out, HostResult* host_res, unsigned int host_seq);
 cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
                            const float* vals, int k, int dense, int32_t* out_ids, float* out_scores);
 cudaError_t setup_forward(Ctx* c);   // chooses the dedup path and the shared-memory layout
@@ -168,13 +177,17 @@ struct Ctx {
 
   // staging for the host-buffer entry point
   // host-buffer entry points: two sets of (device buffer, pinned host buffer, pinned result, event), used in turn
-  unsigned char *st_dev[2], *st_host[2];
-  int64_t st_cap[2];
-  float* st_result[2];        // pinned: {sticky status (int bits), mean loss} of the step that used the set
-  cudaEvent_t st_event[2];    // recorded after that step's result copy
-  cudaEvent_t st_in[2], st_done[2];   // input copy finished / kernels of the step finished
-  cudaStream_t st_copy_in, st_copy_out;   // the copies run beside the kernels of the neighbouring steps
-  int st_pending[2];          // a step was enqueued on the set and its result has not been handed out yet
+  // Three sets in rotation: when step t is packed, the result of step t - 2 has been collected, which proves
+  // that every kernel up to the forward kernel of step t - 2 has finished -- so the set of step t - 3 is free,
+  // while the update kernel of step t - 2 may still be reading its own.
+  unsigned char *st_dev[ST_SETS], *st_host[ST_SETS];
+  int64_t st_cap[ST_SETS];
+  HostResult *st_res[ST_SETS], *st_res_dev[ST_SETS];   // pinned, device-mapped: what the update kernel reports of the step that used the set
+  unsigned int st_seq[ST_SETS];                  // sequence number that step was given
+  unsigned int st_counter;                 // sequence numbers handed out so far
+  cudaEvent_t st_in[ST_SETS];                    // input copy finished
+  cudaStream_t st_copy_in;                 // the input copy runs beside the kernels of the previous step
+  int st_pending[ST_SETS];          // a step was enqueued on the set and its result has not been handed out yet
   int st_next;                // set the next host-buffer step uses
 
   int64_t t_host, r_host, next_rebuild;

@@ -49,6 +49,8 @@ struct UpdParams {
   int* hot_done;
   DevState* st;
   float* loss_out;
+  HostResult* host_res;        // mapped host memory that receives {status, loss, sequence number}, or null
+  unsigned int host_seq;
   int B, H, N, D, Wd, act_stride, dense, parity;
   float lr, beta1, beta2, eps, rb1, rb2;
 };
@@ -337,6 +339,12 @@ __device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
     for (int w = 0; w < UPD_WARPS; ++w) r += sm_part[w];
     if (p.loss_out) *p.loss_out = r / (float)B;
     DevState* st = p.st;
+    if (p.host_res) {            // the forward kernel has finished: the sticky status covers this step
+      p.host_res->status = st->status;
+      p.host_res->loss = r / (float)B;
+      __threadfence_system();
+      *reinterpret_cast<volatile unsigned int*>(&p.host_res->seq) = p.host_seq;
+    }
     const int q = p.parity, o = q ^ 1;
     st->last[0] = st->acc[q][0]; st->last[1] = st->acc[q][1]; st->last[2] = st->acc[q][2];
     st->cum[0] += 1ull; st->cum[1] += st->acc[q][0]; st->cum[4] += st->acc[q][1]; st->cum[5] += st->acc[q][2];
@@ -601,7 +609,7 @@ static cudaError_t launch_k_update(Ctx* c, const UpdParams& p, int smem) {
 }
 
 cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
-                          float* loss_out) {
+                          float* loss_out, HostResult* host_res, unsigned int host_seq) {
   UpdParams p;
   p.W1 = c->W1; p.mW1 = c->mW1; p.vW1 = c->vW1; p.b1 = c->b1; p.mb1 = c->mb1; p.vb1 = c->vb1;
   p.W2 = c->W2; p.mW2 = c->mW2; p.vW2 = c->vW2;
@@ -610,7 +618,7 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   p.mask1 = c->mask1; p.mask2 = c->mask2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
   p.own1 = c->own1; p.own2 = c->own2;
   p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.hot_part = c->hot_part; p.hot_done = c->hot_done;
-  p.st = c->dstate; p.loss_out = loss_out;
+  p.st = c->dstate; p.loss_out = loss_out; p.host_res = host_res; p.host_seq = host_seq;
   p.B = batch; p.H = c->H; p.N = c->N; p.D = c->D; p.Wd = c->Wd; p.act_stride = c->act_stride; p.dense = c->dense;
   p.parity = (int)(c->t_host & 1);
   p.lr = c->cfg.lr; p.beta1 = c->cfg.beta1; p.beta2 = c->cfg.beta2; p.eps = c->cfg.eps;
