@@ -143,8 +143,9 @@ dslide_status dslide_train_step_host(dslide_ctx* ctx, int32_t batch, const int32
                                      float* loss_out);
 
 /* The same step, pipelined: the call packs and enqueues this batch and returns as soon as the PREVIOUS
- * host-buffer step has finished, handing out that step's mean loss (*prev_loss_out, may be NULL) and sticky
- * status (the return value); *have_prev (may be NULL) tells whether there was a previous step to report.
+ * host-buffer step has reported -- its loss and status are known, its weight update may still be running --
+ * handing out that step's mean loss (*prev_loss_out, may be NULL) and sticky status (the return value);
+ * *have_prev (may be NULL) tells whether there was a previous step to report.
  * The device therefore always has one step queued while the host prepares the next.  The arrays are copied
  * into the library's pinned buffer before the call returns, so the caller may reuse them at once.
  * dslide_host_result waits for the newest pipelined step and hands out its loss and status (*have = 0 and
