@@ -38,9 +38,19 @@ from paper_2201_12667_b200 import workloads  # noqa: E402
 METRIC = "train samples/s at 670K-class shape on 1 B200; achieved HBM GB/s vs peak"
 REBUILD_PERIOD = 50
 REF_BATCH = 32            # samples per step of the CPU-oracle arm (a bounded sample of the 256-sample batch)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (None until a capture of the current kernel exists)
-NCU_TRAFFIC_BYTES = {"adam": 106.5e6, "forward": 34.3e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/, taken
+# on early steps of this workload (more rows touched than in the timed window) and therefore kept as a ratio to
+# the bytes that scale with the rows of the launch: update kernel 107.8 MB measured against 149.5 MB algorithmic;
+# forward kernel 34.4 MB measured against the 32.2 MB of W1 / W2 rows it gathers.
+NCU_TRAFFIC_RATIO = {"adam": 107.8 / 149.5, "forward": 34.4 / 32.2}
+
+
+def ncu_traffic(kernel, c, per_step, model):
+    if kernel == "adam":
+        return NCU_TRAFFIC_RATIO["adam"] * model["adam"]
+    if kernel == "forward":
+        return NCU_TRAFFIC_RATIO["forward"] * 4 * c["H"] * (per_step["nnz"] + per_step["sum_active"])
+    return None
 
 
 def parse_args():
@@ -354,7 +364,7 @@ def run_dslide(args):
         model_prof = byte_model(c, B, per_step_prof, labels_per_step, args.rebuild_period)
         achieved = model_prof[dominant] / dur / 1e9
         roofline = {"bound": "hbm", "kernel": "k_" + dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                    "frac": achieved / peak, "traffic": ncu_traffic(dominant, c, per_step_prof, model_prof),
                     "algorithmic_bytes_per_launch": model_prof[dominant], "us_per_launch": dur * 1e6,
                     "peak_source": "MEASURED_PEAKS.json hbm_gbs (of %s)" % peak_kind}
         step_gbs = model["total"] / (ms * 1e-3 / K) / 1e9
