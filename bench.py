@@ -41,16 +41,12 @@ REF_BATCH = 32            # samples per step of the CPU-oracle arm (a bounded sa
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/, taken
 # on early steps of this workload (more rows touched than in the timed window) and therefore kept as a ratio to
 # the bytes that scale with the rows of the launch: update kernel 107.8 MB measured against 149.5 MB algorithmic;
-# forward kernel 34.4 MB measured against the 32.2 MB of W1 / W2 rows it gathers.
-NCU_TRAFFIC_RATIO = {"adam": 107.8 / 149.5, "forward": 34.4 / 32.2}
+# forward kernel 34.4 MB measured against 33.3 MB (the rows of W1 / W2 it gathers, tables, batch).
+NCU_TRAFFIC_RATIO = {"adam": 107.8 / 149.5, "forward": 34.4 / 33.3}
 
 
-def ncu_traffic(kernel, c, per_step, model):
-    if kernel == "adam":
-        return NCU_TRAFFIC_RATIO["adam"] * model["adam"]
-    if kernel == "forward":
-        return NCU_TRAFFIC_RATIO["forward"] * 4 * c["H"] * (per_step["nnz"] + per_step["sum_active"])
-    return None
+def ncu_traffic(kernel, model):
+    return NCU_TRAFFIC_RATIO[kernel] * model[kernel] if kernel in NCU_TRAFFIC_RATIO else None
 
 
 def parse_args():
@@ -96,9 +92,11 @@ def byte_model(c, B, per_step, labels_per_step, gap):
     hid = 2 * 4 * B * H
     rebuild = (4 * H * N + 4 * N * L + 4 * L * (2 ** code_bits(c) + 1)) / gap if gap else 0.0
     total = csr + lab + w1 + w2 + b1 + tables + act + hid + rebuild
+    # per kernel: the update kernel is booked the rows (read and write of w, m, v); the forward kernel, being a kernel
+    # of its own, cannot be served those rows on chip, so its figure adds the rows it gathers (once each per use)
     return dict(total=total, rebuild=rebuild,
                 adam=w1 + w2 + b1 + act / 2 + hid / 2,
-                forward=csr + lab + tables + act / 2 + hid / 2)
+                forward=csr + lab + tables + act / 2 + hid / 2 + 4 * H * nnz + 4 * (H + 1) * sumA)
 
 
 class ClockSampler:
@@ -364,7 +362,7 @@ def run_dslide(args):
         model_prof = byte_model(c, B, per_step_prof, labels_per_step, args.rebuild_period)
         achieved = model_prof[dominant] / dur / 1e9
         roofline = {"bound": "hbm", "kernel": "k_" + dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": ncu_traffic(dominant, c, per_step_prof, model_prof),
+                    "frac": achieved / peak, "traffic": ncu_traffic(dominant, model_prof),
                     "algorithmic_bytes_per_launch": model_prof[dominant], "us_per_launch": dur * 1e6,
                     "peak_source": "MEASURED_PEAKS.json hbm_gbs (of %s)" % peak_kind}
         step_gbs = model["total"] / (ms * 1e-3 / K) / 1e9
