@@ -24,6 +24,13 @@ CONFIGS = {
                  batch=256, mean_nnz=42, mean_labels=3, dist="zipf", lr=1e-4, max_labels=16),
     "1b": dict(D=200000, H=256, N=4000000, family=DWTA, K=7, L=64, bin_size=8, srp_nnz=0, bucket_cap=256,
                batch=512, mean_nnz=100, mean_labels=4, dist="zipf", lr=1e-4, max_labels=16),
+    # the paper's second dataset (Table 1: 253,855 words in and out, about one nonzero per sample; Table 3: hidden
+    # layer 200, batch 1024 or 2048): one-hot inputs, a few context words as labels
+    "text8": dict(D=253855, H=200, N=253855, family=SIMHASH, K=9, L=50, bin_size=8, srp_nnz=0, bucket_cap=128,
+                  batch=1024, mean_nnz=1, fixed_nnz=1, mean_labels=4, dist="zipf", lr=1e-4, max_labels=16),
+    # the 670K shape with the large hidden layer and batch of Table 3
+    "670k-h1024": dict(D=135909, H=1024, N=670091, family=DWTA, K=6, L=50, bin_size=8, srp_nnz=0, bucket_cap=128,
+                       batch=1024, mean_nnz=76, mean_labels=5, dist="zipf", lr=1e-4, max_labels=16),
     # a mid-size shape for parity tests: several tiles, ragged tails, both dedup paths
     "mid": dict(D=5003, H=128, N=20011, family=DWTA, K=3, L=10, bin_size=8, srp_nnz=0, bucket_cap=16,
                 batch=48, mean_nnz=30, mean_labels=3, dist="zipf", lr=1e-3, max_labels=16),
@@ -88,7 +95,7 @@ class Workload:
                 ny = int(rng.integers(1, c["max_labels"] + 1))
                 y = rng.choice(c["N"], size=ny, replace=False).astype(np.int32)
             else:
-                nnz = int(np.clip(rng.poisson(c["mean_nnz"]), 1, min(4 * c["mean_nnz"], c["D"])))
+                nnz = c.get("fixed_nnz") or int(np.clip(rng.poisson(c["mean_nnz"]), 1, min(4 * c["mean_nnz"], c["D"])))
                 ids = self.feat.distinct(rng, nnz)
                 v = np.exp(rng.standard_normal(nnz))
                 v = (v / np.sqrt(np.sum(v * v))).astype(np.float32)

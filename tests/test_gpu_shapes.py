@@ -189,3 +189,18 @@ def test_same_step_repeated_gives_the_same_outputs(H):
                 assert np.array_equal(cur[n], ref[n]), (it, n)
     finally:
         pr.close()
+
+
+def test_one_hot_inputs_and_hidden_layer_of_200():
+    """The shape of the paper's second dataset at a reduced vocabulary (Table 1, Table 3): one nonzero per sample,
+    hidden layer 200 (fifty 16-byte pieces per row: the two-piece register layout of the update kernel with a
+    ragged second piece), batch 64 -- words repeat within a batch, so rows of W1 are shared by several samples."""
+    V = 20011
+    pr = Pair(D=V, H=200, N=V, family=SIMHASH, K=6, L=8, bucket_cap=32, max_batch=64, max_labels=16, lr=1e-3, seed=8)
+    try:
+        wl = workloads.Workload(workloads.config("text8", D=V, N=V), seed=15)
+        batches = [wl.batch(i, batch_size=64) for i in range(2)]
+        assert all(np.all(np.diff(b[0]) == 1) for b in batches)
+        one_and_two_steps(pr, batches)
+    finally:
+        pr.close()
