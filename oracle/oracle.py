@@ -41,7 +41,7 @@ class OrcConfig(C.Structure):
         ("family", C.c_int32), ("K", C.c_int32), ("L", C.c_int32),
         ("bin_size", C.c_int32), ("srp_nnz", C.c_int32), ("bucket_cap", C.c_int32),
         ("rebuild_period0", C.c_int32), ("redraw", C.c_int32), ("force_dense", C.c_int32),
-        ("max_active", C.c_int32),
+        ("max_active", C.c_int32), ("densify", C.c_int32),
         ("rebuild_lambda", C.c_double),
         ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
         ("init_std", C.c_double),
@@ -86,6 +86,7 @@ def _load(real):
         lib.orc_build_tables.argtypes = [C.c_void_p]
         lib.orc_rebuild_tables.argtypes = [C.c_void_p]
         lib.orc_hash_vec.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.orc_hash_query.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.orc_forward.restype = C.c_int32
         lib.orc_forward.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 5
         lib.orc_backward.argtypes = [C.c_void_p]
@@ -117,7 +118,7 @@ class Oracle:
         self.dtype = np.float32 if real == "float" else np.float64
         self.lib = _load(real)
         d = dict(family=SIMHASH, bin_size=8, srp_nnz=0, bucket_cap=128, rebuild_period0=0, redraw=1,
-                 force_dense=0, max_active=0, rebuild_lambda=0.0, lr=1e-4, beta1=0.9, beta2=0.999,
+                 force_dense=0, max_active=0, densify=0, rebuild_lambda=0.0, lr=1e-4, beta1=0.9, beta2=0.999,
                  eps=1e-8, init_std=0.01, seed=0)
         d.update(kw)
         self.cfg = OrcConfig(**d)
@@ -194,6 +195,14 @@ class Oracle:
         assert v.shape == (self.H,)
         out = np.zeros(self.L, dtype=np.uint32)
         self.lib.orc_hash_vec(self.o, _p(v), _p(out))
+        return out
+
+    def hash_query(self, v):
+        """Codes of a query (a hidden activation): as hash_vec, plus densification of all-zero DWTA bins when set."""
+        v = np.ascontiguousarray(v, dtype=self.dtype)
+        assert v.shape == (self.H,)
+        out = np.zeros(self.L, dtype=np.uint32)
+        self.lib.orc_hash_query(self.o, _p(v), _p(out))
         return out
 
     def _batch(self, row_ptr, col_idx, vals, label_ptr=None, labels=None):

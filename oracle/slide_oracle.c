@@ -48,6 +48,7 @@ typedef struct {
   int32_t redraw;           /* draw new hash functions at every rebuild (Algorithm 1, last line) */
   int32_t force_dense;      /* "sparsity is 1" (Section 3.6): every output neuron is active      */
   int32_t max_active;       /* 0 = no limit; otherwise a larger active set is an error           */
+  int32_t densify;          /* DWTA: an all-zero bin of a query borrows another bin's position   */
   double rebuild_lambda;    /* gap_i = max(1, floor(p0 * exp(lambda * i)))                       */
   double lr, beta1, beta2, eps;   /* Adam (Section 4.1)                                          */
   double init_std;
@@ -102,7 +103,8 @@ uint64_t orc_rng(uint64_t seed, uint64_t stream, uint64_t r, uint64_t ctr) {
   uint64_t b = mix64(a + GOLD * (r + 1));
   return mix64(b + GOLD * (ctr + 1));
 }
-enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2 };
+enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3 };
+enum { DENSIFY_ATTEMPTS = 16 };
 
 static double u01(uint64_t x) { return ((double)(x >> 11) + 0.5) * (1.0 / 9007199254740992.0); }
 
@@ -177,9 +179,29 @@ void orc_draw_hash(orc *o, int64_t r) {
  * bit = (s >= 0); code = sum_k bit_k << k.
  * DWTA, reading: position of the maximum inside the bin, the lowest
  * position winning ties (so an all-equal bin gives 0);
- * code = sum_k pos_k << (k * log2(bin)). */
-void orc_hash_vec(const orc *o, const REAL *v, uint32_t *codes) {
+ * code = sum_k pos_k << (k * log2(bin)).
+ * Densification (the "D" of DWTA, Section 4.1 names it only; reading, used
+ * for queries when the flag is set): a bin of a query whose values are all
+ * zero carries no information, so function p borrows the position of another
+ * function's bin: it probes the functions p + 1 + (rng(seed, STREAM_PROBE,
+ * r, p * DENSIFY_ATTEMPTS + a) mod (K*L - 1)) (mod K*L), a = 0, 1, ...,
+ * DENSIFY_ATTEMPTS - 1, and takes the position of the first one whose own bin
+ * is not all zero (never a borrowed one); when every probe fails, 0. */
+static int dwta_position(const orc *o, const REAL *v, int p, int *all_zero) {
+  const int bs = o->c.bin_size;
+  const int32_t *idx = o->hash_idx + (size_t)p * bs;
+  int best = 0, zero = 1;
+  for (int i = 0; i < bs; ++i) {
+    if (v[idx[i]] != 0) zero = 0;
+    if (i >= 1 && v[idx[i]] > v[idx[best]]) best = i;
+  }
+  *all_zero = zero;
+  return best;
+}
+
+static void hash_vec(const orc *o, const REAL *v, uint32_t *codes, int is_query) {
   const orc_config *c = &o->c;
+  const int KL = c->K * c->L;
   for (int t = 0; t < c->L; ++t) {
     uint32_t code = 0;
     for (int k = 0; k < c->K; ++k) {
@@ -195,16 +217,29 @@ void orc_hash_vec(const orc *o, const REAL *v, uint32_t *codes) {
       } else {
         int bs = c->bin_size, lg = 0;
         while ((1 << lg) < bs) ++lg;
-        const int32_t *idx = o->hash_idx + (size_t)p * bs;
-        int best = 0;
-        for (int i = 1; i < bs; ++i)
-          if (v[idx[i]] > v[idx[best]]) best = i;
+        int zero;
+        int best = dwta_position(o, v, p, &zero);
+        if (zero && is_query && c->densify && KL > 1) {
+          best = 0;
+          for (int a = 0; a < DENSIFY_ATTEMPTS; ++a) {
+            uint64_t u = orc_rng(c->seed, STREAM_PROBE, (uint64_t)o->r, (uint64_t)p * DENSIFY_ATTEMPTS + (uint64_t)a);
+            int g = (int)(((uint64_t)p + 1u + u % (uint64_t)(KL - 1)) % (uint64_t)KL);
+            int gz;
+            int gb = dwta_position(o, v, g, &gz);
+            if (!gz) { best = gb; break; }
+          }
+        }
         code |= (uint32_t)best << (k * lg);
       }
     }
     codes[t] = code;
   }
 }
+
+/* codes of a neuron's weight row */
+void orc_hash_vec(const orc *o, const REAL *v, uint32_t *codes) { hash_vec(o, v, codes, 0); }
+/* codes of a query (a hidden activation) */
+void orc_hash_query(const orc *o, const REAL *v, uint32_t *codes) { hash_vec(o, v, codes, 1); }
 
 /* Section 2.1 phase 1 / Algorithm 1 "Hash weights to hash tables":
  * bucket (t, code) lists, in ascending id, every neuron whose weight row has
@@ -396,7 +431,7 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
     REAL *h = o->h + (size_t)s * H;
     hidden_layer(o, row_ptr[s + 1] - row_ptr[s], col_idx + row_ptr[s], vals + row_ptr[s], h);
     uint32_t *codes = o->codes + (size_t)s * c->L;
-    orc_hash_vec(o, h, codes);
+    orc_hash_query(o, h, codes);
     const int32_t *lab = label_ptr ? labels + label_ptr[s] : NULL;
     int32_t nl = label_ptr ? label_ptr[s + 1] - label_ptr[s] : 0;
     int64_t na = select_active(o, codes, lab, nl, &buf, &bufcap);

@@ -262,3 +262,60 @@ def test_rebuild_schedule_closed_form():
             if o.r != before:
                 seen.append(step)
         assert seen == want
+
+
+# ---------------------------------------------------------------- densification of all-zero DWTA bins
+def brute_densified_codes(o, v, K, L, bs, seed, r, attempts=16, stream=3):
+    """The definition written out: positions of all bins first, then every all-zero bin borrows."""
+    idx = o.get("hash_idx").reshape(K * L, bs)
+    vals = v[idx]                                       # [KL][bs]
+    pos = np.argmax(vals, axis=1)                       # first maximum = lowest position on ties
+    empty = np.all(vals == 0, axis=1)
+    KL = K * L
+    out = pos.copy()
+    for p in np.nonzero(empty)[0]:
+        out[p] = 0
+        for a in range(attempts):
+            g = (int(p) + 1 + orc_rng(seed, stream, r, int(p) * attempts + a) % (KL - 1)) % KL
+            if not empty[g]:
+                out[p] = pos[g]
+                break
+    lg = int(np.log2(bs))
+    return np.array([sum(int(out[t * K + k]) << (k * lg) for k in range(K)) for t in range(L)], dtype=np.uint32)
+
+
+def test_densified_query_codes_match_the_definition_written_out():
+    rs = np.random.default_rng(11)
+    o = make(DWTA, H=64, K=3, L=7, bin_size=8, densify=1, seed=5)
+    saw_empty = saw_borrow = 0
+    for trial in range(40):
+        v = np.maximum(rs.standard_normal(64), 0).astype(np.float32)
+        v[rs.random(64) < 0.6] = 0.0                    # ReLU output with most units off
+        want = brute_densified_codes(o, v, 3, 7, 8, 5, 0)
+        got = o.hash_query(v)
+        assert np.array_equal(got, want)
+        plain = o.hash_vec(v)                           # neurons' rows are never densified
+        idx = o.get("hash_idx").reshape(21, 8)
+        empty = np.all(v[idx] == 0, axis=1)
+        saw_empty += int(empty.sum())
+        saw_borrow += int(np.any(got != plain))
+        # a function whose own bin is not empty keeps its position
+        for t in range(7):
+            for k in range(3):
+                if not empty[t * 3 + k]:
+                    assert (got[t] >> (3 * k)) & 7 == (plain[t] >> (3 * k)) & 7
+    assert saw_empty > 20 and saw_borrow > 5
+
+
+def test_densification_needs_the_flag_and_a_nonzero_bin_somewhere():
+    v = np.zeros(64, dtype=np.float32)
+    on = make(DWTA, H=64, K=3, L=7, bin_size=8, densify=1, seed=5)
+    off = make(DWTA, H=64, K=3, L=7, bin_size=8, densify=0, seed=5)
+    assert np.all(on.hash_query(v) == 0)                # every probe finds an empty bin
+    v[on.get("hash_idx")[0]] = 2.0                      # one unit on: only the bins holding it are not empty
+    assert np.array_equal(off.hash_query(v), off.hash_vec(v))
+    assert np.array_equal(on.hash_vec(v), off.hash_vec(v))
+    # the probe sequence is drawn again with the hash functions
+    on.draw_hash(1)
+    on.set_counters(0, 1, 0)
+    assert np.array_equal(on.hash_query(v), brute_densified_codes(on, v, 3, 7, 8, 5, 1))
