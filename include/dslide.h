@@ -69,6 +69,11 @@ typedef struct {
   int32_t device;                            /* CUDA device ordinal                                             */
   int32_t dedup_mode;                        /* 0 auto; 1 bitmap in shared memory; 2 sort in shared memory      */
   void* stream;                              /* cudaStream_t the context enqueues on (NULL = default stream)    */
+  int32_t dwta_densify;                      /* 1: DWTA densification for queries (Section 4.1 names the family):
+                                                a bin of the hidden activation whose values are all zero borrows
+                                                the position of the first non-empty bin along a seeded probe
+                                                sequence of 16 other functions (0 when all are empty); 0: such a
+                                                bin yields position 0.  Weight rows are never densified.          */
 } dslide_config;
 
 /* Tensors readable and writable through dslide_get_tensor / dslide_set_tensor. */

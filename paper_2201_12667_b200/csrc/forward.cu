@@ -49,6 +49,8 @@ struct FwdParams {
   int act_stride, Wd, dense, dedup_mode, max_labels, sort_cap, topk, parity;
   int stage_bytes;     // bytes of the staging region (it starts at off_dedup and overlays the dedup work space)
   int hid_rows;        // rows of W1 staged per chunk of the hidden layer
+  int densify;         // DWTA: all-zero bins of the query borrow another bin's position
+  unsigned long long seed, rcount;   // for the probe sequence of the densification: the model's seed, rebuilds so far
   int hash_sm_off;     // where in the staging region the hash functions' index tables are mirrored (-1: read from global memory)
   int hash_sm_bytes;
   int sort_small;      // candidate sets up to this size are deduplicated by sorting even when a bitmap is available
@@ -419,6 +421,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         if (v6 > bv) { bv = v6; best = 6; }
         if (v7 > bv) { bv = v7; best = 7; }
         sh_part[f] = (unsigned char)best;
+        sh_part[p.KL + f] = bv == 0.f ? 1 : 0;     // activations are not negative: a maximum of zero is a bin of zeros
       } else {
         int best = 0;
         float bv = sh_h[ix[0]];
@@ -427,6 +430,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
           if (v > bv) { bv = v; best = i; }       // strict: the lowest position wins ties
         }
         sh_part[f] = (unsigned char)best;
+        sh_part[p.KL + f] = bv == 0.f ? 1 : 0;
       }
     }
     __syncthreads();
@@ -434,7 +438,20 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     const int shift = p.family == DSLIDE_SIMHASH ? 1 : p.lg_bin;
     for (int t = tid; t < p.L; t += FWD_THREADS) {
       uint32_t code = 0;
-      for (int k = 0; k < p.K; ++k) code |= (uint32_t)sh_part[t * p.K + k] << (k * shift);
+      for (int k = 0; k < p.K; ++k) {
+        const int f = t * p.K + k;
+        uint32_t pos = sh_part[f];
+        if (p.densify && p.family == DSLIDE_DWTA && sh_part[p.KL + f] && p.KL > 1) {
+          // a bin of zeros: the position of the first probed function whose own bin is not all zero, else 0
+          pos = 0;
+          for (int a = 0; a < DENSIFY_ATTEMPTS; ++a) {
+            const uint64_t u = ctr_rng(p.seed, RNG_PROBE, p.rcount, (uint64_t)f * DENSIFY_ATTEMPTS + (uint64_t)a);
+            const int g = (int)(((uint64_t)f + 1u + u % (uint64_t)(p.KL - 1)) % (uint64_t)p.KL);
+            if (!sh_part[p.KL + g]) { pos = sh_part[g]; break; }
+          }
+        }
+        code |= pos << (k * shift);
+      }
       sh_code[t] = code;
       if (MODE == 0) p.codes[(size_t)s * p.L + t] = code;
       const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1) + code;
@@ -941,7 +958,7 @@ static FwdLayout fwd_layout(const Ctx* c) {
   int o = align16(c->H * 4);
   l.off_dh = o;      o = align16(o + FWD_WARPS * c->H * 4);
   l.off_code = o;    o = align16(o + c->L * 4);
-  l.off_part = o;    o = align16(o + c->KL);
+  l.off_part = o;    o = align16(o + 2 * c->KL);     // position and all-zero flag of every function's bin
   l.off_misc = o;    o = align16(o + 32 * 4);
   l.off_lab = o;     o = align16(o + (c->cfg.max_labels > 0 ? c->cfg.max_labels : 1) * 4);
   l.off_tbase = o;   o = align16(o + (c->L + 1) * 4);
@@ -1028,6 +1045,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.max_labels = c->cfg.max_labels; p.sort_cap = c->sort_cap; p.topk = 1;
   FwdLayout l = fwd_layout(c);
   p.stage_bytes = c->fwd_stage_bytes; p.hid_rows = l.hid_rows; p.sort_small = c->fwd_sort_small;
+  p.densify = c->cfg.dwta_densify; p.seed = c->cfg.seed; p.rcount = (unsigned long long)c->r_host;
   p.hash_sm_off = c->fwd_hash_sm_off; p.hash_sm_bytes = c->fwd_hash_sm_bytes;
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
   p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;

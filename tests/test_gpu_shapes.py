@@ -204,3 +204,25 @@ def test_one_hot_inputs_and_hidden_layer_of_200():
         one_and_two_steps(pr, batches)
     finally:
         pr.close()
+
+
+def test_densified_dwta_queries():
+    """Most hidden units off (a negative hidden bias): about a quarter of the bins of a query are all zero and borrow
+    a position along the probe sequence; a scheduled rebuild after the first step draws a new sequence.  Codes and
+    active sets must match the oracle bit for bit, with the flag and without it."""
+    for densify in (1, 0):
+        pr = Pair(D=5003, H=128, N=20011, family=DWTA, K=3, L=10, bucket_cap=16, max_batch=48, max_labels=16, lr=1e-3,
+                  seed=9, densify=densify, rebuild_period0=1)
+        try:
+            pr.o.set("b1", np.full(128, -0.05, dtype=np.float32))
+            pr.push_state()
+            wl = workloads.Workload(workloads.config("mid"), seed=16)
+            batches = [wl.batch(i, batch_size=48) for i in range(3)]
+            one_and_two_steps(pr, batches)
+            if densify:
+                h = ds.dslide_get_last(pr.ctx, "hidden", 48).reshape(48, 128)
+                idx = ds.dslide_get_tensor(pr.ctx, "hash_idx").reshape(30, 8)
+                empty = np.all(h[:, idx] == 0, axis=2)
+                assert 0.05 < empty.mean() < 0.9
+        finally:
+            pr.close()
