@@ -49,6 +49,7 @@ typedef struct {
   int32_t force_dense;      /* "sparsity is 1" (Section 3.6): every output neuron is active      */
   int32_t max_active;       /* 0 = no limit; otherwise a larger active set is an error           */
   int32_t densify;          /* DWTA: an all-zero bin of a query borrows another bin's position   */
+  int32_t budget;           /* Section 3.7: active neurons per sample, labels included; 0 = off   */
   double rebuild_lambda;    /* gap_i = max(1, floor(p0 * exp(lambda * i)))                       */
   double lr, beta1, beta2, eps;   /* Adam (Section 4.1)                                          */
   double init_std;
@@ -103,7 +104,7 @@ uint64_t orc_rng(uint64_t seed, uint64_t stream, uint64_t r, uint64_t ctr) {
   uint64_t b = mix64(a + GOLD * (r + 1));
   return mix64(b + GOLD * (ctr + 1));
 }
-enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3 };
+enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3, STREAM_SAMPLE = 4 };
 enum { DENSIFY_ATTEMPTS = 16 };
 
 static double u01(uint64_t x) { return ((double)(x >> 11) + 0.5) * (1.0 / 9007199254740992.0); }
@@ -373,8 +374,50 @@ static void hidden_layer(const orc *o, int32_t nnz, const int32_t *col, const RE
  * input, take the union of the retrieved buckets (at most bucket_cap lowest
  * ids of each), add the labels when given (reading: labels are always
  * active), sort, remove duplicates.  Returns the count, or -1 on overflow. */
+/* Section 3.7: when the neurons retrieved for a sample exceed the sampling
+ * budget, reservoir sampling controls how many are kept; when they do not,
+ * reading: the set is left as it is (the paper's "stop with the current set
+ * of neurons"; its other option, a uniform random fill, is not built).
+ * reading: the budget counts the sample's labels, which are always active,
+ * so m = max(0, budget - |Y|) of the other retrieved neurons are kept.  The
+ * candidates C_0 < C_1 < ... (retrieved ids that are not labels, ascending)
+ * go through the textbook reservoir algorithm: the first m fill the
+ * reservoir; candidate i >= m draws j uniform in [0, i] and replaces
+ * reservoir[j] when j < m.  j = rng(seed, STREAM_SAMPLE, steps taken so far,
+ * sample * 2^32 + i) mod (i + 1).  act[] (ascending, n entries) is rewritten
+ * with the labels and the reservoir, ascending; returns the new count. */
+static int is_label(int32_t id, const int32_t *lab, int32_t nlab) {
+  for (int32_t i = 0; i < nlab; ++i) if (lab[i] == id) return 1;
+  return 0;
+}
+
+static int64_t apply_budget(const orc *o, int32_t *act, int64_t n, const int32_t *lab, int32_t nlab, int32_t s) {
+  const orc_config *c = &o->c;
+  int64_t ny = 0, nc = 0;
+  for (int64_t a = 0; a < n; ++a) { if (is_label(act[a], lab, nlab)) ++ny; else ++nc; }
+  int64_t m = c->budget - ny;
+  if (m < 0) m = 0;
+  if (nc <= m) return n;
+  int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nc > 0 ? nc : 1));
+  int32_t *res = (int32_t *)malloc(sizeof(int32_t) * (size_t)(m > 0 ? m : 1));
+  int64_t k = 0;
+  for (int64_t a = 0; a < n; ++a) if (!is_label(act[a], lab, nlab)) cand[k++] = act[a];
+  for (int64_t i = 0; i < nc; ++i) {
+    if (i < m) { res[i] = cand[i]; continue; }
+    uint64_t u = orc_rng(c->seed, STREAM_SAMPLE, (uint64_t)o->t, ((uint64_t)(uint32_t)s << 32) + (uint64_t)i);
+    uint64_t j = u % (uint64_t)(i + 1);
+    if (j < (uint64_t)m) res[j] = cand[i];
+  }
+  int64_t out = 0;
+  for (int64_t a = 0; a < n; ++a) if (is_label(act[a], lab, nlab)) act[out++] = act[a];
+  for (int64_t j = 0; j < m; ++j) act[out++] = res[j];
+  qsort(act, (size_t)out, sizeof(int32_t), cmp_i32);
+  free(cand); free(res);
+  return out;
+}
+
 static int64_t select_active(const orc *o, const uint32_t *codes, const int32_t *lab, int32_t nlab,
-                             int32_t **buf, int64_t *bufcap) {
+                             int32_t **buf, int64_t *bufcap, int32_t s) {
   const orc_config *c = &o->c;
   int64_t n = 0;
   if (c->force_dense) {
@@ -397,6 +440,7 @@ static int64_t select_active(const orc *o, const uint32_t *codes, const int32_t 
   int64_t u = 0;
   for (int64_t i = 0; i < n; ++i)
     if (u == 0 || (*buf)[u - 1] != (*buf)[i]) (*buf)[u++] = (*buf)[i];
+  if (c->budget > 0) u = apply_budget(o, *buf, u, lab, nlab, s);
   return u;
 }
 
@@ -434,7 +478,7 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
     orc_hash_query(o, h, codes);
     const int32_t *lab = label_ptr ? labels + label_ptr[s] : NULL;
     int32_t nl = label_ptr ? label_ptr[s + 1] - label_ptr[s] : 0;
-    int64_t na = select_active(o, codes, lab, nl, &buf, &bufcap);
+    int64_t na = select_active(o, codes, lab, nl, &buf, &bufcap, s);
     if (c->max_active > 0 && na > c->max_active) { o->error = 4; free(buf); return o->error; }
     int64_t base = o->act_ptr[s];
     ensure_act(o, base + na);

@@ -246,3 +246,75 @@ def test_float_and_double_oracles_agree():
     if all(np.array_equal(a, b) for a, b in zip(of.active_sets(), od.active_sets())):
         assert abs(lf - ld) < 1e-5 * abs(ld)
         np.testing.assert_allclose(of.get("W2"), od.get("W2"), rtol=2e-3, atol=1e-6)
+
+
+# ---------------------------------------------------------------- sampling budget (Section 3.7)
+def _sets_with_and_without_budget(budget, seed=4, t=0, B=6, **kw):
+    rs = np.random.default_rng(21)
+    cfg = dict(D=60, H=16, N=400, family=SIMHASH, K=2, L=6, bucket_cap=40, seed=seed, init_std=0.5)
+    cfg.update(kw)
+    batch = small_batch(rs, B, 60, 400, 8, max_labels=3, dtype=np.float32)
+    free = Oracle("float", **cfg)
+    capped = Oracle("float", budget=budget, **cfg)
+    capped.set_counters(t, 0, 0)
+    free.set_counters(t, 0, 0)
+    free.forward(*batch)
+    capped.forward(*batch)
+    labels = [np.unique(batch[4][batch[3][s]:batch[3][s + 1]]) for s in range(B)]
+    return free.active_sets(), capped.active_sets(), labels, capped
+
+
+def test_budget_keeps_labels_and_the_reservoir_of_the_other_candidates():
+    """Algorithm R written out in Python over the candidates in ascending order, with the oracle's generator."""
+    from oracle.oracle import rng as orc_rng
+    budget, seed, t = 30, 4, 7
+    full, capped, labels, _ = _sets_with_and_without_budget(budget, seed=seed, t=t)
+    over = 0
+    for s, (a0, a1, y) in enumerate(zip(full, capped, labels)):
+        cand = [j for j in a0 if j not in set(y)]
+        m = max(0, budget - len(y))
+        if len(cand) <= m:
+            assert np.array_equal(a0, a1)
+            continue
+        over += 1
+        res = cand[:m]
+        for i in range(m, len(cand)):
+            j = orc_rng(seed, 4, t, (s << 32) + i) % (i + 1)
+            if j < m:
+                res[j] = cand[i]
+        want = np.array(sorted(set(res) | set(y)), dtype=np.int32)
+        assert np.array_equal(a1, want)
+        assert len(a1) == budget and set(y) <= set(a1) and set(a1) <= set(a0)
+        assert np.all(np.diff(a1) > 0)
+    assert over >= 3                                     # the case was exercised
+
+
+def test_budget_above_the_retrieved_count_changes_nothing_and_below_the_labels_keeps_labels_only():
+    full, capped, labels, _ = _sets_with_and_without_budget(10 ** 6)
+    for a0, a1 in zip(full, capped):
+        assert np.array_equal(a0, a1)
+    full, capped, labels, _ = _sets_with_and_without_budget(1)
+    for a1, y in zip(capped, labels):
+        assert np.array_equal(a1, y)                     # m = max(0, 1 - |Y|) = 0 other neurons
+
+
+def test_reservoir_keeps_every_candidate_with_probability_m_over_n():
+    """The property the reservoir algorithm is known for, over 400 values of the step counter (each draws afresh)."""
+    budget = 12
+    counts, ncand, m = None, None, None
+    for t in range(400):
+        full, capped, labels, _ = _sets_with_and_without_budget(budget, t=t, B=1, bucket_cap=60)
+        y = set(labels[0])
+        cand = [j for j in full[0] if j not in y]
+        if counts is None:
+            ncand, m = len(cand), budget - len(y)
+            assert ncand > 3 * m
+            counts = {j: 0 for j in cand}
+        for j in capped[0]:
+            if j not in y:
+                counts[j] += 1
+    freq = np.array(list(counts.values())) / 400.0
+    p = m / ncand
+    sigma = np.sqrt(p * (1 - p) / 400)
+    assert abs(freq.mean() - p) < 1e-12                  # exactly m kept every time
+    assert np.all(np.abs(freq - p) < 5 * sigma)          # no candidate favoured (first or last positions included)
