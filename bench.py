@@ -61,6 +61,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--rebuild-period", type=int, default=REBUILD_PERIOD)
+    ap.add_argument("--budget", type=int, default=0, help="sampling budget per sample (Section 3.7); 0 = none, as in the headline")
     return ap.parse_args()
 
 
@@ -212,7 +213,7 @@ def workload_config(c, B, args, nb):
                         "~%d labels/sample" % (c["name"], c["D"], c["H"], c["N"],
                                                "DWTA" if c["family"] == workloads.DWTA else "SimHash", c["K"], c["L"],
                                                c["bucket_cap"], B, c["mean_nnz"], c["mean_labels"]),
-            "batch": B, "rebuild_every": args.rebuild_period, "distinct_batches": nb,
+            "batch": B, "rebuild_every": args.rebuild_period, "distinct_batches": nb, "sampling_budget": args.budget,
             "l2": "inputs larger than L2: 1.3 GB of model state, a different batch (and so different rows) every step"}
 
 
@@ -258,7 +259,8 @@ def run_dslide(args):
     cfg = ds.make_config(input_dim=c["D"], hidden_dim=c["H"], output_dim=c["N"], hash_family=c["family"], K=c["K"],
                          L=c["L"], dwta_bin_size=c["bin_size"], bucket_cap=c["bucket_cap"],
                          rebuild_period0=args.rebuild_period, rebuild_growth_lambda=0.0, redraw_hash_fns=1,
-                         max_batch=B, max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0, device=local)
+                         max_batch=B, max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0, device=local,
+                         sample_budget=args.budget)
     ctx = ds.dslide_init(cfg)
 
     wl = workloads.Workload(c, seed=shard_seed(rank))

@@ -74,6 +74,13 @@ typedef struct {
                                                 the position of the first non-empty bin along a seeded probe
                                                 sequence of 16 other functions (0 when all are empty); 0: such a
                                                 bin yields position 0.  Weight rows are never densified.          */
+  int32_t sample_budget;                     /* Section 3.7: active neurons kept per sample, the sample's labels
+                                                included; when more are retrieved, reservoir sampling (draws
+                                                numbered by step, sample and candidate) keeps budget - labels of
+                                                the others; fewer are left as they are.  0 = no budget.  The
+                                                work space must fit the forward kernel's shared memory: about
+                                                5 * (L * bucket_cap) + 8 * budget bytes <= 64 KB, else
+                                                dslide_init returns DSLIDE_ERR_INVALID_ARG.                       */
 } dslide_config;
 
 /* Tensors readable and writable through dslide_get_tensor / dslide_set_tensor. */

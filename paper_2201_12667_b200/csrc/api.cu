@@ -154,7 +154,7 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   if (!(k.lr > 0.f) || !(k.beta1 >= 0.f && k.beta1 < 1.f) || !(k.beta2 >= 0.f && k.beta2 < 1.f) || !(k.eps > 0.f))
     return DSLIDE_ERR_INVALID_ARG;
   if (k.rebuild_period0 < 0 || k.init_std < 0.f || k.dedup_mode < 0 || k.dedup_mode > 2) return DSLIDE_ERR_INVALID_ARG;
-  if (k.dwta_densify < 0 || k.dwta_densify > 1) return DSLIDE_ERR_INVALID_ARG;
+  if (k.dwta_densify < 0 || k.dwta_densify > 1 || k.sample_budget < 0) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_bin_size == 0) k.dwta_bin_size = 8;
   if (k.srp_nnz == 0) k.srp_nnz = (k.hidden_dim + 2) / 3;
   int lg_bin = 0, bits = 0, fn_len = 0;

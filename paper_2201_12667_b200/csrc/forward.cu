@@ -49,6 +49,8 @@ struct FwdParams {
   int act_stride, Wd, dense, dedup_mode, max_labels, sort_cap, topk, parity;
   int stage_bytes;     // bytes of the staging region (it starts at off_dedup and overlays the dedup work space)
   int hid_rows;        // rows of W1 staged per chunk of the hidden layer
+  int budget;          // Section 3.7: active neurons kept per sample, labels included (0 = no budget)
+  unsigned long long tcount;   // steps taken so far (the reservoir's draws are numbered by step, sample and candidate)
   int densify;         // DWTA: all-zero bins of the query borrow another bin's position
   unsigned long long seed, rcount;   // for the probe sequence of the densification: the model's seed, rebuilds so far
   int hash_sm_off;     // where in the staging region the hash functions' index tables are mirrored (-1: read from global memory)
@@ -220,6 +222,67 @@ __device__ __forceinline__ void rank_sort(const uint32_t* src, uint32_t* dst, in
     for (int u = 0; u < PER; ++u)
       if (tid + u * FWD_THREADS < n) dst[pos[u]] = v[u];
   }
+}
+
+// Section 3.7: the sample's retrieved neurons exceed the sampling budget -> reservoir sampling keeps
+// m = max(0, budget - labels) of those that are not labels.  The textbook algorithm runs over the candidates in
+// ascending id order: the first m fill the reservoir, candidate i >= m draws j uniform in [0, i] and replaces slot j
+// when j < m.  Its outcome is fixed by the draws alone -- slot j ends with the LAST candidate that drew j, or with
+// candidate j itself -- so the block evaluates all draws at once and settles every slot with a shared-memory max.
+// ids[0 .. na) (ascending, mirrored in sh_ids up to ACT_SM) is rewritten with the labels and the reservoir,
+// ascending; returns the new count.  work: 4 * na + 4 * m + nc + 4 * (m + labels) bytes of shared memory.
+// Called by the whole block; kept out of line because most configurations never run it.
+__device__ __noinline__ int budget_select(int budget, uint64_t seed, uint64_t tcount, int s, int32_t* ids, int* sh_ids,
+                                          int na, const int32_t* lab, int nlab, unsigned char* work, int* sh_scan) {
+  const int tid = threadIdx.x;
+  int* cidx = reinterpret_cast<int*>(work);                 // [na] index among the candidates, -1 for a label
+  const int chunk = (na + FWD_THREADS - 1) / FWD_THREADS;
+  const int a0 = min(na, tid * chunk), a1 = min(na, a0 + chunk);
+  int cnt = 0;
+  for (int a = a0; a < a1; ++a) {
+    const int id = a < ACT_SM ? sh_ids[a] : ids[a];
+    bool isl = false;
+    for (int i = 0; i < nlab; ++i) isl = isl || lab[i] == id;
+    cidx[a] = isl ? -1 : 0;
+    cnt += isl ? 0 : 1;
+  }
+  int nc = 0;
+  int at = block_excl_scan(cnt, sh_scan, &nc);
+  const int ny = na - nc;
+  const int m = max(0, budget - ny);
+  if (nc <= m) return na;                                    // uniform over the block
+  for (int a = a0; a < a1; ++a)
+    if (cidx[a] == 0) cidx[a] = at++;
+  int* win = cidx + na;                                      // [m] the last candidate that drew the slot
+  unsigned char* sel = reinterpret_cast<unsigned char*>(win + m);        // [nc]
+  int* out = reinterpret_cast<int*>(work + (((size_t)4 * na + (size_t)4 * m + nc + 15) & ~(size_t)15));  // [m + ny]
+  for (int j = tid; j < m; j += FWD_THREADS) win[j] = -1;
+  for (int i = tid; i < nc; i += FWD_THREADS) sel[i] = 0;
+  __syncthreads();
+  for (int a = a0; a < a1; ++a) {
+    const int i = cidx[a];
+    if (i >= m) {
+      const uint64_t u = ctr_rng(seed, RNG_SAMPLE, tcount, ((uint64_t)(uint32_t)s << 32) + (uint64_t)i);
+      const int j = (int)(u % (uint64_t)(i + 1));
+      if (j < m) atomicMax(&win[j], i);
+    }
+  }
+  __syncthreads();
+  for (int j = tid; j < m; j += FWD_THREADS) sel[win[j] >= 0 ? win[j] : j] = 1;
+  __syncthreads();
+  cnt = 0;
+  for (int a = a0; a < a1; ++a) cnt += (cidx[a] < 0 || sel[cidx[a]]) ? 1 : 0;
+  int total = 0;
+  at = block_excl_scan(cnt, sh_scan, &total);
+  for (int a = a0; a < a1; ++a)
+    if (cidx[a] < 0 || sel[cidx[a]]) out[at++] = a < ACT_SM ? sh_ids[a] : ids[a];
+  __syncthreads();
+  for (int a = tid; a < total; a += FWD_THREADS) {
+    ids[a] = out[a];
+    if (a < ACT_SM) sh_ids[a] = out[a];
+  }
+  __syncthreads();
+  return total;
 }
 
 // The sample is skipped: no loss, no gradient, nothing touched (predict: no candidates).
@@ -606,6 +669,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
     na = total;
     __syncthreads();                 // ids visible to the block; the dedup work space is free from here on
+    if (p.budget > 0) na = budget_select(p.budget, p.seed, p.tcount, s, ids, sh_ids, na, MODE == 0 ? p.labels + lbeg : nullptr, nlab, smem + p.off_dedup, sh_misc);
   }
   if (MODE == 0 && tid == 0) p.act_cnt[s] = na;
   const bool small = !dense && na <= ACT_SM;      // ids and logits mirrored in shared memory
@@ -1019,6 +1083,11 @@ cudaError_t setup_forward(Ctx* c) {
       c->fwd_hash_sm_off = (c->fwd_stage_bytes - (int)hb) & ~15;
     }
   }
+  if (c->cfg.sample_budget > 0 && !c->dense) {
+    // the reservoir's work space (an index per retrieved id, a slot per kept one, flags, the kept ids) overlays the staging region
+    const long long a = c->act_stride, m = c->cfg.sample_budget < c->act_stride ? c->cfg.sample_budget : c->act_stride;
+    if (4 * a + 4 * m + a + 16 + 4 * (m + c->cfg.max_labels) > (long long)c->fwd_stage_bytes) return cudaErrorInvalidValue;
+  }
   c->fwd_smem = l.fixed_bytes + c->fwd_stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(k_forward<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<0, MAX_KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -1046,6 +1115,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   FwdLayout l = fwd_layout(c);
   p.stage_bytes = c->fwd_stage_bytes; p.hid_rows = l.hid_rows; p.sort_small = c->fwd_sort_small;
   p.densify = c->cfg.dwta_densify; p.seed = c->cfg.seed; p.rcount = (unsigned long long)c->r_host;
+  p.budget = c->cfg.sample_budget; p.tcount = (unsigned long long)c->t_host;
   p.hash_sm_off = c->fwd_hash_sm_off; p.hash_sm_bytes = c->fwd_hash_sm_bytes;
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
   p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;

@@ -226,3 +226,37 @@ def test_densified_dwta_queries():
                 assert 0.05 < empty.mean() < 0.9
         finally:
             pr.close()
+
+
+@pytest.mark.parametrize("family,K,L,cap,budget", [
+    (SIMHASH, 3, 12, 40, 100),     # 300-480 retrieved per sample, 100 kept
+    (SIMHASH, 2, 12, 400, 1100),   # well over a thousand retrieved: sets past the shared-memory mirror of the ids
+    (DWTA, 3, 10, 16, 40),         # some samples over, some under the budget
+    (DWTA, 3, 10, 16, 2),          # fewer than some label lists: those samples keep their labels only
+])
+def test_sampling_budget(family, K, L, cap, budget):
+    """Section 3.7: reservoir sampling over the retrieved neurons.  The kept sets must be the oracle's bit for bit
+    (the same draws decide), at two consecutive steps (the draws are numbered by step), and the step built on
+    them must match as usual."""
+    pr = Pair(D=3001, H=128, N=12007, family=family, K=K, L=L, bucket_cap=cap, max_batch=16, max_labels=16, lr=1e-3,
+              seed=10, budget=budget)
+    try:
+        wl = workloads.Workload(workloads.config("mid", D=3001, N=12007), seed=17)
+        batches = [wl.batch(i, batch_size=16) for i in range(2)]
+        one_and_two_steps(pr, batches)
+        cnt = ds.dslide_get_last(pr.ctx, "act_count", 16)
+        nlab = np.array([len(np.unique(batches[1][4][batches[1][3][s]:batches[1][3][s + 1]])) for s in range(16)])
+        assert np.all(cnt <= np.maximum(budget, nlab))
+        if budget >= 40:
+            assert np.any(cnt == budget)                 # the budget was reached by some sample
+        # inference applies the same budget
+        k = 5
+        ids_o, sc_o = pr.o.predict_topk(*batches[1][:3], k)
+        dev = [torch.from_numpy(a).cuda() for a in batches[1][:3]]
+        out_ids = torch.zeros(16 * k, dtype=torch.int32, device="cuda")
+        out_sc = torch.zeros(16 * k, dtype=torch.float32, device="cuda")
+        ds.dslide_predict_topk(pr.ctx, 16, *dev, k, False, out_ids, out_sc)
+        ds.dslide_sync(pr.ctx)
+        assert np.array_equal(out_ids.cpu().numpy().reshape(16, k), ids_o)
+    finally:
+        pr.close()
