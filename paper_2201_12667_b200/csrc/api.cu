@@ -60,7 +60,7 @@ cudaError_t dalloc(T** p, size_t n, cudaStream_t st, bool zero) {
 void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->hdr1, c->hdr2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
-                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1,
+                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1, c->ovf1, c->ovf2,
                   c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
                   c->st_dev[0], c->st_dev[1], c->st_dev[2]};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -215,12 +215,13 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(hash_idx, (size_t)c->KL * fn_len, true); A(hash_sign, (size_t)c->KL * fn_len, true);
   A(h, B * H, true); A(dh, B * H, true); A(loss, B, true); A(codes, B * c->L, true);
   A(act_cnt, B, true); A(act_z, B * S, true); A(act_p, B * S, true); A(act_g, B * S, true);
-  A(hdr1, D, true); A(mask1, D * c->Wd, true); A(own1, D, true);
+  A(hdr1, D, true); A(mask1, D * c->Wd, true); A(own1, D, true); A(ovf1, D * HOT_T, false);
   A(hot_rows, HOT_CAP, true); A(med_rows, MED_CAP, true); A(hot_done, HOT_CAP, true); A(hot_part, (size_t)HOT_CAP * HOT_SLICES * (H + 4), true);
   A(dstate, 1, true);
   if (!c->dense) {
     A(act_ids, B * S, true);
     A(mask2, N * c->Wd, true);
+    A(ovf2, N * HOT_T, false);
     A(own2, N, true);
     A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
     A(keysA, (size_t)c->L * N, false);

@@ -149,6 +149,7 @@ struct Ctx {
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;         // per row of W1 / W2: which samples of the batch touch it
+  int2 *ovf1, *ovf2;               // per row: the (sample, coefficient) pairs of touches ROW_SLOTS .. HOT_T - 1, at [row][touch]
   int2 *own1, *own2;               // the distinct touched rows of W1 / W2 with their first-touching sample, in no particular order
   int32_t* hot_rows;               // rows touched by many samples: row of W2, or ~row of W1
   int32_t* med_rows;               // rows touched by more than ROW_SLOTS samples, same encoding

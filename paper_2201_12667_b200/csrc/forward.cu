@@ -38,6 +38,7 @@ struct FwdParams {
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;
+  int2 *ovf1, *ovf2;
   RowHdr *hdr1, *hdr2;
   int2 *own1, *own2;
   int32_t *hot_rows, *med_rows;
@@ -111,13 +112,17 @@ __device__ __forceinline__ void list_row(const FwdParams& p, uint32_t* cnt, int 
 // (nth = touches before this one): the (sample, coefficient) pair goes into the row's slot nth, or, past the
 // slots, the sample's bit into the row's mask; the first toucher enters (row, its own sample) in the list of
 // distinct rows (positions handed out per warp), so that the update kernel can fetch that sample's row at once.  Called by whole warps; `live` tells whether this thread has a touch.
-__device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int2* own,
+__device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int2* ovfrow, int2* own,
                                              unsigned int* n_own, int row, int code, unsigned nth, int s, float coef) {
   const int lane = threadIdx.x & 31;
   bool first = false;
   if (live) {
     if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(coef));
-    else atomicOr(maskrow + (s >> 5), 1u << (s & 31));
+    else {
+      atomicOr(maskrow + (s >> 5), 1u << (s & 31));
+      // up to HOT_T touches keep their pair as well, so that a row with that many is summed without any search
+      if (nth < (unsigned)HOT_T) ovfrow[nth] = make_int2(s, __float_as_int(coef));
+    }
     first = nth == 0u;
     list_row(p, &hd->cnt, code, nth);
   }
@@ -749,7 +754,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
             x = __ldg(p.vals + rbeg + i);
             nth = atomicAdd(&p.hdr1[c].cnt, 1u) & CNT_MASK;
           }
-          finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
+          finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.ovf1 + (size_t)c * HOT_T, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
         }
     }
     if (!mbar_wait(sh_bar, phase)) timed_out = true;
@@ -978,7 +983,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
 #pragma unroll
     for (int u = 0; u < HO_PER; ++u)
       if (u * FWD_THREADS < na)            // uniform over the block
-        finish_touch(p, tid + u * FWD_THREADS < na, p.hdr2 + jj0[u], p.mask2 + (size_t)jj0[u] * p.Wd, p.own2,
+        finish_touch(p, tid + u * FWD_THREADS < na, p.hdr2 + jj0[u], p.mask2 + (size_t)jj0[u] * p.Wd,
+                     p.ovf2 + (size_t)jj0[u] * HOT_T, p.own2,
                      &p.st->n_own[p.parity][0], jj0[u], jj0[u], nth0[u], s, ga0[u]);
     for (int a0 = HO_PER * FWD_THREADS; a0 < na; a0 += FWD_THREADS) {
       const int a = a0 + tid;
@@ -991,7 +997,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         ga = gp[a];
         nth = atomicAdd(&p.hdr2[jj].cnt, 1u) & CNT_MASK;
       }
-      finish_touch(p, live, p.hdr2 + jj, p.mask2 + (size_t)jj * p.Wd, p.own2, &p.st->n_own[p.parity][0], jj, jj, nth, s, ga);
+      finish_touch(p, live, p.hdr2 + jj, p.mask2 + (size_t)jj * p.Wd, p.ovf2 + (size_t)jj * HOT_T, p.own2, &p.st->n_own[p.parity][0], jj, jj, nth, s, ga);
     }
   }
   if (tid == 0) {
@@ -1104,7 +1110,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals; p.label_ptr = label_ptr; p.labels = labels;
   p.h = c->h; p.dh = c->dh; p.loss = c->loss; p.codes = c->codes;
   p.act_cnt = c->act_cnt; p.act_ids = c->act_ids; p.act_z = c->act_z; p.act_p = c->act_p; p.act_g = c->act_g;
-  p.mask1 = c->mask1; p.mask2 = c->mask2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.ovf1 = c->ovf1; p.ovf2 = c->ovf2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
   p.own1 = c->own1; p.own2 = c->own2; p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.parity = (int)(c->t_host & 1);
   p.st = c->dstate; p.out_ids = nullptr; p.out_scores = nullptr;
   p.nb = c->nb;

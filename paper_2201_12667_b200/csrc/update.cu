@@ -42,6 +42,7 @@ struct UpdParams {
   const int32_t *row_ptr, *col_idx;
   const float* vals;
   uint32_t *mask1, *mask2;
+  const int2 *ovf1, *ovf2;
   RowHdr *hdr1, *hdr2;
   const int2 *own1, *own2;
   const int32_t *hot_rows, *med_rows;
@@ -78,6 +79,7 @@ struct Side {
   float *W, *M, *V;
   const float* src;
   uint32_t* mask;
+  const int2* ovf;
   RowHdr* hdr;
   int is_w2;
 };
@@ -87,6 +89,7 @@ __device__ __forceinline__ Side make_side(const UpdParams& p, bool w2) {
   sd.W = w2 ? p.W2 : p.W1; sd.M = w2 ? p.mW2 : p.mW1; sd.V = w2 ? p.vW2 : p.vW1;
   sd.src = w2 ? p.h : p.dh;
   sd.mask = w2 ? p.mask2 : p.mask1;
+  sd.ovf = w2 ? p.ovf2 : p.ovf1;
   sd.hdr = w2 ? p.hdr2 : p.hdr1;
   sd.is_w2 = w2 ? 1 : 0;
   return sd;
@@ -429,7 +432,11 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowpt
   const int2 hv = load_hdr(sd.hdr + row, lane);
   const unsigned cv = (unsigned)__shfl_sync(FULL, hv.x, 0);
   if ((cv & CNT_HOT) || (cv & CNT_MASK) == 0u) return;
-  const int slot_s = hdr_slots(hv).x;
+  const int2 sl = hdr_slots(hv);
+  const int total = (int)(cv & CNT_MASK);
+  // the pairs of touches ROW_SLOTS .. HOT_T - 1, asked for together with the rows
+  int2 pair = sl;
+  if (total <= HOT_T && lane >= ROW_SLOTS && lane < total) pair = sd.ovf[(size_t)row * HOT_T + lane];
   float4 w[NCH], m[NCH], v[NCH], acc[NCH];
   load_row<NCH>(sd.W, (size_t)row, H, H4, lane, w);
   load_row<NCH>(sd.M, (size_t)row, H, H4, lane, m);
@@ -437,7 +444,25 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowpt
 #pragma unroll
   for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   float csum = 0.f;
-  sum_masked<NCH>(p, sd, rowptr, row, slot_s, 0, nwB, scr, acc, csum, H, H4, lane);
+  if (total <= HOT_T) {
+    // every touch has its pair: lane k holds touch k; put them in ascending sample order (each sample touches a
+    // row once, so the samples are distinct) and add; the mask only has to be cleared
+    const int s_me = lane < total ? pair.x : 0x7fffffff;
+    int rank = 0;
+    for (int k = 0; k < total; ++k) rank += __shfl_sync(FULL, s_me, k) < s_me ? 1 : 0;
+    __syncwarp();
+    if (lane < total) { scr[rank] = pair.x; scr[32 + rank] = pair.y; }
+    __syncwarp();
+    const int s_mine = lane < total ? scr[lane] : 0;
+    const float g_mine = lane < total ? __int_as_float(scr[32 + lane]) : 0.f;
+    accumulate_list<NCH>(acc, csum, total, s_mine, g_mine, sd.src, H, H4, lane);
+    __syncwarp();
+    uint32_t* mrow = sd.mask + (size_t)row * p.Wd;
+    for (int wi = lane; wi < nwB; wi += 32)
+      if (mrow[wi]) mrow[wi] = 0u;
+  } else {
+    sum_masked<NCH>(p, sd, rowptr, row, sl.x, 0, nwB, scr, acc, csum, H, H4, lane);
+  }
   adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
   finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
 }
@@ -615,7 +640,7 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   p.W2 = c->W2; p.mW2 = c->mW2; p.vW2 = c->vW2;
   p.h = c->h; p.dh = c->dh; p.act_g = c->act_g; p.loss = c->loss; p.act_cnt = c->act_cnt; p.act_ids = c->act_ids;
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals;
-  p.mask1 = c->mask1; p.mask2 = c->mask2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.ovf1 = c->ovf1; p.ovf2 = c->ovf2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
   p.own1 = c->own1; p.own2 = c->own2;
   p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.hot_part = c->hot_part; p.hot_done = c->hot_done;
   p.st = c->dstate; p.loss_out = loss_out; p.host_res = host_res; p.host_seq = host_seq;
