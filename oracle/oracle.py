@@ -41,7 +41,7 @@ class OrcConfig(C.Structure):
         ("family", C.c_int32), ("K", C.c_int32), ("L", C.c_int32),
         ("bin_size", C.c_int32), ("srp_nnz", C.c_int32), ("bucket_cap", C.c_int32),
         ("rebuild_period0", C.c_int32), ("redraw", C.c_int32), ("force_dense", C.c_int32),
-        ("max_active", C.c_int32), ("densify", C.c_int32), ("budget", C.c_int32),
+        ("max_active", C.c_int32), ("densify", C.c_int32), ("budget", C.c_int32), ("budget_fill", C.c_int32),
         ("rebuild_lambda", C.c_double),
         ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
         ("init_std", C.c_double),
@@ -118,7 +118,7 @@ class Oracle:
         self.dtype = np.float32 if real == "float" else np.float64
         self.lib = _load(real)
         d = dict(family=SIMHASH, bin_size=8, srp_nnz=0, bucket_cap=128, rebuild_period0=0, redraw=1,
-                 force_dense=0, max_active=0, densify=0, budget=0, rebuild_lambda=0.0, lr=1e-4, beta1=0.9, beta2=0.999,
+                 force_dense=0, max_active=0, densify=0, budget=0, budget_fill=0, rebuild_lambda=0.0, lr=1e-4, beta1=0.9, beta2=0.999,
                  eps=1e-8, init_std=0.01, seed=0)
         d.update(kw)
         self.cfg = OrcConfig(**d)

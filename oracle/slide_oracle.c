@@ -50,6 +50,7 @@ typedef struct {
   int32_t max_active;       /* 0 = no limit; otherwise a larger active set is an error           */
   int32_t densify;          /* DWTA: an all-zero bin of a query borrows another bin's position   */
   int32_t budget;           /* Section 3.7: active neurons per sample, labels included; 0 = off   */
+  int32_t budget_fill;      /* Section 3.7: an under-full set is topped up with uniform draws     */
   double rebuild_lambda;    /* gap_i = max(1, floor(p0 * exp(lambda * i)))                       */
   double lr, beta1, beta2, eps;   /* Adam (Section 4.1)                                          */
   double init_std;
@@ -104,7 +105,7 @@ uint64_t orc_rng(uint64_t seed, uint64_t stream, uint64_t r, uint64_t ctr) {
   uint64_t b = mix64(a + GOLD * (r + 1));
   return mix64(b + GOLD * (ctr + 1));
 }
-enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3, STREAM_SAMPLE = 4 };
+enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3, STREAM_SAMPLE = 4, STREAM_FILL = 5 };
 enum { DENSIFY_ATTEMPTS = 16 };
 
 static double u01(uint64_t x) { return ((double)(x >> 11) + 0.5) * (1.0 / 9007199254740992.0); }
@@ -391,13 +392,36 @@ static int is_label(int32_t id, const int32_t *lab, int32_t nlab) {
   return 0;
 }
 
+/* Section 3.7, the other option for a set below the budget: "fill the rest of
+ * the sampling budget with uniformly sampled neurons".  reading: neurons are
+ * drawn one after the other, id_k = rng(seed, STREAM_FILL, steps taken so
+ * far, sample * 2^32 + k) mod N, k = 0, 1, ...; a draw that is already in the
+ * set (retrieved, label, or drawn before) is passed over; drawing stops when
+ * the set has min(budget, N) members or after 2 * (missing members) + 64
+ * draws.  act[] must have room for budget entries; it is returned ascending. */
+static int64_t fill_budget(const orc *o, int32_t *act, int64_t n, int32_t s) {
+  const orc_config *c = &o->c;
+  int64_t target = c->budget < c->N ? c->budget : c->N;
+  if (n >= target) return n;
+  int64_t need = target - n, draws = 2 * need + 64, got = 0;
+  for (int64_t k = 0; k < draws && got < need; ++k) {
+    uint64_t u = orc_rng(c->seed, STREAM_FILL, (uint64_t)o->t, ((uint64_t)(uint32_t)s << 32) + (uint64_t)k);
+    int32_t id = (int32_t)(u % (uint64_t)c->N);
+    int seen = 0;
+    for (int64_t a = 0; a < n + got; ++a) if (act[a] == id) { seen = 1; break; }
+    if (!seen) act[n + got++] = id;
+  }
+  qsort(act, (size_t)(n + got), sizeof(int32_t), cmp_i32);
+  return n + got;
+}
+
 static int64_t apply_budget(const orc *o, int32_t *act, int64_t n, const int32_t *lab, int32_t nlab, int32_t s) {
   const orc_config *c = &o->c;
   int64_t ny = 0, nc = 0;
   for (int64_t a = 0; a < n; ++a) { if (is_label(act[a], lab, nlab)) ++ny; else ++nc; }
   int64_t m = c->budget - ny;
   if (m < 0) m = 0;
-  if (nc <= m) return n;
+  if (nc <= m) return c->budget_fill ? fill_budget(o, act, n, s) : n;
   int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nc > 0 ? nc : 1));
   int32_t *res = (int32_t *)malloc(sizeof(int32_t) * (size_t)(m > 0 ? m : 1));
   int64_t k = 0;
@@ -426,6 +450,7 @@ static int64_t select_active(const orc *o, const uint32_t *codes, const int32_t 
     return c->N;
   }
   int64_t worst = (int64_t)c->L * c->bucket_cap + nlab;
+  if (c->budget_fill && worst < c->budget) worst = c->budget;
   if (*bufcap < worst) { *buf = (int32_t *)realloc(*buf, sizeof(int32_t) * (size_t)worst); *bufcap = worst; }
   int64_t nb = (int64_t)1 << o->bits;
   for (int t = 0; t < c->L; ++t) {

@@ -318,3 +318,39 @@ def test_reservoir_keeps_every_candidate_with_probability_m_over_n():
     sigma = np.sqrt(p * (1 - p) / 400)
     assert abs(freq.mean() - p) < 1e-12                  # exactly m kept every time
     assert np.all(np.abs(freq - p) < 5 * sigma)          # no candidate favoured (first or last positions included)
+
+
+def test_budget_fill_tops_an_under_full_set_up_with_uniform_draws():
+    """The fill written out in Python: draws in order, already-present ids passed over, stop when full or after
+    2 * missing + 64 draws."""
+    from oracle.oracle import rng as orc_rng
+    seed, t = 4, 3
+    for budget, N in ((150, 400), (395, 400), (10 ** 4, 400)):
+        free, filled, labels, _ = _sets_with_and_without_budget(budget, seed=seed, t=t, budget_fill=1, N=N)
+        nofill, _, _, _ = _sets_with_and_without_budget(budget, seed=seed, t=t, N=N)
+        topped = 0
+        for s, (a0, a1) in enumerate(zip(free, filled)):
+            target = min(budget, N)
+            if len(a0) >= target:
+                continue                                  # over the budget: the reservoir's business
+            have = list(a0)
+            need = target - len(a0)
+            for k in range(2 * need + 64):
+                if len(have) == target:
+                    break
+                j = orc_rng(seed, 5, t, (s << 32) + k) % N
+                if j not in have:
+                    have.append(j)
+            assert np.array_equal(a1, np.array(sorted(have), dtype=np.int32))
+            assert set(a0) <= set(a1) and np.all(np.diff(a1) > 0)
+            topped += 1
+            if budget == 150:
+                assert len(a1) == 150                     # far from N, the draws always suffice
+        assert topped >= 3
+
+
+def test_budget_fill_off_leaves_under_full_sets_alone():
+    free, capped, labels, _ = _sets_with_and_without_budget(150)
+    for a0, a1 in zip(free, capped):
+        if len(a0) <= 150:
+            assert np.array_equal(a0, a1)
