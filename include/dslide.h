@@ -81,6 +81,14 @@ typedef struct {
                                                 work space must fit the forward kernel's shared memory: about
                                                 5 * (L * bucket_cap) + 8 * budget bytes <= 64 KB, else
                                                 dslide_init returns DSLIDE_ERR_INVALID_ARG.                       */
+  int32_t budget_fill;                       /* 1 (needs sample_budget > 0 and max_active_per_sample = 0): a
+                                                sample whose retrieved neurons and labels are fewer than the
+                                                budget is topped up with uniformly drawn neurons (Section 3.7):
+                                                ids drawn one after the other, repeats and members passed over,
+                                                until min(budget, N) members or 2 * missing + 64 draws.  The
+                                                per-sample arrays then hold up to budget entries; the work space
+                                                (about 80 bytes per budgeted neuron) must fit the forward
+                                                kernel's shared memory, else DSLIDE_ERR_INVALID_ARG.              */
 } dslide_config;
 
 /* Tensors readable and writable through dslide_get_tensor / dslide_set_tensor. */

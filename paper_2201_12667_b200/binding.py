@@ -42,7 +42,7 @@ class Config(C.Structure):
         ("max_batch", C.c_int32), ("max_labels", C.c_int32), ("max_active_per_sample", C.c_int32),
         ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
         ("init_std", C.c_float), ("seed", C.c_uint64), ("device", C.c_int32), ("dedup_mode", C.c_int32),
-        ("stream", C.c_void_p), ("dwta_densify", C.c_int32), ("sample_budget", C.c_int32),
+        ("stream", C.c_void_p), ("dwta_densify", C.c_int32), ("sample_budget", C.c_int32), ("budget_fill", C.c_int32),
     ]
 
 
@@ -100,13 +100,13 @@ def _dptr(t):
 def make_config(*, input_dim, hidden_dim, output_dim, hash_family=DWTA, K=6, L=50, dwta_bin_size=8, srp_nnz=0,
                 bucket_cap=128, rebuild_period0=50, rebuild_growth_lambda=0.0, redraw_hash_fns=1, force_dense=0,
                 max_batch=256, max_labels=16, max_active_per_sample=0, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8,
-                init_std=0.01, seed=0, device=0, dedup_mode=0, stream=None, dwta_densify=0, sample_budget=0):
+                init_std=0.01, seed=0, device=0, dedup_mode=0, stream=None, dwta_densify=0, sample_budget=0, budget_fill=0):
     if stream is None:
         import torch
         stream = torch.cuda.current_stream(device).cuda_stream
     return Config(input_dim, hidden_dim, output_dim, hash_family, K, L, dwta_bin_size, srp_nnz, bucket_cap,
                   rebuild_period0, rebuild_growth_lambda, redraw_hash_fns, force_dense, max_batch, max_labels,
-                  max_active_per_sample, lr, beta1, beta2, eps, init_std, seed, device, dedup_mode, stream, dwta_densify, sample_budget)
+                  max_active_per_sample, lr, beta1, beta2, eps, init_std, seed, device, dedup_mode, stream, dwta_densify, sample_budget, budget_fill)
 
 
 # ---- the C entry points, same names ---------------------------------------------------------

@@ -155,6 +155,8 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     return DSLIDE_ERR_INVALID_ARG;
   if (k.rebuild_period0 < 0 || k.init_std < 0.f || k.dedup_mode < 0 || k.dedup_mode > 2) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_densify < 0 || k.dwta_densify > 1 || k.sample_budget < 0) return DSLIDE_ERR_INVALID_ARG;
+  if (k.budget_fill < 0 || k.budget_fill > 1) return DSLIDE_ERR_INVALID_ARG;
+  if (k.budget_fill && (k.sample_budget < 1 || k.max_active_per_sample != 0 || k.force_dense)) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_bin_size == 0) k.dwta_bin_size = 8;
   if (k.srp_nnz == 0) k.srp_nnz = (k.hidden_dim + 2) / 3;
   int lg_bin = 0, bits = 0, fn_len = 0;
@@ -175,6 +177,7 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
                                                       : (int64_t)k.L * k.bucket_cap + k.max_labels);
   if (!k.force_dense && act_stride > (int64_t)k.L * k.bucket_cap + k.max_labels)
     act_stride = (int64_t)k.L * k.bucket_cap + k.max_labels;
+  if (k.budget_fill && act_stride < k.sample_budget) act_stride = k.sample_budget;     // a filled set has up to budget members
   if (act_stride > k.output_dim) act_stride = k.output_dim;
   if (act_stride < 1) return DSLIDE_ERR_INVALID_ARG;
 

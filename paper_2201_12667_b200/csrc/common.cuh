@@ -24,7 +24,7 @@ __host__ __device__ inline uint64_t ctr_rng(uint64_t seed, uint64_t stream, uint
   uint64_t b = sm64(a + g * (r + 1));
   return sm64(b + g * (ctr + 1));
 }
-enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2, RNG_PROBE = 3, RNG_SAMPLE = 4 };
+enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2, RNG_PROBE = 3, RNG_SAMPLE = 4, RNG_FILL = 5 };
 constexpr int DENSIFY_ATTEMPTS = 16;     // functions an all-zero DWTA bin of a query probes for a position to borrow
 
 // Device-resident step state (read and written by kernels only; the host reads it

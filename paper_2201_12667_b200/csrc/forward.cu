@@ -51,6 +51,7 @@ struct FwdParams {
   int stage_bytes;     // bytes of the staging region (it starts at off_dedup and overlays the dedup work space)
   int hid_rows;        // rows of W1 staged per chunk of the hidden layer
   int budget;          // Section 3.7: active neurons kept per sample, labels included (0 = no budget)
+  int budget_fill;     // Section 3.7: a set below the budget is topped up with uniform draws
   unsigned long long tcount;   // steps taken so far (the reservoir's draws are numbered by step, sample and candidate)
   int densify;         // DWTA: all-zero bins of the query borrow another bin's position
   unsigned long long seed, rcount;   // for the probe sequence of the densification: the model's seed, rebuilds so far
@@ -229,6 +230,107 @@ __device__ __forceinline__ void rank_sort(const uint32_t* src, uint32_t* dst, in
   }
 }
 
+// Section 3.7, the fill option: a set below the budget is topped up with neurons drawn one after the other,
+// id_k = rng(seed, RNG_FILL, steps taken, sample * 2^32 + k) mod N; a draw already in the set (retrieved, label, or
+// drawn before) is passed over; drawing stops when the set has min(budget, N) members or after 2 * missing + 64
+// draws.  All draws are evaluated at once: a shared-memory hash set records the first draw of every id, a search in
+// the (ascending) set tells which ids are new, and the running count in draw order says which of them still fit.
+// The accepted ids are put in order and merged with the set.  Returns the new count.
+__device__ __forceinline__ int fill_work_bytes(int need) {
+  const int D = 2 * need + 64;
+  int ts = 64;
+  while (ts < 2 * D) ts <<= 1;
+  return 4 * D + ((D + 3) & ~3) + 8 * ts + 8 * need;       // draws, flags, hash set (ids, first draws), accepted ids twice
+}
+__device__ __noinline__ int budget_fill(int budget, int N, uint64_t seed, uint64_t tcount, int s, int32_t* ids, int* sh_ids,
+                                        int na, unsigned char* work, int work_bytes, int* sh_scan, DevState* st) {
+  const int tid = threadIdx.x;
+  const int target = min(budget, N);
+  if (na >= target) return na;
+  const int need = target - na;
+  const int D = 2 * need + 64;
+  int ts = 64;
+  while (ts < 2 * D) ts <<= 1;
+  if (fill_work_bytes(need) + 4 * target > work_bytes) {     // cannot happen with the sizes checked at start-up
+    if (tid == 0) set_status(st, DSLIDE_ERR_OVERFLOW);
+    return na;
+  }
+  int* draw = reinterpret_cast<int*>(work);                 // [D]
+  unsigned char* okf = reinterpret_cast<unsigned char*>(draw + D);       // [D]
+  int* keys = reinterpret_cast<int*>(okf + ((D + 3) & ~3)); // [ts] ids seen, -1 = empty
+  int* mink = keys + ts;                                    // [ts] the first draw of that id
+  int* F = mink + ts;                                       // [need] accepted ids in draw order
+  int* Fs = F + need;                                       // [need] ascending
+  int* out = Fs + need;                                     // [target]
+  const int lg = 31 - __clz(ts);
+  for (int h = tid; h < ts; h += FWD_THREADS) { keys[h] = -1; mink[h] = 0x7fffffff; }
+  for (int k = tid; k < D; k += FWD_THREADS)
+    draw[k] = (int)(ctr_rng(seed, RNG_FILL, tcount, ((uint64_t)(uint32_t)s << 32) + (uint64_t)k) % (uint64_t)N);
+  __syncthreads();
+  for (int k = tid; k < D; k += FWD_THREADS) {
+    const int id = draw[k];
+    unsigned h = ((unsigned)id * 2654435761u) >> (32 - lg);
+    for (int it = 0; it < ts; ++it) {
+      const int prev = atomicCAS(&keys[h], -1, id);
+      if (prev == -1 || prev == id) { atomicMin(&mink[h], k); break; }
+      h = (h + 1) & (unsigned)(ts - 1);
+    }
+  }
+  __syncthreads();
+  for (int k = tid; k < D; k += FWD_THREADS) {
+    const int id = draw[k];
+    unsigned h = ((unsigned)id * 2654435761u) >> (32 - lg);
+    bool first = false;
+    for (int it = 0; it < ts; ++it) {
+      if (keys[h] == id) { first = mink[h] == k; break; }
+      h = (h + 1) & (unsigned)(ts - 1);
+    }
+    int lo = 0, hi = na;                                    // is the id in the set already?
+    while (lo < hi) { const int mid = (lo + hi) >> 1; const int v = mid < ACT_SM ? sh_ids[mid] : ids[mid]; if (v < id) lo = mid + 1; else hi = mid; }
+    const bool in_set = lo < na && (lo < ACT_SM ? sh_ids[lo] : ids[lo]) == id;
+    okf[k] = (first && !in_set) ? 1 : 0;
+  }
+  __syncthreads();
+  // running count in draw order: the first `need` new ids are accepted
+  const int chunk = (D + FWD_THREADS - 1) / FWD_THREADS;
+  const int k0 = min(D, tid * chunk), k1 = min(D, k0 + chunk);
+  int cnt = 0;
+  for (int k = k0; k < k1; ++k) cnt += okf[k];
+  int total_ok = 0;
+  int at = block_excl_scan(cnt, sh_scan, &total_ok);
+  for (int k = k0; k < k1; ++k)
+    if (okf[k]) { if (at < need) F[at] = draw[k]; ++at; }
+  const int got = min(total_ok, need);
+  __syncthreads();
+  for (int j = tid; j < got; j += FWD_THREADS) {            // ascending order by counting (the ids are distinct)
+    const int v = F[j];
+    int r = 0;
+    for (int q = 0; q < got; ++q) r += F[q] < v ? 1 : 0;
+    Fs[r] = v;
+  }
+  __syncthreads();
+  for (int i = tid; i < na; i += FWD_THREADS) {             // merge: each element lands after the smaller ones of both lists
+    const int v = i < ACT_SM ? sh_ids[i] : ids[i];
+    int lo = 0, hi = got;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (Fs[mid] < v) lo = mid + 1; else hi = mid; }
+    out[i + lo] = v;
+  }
+  for (int j = tid; j < got; j += FWD_THREADS) {
+    const int v = Fs[j];
+    int lo = 0, hi = na;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; const int w = mid < ACT_SM ? sh_ids[mid] : ids[mid]; if (w < v) lo = mid + 1; else hi = mid; }
+    out[j + lo] = v;
+  }
+  __syncthreads();
+  const int total = na + got;
+  for (int a = tid; a < total; a += FWD_THREADS) {
+    ids[a] = out[a];
+    if (a < ACT_SM) sh_ids[a] = out[a];
+  }
+  __syncthreads();
+  return total;
+}
+
 // Section 3.7: the sample's retrieved neurons exceed the sampling budget -> reservoir sampling keeps
 // m = max(0, budget - labels) of those that are not labels.  The textbook algorithm runs over the candidates in
 // ascending id order: the first m fill the reservoir, candidate i >= m draws j uniform in [0, i] and replaces slot j
@@ -237,8 +339,9 @@ __device__ __forceinline__ void rank_sort(const uint32_t* src, uint32_t* dst, in
 // ids[0 .. na) (ascending, mirrored in sh_ids up to ACT_SM) is rewritten with the labels and the reservoir,
 // ascending; returns the new count.  work: 4 * na + 4 * m + nc + 4 * (m + labels) bytes of shared memory.
 // Called by the whole block; kept out of line because most configurations never run it.
-__device__ __noinline__ int budget_select(int budget, uint64_t seed, uint64_t tcount, int s, int32_t* ids, int* sh_ids,
-                                          int na, const int32_t* lab, int nlab, unsigned char* work, int* sh_scan) {
+__device__ __noinline__ int budget_select(int budget, int fill, int N, uint64_t seed, uint64_t tcount, int s, int32_t* ids,
+                                          int* sh_ids, int na, const int32_t* lab, int nlab, unsigned char* work,
+                                          int work_bytes, int* sh_scan, DevState* st) {
   const int tid = threadIdx.x;
   int* cidx = reinterpret_cast<int*>(work);                 // [na] index among the candidates, -1 for a label
   const int chunk = (na + FWD_THREADS - 1) / FWD_THREADS;
@@ -255,7 +358,8 @@ __device__ __noinline__ int budget_select(int budget, uint64_t seed, uint64_t tc
   int at = block_excl_scan(cnt, sh_scan, &nc);
   const int ny = na - nc;
   const int m = max(0, budget - ny);
-  if (nc <= m) return na;                                    // uniform over the block
+  if (nc <= m)                                               // uniform over the block
+    return fill ? budget_fill(budget, N, seed, tcount, s, ids, sh_ids, na, work, work_bytes, sh_scan, st) : na;
   for (int a = a0; a < a1; ++a)
     if (cidx[a] == 0) cidx[a] = at++;
   int* win = cidx + na;                                      // [m] the last candidate that drew the slot
@@ -674,7 +778,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
     na = total;
     __syncthreads();                 // ids visible to the block; the dedup work space is free from here on
-    if (p.budget > 0) na = budget_select(p.budget, p.seed, p.tcount, s, ids, sh_ids, na, MODE == 0 ? p.labels + lbeg : nullptr, nlab, smem + p.off_dedup, sh_misc);
+    if (p.budget > 0)
+      na = budget_select(p.budget, p.budget_fill, N, p.seed, p.tcount, s, ids, sh_ids, na, MODE == 0 ? p.labels + lbeg : nullptr,
+                         nlab, smem + p.off_dedup, p.stage_bytes, sh_misc, p.st);
   }
   if (MODE == 0 && tid == 0) p.act_cnt[s] = na;
   const bool small = !dense && na <= ACT_SM;      // ids and logits mirrored in shared memory
@@ -1093,6 +1199,13 @@ cudaError_t setup_forward(Ctx* c) {
     // the reservoir's work space (an index per retrieved id, a slot per kept one, flags, the kept ids) overlays the staging region
     const long long a = c->act_stride, m = c->cfg.sample_budget < c->act_stride ? c->cfg.sample_budget : c->act_stride;
     if (4 * a + 4 * m + a + 16 + 4 * (m + c->cfg.max_labels) > (long long)c->fwd_stage_bytes) return cudaErrorInvalidValue;
+    if (c->cfg.budget_fill) {
+      // the fill's work space for the largest number of missing ids (the whole budget): draws, flags, hash set, ids
+      const long long b = c->cfg.sample_budget < c->N ? c->cfg.sample_budget : c->N, D = 2 * b + 64;
+      long long ts = 64;
+      while (ts < 2 * D) ts <<= 1;
+      if (4 * D + D + 4 + 8 * ts + 8 * b + 4 * b > (long long)c->fwd_stage_bytes) return cudaErrorInvalidValue;
+    }
   }
   c->fwd_smem = l.fixed_bytes + c->fwd_stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(k_forward<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -1121,7 +1234,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   FwdLayout l = fwd_layout(c);
   p.stage_bytes = c->fwd_stage_bytes; p.hid_rows = l.hid_rows; p.sort_small = c->fwd_sort_small;
   p.densify = c->cfg.dwta_densify; p.seed = c->cfg.seed; p.rcount = (unsigned long long)c->r_host;
-  p.budget = c->cfg.sample_budget; p.tcount = (unsigned long long)c->t_host;
+  p.budget = c->cfg.sample_budget; p.budget_fill = c->cfg.budget_fill; p.tcount = (unsigned long long)c->t_host;
   p.hash_sm_off = c->fwd_hash_sm_off; p.hash_sm_bytes = c->fwd_hash_sm_bytes;
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
   p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;

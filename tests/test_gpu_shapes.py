@@ -260,3 +260,45 @@ def test_sampling_budget(family, K, L, cap, budget):
         assert np.array_equal(out_ids.cpu().numpy().reshape(16, k), ids_o)
     finally:
         pr.close()
+
+
+@pytest.mark.parametrize("family,K,L,cap,budget", [
+    (DWTA, 3, 10, 16, 200),        # every sample under the budget: 40-150 retrieved, topped up to 200
+    (DWTA, 3, 10, 16, 60),         # some over (reservoir), some under (fill)
+    (SIMHASH, 2, 12, 400, 1100),   # sets topped up past the shared-memory mirror of the ids
+])
+def test_sampling_budget_with_fill(family, K, L, cap, budget):
+    """Section 3.7's other option: sets below the budget are filled with uniform draws.  Same bar as above: the sets
+    are the oracle's bit for bit at two consecutive steps and at inference."""
+    pr = Pair(D=3001, H=128, N=12007, family=family, K=K, L=L, bucket_cap=cap, max_batch=16, max_labels=16, lr=1e-3,
+              seed=11, budget=budget, budget_fill=1)
+    try:
+        wl = workloads.Workload(workloads.config("mid", D=3001, N=12007), seed=18)
+        batches = [wl.batch(i, batch_size=16) for i in range(2)]
+        one_and_two_steps(pr, batches)
+        cnt = ds.dslide_get_last(pr.ctx, "act_count", 16)
+        assert np.all(cnt == budget)                      # far from N, the draws always suffice
+        k = 5
+        ids_o, sc_o = pr.o.predict_topk(*batches[1][:3], k)
+        dev = [torch.from_numpy(a).cuda() for a in batches[1][:3]]
+        out_ids = torch.zeros(16 * k, dtype=torch.int32, device="cuda")
+        out_sc = torch.zeros(16 * k, dtype=torch.float32, device="cuda")
+        ds.dslide_predict_topk(pr.ctx, 16, *dev, k, False, out_ids, out_sc)
+        ds.dslide_sync(pr.ctx)
+        assert np.array_equal(out_ids.cpu().numpy().reshape(16, k), ids_o)
+    finally:
+        pr.close()
+
+
+def test_fill_that_cannot_reach_the_budget():
+    """A budget of all N neurons: the draws run out (2 * missing + 64 of them) before every neuron has come up."""
+    pr = Pair(D=300, H=32, N=257, family=SIMHASH, K=2, L=2, bucket_cap=8, max_batch=8, max_labels=4, lr=1e-3, seed=12,
+              budget=257, budget_fill=1)
+    try:
+        wl = workloads.Workload(workloads.config("tiny", D=300, N=257, max_labels=3), seed=19)
+        batches = [wl.batch(i, batch_size=8) for i in range(2)]
+        one_and_two_steps(pr, batches)
+        cnt = ds.dslide_get_last(pr.ctx, "act_count", 8)
+        assert np.all(cnt < 257) and np.all(cnt > 128)
+    finally:
+        pr.close()
