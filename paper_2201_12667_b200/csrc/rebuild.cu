@@ -315,6 +315,8 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
 // counts[t][0] = 0, counts[t][c + 1] = size of bucket c  ->  inclusive running sum = bucket offsets.
 // Two kernels over chunks of BS_CHUNK counters: the sum of every chunk, then per chunk the sum of the
 // table's earlier chunks plus a scan inside the chunk.
+constexpr int ORD_SMALL = 16;     // buckets up to this size are put in order in registers
+constexpr int ORD_BLOCK = 4096;   // up to this size by one block in shared memory
 constexpr int BS_THREADS = 256;
 constexpr int BS_PER = 16;
 constexpr int BS_CHUNK = BS_THREADS * BS_PER;
@@ -340,7 +342,10 @@ __global__ void __launch_bounds__(BS_THREADS) k_bucket_sums(const int32_t* off, 
   }
 }
 
-__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks) {
+// With cnt != null the buckets of more than min_n (>= ORD_SMALL) ids are entered in the lists of the block-wide and
+// the ordered-pass ordering kernels on the way (cnt[0] / cnt[1] are the lists' lengths).
+__global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long long nb, const int32_t* part, int nchunks,
+                                                            int min_n, int2* mid, int2* big, int* cnt) {
   __shared__ int sh[BS_THREADS / 32 + 1];
   int32_t* o = off + (size_t)blockIdx.y * (size_t)(nb + 1);
   const long long n = nb + 1, base = (long long)blockIdx.x * BS_CHUNK;
@@ -381,6 +386,10 @@ __global__ void __launch_bounds__(BS_THREADS) k_bucket_scan(int32_t* off, long l
     }
     const long long i = wbase + u * 32 + lane;
     if (i < n) o[i] = run + incl;
+    if (cnt && i >= 1 && i < n && v[u] > min_n) {          // word i counts bucket i - 1
+      if (v[u] <= ORD_BLOCK) mid[atomicAdd(cnt, 1)] = make_int2((int)blockIdx.y, (int)(i - 1));
+      else big[atomicAdd(cnt + 1, 1)] = make_int2((int)blockIdx.y, (int)(i - 1));
+    }
     run += __shfl_sync(0xffffffffu, incl, 31);
   }
 }
@@ -557,8 +566,6 @@ k_sort_scatter(const uint32_t* keys_in, const int32_t* vals_in, uint32_t* keys_o
 // order where they stand: in registers for
 // buckets of up to ORD_SMALL ids, by a block-wide sort in shared memory up to ORD_BLOCK, and for a larger bucket by
 // one ordered pass over the table's codes that writes the matching ids out again.
-constexpr int ORD_SMALL = 16;
-constexpr int ORD_BLOCK = 4096;
 constexpr int ORD_THREADS = 256;
 
 __global__ void __launch_bounds__(256) k_place_ids(const uint32_t* keys, const uint32_t* ranks, const int32_t* off, int32_t* ids,
@@ -670,19 +677,24 @@ __global__ void __launch_bounds__(ORD_THREADS) k_order_big(const uint32_t* keys,
   }
 }
 
-// Puts the ids of every bucket with more than min_n ids in ascending order (place path only).
-cudaError_t launch_order_buckets(Ctx* c, int min_n) {
+// Puts the ids of every bucket with more than min_n ids in ascending order (place path only).  With `listed`, the
+// offset scan has already entered those buckets in the lists (all of them larger than ORD_SMALL).
+static cudaError_t order_buckets(Ctx* c, int min_n, bool listed) {
   if (min_n < 1) min_n = 1;
-  cudaError_t e = cudaMemsetAsync(c->ord_cnt, 0, 2 * sizeof(int), c->stream);
-  if (e != cudaSuccess) return e;
   LaunchScope ls(c, KID_ORDER_BUCKETS);
-  dim3 grid((unsigned)min((long long)((c->nb + 255) / 256), 2048LL), c->L);
-  k_order_small<<<grid, 256, 0, c->stream>>>(c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_mid, c->ord_big, c->ord_cnt, min_n);
+  if (!listed) {
+    cudaError_t e = cudaMemsetAsync(c->ord_cnt, 0, 2 * sizeof(int), c->stream);
+    if (e != cudaSuccess) return e;
+    dim3 grid((unsigned)min((long long)((c->nb + 255) / 256), 2048LL), c->L);
+    k_order_small<<<grid, 256, 0, c->stream>>>(c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_mid, c->ord_big, c->ord_cnt, min_n);
+  }
   k_order_mid<<<c->num_sms * 4, ORD_THREADS, 0, c->stream>>>(c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_mid, c->ord_cnt);
   k_order_big<<<c->num_sms, ORD_THREADS, 0, c->stream>>>(c->keysA, c->bucket_off, c->bucket_ids, c->N, c->nb, c->ord_big,
                                                           c->ord_cnt);
   return cudaGetLastError();
 }
+
+cudaError_t launch_order_buckets(Ctx* c, int min_n) { return order_buckets(c, min_n, false); }
 
 cudaError_t launch_build_tables(Ctx* c) {
   const size_t off_bytes = (size_t)c->L * (size_t)(c->nb + 1) * sizeof(int32_t);
@@ -722,12 +734,17 @@ cudaError_t launch_build_tables(Ctx* c) {
                                                              c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  const bool list_in_scan = c->place_path && c->cap >= ORD_SMALL;
   {
     const int nchunks = (int)((c->nb + 1 + BS_CHUNK - 1) / BS_CHUNK);
     dim3 grid(nchunks, c->L);
+    // on the place path, with a cap of at least ORD_SMALL, the buckets that must be in order for the step (those
+    // above the cap) are listed by the scan itself: no separate pass over all bucket sizes
+    if (list_in_scan && (e = cudaMemsetAsync(c->ord_cnt, 0, 2 * sizeof(int), c->stream)) != cudaSuccess) return e;
     LaunchScope ls(c, KID_BUCKET_SCAN);
     k_bucket_sums<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
-    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks);
+    k_bucket_scan<<<grid, BS_THREADS, 0, c->stream>>>(c->bucket_off, c->nb, c->bucket_part, nchunks, c->cap, c->ord_mid,
+                                                      c->ord_big, list_in_scan ? c->ord_cnt : nullptr);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
@@ -742,7 +759,7 @@ cudaError_t launch_build_tables(Ctx* c) {
     // order afterwards anyway: only buckets larger than the cap must be in ascending order for the step.  The
     // smaller ones are ordered when the table is read back (launch_order_buckets(c, 1)).
     c->ids_ordered_above = c->cap;
-    return launch_order_buckets(c, c->cap);
+    return order_buckets(c, c->cap, list_in_scan);
   }
 
   if ((e = cudaFuncSetAttribute(k_sort_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, SORT_SMEM)) != cudaSuccess) return e;
