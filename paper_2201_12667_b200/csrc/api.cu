@@ -218,13 +218,13 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(hash_idx, (size_t)c->KL * fn_len, true); A(hash_sign, (size_t)c->KL * fn_len, true);
   A(h, B * H, true); A(dh, B * H, true); A(loss, B, true); A(codes, B * c->L, true);
   A(act_cnt, B, true); A(act_z, B * S, true); A(act_p, B * S, true); A(act_g, B * S, true);
-  A(hdr1, D, true); A(mask1, D * c->Wd, true); A(own1, D, true); A(ovf1, D * HOT_T, false);
+  A(hdr1, D, true); A(mask1, D * c->Wd, true); A(own1, D, true); A(ovf1, D * PAIR_T, false);
   A(hot_rows, HOT_CAP, true); A(med_rows, MED_CAP, true); A(hot_done, HOT_CAP, true); A(hot_part, (size_t)HOT_CAP * HOT_SLICES * (H + 4), true);
   A(dstate, 1, true);
   if (!c->dense) {
     A(act_ids, B * S, true);
     A(mask2, N * c->Wd, true);
-    A(ovf2, N * HOT_T, false);
+    A(ovf2, N * PAIR_T, false);
     A(own2, N, true);
     A(bucket_off, (size_t)c->L * (size_t)(c->nb + 1), true); A(bucket_ids, (size_t)c->L * N, true);
     A(keysA, (size_t)c->L * N, false);

@@ -60,6 +60,8 @@ constexpr int ROW_SLOTS = 6;
 // count set) and summed in HOT_SLICES slices by different warps; at most HOT_CAP rows are listed, further
 // ones are summed by a single warp.
 constexpr int HOT_T = 32;
+// Touches of a row up to this many keep their (sample, coefficient) pair (the first ROW_SLOTS in the row record).
+constexpr int PAIR_T = 32;
 constexpr int HOT_SLICES = 8;
 constexpr int HOT_CAP = 1024;
 // Rows touched by more than ROW_SLOTS samples are listed too (at most MED_CAP of them; further ones are found
@@ -149,7 +151,7 @@ struct Ctx {
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;         // per row of W1 / W2: which samples of the batch touch it
-  int2 *ovf1, *ovf2;               // per row: the (sample, coefficient) pairs of touches ROW_SLOTS .. HOT_T - 1, at [row][touch]
+  int2 *ovf1, *ovf2;               // per row: the (sample, coefficient) pairs of touches ROW_SLOTS .. PAIR_T - 1, at [row][touch]
   int2 *own1, *own2;               // the distinct touched rows of W1 / W2 with their first-touching sample, in no particular order
   int32_t* hot_rows;               // rows touched by many samples: row of W2, or ~row of W1
   int32_t* med_rows;               // rows touched by more than ROW_SLOTS samples, same encoding

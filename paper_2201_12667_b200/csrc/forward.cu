@@ -121,8 +121,8 @@ __device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowH
     if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(coef));
     else {
       atomicOr(maskrow + (s >> 5), 1u << (s & 31));
-      // up to HOT_T touches keep their pair as well, so that a row with that many is summed without any search
-      if (nth < (unsigned)HOT_T) ovfrow[nth] = make_int2(s, __float_as_int(coef));
+      // up to PAIR_T touches keep their pair as well, so that a row with that many is summed without any search
+      if (nth < (unsigned)PAIR_T) ovfrow[nth] = make_int2(s, __float_as_int(coef));
     }
     first = nth == 0u;
     list_row(p, &hd->cnt, code, nth);
@@ -860,7 +860,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
             x = __ldg(p.vals + rbeg + i);
             nth = atomicAdd(&p.hdr1[c].cnt, 1u) & CNT_MASK;
           }
-          finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.ovf1 + (size_t)c * HOT_T, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
+          finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.ovf1 + (size_t)c * PAIR_T, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
         }
     }
     if (!mbar_wait(sh_bar, phase)) timed_out = true;
@@ -1090,7 +1090,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     for (int u = 0; u < HO_PER; ++u)
       if (u * FWD_THREADS < na)            // uniform over the block
         finish_touch(p, tid + u * FWD_THREADS < na, p.hdr2 + jj0[u], p.mask2 + (size_t)jj0[u] * p.Wd,
-                     p.ovf2 + (size_t)jj0[u] * HOT_T, p.own2,
+                     p.ovf2 + (size_t)jj0[u] * PAIR_T, p.own2,
                      &p.st->n_own[p.parity][0], jj0[u], jj0[u], nth0[u], s, ga0[u]);
     for (int a0 = HO_PER * FWD_THREADS; a0 < na; a0 += FWD_THREADS) {
       const int a = a0 + tid;
@@ -1103,7 +1103,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         ga = gp[a];
         nth = atomicAdd(&p.hdr2[jj].cnt, 1u) & CNT_MASK;
       }
-      finish_touch(p, live, p.hdr2 + jj, p.mask2 + (size_t)jj * p.Wd, p.ovf2 + (size_t)jj * HOT_T, p.own2, &p.st->n_own[p.parity][0], jj, jj, nth, s, ga);
+      finish_touch(p, live, p.hdr2 + jj, p.mask2 + (size_t)jj * p.Wd, p.ovf2 + (size_t)jj * PAIR_T, p.own2, &p.st->n_own[p.parity][0], jj, jj, nth, s, ga);
     }
   }
   if (tid == 0) {

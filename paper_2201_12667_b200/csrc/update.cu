@@ -434,9 +434,9 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowpt
   if ((cv & CNT_HOT) || (cv & CNT_MASK) == 0u) return;
   const int2 sl = hdr_slots(hv);
   const int total = (int)(cv & CNT_MASK);
-  // the pairs of touches ROW_SLOTS .. HOT_T - 1, asked for together with the rows
+  // the pairs of touches ROW_SLOTS .. PAIR_T - 1, asked for together with the rows
   int2 pair = sl;
-  if (total <= HOT_T && lane >= ROW_SLOTS && lane < total) pair = sd.ovf[(size_t)row * HOT_T + lane];
+  if (total <= PAIR_T && lane >= ROW_SLOTS && lane < total) pair = sd.ovf[(size_t)row * PAIR_T + lane];
   float4 w[NCH], m[NCH], v[NCH], acc[NCH];
   load_row<NCH>(sd.W, (size_t)row, H, H4, lane, w);
   load_row<NCH>(sd.M, (size_t)row, H, H4, lane, m);
@@ -444,7 +444,7 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowpt
 #pragma unroll
   for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   float csum = 0.f;
-  if (total <= HOT_T) {
+  if (total <= PAIR_T) {
     // every touch has its pair: lane k holds touch k; put them in ascending sample order (each sample touches a
     // row once, so the samples are distinct) and add; the mask only has to be cleared
     const int s_me = lane < total ? pair.x : 0x7fffffff;
