@@ -9,11 +9,12 @@
 // The same kernel in predict mode stops after the logits and selects the top k.
 //
 // Every phase is a short chain of memory rounds, so each round puts as much in flight as it can:
-// the rows of W1 of a chunk of nonzeros are fetched by all threads at once into shared memory and
-// then summed in the stored order; the L bucket offsets are fetched in one round and all bucket
-// entries in a second; the active rows of W2 are copied by the bulk-copy engine (cp.async.bulk,
-// completion on an mbarrier) into the shared memory the dedup work space no longer needs, and
-// serve both the logits and the back-propagated error.
+// the rows of W1 of a chunk of nonzeros arrive by one bulk copy each (cp.async.bulk, completion on an
+// mbarrier) and are then summed in the stored order; the L bucket offsets are fetched in one round and
+// all bucket entries in a second; the active rows of W2 are copied the same way into the shared memory
+// the dedup work space no longer needs, and serve both the logits and the back-propagated error (in
+// one pass when the set is larger than that space).  Optional steps of the selection: densification
+// of all-zero DWTA bins of the query (Section 4.1) and the sampling budget of Section 3.7.
 #include "common.cuh"
 
 namespace dslide {

@@ -5,23 +5,24 @@
 // The forward kernel leaves, per step and per touched row of W2 / W1: in the row's 64-byte record the
 // number of samples that touch the row and the (sample, coefficient) pairs of its first ROW_SLOTS
 // touches (the record also holds the bias of a row of W2 with its moments, so one line brings all of
-// it); a bit mask of the samples of any further touches; and two lists of (row, first-touching sample)
-// for the distinct touched rows.
+// it); a bit mask of the samples of any further touches, whose pairs up to touch PAIR_T are kept in a
+// side array as well; and two lists of (row, first-touching sample) for the distinct touched rows.
 //
 //   k_update : a warp works on two rows of the row lists at a time; the loads of a row's weights and
 //              moments, of its record and of the first-touching sample's row (h for W2, dh for W1) are
 //              all issued together.  A row touched by one sample takes its gradient from slot 0; a row
 //              touched by up to ROW_SLOTS samples from its slots, put in ascending sample order; a row
-//              touched by more from slots and mask (the sample's coefficient for this row is found by
-//              binary search in the sample's ascending id list), again in ascending sample order.  So
+//              touched by up to PAIR_T samples from its slots and kept pairs, likewise; a row touched by
+//              more from slots and mask (the sample's coefficient for this row is found by binary
+//              search in the sample's ascending id list), again in ascending sample order.  So
 //              the sums do not depend on the order in which the forward kernel's blocks ran, and no
 //              floating-point atomics are used.  Rows touched by more than ROW_SLOTS samples were
 //              listed by the forward kernel and are summed by a warp each; rows touched by more than
 //              HOT_T samples were listed a second time: each is cut into HOT_SLICES slices of its mask,
 //              summed by different warps, and the warp that finishes a row's last slice adds the slice
-//              sums in slice order.  Warps draw tickets (the first one is the warp's own number, the
-//              others come from a counter): hot slices, then listed rows, then the ordinary rows four
-//              at a time.  Adam is applied to the touched rows only; untouched rows are neither read
+//              sums in slice order.  Warps draw tickets (the first two are fixed by the warp's number,
+//              the others come from a counter): hot slices, then listed rows, then the ordinary rows four
+//              at a time, the last few thousand two at a time.  Adam is applied to the touched rows only; untouched rows are neither read
 //              nor written.  The warp that updates a row resets its count and mask for the next step.
 //              The first blocks of the grid update the hidden bias and reduce the batch loss.
 //   k_adam_dense : the output layer when every neuron is active (no lists, no masks).
