@@ -62,7 +62,7 @@ void free_all(Ctx* c) {
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1, c->ovf1, c->ovf2,
                   c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
-                  c->st_dev[0], c->st_dev[1], c->st_dev[2]};
+                  c->st_dev[0], c->st_dev[1], c->st_dev[2], c->pd_part};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (int b = 0; b < ST_SETS; ++b) {
     if (c->st_host[b]) cudaFreeHost(c->st_host[b]);

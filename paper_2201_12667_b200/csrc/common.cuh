@@ -197,6 +197,8 @@ struct Ctx {
   int64_t t_host, r_host, next_rebuild;
   int64_t launches;
   int profiling;
+  void* pd_part;       // dense inference: the slices' best-k lists (ids, then scores), grown on demand
+  size_t pd_cap;
   void* prof;          // std::vector of event pairs while profiling
 };
 

@@ -545,9 +545,10 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     if (k < H) {
       const float hv = acc[u] > 0.f ? acc[u] : 0.f;
       sh_h[k] = hv;
-      if (MODE == 0) p.h[(size_t)s * H + k] = hv;
+      if (MODE == 0 || p.dense) p.h[(size_t)s * H + k] = hv;
     }
   }
+  if (MODE == 1 && p.dense) return;        // inference over all neurons: the logits are taken by k_predict_dense
   __syncthreads();
 
   const bool dense = p.dense != 0;
@@ -1114,6 +1115,175 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   }
 }
 
+
+// ---------------------------------------------------------------------------
+// Inference over all N neurons (no tables): logits of PD_SG samples at a time against a slice of W2
+// ---------------------------------------------------------------------------
+// A block takes PD_SG samples and one slice of the neurons: the samples' hidden activations sit in shared memory, the
+// slice's rows pass through the staging space (one bulk copy per row) and every thread takes one staged row against
+// all PD_SG activations, so a row is fetched once per PD_SG samples instead of once per sample (PD_SG = 32, 16 or 8,
+// the largest whose lists of k fit).  Every warp keeps the
+// best k (logit descending, id ascending) per sample in shared memory: a lane offers its logit only when it beats the
+// list's last entry.  The block's lists are merged per sample and written out; k_predict_merge merges the slices.
+struct PredDenseParams {
+  const float* W2;
+  const RowHdr* hdr2;
+  const float* h;
+  DevState* st;
+  int32_t* part_ids;     // [nslices][B][k]
+  float* part_z;
+  int B, H, N, k, nslices, rows_per_round;
+};
+
+template <int PD_SG>      // samples per block: more of them means fewer passes over W2, and longer lists in shared memory
+__global__ void __launch_bounds__(FWD_THREADS) k_predict_dense(const PredDenseParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = p.H, H4 = H >> 2, k = p.k, ldr = H + 4;
+  float* hs = reinterpret_cast<float*>(smem);                                   // [PD_SG][H]
+  float* lz = hs + (size_t)PD_SG * H;                                           // [FWD_WARPS][PD_SG][k]
+  int* li = reinterpret_cast<int*>(lz + (size_t)FWD_WARPS * PD_SG * k);
+  uint64_t* bar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(li + (size_t)FWD_WARPS * PD_SG * k) + 15) & ~(uintptr_t)15);
+  float* stage = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(bar) + 16);   // [rows_per_round][ldr]
+  const int s0 = blockIdx.y * PD_SG;
+  const int ns = min(PD_SG, p.B - s0);
+  const int per = (p.N + p.nslices - 1) / p.nslices;
+  const int jb = min(p.N, (int)blockIdx.x * per), je = min(p.N, jb + per);
+  for (int e = tid; e < PD_SG * H; e += FWD_THREADS) {
+    const int s = e / H;
+    hs[e] = s < ns ? p.h[(size_t)(s0 + s) * H + (e - s * H)] : 0.f;
+  }
+  if (tid == 0) { mbar_init(bar, 1); asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+  int cnt[PD_SG];                          // lane 0: entries in the warp's list of each sample
+#pragma unroll
+  for (int s = 0; s < PD_SG; ++s) cnt[s] = 0;
+  const float4* hs4 = reinterpret_cast<const float4*>(hs);
+  uint32_t phase = 0;
+  bool timed_out = false;
+  for (int r0 = jb; r0 < je; r0 += p.rows_per_round) {
+    const int nr = min(p.rows_per_round, je - r0);
+    __syncthreads();
+    if (tid == 0) mbar_expect_tx(bar, (uint32_t)nr * (uint32_t)H * 4u);
+    fence_proxy_async();
+    __syncthreads();
+    for (int r = tid; r < nr; r += FWD_THREADS)
+      bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)(r0 + r) * H, (uint32_t)H * 4u, bar);
+    if (!mbar_wait(bar, phase)) timed_out = true;
+    phase ^= 1u;
+    if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
+    for (int ab = 0; ab < nr; ab += FWD_THREADS) {
+      const int a = ab + tid;
+      const bool live = a < nr;
+      float d[PD_SG];
+#pragma unroll
+      for (int s = 0; s < PD_SG; ++s) d[s] = 0.f;
+      float bias = 0.f;
+      if (live) {
+        bias = __ldg(&p.hdr2[r0 + a].b);
+        const float4* row = reinterpret_cast<const float4*>(stage + (size_t)a * ldr);
+        for (int c = 0; c < H4; ++c) {
+          const float4 w = row[c];
+#pragma unroll
+          for (int s = 0; s < PD_SG; ++s) {
+            const float4 x = hs4[s * H4 + c];
+            d[s] = fmaf(w.x, x.x, d[s]); d[s] = fmaf(w.y, x.y, d[s]); d[s] = fmaf(w.z, x.z, d[s]); d[s] = fmaf(w.w, x.w, d[s]);
+          }
+        }
+      }
+      const int j = r0 + a;
+#pragma unroll
+      for (int s = 0; s < PD_SG; ++s) {
+        if (s >= ns) break;                                   // uniform
+        const float z = bias + d[s];
+        float* wz = lz + ((size_t)warp * PD_SG + s) * k;
+        int* wi = li + ((size_t)warp * PD_SG + s) * k;
+        const int n = __shfl_sync(FULLM, cnt[s], 0);
+        const bool offer = live && (n < k || topk_better(z, j, wz[k - 1], wi[k - 1]));
+        unsigned m = __ballot_sync(FULLM, offer);
+        while (m) {                                           // rare once the lists have filled
+          const int l = __ffs(m) - 1;
+          m &= m - 1;
+          const float zl = __shfl_sync(FULLM, z, l);
+          const int jl = __shfl_sync(FULLM, j, l);
+          if (lane == 0 && (cnt[s] < k || topk_better(zl, jl, wz[cnt[s] - 1], wi[cnt[s] - 1]))) {
+            int q = cnt[s] < k ? cnt[s]++ : k - 1;
+            while (q > 0 && topk_better(zl, jl, wz[q - 1], wi[q - 1])) { wz[q] = wz[q - 1]; wi[q] = wi[q - 1]; --q; }
+            wz[q] = zl; wi[q] = jl;
+          }
+          __syncwarp();
+        }
+      }
+    }
+  }
+  if (timed_out) {
+    mbar_wait(bar, phase ^ 1u);
+    if (tid == 0) set_status(p.st, DSLIDE_ERR_TIMEOUT);
+  }
+  // the eight warps' lists of a sample, merged by one thread per sample: k rounds over the list heads
+  int* sh_cnt = reinterpret_cast<int*>(stage);                // [FWD_WARPS][PD_SG] (the staging space is free now)
+  __syncthreads();
+  if (lane == 0)
+#pragma unroll
+    for (int s = 0; s < PD_SG; ++s) sh_cnt[warp * PD_SG + s] = timed_out ? 0 : cnt[s];
+  __syncthreads();
+  if (tid < ns) {
+    const int s = tid;
+    int head[FWD_WARPS];
+    for (int w = 0; w < FWD_WARPS; ++w) head[w] = 0;
+    int32_t* oi = p.part_ids + ((size_t)blockIdx.x * p.B + (s0 + s)) * k;
+    float* oz = p.part_z + ((size_t)blockIdx.x * p.B + (s0 + s)) * k;
+    for (int q = 0; q < k; ++q) {
+      int bw = -1;
+      for (int w = 0; w < FWD_WARPS; ++w) {
+        if (head[w] >= sh_cnt[w * PD_SG + s]) continue;
+        const float* wz = lz + ((size_t)w * PD_SG + s) * k;
+        const int* wi = li + ((size_t)w * PD_SG + s) * k;
+        if (bw < 0) { bw = w; continue; }
+        const float* bz = lz + ((size_t)bw * PD_SG + s) * k;
+        const int* bi = li + ((size_t)bw * PD_SG + s) * k;
+        if (topk_better(wz[head[w]], wi[head[w]], bz[head[bw]], bi[head[bw]])) bw = w;
+      }
+      if (bw >= 0) {
+        oi[q] = li[((size_t)bw * PD_SG + s) * k + head[bw]];
+        oz[q] = lz[((size_t)bw * PD_SG + s) * k + head[bw]];
+        head[bw]++;
+      } else {
+        oi[q] = -1;
+        oz[q] = -INFINITY;
+      }
+    }
+  }
+}
+
+// One thread per sample merges the slices' lists (each in order, padded with id -1).
+__global__ void k_predict_merge(const int32_t* part_ids, const float* part_z, int B, int k, int nslices, int32_t* out_ids,
+                                float* out_scores) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= B) return;
+  int head[64];
+  for (int w = 0; w < nslices; ++w) head[w] = 0;
+  for (int q = 0; q < k; ++q) {
+    int bw = -1;
+    for (int w = 0; w < nslices; ++w) {
+      if (head[w] >= k) continue;
+      const size_t at = ((size_t)w * B + s) * k + head[w];
+      if (part_ids[at] < 0) continue;
+      if (bw < 0) { bw = w; continue; }
+      const size_t bt = ((size_t)bw * B + s) * k + head[bw];
+      if (topk_better(part_z[at], part_ids[at], part_z[bt], part_ids[bt])) bw = w;
+    }
+    if (bw >= 0) {
+      const size_t bt = ((size_t)bw * B + s) * k + head[bw];
+      out_ids[(size_t)s * k + q] = part_ids[bt];
+      out_scores[(size_t)s * k + q] = part_z[bt];
+      head[bw]++;
+    } else {
+      out_ids[(size_t)s * k + q] = -1;
+      out_scores[(size_t)s * k + q] = -INFINITY;
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------
 // Host side: shared-memory layout and launches
 // ---------------------------------------------------------------------------
@@ -1264,11 +1434,43 @@ cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int3
   p.out_ids = out_ids;
   p.out_scores = out_scores;
   if (dense) p.dense = 1;
-  {
-    LaunchScope ls(c, KID_PREDICT);
-    if (c->H <= FWD_THREADS) k_forward<1, 1><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
-    else k_forward<1, MAX_KPT><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+  LaunchScope ls(c, KID_PREDICT);
+  if (c->H <= FWD_THREADS) k_forward<1, 1><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+  else k_forward<1, MAX_KPT><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || !dense) return e;
+  // over all neurons: the kernel above has left the hidden activations; groups of sg samples x slices of W2
+  const int sg = k <= 8 ? 32 : (k <= 16 ? 16 : 8);
+  const int ngroups = (batch + sg - 1) / sg;
+  int nslices = (2 * c->num_sms + ngroups - 1) / ngroups;
+  if (nslices > 64) nslices = 64;
+  if (nslices > c->N) nslices = c->N;
+  if (nslices < 1) nslices = 1;
+  const size_t need = (size_t)nslices * batch * k * 8;
+  if (need > c->pd_cap) {
+    if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) return e;
+    if (c->pd_part) cudaFree(c->pd_part);
+    c->pd_part = nullptr; c->pd_cap = 0;
+    if ((e = cudaMalloc(&c->pd_part, need)) != cudaSuccess) return e;
+    c->pd_cap = need;
   }
+  PredDenseParams q;
+  q.W2 = c->W2; q.hdr2 = c->hdr2; q.h = c->h; q.st = c->dstate;
+  q.part_ids = reinterpret_cast<int32_t*>(c->pd_part);
+  q.part_z = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(c->pd_part) + (size_t)nslices * batch * k * 4);
+  q.B = batch; q.H = c->H; q.N = c->N; q.k = k; q.nslices = nslices;
+  const size_t fixed = (size_t)sg * c->H * 4 + (size_t)FWD_WARPS * sg * k * 8 + 48;
+  const size_t row = (size_t)(c->H + 4) * 4;
+  long long rows = ((long long)(227 * 1024) / 2 - (long long)fixed - 1024) / (long long)row;     // two blocks per multiprocessor
+  if (rows < 8) rows = ((long long)(227 * 1024) - (long long)fixed - 1024) / (long long)row;
+  if (rows < 1) return cudaErrorInvalidValue;
+  if (rows > 512) rows = 512;
+  q.rows_per_round = (int)rows;
+  const size_t smem = fixed + (size_t)rows * row;
+  auto kern = sg == 32 ? k_predict_dense<32> : (sg == 16 ? k_predict_dense<16> : k_predict_dense<8>);
+  if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess) return e;
+  kern<<<dim3(nslices, ngroups), FWD_THREADS, smem, c->stream>>>(q);
+  k_predict_merge<<<(batch + 127) / 128, 128, 0, c->stream>>>(q.part_ids, q.part_z, batch, k, nslices, out_ids, out_scores);
   return cudaGetLastError();
 }
 

@@ -318,15 +318,15 @@ def test_force_dense_matches_oracle_and_dense_softmax():
 
 
 # ------------------------------------------------------------------ inference
-@pytest.mark.parametrize("dense", [0, 1])
-def test_predict_topk(dense):
+@pytest.mark.parametrize("dense,k", [(0, 5), (1, 5), (1, 12), (1, 40)])   # over all neurons: 32, 16, 8 samples per block
+def test_predict_topk(dense, k):
     pr = mid_pair()
     try:
         pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.05)
         pr.push_state()
         wl = workloads.Workload(workloads.config("mid"), seed=7)
         batch = wl.batch(0)
-        B, k = len(batch[0]) - 1, 5
+        B = len(batch[0]) - 1
         ids_o, sc_o = pr.o.predict_topk(batch[0], batch[1], batch[2], k, dense=bool(dense))
         dev = to_dev(batch[:3])
         ids_g = torch.empty(B * k, dtype=torch.int32, device="cuda")
