@@ -906,14 +906,20 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         if (live) { j = dense ? c0 + a : idp[c0 + a]; zv = __ldg(&p.hdr2[j].b) + dot; }
         float* lz = tk_z + warp * p.topk;
         int* li = tk_id + warp * p.topk;
-        for (int l = 0; l < 32; ++l) {
+        // a lane offers its logit only when the list is not full yet or the logit beats the list's last entry
+        const int n = __shfl_sync(FULLM, tk_cnt, 0);
+        unsigned m = __ballot_sync(FULLM, j >= 0 && (n < p.topk || topk_better(zv, j, lz[p.topk - 1], li[p.topk - 1])));
+        while (m) {
+          const int l = __ffs(m) - 1;
+          m &= m - 1;
           const int jl = __shfl_sync(FULLM, j, l);
           const float zl = __shfl_sync(FULLM, zv, l);
-          if (lane == 0 && jl >= 0 && (tk_cnt < p.topk || topk_better(zl, jl, lz[tk_cnt - 1], li[tk_cnt - 1]))) {
+          if (lane == 0 && (tk_cnt < p.topk || topk_better(zl, jl, lz[tk_cnt - 1], li[tk_cnt - 1]))) {
             int q = tk_cnt < p.topk ? tk_cnt++ : p.topk - 1;
             while (q > 0 && topk_better(zl, jl, lz[q - 1], li[q - 1])) { lz[q] = lz[q - 1]; li[q] = li[q - 1]; --q; }
             lz[q] = zl; li[q] = jl;
           }
+          __syncwarp();
         }
       }
     }
