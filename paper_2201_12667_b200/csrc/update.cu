@@ -621,6 +621,9 @@ static cudaError_t launch_k_update(Ctx* c, const UpdParams& p, int smem) {
     e = cudaFuncSetAttribute(k_update<NCH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
+  // the kernel needs little shared memory: the rest of the unified store serves as cache for the h / dh rows
+  e = cudaFuncSetAttribute(k_update<NCH, G>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxL1);
+  if (e != cudaSuccess) return e;
   // one wave: the blocks for the hidden bias come first, the rest fill the remaining block slots of the device
   const int naux = (c->H + 31) / 32;
   int per_sm = 0;
