@@ -6,8 +6,8 @@
  * The operations follow "Distributed SLIDE" (arXiv 2201.12667): Section 2.1 (the
  * three phases of SLIDE), Algorithm 1 (training procedure), Section 3.5 (Adam
  * moments per weight and bias array), Section 3.6 (layer operations and the
- * per-sample snapshot of active neurons), Section 4.1 (hash families, K, L, Adam
- * constants).  Nothing is sharded or communicated between GPUs.
+ * per-sample snapshot of active neurons), Section 3.7 (sampling budget), Section 4.1
+ * (hash families, K, L, Adam constants).  Nothing is sharded or communicated between GPUs.
  *
  * Conventions
  *  - Every function returns a dslide_status.  No exceptions, no abort, no output.
@@ -181,7 +181,10 @@ dslide_status dslide_host_result(dslide_ctx* ctx, float* loss_out, int32_t* have
  * (dense = 1) -> logits -> the k largest by (logit descending, id ascending).
  * out_ids [batch*k] (device, -1 where fewer than k candidates), out_scores [batch*k]
  * (device, -inf there).  1 <= k <= 64.  The paper reports accuracy but not how it
- * evaluates; this is the reading taken. */
+ * evaluates; this is the reading taken.  With dense = 1 the first call (and any call
+ * with a larger batch * k) allocates device work space for the partial lists after
+ * waiting for the stream; the hidden activations of the batch replace those the last
+ * training step left for dslide_get_last. */
 dslide_status dslide_predict_topk(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
                                   const int32_t* col_idx, const float* vals, int32_t k,
                                   int32_t dense, int32_t* out_ids, float* out_scores);
