@@ -60,7 +60,7 @@ cudaError_t dalloc(T** p, size_t n, cudaStream_t st, bool zero) {
 void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->hdr1, c->hdr2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
-                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1, c->ovf1, c->ovf2,
+                  c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1, c->ovf1, c->ovf2, c->hotmap1, c->hotcoef1,
                   c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
                   c->st_dev[0], c->st_dev[1], c->st_dev[2], c->pd_part};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -221,6 +221,8 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(hdr1, D, true); A(mask1, D * c->Wd, true); A(own1, D, true); A(ovf1, D * PAIR_T, false);
   A(hot_rows, HOT_CAP, true); A(med_rows, MED_CAP, true); A(hot_done, HOT_CAP, true); A(hot_part, (size_t)HOT_CAP * HOT_SLICES * (H + 4), true);
   A(dstate, 1, true);
+  A(hotmap1, D, false); A(hotcoef1, (size_t)HOTMAP_CAP * B, false);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->hotmap1, 0xff, D * sizeof(int32_t), st);
   if (!c->dense) {
     A(act_ids, B * S, true);
     A(mask2, N * c->Wd, true);

@@ -38,6 +38,7 @@ struct DevState {
   unsigned int n_hot[2];           // rows touched by more than HOT_T samples (entries of the hot-row list)
   unsigned int n_med[2];           // rows touched by more than ROW_SLOTS samples (entries of the medium-row list)
   unsigned int ticket[2];          // work tickets handed out by the update kernel
+  unsigned int n_hotslots;         // rows of W1 that were given a line of the coefficient table so far (not per step)
   unsigned long long acc[2][3];    // forward kernel: sum of active-set sizes, nonzeros, bucket entries read
   unsigned long long last[3];      // acc of the last finished step
   unsigned long long cum[6];       // since the last reset: steps, sum_active, U2, U1, nnz, fetched
@@ -62,6 +63,9 @@ constexpr int ROW_SLOTS = 6;
 constexpr int HOT_T = 32;
 // Touches of a row up to this many keep their (sample, coefficient) pair (the first ROW_SLOTS in the row record).
 constexpr int PAIR_T = 32;
+// Rows of W1 that have been hot once (frequent features stay frequent) own a line of a coefficient table: every
+// later touch leaves its value there, indexed by sample, and the slices of the row read it instead of searching.
+constexpr int HOTMAP_CAP = 4096;
 constexpr int HOT_SLICES = 8;
 constexpr int HOT_CAP = 1024;
 // Rows touched by more than ROW_SLOTS samples are listed too (at most MED_CAP of them; further ones are found
@@ -151,6 +155,8 @@ struct Ctx {
   int32_t *act_cnt, *act_ids;
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;         // per row of W1 / W2: which samples of the batch touch it
+  int32_t* hotmap1;                // per row of W1: its line of hotcoef1, or -1
+  float* hotcoef1;                 // [HOTMAP_CAP][max_batch]
   int2 *ovf1, *ovf2;               // per row: the (sample, coefficient) pairs of touches ROW_SLOTS .. PAIR_T - 1, at [row][touch]
   int2 *own1, *own2;               // the distinct touched rows of W1 / W2 with their first-touching sample, in no particular order
   int32_t* hot_rows;               // rows touched by many samples: row of W2, or ~row of W1

@@ -40,6 +40,9 @@ struct FwdParams {
   float *act_z, *act_p, *act_g;
   uint32_t *mask1, *mask2;
   int2 *ovf1, *ovf2;
+  const int32_t* hotmap1;   // rows of W1 with a line of the coefficient table
+  float* hotcoef1;
+  int bstride;              // samples per line of that table
   RowHdr *hdr1, *hdr2;
   int2 *own1, *own2;
   int32_t *hot_rows, *med_rows;
@@ -861,6 +864,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
             c = __ldg(p.col_idx + rbeg + i);
             x = __ldg(p.vals + rbeg + i);
             nth = atomicAdd(&p.hdr1[c].cnt, 1u) & CNT_MASK;
+            const int line = __ldg(p.hotmap1 + c);          // a feature that has been hot before: its value goes to its line
+            if (line >= 0) p.hotcoef1[(size_t)line * p.bstride + s] = x;
           }
           finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.ovf1 + (size_t)c * PAIR_T, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
         }
@@ -1400,7 +1405,8 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals; p.label_ptr = label_ptr; p.labels = labels;
   p.h = c->h; p.dh = c->dh; p.loss = c->loss; p.codes = c->codes;
   p.act_cnt = c->act_cnt; p.act_ids = c->act_ids; p.act_z = c->act_z; p.act_p = c->act_p; p.act_g = c->act_g;
-  p.mask1 = c->mask1; p.mask2 = c->mask2; p.ovf1 = c->ovf1; p.ovf2 = c->ovf2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.ovf1 = c->ovf1; p.ovf2 = c->ovf2;
+  p.hotmap1 = c->hotmap1; p.hotcoef1 = c->hotcoef1; p.bstride = c->cfg.max_batch; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
   p.own1 = c->own1; p.own2 = c->own2; p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.parity = (int)(c->t_host & 1);
   p.st = c->dstate; p.out_ids = nullptr; p.out_scores = nullptr;
   p.nb = c->nb;

@@ -20,7 +20,8 @@
 //              listed by the forward kernel and are summed by a warp each; rows touched by more than
 //              HOT_T samples were listed a second time: each is cut into HOT_SLICES slices of its mask,
 //              summed by different warps, and the warp that finishes a row's last slice adds the slice
-//              sums in slice order.  Warps draw tickets (the first two are fixed by the warp's number,
+//              sums in slice order (rows of W1 that have been hot before find their coefficients in a
+//              table line the forward kernel fills, instead of searching).  Warps draw tickets (the first two are fixed by the warp's number,
 //              the others come from a counter): hot slices, then listed rows, then the ordinary rows four
 //              at a time, the last few thousand two at a time.  Adam is applied to the touched rows only; untouched rows are neither read
 //              nor written.  The warp that updates a row resets its count and mask for the next step.
@@ -44,6 +45,9 @@ struct UpdParams {
   const float* vals;
   uint32_t *mask1, *mask2;
   const int2 *ovf1, *ovf2;
+  int32_t* hotmap1;
+  const float* hotcoef1;
+  int bstride;
   RowHdr *hdr1, *hdr2;
   const int2 *own1, *own2;
   const int32_t *hot_rows, *med_rows;
@@ -202,7 +206,7 @@ __device__ __forceinline__ void sum_slots(const Side& sd, int2 sl, int total, in
 template <int NCH>
 __device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, const int* rowptr, int row,
                                            int slot_s, int w0, int w1, int* scr, float4 (&acc)[NCH], float& csum,
-                                           int H, int H4, int lane) {
+                                           int H, int H4, int lane, const float* line = nullptr) {
   uint32_t* mrow = sd.mask + (size_t)row * p.Wd;
   int fill = 0;
   const unsigned lt = (1u << lane) - 1u;
@@ -224,7 +228,7 @@ __device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, c
       if (fill + nb > 32) {
         __syncwarp();
         const int s_mine = lane < fill ? scr[lane] : 0;
-        const float g_mine = lane < fill ? find_coef(p, sd, rowptr, row, s_mine) : 0.f;
+        const float g_mine = lane < fill ? (line ? line[s_mine] : find_coef(p, sd, rowptr, row, s_mine)) : 0.f;
         accumulate_list<NCH>(acc, csum, fill, s_mine, g_mine, sd.src, H, H4, lane);
         fill = 0;
         __syncwarp();
@@ -236,7 +240,7 @@ __device__ __forceinline__ void sum_masked(const UpdParams& p, const Side& sd, c
   __syncwarp();
   if (fill > 0) {
     const int s_mine = lane < fill ? scr[lane] : 0;
-    const float g_mine = lane < fill ? find_coef(p, sd, rowptr, row, s_mine) : 0.f;
+    const float g_mine = lane < fill ? (line ? line[s_mine] : find_coef(p, sd, rowptr, row, s_mine)) : 0.f;
     accumulate_list<NCH>(acc, csum, fill, s_mine, g_mine, sd.src, H, H4, lane);
   }
   __syncwarp();
@@ -379,7 +383,11 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* rowptr, 
   for (int u = 0; u < NCH; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
   float csum = 0.f;
   const int2 hv = load_hdr(sd.hdr + row, lane);
-  sum_masked<NCH>(p, sd, rowptr, row, hdr_slots(hv).x, w0, w1, scr, acc, csum, H, H4, lane);
+  // a row of W1 that has been hot before has its coefficients in its line of the table (left there by the forward
+  // kernel of this step), indexed by sample: no search
+  const int hline = w2 ? -1 : p.hotmap1[row];
+  sum_masked<NCH>(p, sd, rowptr, row, hdr_slots(hv).x, w0, w1, scr, acc, csum, H, H4, lane,
+                  hline >= 0 ? p.hotcoef1 + (size_t)hline * p.bstride : nullptr);
   const int ld = H + 4;
   float* part = p.hot_part + (size_t)hrow * HOT_SLICES * ld;
   float4* mine = reinterpret_cast<float4*>(part + (size_t)slice * ld);
@@ -417,7 +425,13 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* rowptr, 
   }
   adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
   finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
-  if (lane == 0) p.hot_done[hrow] = 0;
+  if (lane == 0) {
+    p.hot_done[hrow] = 0;
+    if (!w2 && hline < 0) {           // hot for the first time: a line for the steps to come (every slice of this step has read -1)
+      const unsigned at = atomicAdd(&p.st->n_hotslots, 1u);
+      if (at < (unsigned)HOTMAP_CAP) p.hotmap1[row] = (int)at;
+    }
+  }
 }
 
 // A row touched by more than ROW_SLOTS samples that the forward kernel listed: one warp sums it from slots and
@@ -644,7 +658,8 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   p.W2 = c->W2; p.mW2 = c->mW2; p.vW2 = c->vW2;
   p.h = c->h; p.dh = c->dh; p.act_g = c->act_g; p.loss = c->loss; p.act_cnt = c->act_cnt; p.act_ids = c->act_ids;
   p.row_ptr = row_ptr; p.col_idx = col_idx; p.vals = vals;
-  p.mask1 = c->mask1; p.mask2 = c->mask2; p.ovf1 = c->ovf1; p.ovf2 = c->ovf2; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
+  p.mask1 = c->mask1; p.mask2 = c->mask2; p.ovf1 = c->ovf1; p.ovf2 = c->ovf2;
+  p.hotmap1 = c->hotmap1; p.hotcoef1 = c->hotcoef1; p.bstride = c->cfg.max_batch; p.hdr1 = c->hdr1; p.hdr2 = c->hdr2;
   p.own1 = c->own1; p.own2 = c->own2;
   p.hot_rows = c->hot_rows; p.med_rows = c->med_rows; p.hot_part = c->hot_part; p.hot_done = c->hot_done;
   p.st = c->dstate; p.loss_out = loss_out; p.host_res = host_res; p.host_seq = host_seq;
