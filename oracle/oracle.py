@@ -82,6 +82,8 @@ def _load(real):
             getattr(lib, f).argtypes = [C.c_void_p]
         lib.orc_rng.restype = C.c_uint64
         lib.orc_rng.argtypes = [C.c_uint64] * 4
+        lib.orc_mix64.restype = C.c_uint64
+        lib.orc_mix64.argtypes = [C.c_uint64]
         lib.orc_draw_hash.argtypes = [C.c_void_p, C.c_int64]
         lib.orc_build_tables.argtypes = [C.c_void_p]
         lib.orc_rebuild_tables.argtypes = [C.c_void_p]
@@ -104,6 +106,11 @@ def _load(real):
 
 def rng(seed, stream, r, ctr):
     return int(_load("float").orc_rng(seed, stream, r, ctr))
+
+
+def mix64(z):
+    """The generator's output function alone (pinned against the published splitmix64 outputs)."""
+    return int(_load("float").orc_mix64(z))
 
 
 def _p(a):

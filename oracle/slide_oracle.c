@@ -17,7 +17,7 @@
  * (used by the gradient and dense-limit pins).
  *
  * Where the paper is silent the reading taken is stated next to the code
- * (marked "reading:").  Pins: tests/test_oracle_*.py.  Unpinned: the
+ * (marked "reading:").  Pins: tests/test_oracle_*.py (the generator and the initial weights: tests/test_oracle_rng.py).  Unpinned: the
  * paper's accuracy figures (they need its datasets) -- "parity unpinned"
  * for those; no function in this file is unpinned.
  */
@@ -99,6 +99,10 @@ static uint64_t mix64(uint64_t z) {
   return z ^ (z >> 31);
 }
 static const uint64_t GOLD = 0x9E3779B97F4A7C15ULL;
+
+/* The output function alone, for the pin against the published splitmix64 outputs:
+ * the k-th output of splitmix64 seeded with s is mix64(s + k * GOLD), k = 1, 2, ... */
+uint64_t orc_mix64(uint64_t z) { return mix64(z); }
 
 uint64_t orc_rng(uint64_t seed, uint64_t stream, uint64_t r, uint64_t ctr) {
   uint64_t a = mix64(seed + GOLD * (stream + 1));
@@ -371,22 +375,7 @@ static void hidden_layer(const orc *o, int32_t nnz, const int32_t *col, const RE
   }
 }
 
-/* Section 2.1 feed-forward stage + Fig. 1: query the L tables with the layer
- * input, take the union of the retrieved buckets (at most bucket_cap lowest
- * ids of each), add the labels when given (reading: labels are always
- * active), sort, remove duplicates.  Returns the count, or -1 on overflow. */
-/* Section 3.7: when the neurons retrieved for a sample exceed the sampling
- * budget, reservoir sampling controls how many are kept; when they do not,
- * reading: the set is left as it is (the paper's "stop with the current set
- * of neurons"; its other option, a uniform random fill, is not built).
- * reading: the budget counts the sample's labels, which are always active,
- * so m = max(0, budget - |Y|) of the other retrieved neurons are kept.  The
- * candidates C_0 < C_1 < ... (retrieved ids that are not labels, ascending)
- * go through the textbook reservoir algorithm: the first m fill the
- * reservoir; candidate i >= m draws j uniform in [0, i] and replaces
- * reservoir[j] when j < m.  j = rng(seed, STREAM_SAMPLE, steps taken so far,
- * sample * 2^32 + i) mod (i + 1).  act[] (ascending, n entries) is rewritten
- * with the labels and the reservoir, ascending; returns the new count. */
+/* Is id one of the sample's labels? */
 static int is_label(int32_t id, const int32_t *lab, int32_t nlab) {
   for (int32_t i = 0; i < nlab; ++i) if (lab[i] == id) return 1;
   return 0;
@@ -415,6 +404,19 @@ static int64_t fill_budget(const orc *o, int32_t *act, int64_t n, int32_t s) {
   return n + got;
 }
 
+/* Section 3.7: when the neurons retrieved for a sample exceed the sampling
+ * budget, reservoir sampling controls how many are kept; when they do not,
+ * reading: the set is left as it is (the paper's "stop with the current set
+ * of neurons") unless budget_fill asks for the paper's other option, the
+ * uniform random fill (fill_budget above).
+ * reading: the budget counts the sample's labels, which are always active,
+ * so m = max(0, budget - |Y|) of the other retrieved neurons are kept.  The
+ * candidates C_0 < C_1 < ... (retrieved ids that are not labels, ascending)
+ * go through the textbook reservoir algorithm: the first m fill the
+ * reservoir; candidate i >= m draws j uniform in [0, i] and replaces
+ * reservoir[j] when j < m.  j = rng(seed, STREAM_SAMPLE, steps taken so far,
+ * sample * 2^32 + i) mod (i + 1).  act[] (ascending, n entries) is rewritten
+ * with the labels and the reservoir, ascending; returns the new count. */
 static int64_t apply_budget(const orc *o, int32_t *act, int64_t n, const int32_t *lab, int32_t nlab, int32_t s) {
   const orc_config *c = &o->c;
   int64_t ny = 0, nc = 0;
@@ -440,6 +442,11 @@ static int64_t apply_budget(const orc *o, int32_t *act, int64_t n, const int32_t
   return out;
 }
 
+/* Section 2.1 feed-forward stage + Fig. 1: query the L tables with the layer
+ * input, take the union of the retrieved buckets (at most bucket_cap lowest
+ * ids of each), add the labels when given (reading: labels are always
+ * active), sort, remove duplicates, then apply the sampling budget when one
+ * is set.  Returns the count. */
 static int64_t select_active(const orc *o, const uint32_t *codes, const int32_t *lab, int32_t nlab,
                              int32_t **buf, int64_t *bufcap, int32_t s) {
   const orc_config *c = &o->c;

@@ -354,3 +354,36 @@ def test_budget_fill_off_leaves_under_full_sets_alone():
     for a0, a1 in zip(free, capped):
         if len(a0) <= 150:
             assert np.array_equal(a0, a1)
+
+
+# ---------------------------------------------------------------- the weight bar's floor, measured
+def test_fp32_rounding_alone_moves_weights_by_the_floor_the_gpu_bar_uses():
+    """The GPU parity bar for weights after 10 Adam steps is 1e-3 of max(|a|, |b|, 0.01 * largest magnitude).
+    Why 0.01 and not 0.001: Adam divides by the gradient's magnitude, so fp32 rounding in a cancelling gradient
+    sum moves a weight by a fixed fraction of lr whatever the weight's size.  Measured here with the oracle alone:
+    its fp32 and fp64 builds, same start, same batches, same active sets, differ by about 2e-4 under the 0.01
+    floor and by more than the 1e-3 bar under a 0.001 floor -- i.e. that floor would be below fp32 noise."""
+    from paper_2201_12667_b200 import workloads
+    from tests.helpers import max_rel_err
+    c = workloads.config("mid")
+    kw = dict(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"], L=c["L"], bucket_cap=c["bucket_cap"],
+              lr=c["lr"], init_std=0.05, seed=0)
+    a, b = Oracle("float", **kw), Oracle("double", **kw)
+    try:
+        for n in ("W1", "W2"):
+            b.set(n, a.view(n).astype(np.float64))
+        b.build_tables()
+        wl = workloads.Workload(c, seed=0)
+        for i in range(10):
+            bt = wl.batch(i)
+            a.train_step(*bt)
+            b.train_step(*bt)
+            assert np.array_equal(a.get("act_ids"), b.get("act_ids"))     # no code flipped: same rows touched
+        names = ("W1", "b1", "W2", "b2")
+        wide = max(max_rel_err(a.view(n), b.view(n), 1e-2) for n in names)
+        narrow = max(max_rel_err(a.view(n), b.view(n), 1e-3) for n in names)
+        assert 1e-4 < wide < 4e-4           # fp32 noise sits a factor 3-10 inside the 1e-3 bar
+        assert narrow > 1e-3                # with the smaller floor the noise alone would break the bar
+    finally:
+        a.close()
+        b.close()
