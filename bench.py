@@ -263,7 +263,7 @@ def run_dslide(args):
                          L=c["L"], dwta_bin_size=c["bin_size"], bucket_cap=c["bucket_cap"],
                          rebuild_period0=args.rebuild_period, rebuild_growth_lambda=0.0, redraw_hash_fns=1,
                          max_batch=B, max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0, device=local,
-                         sample_budget=args.budget)
+                         sample_budget=args.budget, inputs_ready=1)
     ctx = ds.dslide_init(cfg)
 
     wl = workloads.Workload(c, seed=shard_seed(rank))

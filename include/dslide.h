@@ -44,7 +44,10 @@ typedef enum {
   DSLIDE_ERR_OVERFLOW = 4,   /* an active set, label list or batch exceeds the configured maximum */
   DSLIDE_ERR_BAD_INDEX = 5,  /* feature id outside [0,D) or label id outside [0,N), seen on the device */
   DSLIDE_ERR_STATE = 6,
-  DSLIDE_ERR_TIMEOUT = 7     /* a bounded wait inside a kernel ran out (the sample concerned is skipped)               */
+  DSLIDE_ERR_TIMEOUT = 7     /* a bounded wait inside a kernel ran out.  The sample concerned is skipped: no loss, no
+                                gradient.  If the wait that ran out was for rows of W2, the sample's rows of W1 had
+                                been handed to the update already: they receive an Adam update with a zero
+                                gradient from this sample (their moments decay), unlike rows nobody touched.    */
 } dslide_status;
 
 enum { DSLIDE_SIMHASH = 0, DSLIDE_DWTA = 1 };
@@ -89,6 +92,15 @@ typedef struct {
                                                 per-sample arrays then hold up to budget entries; the work space
                                                 (about 80 bytes per budgeted neuron) must fit the forward
                                                 kernel's shared memory, else DSLIDE_ERR_INVALID_ARG.              */
+  int32_t inputs_ready;                      /* dslide_train_step only.  0: the batch arrays may still be written by
+                                                work enqueued earlier on the context's stream (a kernel or copy of
+                                                the caller's); the step reads them only after that work has
+                                                completed.  1: the caller promises that the five arrays were
+                                                complete in device memory BEFORE the call (their producer has
+                                                finished, not merely been enqueued); the step then reads them while
+                                                the previous step's update is still draining, which shortens the
+                                                step by a few microseconds.  The host-buffer entry points wait for
+                                                their own copy and always read early.                              */
 } dslide_config;
 
 /* Tensors readable and writable through dslide_get_tensor / dslide_set_tensor. */
@@ -183,8 +195,11 @@ dslide_status dslide_host_result(dslide_ctx* ctx, float* loss_out, int32_t* have
  * (device, -inf there).  1 <= k <= 64.  The paper reports accuracy but not how it
  * evaluates; this is the reading taken.  With dense = 1 the first call (and any call
  * with a larger batch * k) allocates device work space for the partial lists after
- * waiting for the stream; the hidden activations of the batch replace those the last
- * training step left for dslide_get_last. */
+ * waiting for the stream.  A predict call uses the per-sample work space of the training
+ * step: afterwards the snapshot read by dslide_get_last (hidden activations with dense = 1;
+ * active ids and logits with dense = 0, whose counts, codes and losses still belong to the
+ * last training step) is no longer that of the last training step.  The next training step
+ * rewrites all of it. */
 dslide_status dslide_predict_topk(dslide_ctx* ctx, int32_t batch, const int32_t* row_ptr,
                                   const int32_t* col_idx, const float* vals, int32_t k,
                                   int32_t dense, int32_t* out_ids, float* out_scores);
@@ -195,7 +210,8 @@ dslide_status dslide_sync(dslide_ctx* ctx);
 /* State I/O (check-pointing and the parity harness).  Synchronous.  host pointers.
  * nbytes must equal the tensor's size exactly.  Setting weights or hash functions does
  * not rebuild the tables; call dslide_build_tables. */
-dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes);
+enum { DSLIDE_DT_F32 = 0, DSLIDE_DT_I32 = 1, DSLIDE_DT_I64 = 2 };
+dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes, int32_t* dtype /* may be NULL: DSLIDE_DT_* */);
 dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, int64_t nbytes);
 dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host_src, int64_t nbytes);
 
@@ -251,7 +267,9 @@ dslide_status dslide_profile_end(dslide_ctx* ctx, double ms[DSLIDE_K_COUNT], int
  * (once per device, with that device current); make that first call before any stream capture.
  * All calls on a device share the one array, which keeps the last call's contents: the kernel
  * overwrites what it reads, but two calls that overlap on the GPU (different streams, no
- * ordering between them) race on it -- order them. */
+ * ordering between them) race on it -- order them.  The address looked up by the first call is
+ * kept per device ordinal for the life of the process: it is stale after cudaDeviceReset, and
+ * the first call on a device must not race with another first call from a second host thread. */
 #define DSLIDE_STATIC_SORT_MAX_N 262144
 #define DSLIDE_STATIC_SORT_MAX_BITS 18
 dslide_status dslide_bucket_sort_static(const uint32_t* codes, int32_t n, int32_t bits,

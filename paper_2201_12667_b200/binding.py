@@ -43,6 +43,7 @@ class Config(C.Structure):
         ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
         ("init_std", C.c_float), ("seed", C.c_uint64), ("device", C.c_int32), ("dedup_mode", C.c_int32),
         ("stream", C.c_void_p), ("dwta_densify", C.c_int32), ("sample_budget", C.c_int32), ("budget_fill", C.c_int32),
+        ("inputs_ready", C.c_int32),
     ]
 
 
@@ -58,7 +59,7 @@ _SIGS = {
     "dslide_host_result": (_i32, [_vp, C.POINTER(C.c_float), C.POINTER(_i32)]),
     "dslide_predict_topk": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _vp]),
     "dslide_sync": (_i32, [_vp]),
-    "dslide_tensor_info": (_i32, [_vp, _i32, C.POINTER(_i64)]),
+    "dslide_tensor_info": (_i32, [_vp, _i32, C.POINTER(_i64), C.POINTER(_i32)]),
     "dslide_get_tensor": (_i32, [_vp, _i32, _vp, _i64]),
     "dslide_set_tensor": (_i32, [_vp, _i32, _vp, _i64]),
     "dslide_last_info": (_i32, [_vp, _i32, C.POINTER(_i64), C.POINTER(_i32)]),
@@ -100,13 +101,15 @@ def _dptr(t):
 def make_config(*, input_dim, hidden_dim, output_dim, hash_family=DWTA, K=6, L=50, dwta_bin_size=8, srp_nnz=0,
                 bucket_cap=128, rebuild_period0=50, rebuild_growth_lambda=0.0, redraw_hash_fns=1, force_dense=0,
                 max_batch=256, max_labels=16, max_active_per_sample=0, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8,
-                init_std=0.01, seed=0, device=0, dedup_mode=0, stream=None, dwta_densify=0, sample_budget=0, budget_fill=0):
+                init_std=0.01, seed=0, device=0, dedup_mode=0, stream=None, dwta_densify=0, sample_budget=0, budget_fill=0,
+                inputs_ready=0):
     if stream is None:
         import torch
         stream = torch.cuda.current_stream(device).cuda_stream
     return Config(input_dim, hidden_dim, output_dim, hash_family, K, L, dwta_bin_size, srp_nnz, bucket_cap,
                   rebuild_period0, rebuild_growth_lambda, redraw_hash_fns, force_dense, max_batch, max_labels,
-                  max_active_per_sample, lr, beta1, beta2, eps, init_std, seed, device, dedup_mode, stream, dwta_densify, sample_budget, budget_fill)
+                  max_active_per_sample, lr, beta1, beta2, eps, init_std, seed, device, dedup_mode, stream, dwta_densify, sample_budget, budget_fill,
+                  inputs_ready)
 
 
 # ---- the C entry points, same names ---------------------------------------------------------
@@ -169,10 +172,13 @@ def dslide_sync(ctx, check=True):
     return s
 
 
+_DT = [np.float32, np.int32, np.int64]       # DSLIDE_DT_*
+
+
 def dslide_get_tensor(ctx, name):
-    n = _i64()
-    _check(_lib.dslide_tensor_info(ctx, T[name], C.byref(n)), "dslide_tensor_info")
-    dt = np.dtype(_T_DTYPE.get(name, np.float32))
+    n, code = _i64(), _i32()
+    _check(_lib.dslide_tensor_info(ctx, T[name], C.byref(n), C.byref(code)), "dslide_tensor_info")
+    dt = np.dtype(_DT[code.value])
     out = np.empty(n.value // dt.itemsize, dtype=dt)
     if n.value:
         _check(_lib.dslide_get_tensor(ctx, T[name], out.ctypes.data, n.value), "dslide_get_tensor")
@@ -193,13 +199,13 @@ def dslide_get_last(ctx, name, batch):
     total = n.value // dt.itemsize
     if total == 0:
         return np.zeros((batch, 0), dtype=dt)
-    per = total // _max_batch_of(ctx, n.value, dt, name, stride.value)
+    per = total // _max_batch_of(ctx)
     out = np.empty(batch * per, dtype=dt)
     _check(_lib.dslide_get_last(ctx, LAST[name], out.ctypes.data, out.nbytes), "dslide_get_last")
     return out.reshape(batch, per) if per > 1 else out
 
 
-def _max_batch_of(ctx, nbytes, dt, name, stride):
+def _max_batch_of(ctx):
     # rows of the snapshot array = max_batch; recover it from the loss array, which has one float per sample
     n = _i64()
     _check(_lib.dslide_last_info(ctx, LAST["loss"], C.byref(n), None), "dslide_last_info")

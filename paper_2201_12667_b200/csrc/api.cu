@@ -26,7 +26,7 @@ struct dslide_ctx { Ctx c; };
 namespace dslide {
 struct ProfRec { int kid; cudaEvent_t beg, end; };
 
-LaunchScope::LaunchScope(Ctx* c_, int kid_) : c(c_), kid(kid_), rec(nullptr) {
+LaunchScope::LaunchScope(Ctx* c_, int kid_) : c(c_), kid(kid_), rec(-1) {
   c->launches++;
   if (!c->profiling || !c->prof) return;
   auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
@@ -36,10 +36,12 @@ LaunchScope::LaunchScope(Ctx* c_, int kid_) : c(c_), kid(kid_), rec(nullptr) {
   if (cudaEventCreate(&r.end) != cudaSuccess) { cudaEventDestroy(r.beg); return; }
   cudaEventRecord(r.beg, c->stream);
   v->push_back(r);
-  rec = &v->back();
+  rec = (long long)v->size() - 1;      // an index, not a pointer: the vector may grow (and move) before the scope ends
 }
 LaunchScope::~LaunchScope() {
-  if (rec) cudaEventRecord(static_cast<ProfRec*>(rec)->end, c->stream);
+  if (rec < 0 || !c->prof) return;
+  auto* v = static_cast<std::vector<ProfRec>*>(c->prof);
+  if ((size_t)rec < v->size()) cudaEventRecord((*v)[(size_t)rec].end, c->stream);
 }
 }  // namespace dslide
 
@@ -155,7 +157,7 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
     return DSLIDE_ERR_INVALID_ARG;
   if (k.rebuild_period0 < 0 || k.init_std < 0.f || k.dedup_mode < 0 || k.dedup_mode > 2) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_densify < 0 || k.dwta_densify > 1 || k.sample_budget < 0) return DSLIDE_ERR_INVALID_ARG;
-  if (k.budget_fill < 0 || k.budget_fill > 1) return DSLIDE_ERR_INVALID_ARG;
+  if (k.budget_fill < 0 || k.budget_fill > 1 || k.inputs_ready < 0 || k.inputs_ready > 1) return DSLIDE_ERR_INVALID_ARG;
   if (k.budget_fill && (k.sample_budget < 1 || k.max_active_per_sample != 0 || k.force_dense)) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_bin_size == 0) k.dwta_bin_size = 8;
   if (k.srp_nnz == 0) k.srp_nnz = (k.hidden_dim + 2) / 3;
@@ -299,7 +301,8 @@ dslide_status train_step_impl(dslide_ctx* ctx, int32_t batch, const int32_t* row
                               const float* vals, const int32_t* label_ptr, const int32_t* labels, float* loss_out,
                               HostResult* host_res, unsigned int host_seq) {
   Ctx* c = &ctx->c;
-  CU(launch_forward_train(c, batch, row_ptr, col_idx, vals, label_ptr, labels));
+  // a host-buffer step has waited for its own input copy; a device-pointer step reads early only on the caller's word
+  CU(launch_forward_train(c, batch, row_ptr, col_idx, vals, label_ptr, labels, host_res ? 1 : (c->cfg.inputs_ready ? 1 : 0)));
   CU(launch_update(c, batch, row_ptr, col_idx, vals, loss_out, host_res, host_seq));
   c->t_host += 1;
   if (c->cfg.rebuild_period0 > 0 && c->t_host == c->next_rebuild) {
@@ -483,12 +486,15 @@ dslide_status dslide_sync(dslide_ctx* ctx) {
   return (dslide_status)status;
 }
 
-dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes) {
+dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes, int32_t* dtype) {
   if (!ctx || !nbytes) return DSLIDE_ERR_INVALID_ARG;
   TensorRef t = tensor_ref(&ctx->c, which);
   if (t.bytes < 0) return DSLIDE_ERR_INVALID_ARG;
   if (ctx->c.dense && (which == DSLIDE_T_BUCKET_OFF || which == DSLIDE_T_BUCKET_IDS)) t.bytes = 0;
   *nbytes = t.bytes;
+  if (dtype)
+    *dtype = which == DSLIDE_T_COUNTERS ? DSLIDE_DT_I64
+             : (which >= DSLIDE_T_HASH_IDX && which <= DSLIDE_T_BUCKET_IDS) ? DSLIDE_DT_I32 : DSLIDE_DT_F32;
   return DSLIDE_OK;
 }
 
@@ -496,7 +502,7 @@ dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, 
   if (!ctx || !host_dst) return DSLIDE_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   int64_t want = 0;
-  dslide_status s = dslide_tensor_info(ctx, which, &want);
+  dslide_status s = dslide_tensor_info(ctx, which, &want, nullptr);
   if (s != DSLIDE_OK) return s;
   if (nbytes != want) return DSLIDE_ERR_INVALID_ARG;
   if (which == DSLIDE_T_COUNTERS) {
@@ -521,7 +527,7 @@ dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host
   if (!ctx || !host_src) return DSLIDE_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   int64_t want = 0;
-  dslide_status s = dslide_tensor_info(ctx, which, &want);
+  dslide_status s = dslide_tensor_info(ctx, which, &want, nullptr);
   if (s != DSLIDE_OK) return s;
   if (nbytes != want) return DSLIDE_ERR_INVALID_ARG;
   if (which == DSLIDE_T_COUNTERS) {

@@ -112,7 +112,7 @@ enum { KID_FORWARD = 0, KID_ADAM_DENSE, KID_ADAM, KID_DRAW_HASH, KID_HASH_NEURON
 
 // Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event pair around it.
 struct LaunchScope {
-  Ctx* c; int kid; void* rec;
+  Ctx* c; int kid; long long rec;      // rec: index of the event pair in the context's list, -1 when not profiling
   LaunchScope(Ctx* c, int kid);
   ~LaunchScope();
 };
@@ -123,7 +123,7 @@ cudaError_t launch_draw_hash(Ctx* c, int64_t r);
 cudaError_t launch_build_tables(Ctx* c);
 cudaError_t launch_order_buckets(Ctx* c, int min_n);
 cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
-                                 const float* vals, const int32_t* label_ptr, const int32_t* labels);
+                                 const float* vals, const int32_t* label_ptr, const int32_t* labels, int inputs_ready);
 cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
                           float* loss_out, HostResult* host_res, unsigned int host_seq);
 cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,

@@ -62,6 +62,7 @@ struct FwdParams {
   int hash_sm_off;     // where in the staging region the hash functions' index tables are mirrored (-1: read from global memory)
   int hash_sm_bytes;
   int sort_small;      // candidate sets up to this size are deduplicated by sorting even when a bitmap is available
+  int inputs_ready;    // the batch arrays were complete before the launch: they may be read before griddep_wait()
   int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_tbeg, off_topk, off_ids, off_z, off_col, off_val,
       off_dedup;
 };
@@ -437,6 +438,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
 
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = p.H, H4 = H >> 2, N = p.N;
+  // Unless the caller has promised that the batch arrays were complete before the launch, they may still be being
+  // written by the kernel before this one in the stream: wait for it before the first read.
+  bool waited = false;
+  if (!p.inputs_ready) {
+    griddep_wait();
+    waited = true;
+  }
   const int rbeg = p.row_ptr[s], rend = p.row_ptr[s + 1];
   const int nnz = rend - rbeg;
   int lbeg = 0, nlab = 0;
@@ -473,10 +481,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   // ---- hidden layer: bias, then one fused multiply-add per nonzero in stored order, ReLU.  The rows of W1 of a
   //      chunk of nonzeros are fetched together into shared memory; the column ids are checked on the way
   //      (in range, ascending) ----
-  //      Up to here, and through the first chunk's column ids and values, only the caller's batch is read: the
-  //      kernel may run that far while the previous step's update kernel is still finishing (griddep_wait).
+  //      Up to here, and through the first chunk's column ids and values, only the caller's batch is read: with
+  //      inputs_ready the kernel runs that far while the previous step's update kernel is still finishing.
   float acc[KPT];
-  bool waited = false;
   uint32_t phase = 0;                // of sh_bar, which serves the staging of W1 rows here and of W2 rows below
   bool timed_out = false;
   const int R = p.hid_rows;
@@ -1418,7 +1425,7 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.stage_bytes = c->fwd_stage_bytes; p.hid_rows = l.hid_rows; p.sort_small = c->fwd_sort_small;
   p.densify = c->cfg.dwta_densify; p.seed = c->cfg.seed; p.rcount = (unsigned long long)c->r_host;
   p.budget = c->cfg.sample_budget; p.budget_fill = c->cfg.budget_fill; p.tcount = (unsigned long long)c->t_host;
-  p.hash_sm_off = c->fwd_hash_sm_off; p.hash_sm_bytes = c->fwd_hash_sm_bytes;
+  p.hash_sm_off = c->fwd_hash_sm_off; p.hash_sm_bytes = c->fwd_hash_sm_bytes; p.inputs_ready = 1;
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
   p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;
   p.off_ids = l.off_ids; p.off_z = l.off_z; p.off_col = l.off_col; p.off_val = l.off_val; p.off_dedup = l.off_dedup;
@@ -1426,8 +1433,9 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
 }
 
 cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx, const float* vals,
-                                 const int32_t* label_ptr, const int32_t* labels) {
+                                 const int32_t* label_ptr, const int32_t* labels, int inputs_ready) {
   FwdParams p = make_params(c, batch, row_ptr, col_idx, vals, label_ptr, labels);
+  p.inputs_ready = inputs_ready;
   {
     LaunchScope ls(c, KID_FORWARD);
     // hidden layers of up to FWD_THREADS units take the variant with one unit per thread (less code, fewer registers)

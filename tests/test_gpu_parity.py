@@ -438,7 +438,8 @@ def test_full_size_670k_step_against_oracle():
     """One step at the headline shape (D 135,909, H 128, N 670,091, DWTA K=6 L=50, cap 128, batch 256)."""
     c = workloads.config("670k")
     pr = Pair(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"], L=c["L"], bucket_cap=c["bucket_cap"],
-              max_batch=c["batch"], max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0)
+              max_batch=c["batch"], max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0,
+              inputs_ready=1)                    # as the benchmark launches it: batches resident before the call
     try:
         assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_off"), pr.o.get("bucket_off"))
         assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_ids"), pr.o.get("bucket_ids"))
@@ -458,5 +459,60 @@ def test_full_size_670k_step_against_oracle():
         feats = np.unique(batch[1])
         W1g = ds.dslide_get_tensor(pr.ctx, "W1").reshape(pr.D, pr.H)
         assert max_rel_err(W1g[feats], pr.o.view("W1").reshape(pr.D, pr.H)[feats], 1e-2) < W_TOL
+    finally:
+        pr.close()
+
+
+# ------------------------------------------------------------------ batch arrays produced on the stream just before the step
+@pytest.mark.parametrize("inputs_ready_after_sync", [False, True])
+def test_batch_written_by_a_kernel_on_the_same_stream_right_before_the_step(inputs_ready_after_sync):
+    """The five batch arrays live in fixed device buffers that a copy kernel on the context's stream overwrites
+    immediately before every step (no synchronisation in between): the step must see the new batch, not the one
+    the buffers held before.  With inputs_ready = 1 the caller has to finish the producer first (here: a
+    synchronize), and the early-reading path must then give the same results."""
+    pr = mid_pair(inputs_ready=1 if inputs_ready_after_sync else 0)
+    try:
+        wl = workloads.Workload(workloads.config("mid"), seed=21)
+        batches = [wl.batch(i) for i in range(6)]
+        cap = [max(len(b[k]) for b in batches) for k in range(5)]
+        bufs = [torch.zeros(cap[k], dtype=torch.float32 if k == 2 else torch.int32, device="cuda") for k in range(5)]
+        staged = [to_dev(b) for b in batches]
+        torch.cuda.synchronize()
+        loss = torch.zeros(1, device="cuda")
+        for i, b in enumerate(batches):
+            B = len(b[0]) - 1
+            lo = pr.o.train_step(*b)
+            for k in range(5):
+                bufs[k][:len(b[k])].copy_(staged[i][k])          # a kernel on the same stream, just before the step
+            if inputs_ready_after_sync:
+                torch.cuda.synchronize()
+            ds.dslide_train_step(pr.ctx, B, *bufs, loss)
+            ds.dslide_sync(pr.ctx)
+            assert abs(float(loss.item()) - lo) <= 1e-3 * abs(lo)
+            sets_g, _ = pr.gpu_active_sets(B)
+            for s, ref in enumerate(pr.o.active_sets()):
+                assert np.array_equal(sets_g[s], ref), (i, s)
+    finally:
+        pr.close()
+
+
+def test_training_snapshot_is_whole_again_after_a_predict_call():
+    """A predict call borrows the per-sample work space; the next training step must rewrite all of it."""
+    pr = mid_pair()
+    try:
+        wl = workloads.Workload(workloads.config("mid"), seed=5)
+        b0, b1 = wl.batch(0), wl.batch(1)
+        pr.o.train_step(*b0)
+        pr.gpu_step(b0)
+        B = len(b1[0]) - 1
+        dev = to_dev(b1)
+        out_ids = torch.zeros(B * 4, dtype=torch.int32, device="cuda")
+        out_sc = torch.zeros(B * 4, dtype=torch.float32, device="cuda")
+        for dense in (0, 1):
+            ds.dslide_predict_topk(pr.ctx, B, dev[0], dev[1], dev[2], 4, dense, out_ids, out_sc)
+        ds.dslide_sync(pr.ctx)
+        pr.o.train_step(*b1)
+        pr.gpu_step(b1)
+        compare_forward(pr, b1, bit_exact_hidden=False, tol=1e-3)     # second step: each side on its own weights
     finally:
         pr.close()

@@ -70,3 +70,31 @@ def test_static_sort_rejects_sizes_beyond_its_static_array():
     ds.dslide_bucket_sort_static(codes, 8, 1, off, ids)           # still usable; all codes 0 -> one bucket
     torch.cuda.synchronize()
     assert off.cpu().tolist() == [0, 8, 8] and ids.cpu().tolist() == list(range(8))
+
+
+def reference_sort(codes, bits):
+    """An independent statement of the result: stable order of the ids by code, bucket starts by counting."""
+    ids = np.argsort(codes, kind="stable").astype(np.int32)
+    off = np.zeros((1 << bits) + 1, dtype=np.int32)
+    off[1:] = np.cumsum(np.bincount(codes, minlength=1 << bits))
+    return off, ids
+
+
+@pytest.mark.parametrize("n,bits", [(0, 5),                                 # nothing to sort: offsets all zero
+                                    (ds.STATIC_SORT_MAX_N if torch.cuda.is_available() else 262144, 18),   # the whole static array, to its last byte
+                                    (40001, 10), (40001, 13), (40001, 17),  # second pass narrower than the first
+                                    (1, 1), (513, 9)])
+def test_static_sort_against_a_stable_argsort(n, bits):
+    rng = np.random.default_rng(1000 * bits + n % 997)
+    codes = rng.integers(0, 1 << bits, size=n, dtype=np.int64).astype(np.uint32)
+    # high garbage bits above `bits` must be ignored
+    dirty = (codes | (rng.integers(0, 1 << (31 - bits), size=n, dtype=np.int64).astype(np.uint32) << np.uint32(bits))) if bits < 31 else codes
+    want_off, want_ids = reference_sort(codes.astype(np.int64), bits)
+    d_codes = torch.from_numpy(dirty.astype(np.int64).astype(np.int32) if n else np.zeros(1, dtype=np.int32)).cuda()
+    out_off = torch.full(((1 << bits) + 1,), -7, dtype=torch.int32, device="cuda")
+    out_ids = torch.full((max(n, 1),), -7, dtype=torch.int32, device="cuda")
+    for rep in range(2):
+        ds.dslide_bucket_sort_static(d_codes, n, bits, out_off, out_ids)
+        torch.cuda.synchronize()
+        assert np.array_equal(out_off.cpu().numpy(), want_off)
+        assert np.array_equal(out_ids.cpu().numpy()[:n], want_ids)
