@@ -20,18 +20,20 @@ _CFLAGS = ["-O2", "-ffp-contract=off", "-fPIC", "-shared", "-std=c99", "-fno-fas
 
 
 def lib_path(real):
-    return os.path.join(_HERE, "libslide_oracle_%s.so" % ("f32" if real == "float" else "f64"))
+    return os.path.join(_HERE, "libslide_oracle_%s.so" % {"float": "f32", "double": "f64", "float_omp": "f32_omp"}[real])
 
 
 def build(force=False):
-    """Compile both variants of the oracle with gcc (a few seconds)."""
-    for real in ("float", "double"):
+    """Compile the variants of the oracle with gcc (a few seconds): fp32, fp64, and fp32 with OpenMP (the same
+    source; only used to time the oracle on all host cores, and pinned bit-identical to the plain fp32 build)."""
+    for real in ("float", "double", "float_omp"):
         out = lib_path(real)
         if (not force and os.path.exists(out)
                 and os.path.getmtime(out) >= os.path.getmtime(_SRC)):
             continue
         tmp = out + ".tmp%d" % os.getpid()
-        subprocess.check_call(["gcc"] + _CFLAGS + ["-DREAL=%s" % real, _SRC, "-o", tmp, "-lm"])
+        extra = ["-fopenmp"] if real.endswith("_omp") else []
+        subprocess.check_call(["gcc"] + _CFLAGS + extra + ["-DREAL=%s" % real.split("_")[0], _SRC, "-o", tmp, "-lm"])
         os.replace(tmp, out)
 
 
@@ -82,6 +84,8 @@ def _load(real):
             getattr(lib, f).argtypes = [C.c_void_p]
         lib.orc_rng.restype = C.c_uint64
         lib.orc_rng.argtypes = [C.c_uint64] * 4
+        lib.orc_threads.restype = C.c_int32
+        lib.orc_threads.argtypes = []
         lib.orc_mix64.restype = C.c_uint64
         lib.orc_mix64.argtypes = [C.c_uint64]
         lib.orc_draw_hash.argtypes = [C.c_void_p, C.c_int64]
@@ -118,11 +122,11 @@ def _p(a):
 
 
 class Oracle:
-    """One model instance of the CPU oracle.  `real` is "float" or "double"."""
+    """One model instance of the CPU oracle.  `real` is "float", "double" or "float_omp" (fp32 on all cores)."""
 
     def __init__(self, real="float", **kw):
         self.real = real
-        self.dtype = np.float32 if real == "float" else np.float64
+        self.dtype = np.float64 if real == "double" else np.float32
         self.lib = _load(real)
         d = dict(family=SIMHASH, bin_size=8, srp_nnz=0, bucket_cap=128, rebuild_period0=0, redraw=1,
                  force_dense=0, max_active=0, densify=0, budget=0, budget_fill=0, rebuild_lambda=0.0, lr=1e-4, beta1=0.9, beta2=0.999,
@@ -133,6 +137,11 @@ class Oracle:
         if not self.o:
             raise MemoryError("orc_create failed")
         self.H, self.N, self.D, self.L, self.K = d["H"], d["N"], d["D"], d["L"], d["K"]
+
+    @property
+    def threads(self):
+        """Worker threads the library uses (1 unless it is the OpenMP build)."""
+        return int(self.lib.orc_threads())
 
     def close(self):
         if self.o:

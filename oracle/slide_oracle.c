@@ -11,7 +11,11 @@
  * benchmark may call it; the product never does.
  *
  * Every function follows the order of the paper's algorithm and does no
- * blocking, fusion or reordering.  The scalar type REAL is chosen at
+ * blocking, fusion or reordering.  The loops over samples, over neurons and
+ * over touched rows carry OpenMP pragmas that only a second build
+ * (-fopenmp, used to time the oracle on all host cores) honours; each
+ * accumulator still receives the same addends in the same order, so that
+ * build is bit-identical to the plain one (pinned in tests).  The scalar type REAL is chosen at
  * compile time: float (the parity target: the paper's networks are fp32
  * and hash codes depend on the exact fp32 hidden activation) or double
  * (used by the gradient and dense-limit pins).
@@ -25,6 +29,25 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* Which of nthreads workers this one is (0 of 1 in the plain build). */
+static void who_am_i(int *tid, int *nthreads) {
+#ifdef _OPENMP
+  *tid = omp_get_thread_num(); *nthreads = omp_get_num_threads();
+#else
+  *tid = 0; *nthreads = 1;
+#endif
+}
+int32_t orc_threads(void) {
+#ifdef _OPENMP
+  return (int32_t)omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
 
 #ifndef REAL
 #define REAL float
@@ -118,6 +141,7 @@ static double u01(uint64_t x) { return ((double)(x >> 11) + 0.5) * (1.0 / 900719
  * reading: N(0, init_std^2) by Box-Muller over two counter-based uniforms;
  * biases and Adam moments start at zero. */
 static void init_gauss(REAL *w, int64_t n, uint64_t seed, uint64_t stream, double std) {
+#pragma omp parallel for schedule(static)
   for (int64_t i = 0; i < n; ++i) {
     double u1 = u01(orc_rng(seed, stream, 0, 2 * (uint64_t)i));
     double u2 = u01(orc_rng(seed, stream, 0, 2 * (uint64_t)i + 1));
@@ -254,9 +278,11 @@ void orc_build_tables(orc *o) {
   const orc_config *c = &o->c;
   int64_t nb = (int64_t)1 << o->bits;
   uint32_t *codes = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)c->N * (size_t)c->L);
+#pragma omp parallel for schedule(static)
   for (int j = 0; j < c->N; ++j) orc_hash_vec(o, o->W2 + (size_t)j * c->H, codes + (size_t)j * c->L);
-  int32_t *cursor = (int32_t *)malloc(sizeof(int32_t) * (size_t)nb);
+#pragma omp parallel for schedule(dynamic, 1)
   for (int t = 0; t < c->L; ++t) {
+    int32_t *cursor = (int32_t *)malloc(sizeof(int32_t) * (size_t)nb);
     int32_t *off = o->bucket_off + (size_t)t * (size_t)(nb + 1);
     int32_t *ids = o->bucket_ids + (size_t)t * (size_t)c->N;
     memset(off, 0, sizeof(int32_t) * (size_t)(nb + 1));
@@ -264,8 +290,8 @@ void orc_build_tables(orc *o) {
     for (int64_t b = 0; b < nb; ++b) off[b + 1] += off[b];
     for (int64_t b = 0; b < nb; ++b) cursor[b] = off[b];
     for (int j = 0; j < c->N; ++j) ids[cursor[codes[(size_t)j * c->L + t]]++] = j;
+    free(cursor);
   }
-  free(cursor);
   free(codes);
 }
 
@@ -501,8 +527,10 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
   for (int64_t i = 0; i < nlab; ++i)
     if (labels[i] < 0 || labels[i] >= c->N) { o->error = 5; return o->error; }
 
-  int32_t *buf = NULL; int64_t bufcap = 0;
-  o->act_ptr[0] = 0;
+  /* first loop over the samples: hidden activation, codes, active set (kept per sample) */
+  int32_t **sel = (int32_t **)calloc((size_t)B, sizeof(int32_t *));
+  int64_t *na_of = (int64_t *)calloc((size_t)B, sizeof(int64_t));
+#pragma omp parallel for schedule(dynamic, 1)
   for (int32_t s = 0; s < B; ++s) {
     REAL *h = o->h + (size_t)s * H;
     hidden_layer(o, row_ptr[s + 1] - row_ptr[s], col_idx + row_ptr[s], vals + row_ptr[s], h);
@@ -510,11 +538,30 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
     orc_hash_query(o, h, codes);
     const int32_t *lab = label_ptr ? labels + label_ptr[s] : NULL;
     int32_t nl = label_ptr ? label_ptr[s + 1] - label_ptr[s] : 0;
-    int64_t na = select_active(o, codes, lab, nl, &buf, &bufcap, s);
-    if (c->max_active > 0 && na > c->max_active) { o->error = 4; free(buf); return o->error; }
-    int64_t base = o->act_ptr[s];
-    ensure_act(o, base + na);
-    o->act_ptr[s + 1] = base + na;
+    int32_t *buf = NULL; int64_t bufcap = 0;
+    na_of[s] = select_active(o, codes, lab, nl, &buf, &bufcap, s);
+    sel[s] = buf;
+  }
+  /* where each sample's entries go in the snapshot arrays */
+  o->act_ptr[0] = 0;
+  for (int32_t s = 0; s < B; ++s) {
+    if (c->max_active > 0 && na_of[s] > c->max_active) o->error = 4;
+    o->act_ptr[s + 1] = o->act_ptr[s] + na_of[s];
+  }
+  if (o->error) {
+    for (int32_t s = 0; s < B; ++s) free(sel[s]);
+    free(sel); free(na_of);
+    return o->error;
+  }
+  ensure_act(o, o->act_ptr[B]);
+  /* second loop over the samples: activations of the active neurons, softmax, errors */
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int32_t s = 0; s < B; ++s) {
+    const REAL *h = o->h + (size_t)s * H;
+    const int32_t *buf = sel[s];
+    const int32_t *lab = label_ptr ? labels + label_ptr[s] : NULL;
+    int32_t nl = label_ptr ? label_ptr[s + 1] - label_ptr[s] : 0;
+    int64_t base = o->act_ptr[s], na = na_of[s];
     memcpy(o->act_ids + base, buf, sizeof(int32_t) * (size_t)na);
 
     /* feed forward of the second type over the active neurons only (Section 3.6) */
@@ -552,7 +599,8 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
     }
     for (int64_t a = 0; a < na; ++a) g[a] = g[a] / (REAL)B;
   }
-  free(buf);
+  for (int32_t s = 0; s < B; ++s) free(sel[s]);
+  free(sel); free(na_of);
   return 0;
 }
 
@@ -562,6 +610,8 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
 void orc_backward(orc *o) {
   const orc_config *c = &o->c;
   int H = c->H;
+  /* error at the hidden layer, sample by sample */
+#pragma omp parallel for schedule(dynamic, 1)
   for (int32_t s = 0; s < o->B; ++s) {
     const REAL *h = o->h + (size_t)s * H;
     REAL *dh = o->dh + (size_t)s * H;
@@ -570,18 +620,34 @@ void orc_backward(orc *o) {
       int32_t j = o->act_ids[a];
       REAL g = o->act_g[a];
       for (int k = 0; k < H; ++k) dh[k] += g * o->W2[(size_t)j * H + k];
-      for (int k = 0; k < H; ++k) o->dW2[(size_t)j * H + k] += g * h[k];
-      o->db2[j] += g;
-      o->touch2[j] = 1;
     }
     for (int k = 0; k < H; ++k) if (!(h[k] > 0)) dh[k] = 0;   /* ReLU derivative */
-    for (int32_t i = o->row_ptr[s]; i < o->row_ptr[s + 1]; ++i) {
-      int32_t f = o->col_idx[i];
-      REAL x = o->vals[i];
-      for (int k = 0; k < H; ++k) o->dW1[(size_t)f * H + k] += x * dh[k];
-      o->touch1[f] = 1;
+  }
+  /* gradients of the rows, samples in ascending order; a worker adds only into the rows it owns */
+#pragma omp parallel
+  {
+    int tid, nt;
+    who_am_i(&tid, &nt);
+    for (int32_t s = 0; s < o->B; ++s) {
+      const REAL *h = o->h + (size_t)s * H;
+      const REAL *dh = o->dh + (size_t)s * H;
+      for (int64_t a = o->act_ptr[s]; a < o->act_ptr[s + 1]; ++a) {
+        int32_t j = o->act_ids[a];
+        if (j % nt != tid) continue;
+        REAL g = o->act_g[a];
+        for (int k = 0; k < H; ++k) o->dW2[(size_t)j * H + k] += g * h[k];
+        o->db2[j] += g;
+        o->touch2[j] = 1;
+      }
+      for (int32_t i = o->row_ptr[s]; i < o->row_ptr[s + 1]; ++i) {
+        int32_t f = o->col_idx[i];
+        if (f % nt != tid) continue;
+        REAL x = o->vals[i];
+        for (int k = 0; k < H; ++k) o->dW1[(size_t)f * H + k] += x * dh[k];
+        o->touch1[f] = 1;
+      }
+      for (int k = tid; k < H; k += nt) o->db1[k] += dh[k];
     }
-    for (int k = 0; k < H; ++k) o->db1[k] += dh[k];
   }
 }
 
@@ -604,6 +670,7 @@ void orc_adam(orc *o) {
   o->t += 1;
   REAL bc1 = (REAL)(1.0 - pow(c->beta1, (double)o->t));
   REAL bc2 = (REAL)(1.0 - pow(c->beta2, (double)o->t));
+#pragma omp parallel for schedule(static)
   for (int j = 0; j < c->N; ++j) {
     if (!o->touch2[j]) continue;
     for (int k = 0; k < H; ++k) {
@@ -615,6 +682,7 @@ void orc_adam(orc *o) {
     o->db2[j] = 0;
     o->touch2[j] = 0;
   }
+#pragma omp parallel for schedule(static)
   for (int f = 0; f < c->D; ++f) {
     if (!o->touch1[f]) continue;
     for (int k = 0; k < H; ++k) {

@@ -387,3 +387,29 @@ def test_fp32_rounding_alone_moves_weights_by_the_floor_the_gpu_bar_uses():
     finally:
         a.close()
         b.close()
+
+
+# ---------------------------------------------------------------- the all-cores build is the same oracle
+def test_openmp_build_is_bit_identical_to_the_plain_build():
+    """The build that times the oracle on all host cores runs the same source with its loops over samples, neurons
+    and touched rows shared out between threads; every accumulator receives the same addends in the same order, so
+    tables, snapshots and weights must be identical bit for bit."""
+    from paper_2201_12667_b200 import workloads
+    c = workloads.config("mid")
+    kw = dict(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"], L=c["L"], bucket_cap=c["bucket_cap"],
+              lr=c["lr"], init_std=0.05, seed=4, rebuild_period0=2)
+    a, b = Oracle("float", **kw), Oracle("float_omp", **kw)
+    try:
+        assert a.threads == 1 and b.threads >= 1
+        wl = workloads.Workload(c, seed=4)
+        for i in range(3):                       # a scheduled rebuild falls after the second step
+            bt = wl.batch(i)
+            la, lb = a.train_step(*bt), b.train_step(*bt)
+            assert la == lb
+            for n in ("h", "dh", "codes", "act_ptr", "act_ids", "act_z", "act_p", "act_g", "loss"):
+                assert np.array_equal(a.get(n), b.get(n)), (i, n)
+        for n in ("W1", "b1", "W2", "b2", "mW1", "vW1", "mW2", "vW2", "mb2", "vb2", "bucket_off", "bucket_ids", "hash_idx"):
+            assert np.array_equal(a.get(n), b.get(n)), n
+    finally:
+        a.close()
+        b.close()
