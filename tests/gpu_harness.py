@@ -19,8 +19,8 @@ class Pair:
     def __init__(self, D, H, N, family, K, L, bucket_cap, max_batch, bin_size=8, srp_nnz=0, max_labels=16,
                  rebuild_period0=0, rebuild_lambda=0.0, redraw=1, force_dense=0, max_active=0, lr=1e-3,
                  init_std=0.05, seed=0, dedup_mode=0, sync_weights=True, densify=0, budget=0, budget_fill=0,
-                 inputs_ready=0):
-        self.o = Oracle("float", D=D, H=H, N=N, family=family, K=K, L=L, bin_size=bin_size, srp_nnz=srp_nnz,
+                 inputs_ready=0, oracle_build="float"):
+        self.o = Oracle(oracle_build, D=D, H=H, N=N, family=family, K=K, L=L, bin_size=bin_size, srp_nnz=srp_nnz,
                         bucket_cap=bucket_cap, rebuild_period0=rebuild_period0, rebuild_lambda=rebuild_lambda,
                         redraw=redraw, force_dense=force_dense, max_active=max_active, lr=lr, init_std=init_std,
                         seed=seed, densify=densify, budget=budget, budget_fill=budget_fill)

@@ -84,3 +84,27 @@ def test_reference_arm_prints_one_json_line_and_only_on_rank_zero():
     env1 = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
     out1 = subprocess.run(cmd, env=env1, capture_output=True, text=True, timeout=600)
     assert out1.returncode == 0 and out1.stdout.strip() == ""
+
+
+def test_full_step_accounting_never_drops_or_doubles_the_rebuild():
+    # 500 steps at period 50 with the 10 scheduled rebuilds inside: as measured
+    ms, how = bench.full_step_ms(40.0, 500, 10, 0.9, 50)
+    assert ms == pytest.approx(0.08) and how.startswith("as measured")
+    # 20 steps without any rebuild inside: one rebuild per 50 steps is added
+    ms, how = bench.full_step_ms(1.2, 20, 0, 0.9, 50)
+    assert ms == pytest.approx(1.2 / 20 + 0.9 / 50) and "added per 50 steps" in how
+    # 30 steps that happen to hold one rebuild (1 per 30 > 1 per 50): taken out, then charged at 1 per 50
+    ms, _ = bench.full_step_ms(30 * 0.06 + 0.9, 30, 1, 0.9, 50)
+    assert ms == pytest.approx(0.06 + 0.9 / 50)
+    # no schedule
+    assert bench.full_step_ms(2.0, 20, 0, 0.0, 0)[0] == pytest.approx(0.1)
+
+
+def test_sweep_grid_covers_the_batch_and_fraction_axes():
+    assert bench.SWEEP_BATCHES == (64, 128, 256, 512, 1024, 2048)
+    fr = [f for f, _ in bench.SWEEP_FRACTIONS]
+    assert fr[0] == 0.0005 and fr[-1] == 1.0 and bench.SWEEP_FRACTIONS[-1][1] == dict(force_dense=1)
+    N = workloads.config("670k")["N"]
+    for f, over in bench.SWEEP_FRACTIONS[:-1]:
+        per_bucket = min(over["bucket_cap"], N / 8 ** over["K"])
+        assert 0.6 * f * N <= over["L"] * per_bucket <= 1.7 * f * N      # duplicates shrink the union of large buckets

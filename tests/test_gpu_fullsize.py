@@ -1,0 +1,75 @@
+"""GPU-vs-oracle parity at the full size of the larger benchmark shapes, in the launch configuration bench.py times
+(batches resident before the call).  The oracle runs in its all-cores build, which is pinned bit-identical to the
+plain one; both shapes reach kernel paths the small cases only imitate:
+
+  325K-class  SimHash K=9: 512 buckets of ~635 ids per table, capped at 128 -> ~6,100 active neurons per sample,
+              active rows streamed through shared memory in ~32 chunks, dedup through the N-bit bitmap, rows of W2
+              shared by ~15 samples each (listed and hot rows in the update), one 9-bit radix pass in the table build.
+  ~1B         N = 4,000,000 > 2^22 (sort keys cannot be packed with their position), 21-bit codes (place-then-order
+              table build over 2 M buckets per table), hidden width 256 (two 16-byte chunks per lane), the N-bit
+              bitmap does not fit shared memory, batch 512.
+"""
+import numpy as np
+import pytest
+import torch
+
+from tests.helpers import max_rel_err
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2201_12667_b200 import binding as ds
+    from paper_2201_12667_b200 import workloads
+    from tests.gpu_harness import Pair
+    from tests.test_gpu_parity import ACT_TOL, W_TOL, compare_forward
+
+
+def full_size_step(name, sample_rows_every):
+    c = workloads.config(name)
+    pr = Pair(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"], L=c["L"], bucket_cap=c["bucket_cap"],
+              max_batch=c["batch"], max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0, inputs_ready=1,
+              oracle_build="float_omp")
+    try:
+        assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_off"), pr.o.view("bucket_off"))
+        assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_ids"), pr.o.view("bucket_ids"))
+        wl = workloads.Workload(c, seed=0)
+        batch = wl.batch(0)
+        lo = pr.o.train_step(*batch)
+        lg = pr.gpu_step(batch)
+        assert abs(lo - lg) <= ACT_TOL * abs(lo)
+        compare_forward(pr, batch)                 # hidden layer, codes and active sets bit-exact; activations at 1e-4
+        sizes = np.diff(pr.o.get("act_ptr"))
+        act = np.unique(pr.o.get("act_ids"))
+        W2g = ds.dslide_get_tensor(pr.ctx, "W2").reshape(pr.N, pr.H)
+        W2o = pr.o.view("W2").reshape(pr.N, pr.H)
+        assert max_rel_err(W2g[act], W2o[act], 1e-2) < W_TOL
+        b2g, b2o = ds.dslide_get_tensor(pr.ctx, "b2"), pr.o.view("b2")
+        assert max_rel_err(b2g[act], b2o[act], 1e-2) < W_TOL
+        rest = np.setdiff1d(np.arange(0, pr.N, sample_rows_every), act)
+        assert np.array_equal(W2g[rest].view(np.uint32), W2o[rest].view(np.uint32))      # untouched rows: bit-identical
+        del W2g
+        feats = np.unique(batch[1])
+        W1g = ds.dslide_get_tensor(pr.ctx, "W1").reshape(pr.D, pr.H)
+        W1o = pr.o.view("W1").reshape(pr.D, pr.H)
+        assert max_rel_err(W1g[feats], W1o[feats], 1e-2) < W_TOL
+        other = np.setdiff1d(np.arange(0, pr.D, sample_rows_every), feats)
+        assert np.array_equal(W1g[other].view(np.uint32), W1o[other].view(np.uint32))
+        for n in ("mW2", "vW2"):
+            g = ds.dslide_get_tensor(pr.ctx, n).reshape(pr.N, pr.H)
+            assert max_rel_err(g[act], pr.o.view(n).reshape(pr.N, pr.H)[act], 1e-2) < W_TOL, n
+            del g
+        assert max_rel_err(ds.dslide_get_tensor(pr.ctx, "b1"), pr.o.view("b1"), 1e-2) < W_TOL
+        return sizes, len(act)
+    finally:
+        pr.close()
+
+
+def test_full_size_325k_step_against_oracle():
+    sizes, distinct = full_size_step("325k", 89)
+    assert sizes.mean() > 3000               # the large-active-set regime: thousands of neurons per sample
+    assert sizes.sum() > 5 * distinct        # every touched row of W2 is shared by several samples
+
+
+def test_full_size_1b_step_against_oracle():
+    sizes, distinct = full_size_step("1b", 997)
+    assert 20 < sizes.mean() < 2000 and distinct > 2 ** 14
