@@ -77,6 +77,11 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// 16-byte asynchronous copy global -> shared (through L2 only), and the wait for all of a thread's copies
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -114,31 +119,57 @@ __device__ __forceinline__ void list_row(const FwdParams& p, uint32_t* cnt, int 
   }
 }
 
-// Second half of handing a touched row to the update kernel, once the row's touch counter has answered
-// (nth = touches before this one): the (sample, coefficient) pair goes into the row's slot nth, or, past the
-// slots, the sample's bit into the row's mask; the first toucher enters (row, its own sample) in the list of
-// distinct rows (positions handed out per warp), so that the update kernel can fetch that sample's row at once.  Called by whole warps; `live` tells whether this thread has a touch.
+// Handing a touched row to the update kernel, once the row's touch counter has answered (nth = touches before this
+// one).  touch_mark: the (sample, coefficient) pair goes into the row's slot nth, or, past the slots, the sample's bit
+// into the row's mask (and, up to PAIR_T touches, the pair into the side array); the touch that fills the slots or
+// reaches HOT_T lists the row (list_row: an atomic whose answer is needed, so callers on the critical path put it
+// off to the end of the kernel).  own_reserve / own_store: the first toucher enters (row, its own sample) in the list
+// of distinct rows, so that the update kernel can fetch that sample's row at once; positions are handed out per
+// warp by one atomic, asked for by own_reserve and used by own_store (callers put other work in between, so that
+// no warp waits for the answer).  All three are called by whole warps; `live` tells whether this thread has a touch.
+template <bool LIST = true>      // LIST = false: the caller lists the row (list_row) itself, later
+__device__ __forceinline__ void touch_mark(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int2* ovfrow, int code,
+                                           unsigned nth, int s, float coef) {
+  if (!live) return;
+  if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(coef));
+  else {
+    atomicOr(maskrow + (s >> 5), 1u << (s & 31));
+    // up to PAIR_T touches keep their pair as well, so that a row with that many is summed without any search
+    if (nth < (unsigned)PAIR_T) ovfrow[nth] = make_int2(s, __float_as_int(coef));
+  }
+  if (LIST) list_row(p, &hd->cnt, code, nth);
+}
+__device__ __forceinline__ unsigned own_reserve(bool first, unsigned int* n_own) {
+  const unsigned fm = __ballot_sync(FULLM, first);
+  unsigned base = 0;
+  if (fm && (threadIdx.x & 31) == 0) base = atomicAdd(n_own, (unsigned)__popc(fm));
+  return base;                                   // valid in lane 0
+}
+__device__ __forceinline__ void own_store(bool first, unsigned base, int2* own, int row, int s) {
+  const int lane = threadIdx.x & 31;
+  const unsigned fm = __ballot_sync(FULLM, first);
+  if (!fm) return;
+  base = __shfl_sync(FULLM, base, 0);
+  if (first) own[base + __popc(fm & ((1u << lane) - 1u))] = make_int2(row, s);
+}
 __device__ __forceinline__ void finish_touch(const FwdParams& p, bool live, RowHdr* hd, uint32_t* maskrow, int2* ovfrow, int2* own,
                                              unsigned int* n_own, int row, int code, unsigned nth, int s, float coef) {
-  const int lane = threadIdx.x & 31;
-  bool first = false;
-  if (live) {
-    if (nth < (unsigned)ROW_SLOTS) hd->slot[nth] = make_int2(s, __float_as_int(coef));
-    else {
-      atomicOr(maskrow + (s >> 5), 1u << (s & 31));
-      // up to PAIR_T touches keep their pair as well, so that a row with that many is summed without any search
-      if (nth < (unsigned)PAIR_T) ovfrow[nth] = make_int2(s, __float_as_int(coef));
-    }
-    first = nth == 0u;
-    list_row(p, &hd->cnt, code, nth);
-  }
-  const unsigned fm = __ballot_sync(FULLM, first);
-  if (fm) {
-    unsigned base = 0;
-    if (lane == 0) base = atomicAdd(n_own, (unsigned)__popc(fm));
-    base = __shfl_sync(FULLM, base, 0);
-    if (first) own[base + __popc(fm & ((1u << lane) - 1u))] = make_int2(row, s);
-  }
+  touch_mark(p, live, hd, maskrow, ovfrow, code, nth, s, coef);
+  const bool first = live && nth == 0u;
+  const unsigned base = own_reserve(first, n_own);
+  own_store(first, base, own, row, s);
+}
+
+// Maximum / sum over the lanes of a warp in a fixed order (same value in every lane).
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(FULLM, v, d));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(FULLM, v, d);
+  return v;
 }
 
 // Exclusive prefix sum of one int per thread over the block; *total gets the block sum.
@@ -431,6 +462,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   int* sh_tbeg = reinterpret_cast<int*>(smem + p.off_tbeg);          // [L]
   int* sh_ids = reinterpret_cast<int*>(smem + p.off_ids);            // [ACT_SM]
   float* sh_z = reinterpret_cast<float*>(smem + p.off_z);            // [ACT_SM]
+  float* sh_g = reinterpret_cast<float*>(smem + p.off_topk);         // [ACT_SM] training: errors of a small set (predict: its best-k lists)
   int* sh_col = reinterpret_cast<int*>(smem + p.off_col);            // [hid_rows]
   float* sh_val = reinterpret_cast<float*>(smem + p.off_val);        // [hid_rows]
   uint32_t* sh_dd = reinterpret_cast<uint32_t*>(smem + p.off_dedup);
@@ -466,7 +498,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
   }
 
-  // ---- label checks: ids in range, list within the maximum ----
+  // ---- label checks: ids in range, list within the maximum (merged with the column checks by the first barrier) ----
   int bad = 0;
   if (nnz < 0 || nlab < 0) bad = DSLIDE_ERR_BAD_INDEX;
   else if (MODE == 0) {
@@ -476,18 +508,21 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     }
   }
   const bool too_many_labels = MODE == 0 && nnz >= 0 && nlab > p.max_labels;
-  bad = __syncthreads_or(bad);
 
   // ---- hidden layer: bias, then one fused multiply-add per nonzero in stored order, ReLU.  The rows of W1 of a
-  //      chunk of nonzeros are fetched together into shared memory; the column ids are checked on the way
-  //      (in range, ascending) ----
+  //      chunk of nonzeros are copied into shared memory together, 16 bytes per thread and copy (cp.async: all of
+  //      them in flight at once, no registers held), and then summed per hidden unit in the stored order; the
+  //      column ids are checked on the way (in range, ascending) ----
   //      Up to here, and through the first chunk's column ids and values, only the caller's batch is read: with
   //      inputs_ready the kernel runs that far while the previous step's update kernel is still finishing.
   float acc[KPT];
-  uint32_t phase = 0;                // of sh_bar, which serves the staging of W1 rows here and of W2 rows below
-  bool timed_out = false;
+  int c1 = 0, line1 = -1;            // this thread's nonzero (tid-th of the sample), kept for the hand-off to the update kernel
+  float x1 = 0.f;
   const int R = p.hid_rows;
-  for (int c0 = 0; c0 < nnz && !bad; c0 += R) {       // `bad` is uniform over the block here
+  // a thread's place in the copy pattern: 16-byte piece c4 of row r, advancing FWD_THREADS pieces per round
+  const int cp_dr = FWD_THREADS / H4, cp_dc = FWD_THREADS - cp_dr * H4;
+  const int cp_r0 = tid / H4, cp_c0 = tid - cp_r0 * H4;
+  for (int c0 = 0; c0 < nnz; c0 += R) {
     const int nr = min(R, nnz - c0);
     for (int i = tid; i < nr; i += FWD_THREADS) {
       const int c = __ldg(p.col_idx + rbeg + c0 + i);
@@ -495,19 +530,23 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       const bool okc = c >= 0 && c < p.D && prev < c;
       if (!okc) bad = DSLIDE_ERR_BAD_INDEX;
       sh_col[i] = okc ? c : 0;
-      sh_val[i] = __ldg(p.vals + rbeg + c0 + i);
+      const float xv = __ldg(p.vals + rbeg + c0 + i);
+      sh_val[i] = xv;
+      if (c0 + i == tid) { c1 = okc ? c : 0; x1 = xv; }
     }
-    if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * (uint32_t)H * 4u);
-    fence_proxy_async();             // the staging space was read through ordinary loads (the previous chunk)
-    bad = __syncthreads_or(bad);
-    if (bad) break;                  // nothing was copied; the barrier is not used again
+    bad = __syncthreads_or(bad);     // also: the previous chunk's readers of the staging space are done
+    if (bad) break;                  // nothing was copied
     if (!waited) {
       griddep_wait();
       waited = true;
     }
-    // one bulk copy per row of W1: every row of the chunk is in flight at once
-    for (int i = tid; i < nr; i += FWD_THREADS)
-      bulk_g2s(stage + (size_t)i * H, p.W1 + (size_t)sh_col[i] * H, (uint32_t)H * 4u, sh_bar);
+    // a feature that has been hot before has a line of the coefficient table (written by the update kernel)
+    if (MODE == 0 && c0 == 0 && tid < nr) line1 = __ldcg(p.hotmap1 + c1);
+    for (int r = cp_r0, c4 = cp_c0; r < nr;) {
+      cp_async16(stage + (size_t)r * H + 4 * c4, p.W1 + (size_t)sh_col[r] * H + 4 * c4);
+      c4 += cp_dc; r += cp_dr;
+      if (c4 >= H4) { c4 -= H4; ++r; }
+    }
     if (c0 == 0) {
 #pragma unroll
       for (int u = 0; u < KPT; ++u) {
@@ -515,20 +554,21 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         acc[u] = k < H ? p.b1[k] : 0.f;
       }
     }
-    if (!mbar_wait(sh_bar, phase)) timed_out = true;
-    phase ^= 1u;
-    if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
+    cp_async_wait_all();
+    __syncthreads();
 #pragma unroll
     for (int u = 0; u < KPT; ++u) {
       const int k = tid + u * FWD_THREADS;
       if (k < H) {
         float a = acc[u];
+#pragma unroll 8
         for (int i = 0; i < nr; ++i) a = __fmaf_rn(sh_val[i], stage[(size_t)i * H + k], a);
         acc[u] = a;
       }
     }
-    __syncthreads();
+    if (c0 + R < nnz) __syncthreads();       // the next chunk overwrites the column ids and values
   }
+  if (nnz <= 0) bad = __syncthreads_or(bad);       // no chunk, no barrier yet: the label checks are merged here
   if (!waited) {                     // no nonzeros, or a bad column id: nothing of the model has been read yet
     griddep_wait();
 #pragma unroll
@@ -536,13 +576,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       const int k = tid + u * FWD_THREADS;
       acc[u] = k < H ? p.b1[k] : 0.f;
     }
-  }
-  if (timed_out) {                   // a row of W1 did not arrive in time: one more bounded wait, then the sample is given up
-    mbar_wait(sh_bar, phase ^ 1u);
-    if (p.hash_sm_off >= 0 && !p.dense) mbar_wait(sh_bar2, 0u);
-    __syncthreads();
-    skip_sample<MODE>(p, s, DSLIDE_ERR_TIMEOUT);
-    return;
   }
   if (bad || too_many_labels) {
     if (p.hash_sm_off >= 0 && !p.dense) mbar_wait(sh_bar2, 0u);     // no copy into this block may be left in flight
@@ -620,7 +653,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     __syncthreads();
     // ---- codes, and the slice of every table's bucket the sample reads: all offsets in one round ----
     const int shift = p.family == DSLIDE_SIMHASH ? 1 : p.lg_bin;
-    for (int t = tid; t < p.L; t += FWD_THREADS) {
+    auto table_code = [&](int t) -> uint32_t {
       uint32_t code = 0;
       for (int k = 0; k < p.K; ++k) {
         const int f = t * p.K + k;
@@ -636,33 +669,75 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         }
         code |= pos << (k * shift);
       }
-      sh_code[t] = code;
-      if (MODE == 0) p.codes[(size_t)s * p.L + t] = code;
-      const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1) + code;
-      const int beg = __ldg(off);
-      int cnt = __ldg(off + 1) - beg;
-      cnt = cnt < p.cap ? cnt : p.cap;
-      sh_tbeg[t] = beg;
-      sh_tbase[t + 1] = cnt;
-    }
-    __syncthreads();
-    if (warp == 0) {            // running sum of the slice lengths: where each table's candidates start
-      int run = 0;
-      for (int b = 0; b < p.L; b += 32) {
-        const int t = b + lane;
-        const int v = t < p.L ? sh_tbase[t + 1] : 0;
-        int incl = v;
+      return code;
+    };
+    if (p.L <= 64) {
+      // up to 64 tables: one warp fetches all the offsets (two tables per lane) and takes the running sum of the
+      // slice lengths in registers -- one barrier instead of two
+      if (warp == 0) {
+        int beg[2], cnt[2];
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          int n = __shfl_up_sync(FULLM, incl, d);
-          if (lane >= d) incl += n;
+        for (int u = 0; u < 2; ++u) {
+          const int t = lane + 32 * u;
+          beg[u] = 0; cnt[u] = 0;
+          if (t < p.L) {
+            const uint32_t code = table_code(t);
+            sh_code[t] = code;
+            if (MODE == 0) p.codes[(size_t)s * p.L + t] = code;
+            const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1) + code;
+            beg[u] = __ldg(off);
+            cnt[u] = __ldg(off + 1);
+          }
         }
-        if (t < p.L) sh_tbase[t + 1] = run + incl;
-        run += __shfl_sync(FULLM, incl, 31);
+        int run = 0;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int t = lane + 32 * u;
+          int c = cnt[u] - beg[u];
+          c = c < p.cap ? c : p.cap;
+          int incl = c;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            int n = __shfl_up_sync(FULLM, incl, d);
+            if (lane >= d) incl += n;
+          }
+          if (t < p.L) { sh_tbeg[t] = beg[u]; sh_tbase[t + 1] = run + incl; }
+          run += __shfl_sync(FULLM, incl, 31);
+        }
+        if (lane == 0) { sh_tbase[0] = 0; sh_misc[24] = run; }
       }
-      if (lane == 0) { sh_tbase[0] = 0; sh_misc[24] = run; }
+      __syncthreads();
+    } else {
+      for (int t = tid; t < p.L; t += FWD_THREADS) {
+        const uint32_t code = table_code(t);
+        sh_code[t] = code;
+        if (MODE == 0) p.codes[(size_t)s * p.L + t] = code;
+        const int32_t* off = p.bucket_off + (size_t)t * (size_t)(p.nb + 1) + code;
+        const int beg = __ldg(off);
+        int cnt = __ldg(off + 1) - beg;
+        cnt = cnt < p.cap ? cnt : p.cap;
+        sh_tbeg[t] = beg;
+        sh_tbase[t + 1] = cnt;
+      }
+      __syncthreads();
+      if (warp == 0) {            // running sum of the slice lengths: where each table's candidates start
+        int run = 0;
+        for (int b = 0; b < p.L; b += 32) {
+          const int t = b + lane;
+          const int v = t < p.L ? sh_tbase[t + 1] : 0;
+          int incl = v;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            int n = __shfl_up_sync(FULLM, incl, d);
+            if (lane >= d) incl += n;
+          }
+          if (t < p.L) sh_tbase[t + 1] = run + incl;
+          run += __shfl_sync(FULLM, incl, 31);
+        }
+        if (lane == 0) { sh_tbase[0] = 0; sh_misc[24] = run; }
+      }
+      __syncthreads();
     }
-    __syncthreads();
 
     // ---- all bucket entries in one round; union over the tables, labels, duplicates removed, ascending ids.
     //      A small candidate set is cheaper to sort than a bitmap over all N neurons is to clear and scan. ----
@@ -729,23 +804,47 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         else rank_sort<RANK_MAX / FWD_THREADS, false>(sh_dd, srt, n);
       }
       __syncthreads();
-      // thread t looks at the sorted elements PER * t ... PER * t + PER - 1 and keeps the first of each run
+      // element i = u * FWD_THREADS + tid of the sorted list is kept when it is the first of its run; its place is
+      // the number of kept elements before it: whole rounds and warps (counts exchanged through shared memory) plus
+      // the warp's own ballot
       constexpr int PER = RANK_MAX / FWD_THREADS;
-      int cnt = 0;
+      int* sh_cntw = reinterpret_cast<int*>(sh_dh);      // [PER][FWD_WARPS]; the space is not used before the back-propagation
+      const unsigned lt = (1u << lane) - 1u;
+      const int rounds = (n + FWD_THREADS - 1) / FWD_THREADS;
+      unsigned keep[PER];
 #pragma unroll
       for (int u = 0; u < PER; ++u) {
-        const int i = tid * PER + u;
-        cnt += (i < n && (i == 0 || srt[i - 1] != srt[i])) ? 1 : 0;
+        keep[u] = 0u;
+        if (u < rounds) {
+          const int i = u * FWD_THREADS + tid;
+          keep[u] = __ballot_sync(FULLM, i < n && (i == 0 || srt[i - 1] != srt[i]));
+          if (lane == 0) sh_cntw[u * FWD_WARPS + warp] = __popc(keep[u]);
+        }
       }
-      int at = block_excl_scan(cnt, sh_misc, &total);
-      if (total <= p.act_stride && cnt > 0) {
+      __syncthreads();
+      {
+        int before = 0;
+        for (int q = 0; q < rounds * FWD_WARPS; ++q) {
+          const int cq = sh_cntw[q];
+          total += cq;
+          if (q < warp) before += cq;           // round 0; later rounds add their offset below
+        }
+        if (total <= p.act_stride) {
+          int base = before;
 #pragma unroll
-        for (int u = 0; u < PER; ++u) {
-          const int i = tid * PER + u;
-          if (i < n && (i == 0 || srt[i - 1] != srt[i])) {
-            ids[at] = (int)srt[i];
-            if (at < ACT_SM) sh_ids[at] = (int)srt[i];
-            ++at;
+          for (int u = 0; u < PER; ++u) {
+            if (u < rounds) {
+              if (u > 0) {
+                base = 0;
+                for (int q = 0; q < u * FWD_WARPS + warp; ++q) base += sh_cntw[q];
+              }
+              const int i = u * FWD_THREADS + tid;
+              if ((keep[u] >> lane) & 1u) {
+                const int at = base + __popc(keep[u] & lt);
+                ids[at] = (int)srt[i];
+                if (at < ACT_SM) sh_ids[at] = (int)srt[i];
+              }
+            }
           }
         }
       }
@@ -799,7 +898,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   // one pointer per array, to shared or to global memory (a conditional expression over two loads would issue both)
   const int* idp = small ? sh_ids : ids;
   const float* zp = small ? sh_z : p.act_z + (size_t)s * p.act_stride;
-  const float* gp = small ? sh_z : p.act_g + (size_t)s * p.act_stride;
+  const float* gp = small ? sh_g : p.act_g + (size_t)s * p.act_stride;
 
   // ---- positions of the sample's distinct labels inside the active set (needed while the rows are staged) ----
   if (MODE == 0) {
@@ -843,43 +942,53 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   for (int u = 0; u < KPT; ++u) { accS[u] = 0.f; accT[u] = 0.f; }
   const int ngrp = H >= FWD_THREADS ? 1 : min(FWD_WARPS, FWD_THREADS / H);   // groups of H threads (sh_dh holds FWD_WARPS)
   const int grp = H >= FWD_THREADS ? 0 : tid / H;
-  const uint32_t row_bytes = (uint32_t)H * 4u;
+  // hand-off to the update kernel: the touch counters of the sample's rows of W1 (one per thread) and of its first
+  // HO_PER * FWD_THREADS active rows are asked while the first rows of W2 are on their way, the list places after the
+  // first logits, and everything is written at the end -- no warp waits for an answer
+  constexpr int HO_PER = 2;
+  int jj0[HO_PER];
+  unsigned nth1 = 0u, nth0[HO_PER], base1 = 0u, base0[HO_PER];
+  // a thread's place in the copy pattern of the padded rows: H4 + 1 pieces per row
+  const int rp_dr = FWD_THREADS / (H4 + 1), rp_dc = FWD_THREADS - rp_dr * (H4 + 1);
+  const int rp_r0 = tid / (H4 + 1), rp_c0 = tid - rp_r0 * (H4 + 1);
+#pragma unroll
+  for (int u = 0; u < HO_PER; ++u) { jj0[u] = 0; nth0[u] = 0u; base0[u] = 0u; }
   for (int c0 = 0; c0 < na; c0 += stage_rows) {
     const int nr = min(stage_rows, na - c0);
     __syncthreads();                               // earlier readers and writers of the staging space are done
-    if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * row_bytes);
-    fence_proxy_async();
-    __syncthreads();
-    for (int r = tid; r < nr; r += FWD_THREADS) {
+    // 16 bytes per thread and copy, all in flight at once: the H4 pieces of the row, and as piece H4 the head of the
+    // row's record (count, bias, bias moments), which lands in the row's padding
+    for (int r = rp_r0, c4 = rp_c0; r < nr;) {
       const int j = dense ? c0 + r : idp[c0 + r];
-      bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)j * H, row_bytes, sh_bar);
+      const void* src = c4 < H4 ? static_cast<const void*>(p.W2 + (size_t)j * H + 4 * c4) : static_cast<const void*>(p.hdr2 + j);
+      cp_async16(stage + (size_t)r * ldr + 4 * c4, src);
+      c4 += rp_dc; r += rp_dr;
+      if (c4 > H4) { c4 -= H4 + 1; ++r; }
     }
-    if (c0 == 0) {
-      // the biases of a small active set are fetched in the same round, into the logits' place
-      if (small)
-        for (int a = tid; a < na; a += FWD_THREADS) sh_z[a] = __ldg(&p.hdr2[sh_ids[a]].b);
-      // ---- the W1 side of the hand-off to the update kernel runs while the copies are in flight: per touched row
-      //      a count of the touching samples, then (finish_touch) the slot or mask entry and the row list ----
-      if (MODE == 0)
-        for (int i0 = 0; i0 < nnz; i0 += FWD_THREADS) {
-          const int i = i0 + tid;
-          const bool live = i < nnz;
-          int c = 0;
-          unsigned nth = 0u;
-          float x = 0.f;
-          if (live) {
-            c = __ldg(p.col_idx + rbeg + i);
-            x = __ldg(p.vals + rbeg + i);
-            nth = atomicAdd(&p.hdr1[c].cnt, 1u) & CNT_MASK;
-            const int line = __ldg(p.hotmap1 + c);          // a feature that has been hot before: its value goes to its line
-            if (line >= 0) p.hotcoef1[(size_t)line * p.bstride + s] = x;
-          }
-          finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.ovf1 + (size_t)c * PAIR_T, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
+    if (c0 == 0 && MODE == 0) {
+      // the touch counters: this thread's nonzero of the sample, and its first HO_PER active rows
+      if (tid < nnz) {
+        if (tid >= R) {                              // beyond the first chunk: not kept in registers above
+          c1 = __ldg(p.col_idx + rbeg + tid);
+          x1 = __ldg(p.vals + rbeg + tid);
+          line1 = __ldcg(p.hotmap1 + c1);
         }
+        nth1 = atomicAdd(&p.hdr1[c1].cnt, 1u) & CNT_MASK;
+        if (line1 >= 0) p.hotcoef1[(size_t)line1 * p.bstride + s] = x1;
+      }
+      if (!dense) {
+#pragma unroll
+        for (int u = 0; u < HO_PER; ++u) {
+          const int a = tid + u * FWD_THREADS;
+          if (a < na) {
+            jj0[u] = idp[a];
+            nth0[u] = atomicAdd(&p.hdr2[jj0[u]].cnt, 1u) & CNT_MASK;
+          }
+        }
+      }
     }
-    if (!mbar_wait(sh_bar, phase)) timed_out = true;
-    phase ^= 1u;
-    if (__syncthreads_or(timed_out ? 1 : 0)) { timed_out = true; break; }
+    cp_async_wait_all();
+    __syncthreads();
     // one thread per staged row
     for (int ab = 0; ab < nr; ab += FWD_THREADS) {
       const int a = ab + tid;
@@ -900,14 +1009,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
       if (MODE == 0) {
         if (live) {
-          float zv;
-          if (small) {                       // the bias is already in the logit's place
-            zv = sh_z[c0 + a] + dot;
-            sh_z[c0 + a] = zv;
-          } else {
-            const int j = dense ? c0 + a : idp[c0 + a];
-            zv = __ldg(&p.hdr2[j].b) + dot;
-          }
+          const float zv = stage[(size_t)a * ldr + H + 1] + dot;      // the bias came with the row
+          if (small) sh_z[c0 + a] = zv;
           z[c0 + a] = zv;
           if (streaming) sh_ce[a] = zv;
         }
@@ -915,7 +1018,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         // predict: lane 0 of each warp keeps the warp's best k so far, fed one lane's logit at a time
         int j = -1;
         float zv = 0.f;
-        if (live) { j = dense ? c0 + a : idp[c0 + a]; zv = __ldg(&p.hdr2[j].b) + dot; }
+        if (live) { j = dense ? c0 + a : idp[c0 + a]; zv = stage[(size_t)a * ldr + H + 1] + dot; }
         float* lz = tk_z + warp * p.topk;
         int* li = tk_id + warp * p.topk;
         // a lane offers its logit only when the list is not full yet or the logit beats the list's last entry
@@ -933,6 +1036,18 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
           }
           __syncwarp();
         }
+      }
+    }
+    if (MODE == 0 && c0 == 0) {
+      // the touch counters have answered by now.  W1 side: slot / mask entries (the coefficient is the input value);
+      // both sides: places in the lists of distinct rows asked for, used at the end of the kernel
+      touch_mark<false>(p, tid < nnz, p.hdr1 + c1, p.mask1 + (size_t)c1 * p.Wd, p.ovf1 + (size_t)c1 * PAIR_T, ~c1, nth1, s, x1);
+      base1 = own_reserve(tid < nnz && nth1 == 0u, &p.st->n_own[p.parity][1]);
+      if (!dense) {
+#pragma unroll
+        for (int u = 0; u < HO_PER; ++u)
+          if (u * FWD_THREADS < na)          // uniform over the block
+            base0[u] = own_reserve(tid + u * FWD_THREADS < na && nth0[u] == 0u, &p.st->n_own[p.parity][0]);
       }
     }
     if (streaming) {
@@ -974,15 +1089,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
     }
   }
-  if (timed_out) {
-    // a copy did not complete in time: give the copies still in flight one more bounded wait, then give the sample
-    // up (its rows of W1 are already handed over; with dh = 0 they receive a zero gradient)
-    mbar_wait(sh_bar, phase ^ 1u);
-    __syncthreads();
-    skip_sample<MODE>(p, s, DSLIDE_ERR_TIMEOUT);
-    return;
-  }
-
   if (MODE == 1) {
     // ---- merge the per-warp lists: k rounds over the list heads ----
     if (lane == 0) sh_misc[warp] = tk_cnt;
@@ -1011,30 +1117,39 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   }
   __syncthreads();           // logits visible to the block
 
-  // ---- softmax over the ragged active set, loss, errors ----
+  // ---- softmax over the ragged active set, loss, errors.  A small set's logits sit in shared memory: every warp
+  //      takes the maximum and the sum over all of them by itself (same order, same result in every warp), which
+  //      spares the block-wide reductions and their barriers ----
   float* pr = p.act_p + (size_t)s * p.act_stride;
   float* g = p.act_g + (size_t)s * p.act_stride;
   float M = Mrun, E = Erun;                        // known already when the rows were streamed
   if (!streaming) {
-    float m = -INFINITY;
-    for (int a = tid; a < na; a += FWD_THREADS) m = fmaxf(m, zp[a]);
-    M = block_max(m, sh_red);
-    float e = 0.f;
-    for (int a = tid; a < na; a += FWD_THREADS) e += expf(zp[a] - M);
-    E = block_sum(e, sh_red);
+    if (small) {
+      float m = -INFINITY;
+      for (int a = lane; a < na; a += 32) m = fmaxf(m, sh_z[a]);
+      M = warp_max(m);
+      float e = 0.f;
+      for (int a = lane; a < na; a += 32) e += expf(sh_z[a] - M);
+      E = warp_sum(e);
+    } else {
+      float m = -INFINITY;
+      for (int a = tid; a < na; a += FWD_THREADS) m = fmaxf(m, zp[a]);
+      M = block_max(m, sh_red);
+      float e = 0.f;
+      for (int a = tid; a < na; a += FWD_THREADS) e += expf(zp[a] - M);
+      E = block_sum(e, sh_red);
+    }
   }
   const float fB = (float)p.B;
-  if (tid == 0) {
-    const int ny = sh_misc[0];
+  const int ny = sh_misc[0];
+  if (tid == FWD_THREADS - 1) {                    // the last thread has the fewest rows below
     float sum = 0.f;
     const float logE = logf(E);
     for (int i = 0; i < nlab; ++i)
       if (sh_lab[i] >= 0) sum += zp[sh_lab[i]] - M - logE;
     p.loss[s] = ny > 0 ? -sum / (float)ny : 0.f;
   }
-  __syncthreads();           // the logits at the label positions have been read: their places may now take the errors
-  const int ny = sh_misc[0];
-  // when the set is small the error takes the logit's place in shared memory, for the steps below
+  // the errors of a small set go to shared memory as well (beside the logits: no barrier before they are written)
   for (int a = tid; a < na; a += FWD_THREADS) {
     const float pa = expf(zp[a] - M) / E;
     pr[a] = pa;
@@ -1042,76 +1157,84 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     for (int i = 0; i < nlab; ++i)
       if (sh_lab[i] == a) ga = (pa - 1.f / (float)ny) / fB;
     g[a] = ga;
-    if (small) sh_z[a] = ga;
+    if (small) sh_g[a] = ga;
   }
   __syncthreads();
 
-  // ---- the W2 side of the hand-off: the touch counters of the first HO_PER * FWD_THREADS active rows are asked now
-  //      and answered while the back-propagation below runs ----
-  constexpr int HO_PER = 4;
-  int jj0[HO_PER];
-  unsigned nth0[HO_PER];
-  float ga0[HO_PER];
-#pragma unroll
-  for (int u = 0; u < HO_PER; ++u) {
-    const int a = tid + u * FWD_THREADS;
-    jj0[u] = 0; nth0[u] = 0u; ga0[u] = 0.f;
-    if (!dense && a < na) {
-      jj0[u] = idp[a];
-      ga0[u] = gp[a];
-      nth0[u] = atomicAdd(&p.hdr2[jj0[u]].cnt, 1u) & CNT_MASK;
-    }
-  }
-
-  // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update).  A thread
-  //      per hidden unit walks the staged rows; with fewer hidden units than threads the rows are dealt to
-  //      several groups of threads whose sums are then added in group order.  When the rows were streamed the
-  //      sums exist already. ----
+  // ---- error at the hidden layer: dh = [h > 0] * sum_a g_a W2[j_a, :] (weights before the update).  Warp w takes
+  //      the staged rows w, w + 8, ...; a lane holds four consecutive hidden units of every 128; the warps' sums are
+  //      then added in warp order.  When the rows were streamed the sums exist already (per group of threads). ----
   {
-    float accd[KPT];
+    constexpr int NCH = KPT == 1 ? 2 : 2 * MAX_KPT;        // 16-byte pieces of a row per lane: H <= 128 * NCH
+    int nparts = ngrp;
+    if (!streaming) {
+      nparts = FWD_WARPS;
+      float4 av[NCH];
 #pragma unroll
-    for (int u = 0; u < KPT; ++u)
-      accd[u] = streaming ? (accS[u] / E - (ny > 0 ? accT[u] / (float)ny : 0.f)) / fB : 0.f;
-    if (!streaming && grp < ngrp) {
-      const int nr = na;                           // all rows are still staged
+      for (int q = 0; q < NCH; ++q) av[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int a = warp; a < na; a += FWD_WARPS) {
+        const float ga = gp[a];
+        const float4* row = reinterpret_cast<const float4*>(stage + (size_t)a * ldr);
 #pragma unroll
-      for (int u = 0; u < KPT; ++u) {
-        const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
-        if (k < H && (u == 0 || H > FWD_THREADS)) {
-          float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
-          int a = grp;
-          for (; a + 3 * ngrp < nr; a += 4 * ngrp) {
-            v0 = fmaf(gp[a], stage[(size_t)a * ldr + k], v0);
-            v1 = fmaf(gp[a + ngrp], stage[(size_t)(a + ngrp) * ldr + k], v1);
-            v2 = fmaf(gp[a + 2 * ngrp], stage[(size_t)(a + 2 * ngrp) * ldr + k], v2);
-            v3 = fmaf(gp[a + 3 * ngrp], stage[(size_t)(a + 3 * ngrp) * ldr + k], v3);
+        for (int q = 0; q < NCH; ++q) {
+          const int c = lane + 32 * q;
+          if (c < H4) {
+            const float4 w = row[c];
+            av[q].x = fmaf(ga, w.x, av[q].x); av[q].y = fmaf(ga, w.y, av[q].y);
+            av[q].z = fmaf(ga, w.z, av[q].z); av[q].w = fmaf(ga, w.w, av[q].w);
           }
-          for (; a < nr; a += ngrp) v0 = fmaf(gp[a], stage[(size_t)a * ldr + k], v0);
-          accd[u] = (v0 + v1) + (v2 + v3);
         }
       }
-    }
-    if (grp < ngrp) {
+#pragma unroll
+      for (int q = 0; q < NCH; ++q) {
+        const int c = lane + 32 * q;
+        if (c < H4) reinterpret_cast<float4*>(sh_dh + (size_t)warp * H)[c] = av[q];
+      }
+    } else if (grp < ngrp) {
 #pragma unroll
       for (int u = 0; u < KPT; ++u) {
         const int k = (H >= FWD_THREADS ? tid : tid - grp * H) + u * FWD_THREADS;
-        if (k < H && (u == 0 || H > FWD_THREADS)) sh_dh[(size_t)grp * H + k] = accd[u];
+        if (k < H && (u == 0 || H > FWD_THREADS))
+          sh_dh[(size_t)grp * H + k] = (accS[u] / E - (ny > 0 ? accT[u] / (float)ny : 0.f)) / fB;
       }
     }
     __syncthreads();
     for (int k = tid; k < H; k += FWD_THREADS) {
       float v = 0.f;
-      for (int w = 0; w < ngrp; ++w) v += sh_dh[(size_t)w * H + k];
+      for (int w = 0; w < nparts; ++w) v += sh_dh[(size_t)w * H + k];
       p.dh[(size_t)s * H + k] = sh_h[k] > 0.f ? v : 0.f;
     }
+  }
+
+  // ---- the rest of the hand-off: slot / mask entries of the rows of W2 (their coefficient is the error), the
+  //      entries of both lists of distinct rows, and whatever did not fit the registers above ----
+  own_store(tid < nnz && nth1 == 0u, base1, p.own1, c1, s);
+  if (tid < nnz) list_row(p, &p.hdr1[c1].cnt, ~c1, nth1);
+  for (int i0 = FWD_THREADS; i0 < nnz; i0 += FWD_THREADS) {
+    const int i = i0 + tid;
+    const bool live = i < nnz;
+    int c = 0;
+    unsigned nth = 0u;
+    float x = 0.f;
+    if (live) {
+      c = __ldg(p.col_idx + rbeg + i);
+      x = __ldg(p.vals + rbeg + i);
+      nth = atomicAdd(&p.hdr1[c].cnt, 1u) & CNT_MASK;
+      const int line = __ldg(p.hotmap1 + c);
+      if (line >= 0) p.hotcoef1[(size_t)line * p.bstride + s] = x;
+    }
+    finish_touch(p, live, p.hdr1 + c, p.mask1 + (size_t)c * p.Wd, p.ovf1 + (size_t)c * PAIR_T, p.own1, &p.st->n_own[p.parity][1], c, ~c, nth, s, x);
   }
   if (!dense) {
 #pragma unroll
     for (int u = 0; u < HO_PER; ++u)
-      if (u * FWD_THREADS < na)            // uniform over the block
-        finish_touch(p, tid + u * FWD_THREADS < na, p.hdr2 + jj0[u], p.mask2 + (size_t)jj0[u] * p.Wd,
-                     p.ovf2 + (size_t)jj0[u] * PAIR_T, p.own2,
-                     &p.st->n_own[p.parity][0], jj0[u], jj0[u], nth0[u], s, ga0[u]);
+      if (u * FWD_THREADS < na) {          // uniform over the block
+        const int a = tid + u * FWD_THREADS;
+        const bool live = a < na;
+        touch_mark(p, live, p.hdr2 + jj0[u], p.mask2 + (size_t)jj0[u] * p.Wd, p.ovf2 + (size_t)jj0[u] * PAIR_T, jj0[u], nth0[u], s,
+                   live ? gp[a] : 0.f);
+        own_store(live && nth0[u] == 0u, base0[u], p.own2, jj0[u], s);
+      }
     for (int a0 = HO_PER * FWD_THREADS; a0 < na; a0 += FWD_THREADS) {
       const int a = a0 + tid;
       const bool live = a < na;
