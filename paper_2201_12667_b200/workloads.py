@@ -31,6 +31,14 @@ CONFIGS = {
     # the 670K shape with the large hidden layer and batch of Table 3
     "670k-h1024": dict(D=135909, H=1024, N=670091, family=DWTA, K=6, L=50, bin_size=8, srp_nnz=0, bucket_cap=128,
                        batch=1024, mean_nnz=76, mean_labels=5, dist="zipf", lr=1e-4, max_labels=16),
+    # the shape of the low-bandwidth experiment (Section 4.7: hidden layer 256, batch 2048) on the first dataset's dimensions
+    "670k-h256-b2048": dict(D=135909, H=256, N=670091, family=DWTA, K=6, L=50, bin_size=8, srp_nnz=0, bucket_cap=128,
+                            batch=2048, mean_nnz=76, mean_labels=5, dist="zipf", lr=1e-4, max_labels=16),
+    # Table 3's batch of 2048 with the large hidden layer
+    "670k-h1024-b2048": dict(D=135909, H=1024, N=670091, family=DWTA, K=6, L=50, bin_size=8, srp_nnz=0, bucket_cap=128,
+                             batch=2048, mean_nnz=76, mean_labels=5, dist="zipf", lr=1e-4, max_labels=16),
+    "text8-b2048": dict(D=253855, H=200, N=253855, family=SIMHASH, K=9, L=50, bin_size=8, srp_nnz=0, bucket_cap=128,
+                        batch=2048, mean_nnz=1, fixed_nnz=1, mean_labels=4, dist="zipf", lr=1e-4, max_labels=16),
     # a mid-size shape for parity tests: several tiles, ragged tails, both dedup paths
     "mid": dict(D=5003, H=128, N=20011, family=DWTA, K=3, L=10, bin_size=8, srp_nnz=0, bucket_cap=16,
                 batch=48, mean_nnz=30, mean_labels=3, dist="zipf", lr=1e-3, max_labels=16),

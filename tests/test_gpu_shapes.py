@@ -302,3 +302,18 @@ def test_fill_that_cannot_reach_the_budget():
         assert np.all(cnt < 257) and np.all(cnt > 128)
     finally:
         pr.close()
+
+
+@pytest.mark.parametrize("name", ["670k-h256-b2048", "670k-h1024-b2048", "text8-b2048"])
+def test_paper_shapes_with_batch_2048_at_reduced_vocabulary(name):
+    """The hidden widths, batch of 2,048 and hashing of the paper's large-batch and low-bandwidth experiments
+    (Table 3; Section 4.7: hidden layer 256, batch 2048) on a vocabulary the oracle steps through in seconds: every
+    row of W1 is touched by dozens of samples (hot rows, sample masks of 64 words)."""
+    c = workloads.config(name, D=4001, N=30011)
+    pr = Pair(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"] if c["family"] == SIMHASH else 4, L=12,
+              bucket_cap=32, max_batch=c["batch"], max_labels=c["max_labels"], lr=1e-3, seed=5, oracle_build="float_omp")
+    try:
+        wl = workloads.Workload(c, seed=17)
+        one_and_two_steps(pr, [wl.batch(i) for i in range(2)])
+    finally:
+        pr.close()
