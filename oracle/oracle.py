@@ -48,16 +48,19 @@ class OrcConfig(C.Structure):
         ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
         ("init_std", C.c_double),
         ("seed", C.c_uint64),
+        ("hidden_K", C.c_int32), ("hidden_L", C.c_int32), ("hidden_cap", C.c_int32),
     ]
 
 
 # must match the enum in slide_oracle.c
 NAMES = ["W1", "b1", "W2", "b2", "mW1", "vW1", "mb1", "vb1", "mW2", "vW2", "mb2", "vb2",
          "dW1", "db1", "dW2", "db2", "hash_idx", "hash_sign", "bucket_off", "bucket_ids",
-         "h", "dh", "codes", "act_ptr", "act_ids", "act_z", "act_p", "act_g", "loss"]
+         "h", "dh", "codes", "act_ptr", "act_ids", "act_z", "act_p", "act_g", "loss",
+         "proj1", "bucket1_off", "bucket1_ids", "codes1", "hact"]
 _WHICH = {n: i for i, n in enumerate(NAMES)}
 _INT_TYPES = {"hash_idx": np.int32, "hash_sign": np.int32, "bucket_off": np.int32, "bucket_ids": np.int32,
-              "codes": np.uint32, "act_ptr": np.int64, "act_ids": np.int32}
+              "codes": np.uint32, "act_ptr": np.int64, "act_ids": np.int32,
+              "proj1": np.int8, "bucket1_off": np.int32, "bucket1_ids": np.int32, "codes1": np.uint32, "hact": np.uint8}
 
 SIMHASH, DWTA = 0, 1
 
@@ -90,6 +93,8 @@ def _load(real):
         lib.orc_mix64.argtypes = [C.c_uint64]
         lib.orc_draw_hash.argtypes = [C.c_void_p, C.c_int64]
         lib.orc_build_tables.argtypes = [C.c_void_p]
+        lib.orc_build_tables1.argtypes = [C.c_void_p]
+        lib.orc_draw_hash1.argtypes = [C.c_void_p, C.c_int64]
         lib.orc_rebuild_tables.argtypes = [C.c_void_p]
         lib.orc_hash_vec.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.orc_hash_query.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -130,7 +135,7 @@ class Oracle:
         self.lib = _load(real)
         d = dict(family=SIMHASH, bin_size=8, srp_nnz=0, bucket_cap=128, rebuild_period0=0, redraw=1,
                  force_dense=0, max_active=0, densify=0, budget=0, budget_fill=0, rebuild_lambda=0.0, lr=1e-4, beta1=0.9, beta2=0.999,
-                 eps=1e-8, init_std=0.01, seed=0)
+                 eps=1e-8, init_std=0.01, seed=0, hidden_K=0, hidden_L=0, hidden_cap=0)
         d.update(kw)
         self.cfg = OrcConfig(**d)
         self.o = self.lib.orc_create(C.byref(self.cfg))
@@ -202,6 +207,13 @@ class Oracle:
 
     def build_tables(self):
         self.lib.orc_build_tables(self.o)
+
+    def build_tables1(self):
+        """Tables over the hidden neurons (LSH-sampled hidden layer)."""
+        self.lib.orc_build_tables1(self.o)
+
+    def draw_hash1(self, r):
+        self.lib.orc_draw_hash1(self.o, r)
 
     def rebuild_tables(self):
         self.lib.orc_rebuild_tables(self.o)

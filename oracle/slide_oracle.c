@@ -78,6 +78,11 @@ typedef struct {
   double lr, beta1, beta2, eps;   /* Adam (Section 4.1)                                          */
   double init_std;
   uint64_t seed;
+  /* LSH-sampled hidden layer (Algorithm 1: active neurons are retrieved for EVERY layer; Section 3.6: a dense layer is
+   * the case "sparsity is 1").  hidden_L = 0: the hidden layer is dense.  hidden_L > 0: L tables of hidden_K-bit
+   * SimHash codes over the hidden neurons' weight vectors, queried with the sparse input; a query reads at most
+   * hidden_cap ids of a bucket. */
+  int32_t hidden_K, hidden_L, hidden_cap;
 } orc_config;
 
 typedef struct {
@@ -95,6 +100,13 @@ typedef struct {
   int32_t *hash_sign;       /* [K*L][srp_nnz], +1/-1 (SimHash only) */
   int32_t *bucket_off;      /* [L][2^bits + 1] */
   int32_t *bucket_ids;      /* [L][N] */
+  /* hidden layer, when it is LSH-sampled */
+  int8_t *proj1;            /* [D][hidden_K*hidden_L]: +1 / -1 / 0, the first layer's sparse random projections */
+  int32_t *bucket1_off;     /* [hidden_L][2^hidden_K + 1] */
+  int32_t *bucket1_ids;     /* [hidden_L][H] */
+  uint32_t *codes1;         /* [B][hidden_L] codes of the inputs */
+  uint8_t *hact;            /* [B][H] 1 = hidden neuron active for the sample */
+  uint8_t *touch1e;         /* [D][H] 1 = weight touched by the batch (input nonzero and hidden neuron active) */
   /* snapshot of the last forward pass (Section 3.6: active neurons, activations, errors) */
   int32_t B;
   REAL *h, *dh;             /* [B][H] */
@@ -132,7 +144,7 @@ uint64_t orc_rng(uint64_t seed, uint64_t stream, uint64_t r, uint64_t ctr) {
   uint64_t b = mix64(a + GOLD * (r + 1));
   return mix64(b + GOLD * (ctr + 1));
 }
-enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3, STREAM_SAMPLE = 4, STREAM_FILL = 5 };
+enum { STREAM_W1 = 0, STREAM_W2 = 1, STREAM_HASH = 2, STREAM_PROBE = 3, STREAM_SAMPLE = 4, STREAM_FILL = 5, STREAM_HASH1 = 6 };
 enum { DENSIFY_ATTEMPTS = 16 };
 
 static double u01(uint64_t x) { return ((double)(x >> 11) + 0.5) * (1.0 / 9007199254740992.0); }
@@ -296,10 +308,115 @@ void orc_build_tables(orc *o) {
 }
 
 /* An unscheduled rebuild: next rebuild count, new functions if asked, tables. */
+void orc_build_tables1(orc *o);
+void orc_draw_hash1(orc *o, int64_t r);
 void orc_rebuild_tables(orc *o) {
   o->r += 1;
-  if (o->c.redraw) orc_draw_hash(o, o->r);
+  if (o->c.redraw) { orc_draw_hash(o, o->r); orc_draw_hash1(o, o->r); }
   orc_build_tables(o);
+  orc_build_tables1(o);
+}
+
+/* ------------------------------------------------------------------ */
+/* LSH-sampled hidden layer.                                           */
+/* Hash family, reading: sparse random projections in their classic    */
+/* form -- every entry of a projection is drawn by itself: +1 with     */
+/* probability 1/6, -1 with probability 1/6, 0 with probability 2/3    */
+/* (density 1/3, as for the output layer).  Entry (c, p) of rebuild    */
+/* count r: u = rng(seed, STREAM_HASH1, r, c * KL + p); u mod 6 == 0   */
+/* -> +1, == 1 -> -1, else 0.  (The output layer's projections choose   */
+/* exactly ceil(H/3) coordinates by a shuffle; over the D input         */
+/* coordinates a shuffle per projection is no plain definition any     */
+/* more.)  Code of a vector v[D]: s_p = sum over the coordinates c of   */
+/* the projection, ascending, of +-v[c], sequential in REAL;           */
+/* bit = (s_p >= 0); code_t = sum_k bit_{tK+k} << k.                    */
+/* ------------------------------------------------------------------ */
+void orc_draw_hash1(orc *o, int64_t r) {
+  const orc_config *c = &o->c;
+  if (c->hidden_L <= 0) return;
+  int64_t KL = (int64_t)c->hidden_K * c->hidden_L;
+#pragma omp parallel for schedule(static)
+  for (int64_t cc = 0; cc < c->D; ++cc)
+    for (int64_t p = 0; p < KL; ++p) {
+      uint64_t u = orc_rng(c->seed, STREAM_HASH1, (uint64_t)r, (uint64_t)cc * (uint64_t)KL + (uint64_t)p) % 6u;
+      o->proj1[cc * KL + p] = u == 0 ? 1 : (u == 1 ? -1 : 0);
+    }
+}
+
+/* codes of the sparse vector with nonzeros (col[j], val[j]), ascending columns: coordinates outside the vector add
+ * nothing, so the sum over the projection's coordinates is the sum over the vector's nonzeros that it selects */
+static void hash1_sparse(const orc *o, int32_t nnz, const int32_t *col, const REAL *val, uint32_t *codes) {
+  const orc_config *c = &o->c;
+  int64_t KL = (int64_t)c->hidden_K * c->hidden_L;
+  for (int t = 0; t < c->hidden_L; ++t) {
+    uint32_t code = 0;
+    for (int k = 0; k < c->hidden_K; ++k) {
+      int64_t p = (int64_t)t * c->hidden_K + k;
+      REAL s = 0;
+      for (int32_t j = 0; j < nnz; ++j) {
+        int8_t e = o->proj1[(int64_t)col[j] * KL + p];
+        if (e != 0) s = s + (e > 0 ? val[j] : -val[j]);
+      }
+      if (s >= 0) code |= 1u << k;
+    }
+    codes[t] = code;
+  }
+}
+
+/* codes of hidden neuron k: its weight vector is column k of W1 */
+static void hash1_neuron(const orc *o, int k, uint32_t *codes) {
+  const orc_config *c = &o->c;
+  int64_t KL = (int64_t)c->hidden_K * c->hidden_L;
+  for (int t = 0; t < c->hidden_L; ++t) {
+    uint32_t code = 0;
+    for (int q = 0; q < c->hidden_K; ++q) {
+      int64_t p = (int64_t)t * c->hidden_K + q;
+      REAL s = 0;
+      for (int64_t cc = 0; cc < c->D; ++cc) {
+        int8_t e = o->proj1[cc * KL + p];
+        if (e != 0) { REAL w = o->W1[(size_t)cc * c->H + k]; s = s + (e > 0 ? w : -w); }
+      }
+      if (s >= 0) code |= 1u << q;
+    }
+    codes[t] = code;
+  }
+}
+
+/* tables over the hidden neurons: bucket (t, code) lists, ascending, the neurons with that code in table t */
+void orc_build_tables1(orc *o) {
+  const orc_config *c = &o->c;
+  if (c->hidden_L <= 0) return;
+  int64_t nb = (int64_t)1 << c->hidden_K;
+  uint32_t *codes = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)c->H * (size_t)c->hidden_L);
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int k = 0; k < c->H; ++k) hash1_neuron(o, k, codes + (size_t)k * c->hidden_L);
+  for (int t = 0; t < c->hidden_L; ++t) {
+    int32_t *off = o->bucket1_off + (size_t)t * (size_t)(nb + 1);
+    int32_t *ids = o->bucket1_ids + (size_t)t * (size_t)c->H;
+    memset(off, 0, sizeof(int32_t) * (size_t)(nb + 1));
+    for (int k = 0; k < c->H; ++k) off[codes[(size_t)k * c->hidden_L + t] + 1]++;
+    for (int64_t b = 0; b < nb; ++b) off[b + 1] += off[b];
+    int32_t *cursor = (int32_t *)malloc(sizeof(int32_t) * (size_t)nb);
+    for (int64_t b = 0; b < nb; ++b) cursor[b] = off[b];
+    for (int k = 0; k < c->H; ++k) ids[cursor[codes[(size_t)k * c->hidden_L + t]]++] = k;
+    free(cursor);
+  }
+  free(codes);
+}
+
+/* active hidden neurons of one sample: union over the tables of (at most hidden_cap lowest ids of) the buckets its
+ * codes select; act[k] = 1 for an active neuron */
+static void select_hidden(const orc *o, const uint32_t *codes, uint8_t *act) {
+  const orc_config *c = &o->c;
+  int64_t nb = (int64_t)1 << c->hidden_K;
+  memset(act, 0, (size_t)c->H);
+  for (int t = 0; t < c->hidden_L; ++t) {
+    const int32_t *off = o->bucket1_off + (size_t)t * (size_t)(nb + 1);
+    const int32_t *ids = o->bucket1_ids + (size_t)t * (size_t)c->H;
+    int32_t cnt = off[codes[t] + 1] - off[codes[t]];
+    if (cnt > c->hidden_cap) cnt = c->hidden_cap;
+    for (int32_t i = 0; i < cnt; ++i) act[ids[off[codes[t]] + i]] = 1;
+  }
 }
 
 static REAL *zalloc_real(int64_t n) { return (REAL *)calloc((size_t)(n > 0 ? n : 1), sizeof(REAL)); }
@@ -333,10 +450,19 @@ orc *orc_create(const orc_config *cfg) {
   int64_t nb = (int64_t)1 << o->bits;
   o->bucket_off = (int32_t *)calloc((size_t)(c->L * (nb + 1)), sizeof(int32_t));
   o->bucket_ids = (int32_t *)calloc((size_t)((int64_t)c->L * N), sizeof(int32_t));
+  if (c->hidden_L > 0) {
+    int64_t KL1 = (int64_t)c->hidden_K * c->hidden_L, nb1 = (int64_t)1 << c->hidden_K;
+    o->proj1 = (int8_t *)calloc((size_t)(D * KL1), 1);
+    o->bucket1_off = (int32_t *)calloc((size_t)(c->hidden_L * (nb1 + 1)), sizeof(int32_t));
+    o->bucket1_ids = (int32_t *)calloc((size_t)((int64_t)c->hidden_L * H), sizeof(int32_t));
+    o->touch1e = (uint8_t *)calloc((size_t)(D * H), 1);
+  }
   o->t = 0; o->r = 0;
   o->next_rebuild = c->rebuild_period0;
   orc_draw_hash(o, 0);
   orc_build_tables(o);
+  orc_draw_hash1(o, 0);
+  orc_build_tables1(o);
   return o;
 }
 
@@ -351,6 +477,7 @@ void orc_destroy(orc *o) {
   free(o->h); free(o->dh); free(o->codes); free(o->act_ptr); free(o->act_ids);
   free(o->act_z); free(o->act_p); free(o->act_g); free(o->loss);
   free(o->row_ptr); free(o->col_idx); free(o->vals); free(o->label_ptr); free(o->labels);
+  free(o->proj1); free(o->bucket1_off); free(o->bucket1_ids); free(o->codes1); free(o->hact); free(o->touch1e);
   free(o);
 }
 
@@ -364,6 +491,10 @@ static void ensure_batch(orc *o, int32_t B, int64_t nnz, int64_t nlab) {
     o->loss = (REAL *)realloc(o->loss, sizeof(REAL) * (size_t)B);
     o->row_ptr = (int32_t *)realloc(o->row_ptr, sizeof(int32_t) * (size_t)(B + 1));
     o->label_ptr = (int32_t *)realloc(o->label_ptr, sizeof(int32_t) * (size_t)(B + 1));
+    if (o->c.hidden_L > 0) {
+      o->codes1 = (uint32_t *)realloc(o->codes1, sizeof(uint32_t) * (size_t)(B * o->c.hidden_L));
+      o->hact = (uint8_t *)realloc(o->hact, (size_t)(B * H));
+    }
     o->B_capacity = B;
   }
   if (nnz > o->nnz_capacity) {
@@ -392,9 +523,10 @@ static void ensure_act(orc *o, int64_t need) {
  * reading: bias first, then one fused multiply-add per nonzero in stored
  * order, then ReLU.  The order is part of the definition so that the hidden
  * activation, and with it every hash code, has one correct value. */
-static void hidden_layer(const orc *o, int32_t nnz, const int32_t *col, const REAL *val, REAL *h) {
+static void hidden_layer(const orc *o, int32_t nnz, const int32_t *col, const REAL *val, REAL *h, const uint8_t *act) {
   int H = o->c.H;
   for (int k = 0; k < H; ++k) {
+    if (act && !act[k]) { h[k] = 0; continue; }     /* Section 2.1: a neuron that was not retrieved is a NoOp, activation 0 */
     REAL acc = o->b1[k];
     for (int32_t j = 0; j < nnz; ++j) acc = r_fma(val[j], o->W1[(size_t)col[j] * H + k], acc);
     h[k] = acc > 0 ? acc : 0;
@@ -533,7 +665,14 @@ int32_t orc_forward(orc *o, int32_t B, const int32_t *row_ptr, const int32_t *co
 #pragma omp parallel for schedule(dynamic, 1)
   for (int32_t s = 0; s < B; ++s) {
     REAL *h = o->h + (size_t)s * H;
-    hidden_layer(o, row_ptr[s + 1] - row_ptr[s], col_idx + row_ptr[s], vals + row_ptr[s], h);
+    const uint8_t *hact = NULL;
+    if (c->hidden_L > 0) {      /* Algorithm 1: retrieve the layer's active neurons with the layer's input, then feed forward */
+      uint32_t *codes1 = o->codes1 + (size_t)s * c->hidden_L;
+      hash1_sparse(o, row_ptr[s + 1] - row_ptr[s], col_idx + row_ptr[s], vals + row_ptr[s], codes1);
+      select_hidden(o, codes1, o->hact + (size_t)s * H);
+      hact = o->hact + (size_t)s * H;
+    }
+    hidden_layer(o, row_ptr[s + 1] - row_ptr[s], col_idx + row_ptr[s], vals + row_ptr[s], h, hact);
     uint32_t *codes = o->codes + (size_t)s * c->L;
     orc_hash_query(o, h, codes);
     const int32_t *lab = label_ptr ? labels + label_ptr[s] : NULL;
@@ -645,6 +784,10 @@ void orc_backward(orc *o) {
         REAL x = o->vals[i];
         for (int k = 0; k < H; ++k) o->dW1[(size_t)f * H + k] += x * dh[k];
         o->touch1[f] = 1;
+        if (o->touch1e) {     /* sampled hidden layer: only the weights of the sample's active hidden neurons are touched */
+          const uint8_t *hact = o->hact + (size_t)s * H;
+          for (int k = 0; k < H; ++k) if (hact[k]) o->touch1e[(size_t)f * H + k] = 1;
+        }
       }
       for (int k = tid; k < H; k += nt) o->db1[k] += dh[k];
     }
@@ -687,13 +830,20 @@ void orc_adam(orc *o) {
     if (!o->touch1[f]) continue;
     for (int k = 0; k < H; ++k) {
       size_t e = (size_t)f * H + k;
-      adam_elem(o, &o->W1[e], &o->mW1[e], &o->vW1[e], o->dW1[e], bc1, bc2);
+      if (!o->touch1e || o->touch1e[e]) adam_elem(o, &o->W1[e], &o->mW1[e], &o->vW1[e], o->dW1[e], bc1, bc2);
+      if (o->touch1e) o->touch1e[e] = 0;
       o->dW1[e] = 0;
     }
     o->touch1[f] = 0;
   }
   for (int k = 0; k < H; ++k) {
-    adam_elem(o, &o->b1[k], &o->mb1[k], &o->vb1[k], o->db1[k], bc1, bc2);
+    /* a sampled hidden layer: the bias of a neuron that no sample of the batch retrieved is untouched */
+    int touched = 1;
+    if (c->hidden_L > 0) {
+      touched = 0;
+      for (int32_t s = 0; s < o->B; ++s) if (o->hact[(size_t)s * H + k]) { touched = 1; break; }
+    }
+    if (touched) adam_elem(o, &o->b1[k], &o->mb1[k], &o->vb1[k], o->db1[k], bc1, bc2);
     o->db1[k] = 0;
   }
 }
@@ -765,7 +915,8 @@ enum {
   ORC_W1 = 0, ORC_B1, ORC_W2, ORC_B2, ORC_MW1, ORC_VW1, ORC_MB1, ORC_VB1, ORC_MW2, ORC_VW2, ORC_MB2, ORC_VB2,
   ORC_DW1, ORC_DB1, ORC_DW2, ORC_DB2,
   ORC_HASH_IDX, ORC_HASH_SIGN, ORC_BUCKET_OFF, ORC_BUCKET_IDS,
-  ORC_H, ORC_DH, ORC_CODES, ORC_ACT_PTR, ORC_ACT_IDS, ORC_ACT_Z, ORC_ACT_P, ORC_ACT_G, ORC_LOSS
+  ORC_H, ORC_DH, ORC_CODES, ORC_ACT_PTR, ORC_ACT_IDS, ORC_ACT_Z, ORC_ACT_P, ORC_ACT_G, ORC_LOSS,
+  ORC_PROJ1, ORC_BUCKET1_OFF, ORC_BUCKET1_IDS, ORC_CODES1, ORC_HACT
 };
 
 void *orc_ptr(orc *o, int32_t which) {
@@ -780,6 +931,8 @@ void *orc_ptr(orc *o, int32_t which) {
     case ORC_ACT_PTR: return o->act_ptr; case ORC_ACT_IDS: return o->act_ids;
     case ORC_ACT_Z: return o->act_z; case ORC_ACT_P: return o->act_p; case ORC_ACT_G: return o->act_g;
     case ORC_LOSS: return o->loss;
+    case ORC_PROJ1: return o->proj1; case ORC_BUCKET1_OFF: return o->bucket1_off; case ORC_BUCKET1_IDS: return o->bucket1_ids;
+    case ORC_CODES1: return o->codes1; case ORC_HACT: return o->hact;
   }
   return NULL;
 }
@@ -801,6 +954,11 @@ int64_t orc_count(orc *o, int32_t which) {
     case ORC_ACT_PTR: return o->B + 1;
     case ORC_ACT_IDS: case ORC_ACT_Z: case ORC_ACT_P: case ORC_ACT_G: return o->B ? o->act_ptr[o->B] : 0;
     case ORC_LOSS: return o->B;
+    case ORC_PROJ1: return c->hidden_L > 0 ? D * c->hidden_K * c->hidden_L : 0;
+    case ORC_BUCKET1_OFF: return c->hidden_L > 0 ? c->hidden_L * (((int64_t)1 << c->hidden_K) + 1) : 0;
+    case ORC_BUCKET1_IDS: return c->hidden_L > 0 ? (int64_t)c->hidden_L * H : 0;
+    case ORC_CODES1: return c->hidden_L > 0 ? (int64_t)o->B * c->hidden_L : 0;
+    case ORC_HACT: return c->hidden_L > 0 ? (int64_t)o->B * H : 0;
   }
   return -1;
 }
