@@ -101,6 +101,18 @@ typedef struct {
                                                 the previous step's update is still draining, which shortens the
                                                 step by a few microseconds.  The host-buffer entry points wait for
                                                 their own copy and always read early.                              */
+  int32_t hidden_K, hidden_L, hidden_cap;    /* LSH-sampled hidden layer (Algorithm 1 retrieves the active neurons
+                                                of EVERY layer; Section 3.6: the dense layer is the case "sparsity
+                                                is 1").  hidden_L = 0: dense hidden layer.  hidden_L > 0: hidden_L
+                                                tables of hidden_K-bit sparse-random-projection codes over the hidden
+                                                neurons' weight vectors (columns of W1), queried with the sparse
+                                                input; a query reads at most hidden_cap ids of a bucket.  A neuron
+                                                that is not retrieved has activation 0, passes no gradient on, and
+                                                only weights W1[c][k] with input c nonzero and neuron k retrieved
+                                                (for some sample of the batch) are updated; likewise the bias of k.
+                                                Entry (c, p) of the projections: +1, -1, 0 with probability 1/6,
+                                                1/6, 2/3, drawn per entry.  hidden_K <= 16, hidden_L <= 64,
+                                                hidden_K * hidden_L <= 256.  Rebuilt with the output layer's tables. */
 } dslide_config;
 
 /* Tensors readable and writable through dslide_get_tensor / dslide_set_tensor. */
@@ -113,6 +125,9 @@ enum {
   DSLIDE_T_BUCKET_OFF,  /* i32 [L][2^bits + 1], bits = K (SimHash) or K*log2(bin) (DWTA)                        */
   DSLIDE_T_BUCKET_IDS,  /* i32 [L][N]: per table, neuron ids grouped by bucket, ascending inside a bucket       */
   DSLIDE_T_COUNTERS,    /* i64 [3]: Adam step count t, rebuild count r, step of the next scheduled rebuild      */
+  DSLIDE_T_PROJ1,       /* i8 [D][hidden_K * hidden_L]: the hidden layer's projections (+1 / -1 / 0); 0 bytes when dense */
+  DSLIDE_T_BUCKET1_OFF, /* i32 [hidden_L][2^hidden_K + 1]                                                        */
+  DSLIDE_T_BUCKET1_IDS, /* i32 [hidden_L][H]: hidden neuron ids grouped by bucket, ascending inside a bucket     */
   DSLIDE_T_COUNT
 };
 
@@ -127,6 +142,8 @@ enum {
   DSLIDE_LAST_ACT_ERR,    /* f32 [B][stride] (p - [label]/|labels|) / B                         */
   DSLIDE_LAST_LOSS,       /* f32 [B]                                                            */
   DSLIDE_LAST_DHIDDEN,    /* f32 [B][H] error back-propagated to the hidden layer               */
+  DSLIDE_LAST_CODES1,     /* u32 [B][hidden_L] bucket codes of the inputs (sampled hidden layer)  */
+  DSLIDE_LAST_HIDDEN_MASK,/* u32 [B][ceil(H/32)] bit k = hidden neuron k active for the sample    */
   DSLIDE_LAST_COUNT
 };
 
@@ -210,7 +227,7 @@ dslide_status dslide_sync(dslide_ctx* ctx);
 /* State I/O (check-pointing and the parity harness).  Synchronous.  host pointers.
  * nbytes must equal the tensor's size exactly.  Setting weights or hash functions does
  * not rebuild the tables; call dslide_build_tables. */
-enum { DSLIDE_DT_F32 = 0, DSLIDE_DT_I32 = 1, DSLIDE_DT_I64 = 2 };
+enum { DSLIDE_DT_F32 = 0, DSLIDE_DT_I32 = 1, DSLIDE_DT_I64 = 2, DSLIDE_DT_I8 = 3 };
 dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes, int32_t* dtype /* may be NULL: DSLIDE_DT_* */);
 dslide_status dslide_get_tensor(dslide_ctx* ctx, int32_t which, void* host_dst, int64_t nbytes);
 dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host_src, int64_t nbytes);

@@ -23,13 +23,14 @@ OK, ERR_INVALID_ARG, ERR_OOM, ERR_CUDA, ERR_OVERFLOW, ERR_BAD_INDEX, ERR_STATE, 
 SIMHASH, DWTA = 0, 1
 
 T_NAMES = ["W1", "b1", "W2", "b2", "mW1", "vW1", "mb1", "vb1", "mW2", "vW2", "mb2", "vb2",
-           "hash_idx", "hash_sign", "bucket_off", "bucket_ids", "counters"]
+           "hash_idx", "hash_sign", "bucket_off", "bucket_ids", "counters", "proj1", "bucket1_off", "bucket1_ids"]
 T = {n: i for i, n in enumerate(T_NAMES)}
 _T_DTYPE = {"hash_idx": np.int32, "hash_sign": np.int32, "bucket_off": np.int32, "bucket_ids": np.int32,
-            "counters": np.int64}
-LAST_NAMES = ["hidden", "codes", "act_count", "act_ids", "act_logit", "act_prob", "act_err", "loss", "dhidden"]
+            "counters": np.int64, "proj1": np.int8, "bucket1_off": np.int32, "bucket1_ids": np.int32}
+LAST_NAMES = ["hidden", "codes", "act_count", "act_ids", "act_logit", "act_prob", "act_err", "loss", "dhidden",
+              "codes1", "hidden_mask"]
 LAST = {n: i for i, n in enumerate(LAST_NAMES)}
-_LAST_DTYPE = {"codes": np.uint32, "act_count": np.int32, "act_ids": np.int32}
+_LAST_DTYPE = {"codes": np.uint32, "act_count": np.int32, "act_ids": np.int32, "codes1": np.uint32, "hidden_mask": np.uint32}
 
 
 class Config(C.Structure):
@@ -43,7 +44,7 @@ class Config(C.Structure):
         ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
         ("init_std", C.c_float), ("seed", C.c_uint64), ("device", C.c_int32), ("dedup_mode", C.c_int32),
         ("stream", C.c_void_p), ("dwta_densify", C.c_int32), ("sample_budget", C.c_int32), ("budget_fill", C.c_int32),
-        ("inputs_ready", C.c_int32),
+        ("inputs_ready", C.c_int32), ("hidden_K", C.c_int32), ("hidden_L", C.c_int32), ("hidden_cap", C.c_int32),
     ]
 
 
@@ -102,14 +103,14 @@ def make_config(*, input_dim, hidden_dim, output_dim, hash_family=DWTA, K=6, L=5
                 bucket_cap=128, rebuild_period0=50, rebuild_growth_lambda=0.0, redraw_hash_fns=1, force_dense=0,
                 max_batch=256, max_labels=16, max_active_per_sample=0, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8,
                 init_std=0.01, seed=0, device=0, dedup_mode=0, stream=None, dwta_densify=0, sample_budget=0, budget_fill=0,
-                inputs_ready=0):
+                inputs_ready=0, hidden_K=0, hidden_L=0, hidden_cap=0):
     if stream is None:
         import torch
         stream = torch.cuda.current_stream(device).cuda_stream
     return Config(input_dim, hidden_dim, output_dim, hash_family, K, L, dwta_bin_size, srp_nnz, bucket_cap,
                   rebuild_period0, rebuild_growth_lambda, redraw_hash_fns, force_dense, max_batch, max_labels,
                   max_active_per_sample, lr, beta1, beta2, eps, init_std, seed, device, dedup_mode, stream, dwta_densify, sample_budget, budget_fill,
-                  inputs_ready)
+                  inputs_ready, hidden_K, hidden_L, hidden_cap)
 
 
 # ---- the C entry points, same names ---------------------------------------------------------
@@ -172,7 +173,7 @@ def dslide_sync(ctx, check=True):
     return s
 
 
-_DT = [np.float32, np.int32, np.int64]       # DSLIDE_DT_*
+_DT = [np.float32, np.int32, np.int64, np.int8]       # DSLIDE_DT_*
 
 
 def dslide_get_tensor(ctx, name):

@@ -63,7 +63,7 @@ void free_all(Ctx* c) {
   void* ptrs[] = {c->W1, c->b1, c->W2, c->hdr1, c->hdr2, c->mW1, c->vW1, c->mb1, c->vb1, c->mW2, c->vW2,
                   c->hash_idx, c->hash_sign, c->bucket_off, c->bucket_ids, c->h, c->dh, c->loss, c->codes,
                   c->act_cnt, c->act_ids, c->act_z, c->act_p, c->act_g, c->mask1, c->ovf1, c->ovf2, c->hotmap1, c->hotcoef1,
-                  c->mask2, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
+                  c->mask2, c->proj1, c->bucket1_off, c->bucket1_ids, c->codes1n, c->codes1, c->hmask, c->cmask1, c->own1, c->own2, c->hot_rows, c->med_rows, c->hot_part, c->hot_done, c->dstate, c->keysA, c->keysB, c->valsA, c->valsB, c->tile_hist, c->bucket_part, c->ord_mid, c->ord_big, c->ord_cnt,
                   c->st_dev[0], c->st_dev[1], c->st_dev[2], c->pd_part};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (int b = 0; b < ST_SETS; ++b) {
@@ -108,6 +108,9 @@ TensorRef tensor_ref(Ctx* c, int which) {
     case DSLIDE_T_BUCKET_OFF: return {c->bucket_off, (int64_t)c->L * (c->nb + 1) * 4};
     case DSLIDE_T_BUCKET_IDS: return {c->bucket_ids, (int64_t)c->L * N * 4};
     case DSLIDE_T_COUNTERS: return {nullptr, 3 * 8};
+    case DSLIDE_T_PROJ1: return {c->proj1, c->L1 > 0 ? D * c->KL1 : 0};
+    case DSLIDE_T_BUCKET1_OFF: return {c->bucket1_off, c->L1 > 0 ? (int64_t)c->L1 * (((int64_t)1 << c->K1) + 1) * 4 : 0};
+    case DSLIDE_T_BUCKET1_IDS: return {c->bucket1_ids, c->L1 > 0 ? (int64_t)c->L1 * H * 4 : 0};
   }
   return {nullptr, -1};
 }
@@ -120,9 +123,13 @@ dslide_status drain(Ctx* c) {
 dslide_status rebuild(Ctx* c, bool bump) {
   if (bump) {
     c->r_host += 1;
-    if (c->cfg.redraw_hash_fns) CU(launch_draw_hash(c, c->r_host));
+    if (c->cfg.redraw_hash_fns) {
+      if (!c->dense) CU(launch_draw_hash(c, c->r_host));
+      CU(launch_draw_proj1(c, c->r_host));
+    }
   }
   if (!c->dense) CU(launch_build_tables(c));
+  CU(launch_build_tables1(c));        // the hidden layer's tables, when it is LSH-sampled
   return DSLIDE_OK;
 }
 
@@ -158,6 +165,8 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   if (k.rebuild_period0 < 0 || k.init_std < 0.f || k.dedup_mode < 0 || k.dedup_mode > 2) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_densify < 0 || k.dwta_densify > 1 || k.sample_budget < 0) return DSLIDE_ERR_INVALID_ARG;
   if (k.budget_fill < 0 || k.budget_fill > 1 || k.inputs_ready < 0 || k.inputs_ready > 1) return DSLIDE_ERR_INVALID_ARG;
+  if (k.hidden_L < 0 || k.hidden_L > 64) return DSLIDE_ERR_INVALID_ARG;
+  if (k.hidden_L > 0 && (k.hidden_K < 1 || k.hidden_K > 16 || k.hidden_K * k.hidden_L > 256 || k.hidden_cap < 1)) return DSLIDE_ERR_INVALID_ARG;
   if (k.budget_fill && (k.sample_budget < 1 || k.max_active_per_sample != 0 || k.force_dense)) return DSLIDE_ERR_INVALID_ARG;
   if (k.dwta_bin_size == 0) k.dwta_bin_size = 8;
   if (k.srp_nnz == 0) k.srp_nnz = (k.hidden_dim + 2) / 3;
@@ -197,6 +206,8 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   c->nb = (int64_t)1 << bits;
   c->act_stride = (int)act_stride;
   c->Wd = (k.max_batch + 31) / 32;
+  c->L1 = k.hidden_L; c->K1 = k.hidden_L > 0 ? k.hidden_K : 0; c->KL1 = c->K1 * c->L1; c->cap1 = k.hidden_cap;
+  c->Hw = (k.hidden_dim + 31) / 32;
   c->dense = k.force_dense ? 1 : 0;
   c->stream = (cudaStream_t)k.stream;
   c->next_rebuild = k.rebuild_period0;
@@ -225,6 +236,12 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   A(dstate, 1, true);
   A(hotmap1, D, false); A(hotcoef1, (size_t)HOTMAP_CAP * B, false);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->hotmap1, 0xff, D * sizeof(int32_t), st);
+  if (c->L1 > 0) {
+    A(proj1, D * (size_t)c->KL1, true);
+    A(bucket1_off, (size_t)c->L1 * (((size_t)1 << c->K1) + 1), true); A(bucket1_ids, (size_t)c->L1 * H, true);
+    A(codes1n, (size_t)c->L1 * H + ((size_t)c->KL1 * H + 3) / 4 + 1, true);     // codes, then one byte per (projection, neuron)
+    A(codes1, B * (size_t)c->L1, true); A(hmask, B * (size_t)c->Hw, true); A(cmask1, D * (size_t)c->Hw, true);
+  }
   if (!c->dense) {
     A(act_ids, B * S, true);
     A(mask2, N * c->Wd, true);
@@ -262,6 +279,8 @@ dslide_status dslide_init(const dslide_config* cfg, dslide_ctx** out) {
   if (e == cudaSuccess) e = launch_init_gauss(c, c->W2, (int64_t)(N * H), RNG_W2);
   if (e == cudaSuccess && !c->dense) e = launch_draw_hash(c, 0);
   if (e == cudaSuccess && !c->dense) e = launch_build_tables(c);
+  if (e == cudaSuccess) e = launch_draw_proj1(c, 0);
+  if (e == cudaSuccess) e = launch_build_tables1(c);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
     dslide_status s = e == cudaErrorMemoryAllocation ? DSLIDE_ERR_OOM
@@ -494,7 +513,9 @@ dslide_status dslide_tensor_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes
   *nbytes = t.bytes;
   if (dtype)
     *dtype = which == DSLIDE_T_COUNTERS ? DSLIDE_DT_I64
-             : (which >= DSLIDE_T_HASH_IDX && which <= DSLIDE_T_BUCKET_IDS) ? DSLIDE_DT_I32 : DSLIDE_DT_F32;
+             : which == DSLIDE_T_PROJ1 ? DSLIDE_DT_I8
+             : ((which >= DSLIDE_T_HASH_IDX && which <= DSLIDE_T_BUCKET_IDS) || which == DSLIDE_T_BUCKET1_OFF ||
+                which == DSLIDE_T_BUCKET1_IDS) ? DSLIDE_DT_I32 : DSLIDE_DT_F32;
   return DSLIDE_OK;
 }
 
@@ -548,7 +569,13 @@ dslide_status dslide_set_tensor(dslide_ctx* ctx, int32_t which, const void* host
     for (int64_t i = 0; i < want / 4; ++i)
       if (ix[i] < 0 || ix[i] >= c->H) return DSLIDE_ERR_INVALID_ARG;
   }
-  if (which == DSLIDE_T_BUCKET_OFF || which == DSLIDE_T_BUCKET_IDS) return DSLIDE_ERR_INVALID_ARG;  // derived state
+  if (which == DSLIDE_T_BUCKET_OFF || which == DSLIDE_T_BUCKET_IDS || which == DSLIDE_T_BUCKET1_OFF ||
+      which == DSLIDE_T_BUCKET1_IDS) return DSLIDE_ERR_INVALID_ARG;  // derived state
+  if (which == DSLIDE_T_PROJ1) {
+    const signed char* e = (const signed char*)host_src;
+    for (int64_t i = 0; i < want; ++i)
+      if (e[i] < -1 || e[i] > 1) return DSLIDE_ERR_INVALID_ARG;
+  }
   if (want == 0) return DSLIDE_OK;
   const TensorRef tr = tensor_ref(c, which);
   if (tr.pitch) CU(cudaMemcpy2DAsync(tr.ptr, (size_t)tr.pitch, host_src, sizeof(float), sizeof(float), (size_t)want / sizeof(float),
@@ -568,6 +595,8 @@ dslide_status dslide_last_info(dslide_ctx* ctx, int32_t which, int64_t* nbytes, 
     case DSLIDE_LAST_ACT_COUNT: case DSLIDE_LAST_LOSS: *nbytes = B * 4; return DSLIDE_OK;
     case DSLIDE_LAST_ACT_IDS: *nbytes = c->dense ? 0 : B * S * 4; return DSLIDE_OK;
     case DSLIDE_LAST_ACT_LOGIT: case DSLIDE_LAST_ACT_PROB: case DSLIDE_LAST_ACT_ERR: *nbytes = B * S * 4; return DSLIDE_OK;
+    case DSLIDE_LAST_CODES1: *nbytes = B * c->L1 * 4; return DSLIDE_OK;
+    case DSLIDE_LAST_HIDDEN_MASK: *nbytes = c->L1 > 0 ? B * c->Hw * 4 : 0; return DSLIDE_OK;
   }
   return DSLIDE_ERR_INVALID_ARG;
 }
@@ -589,6 +618,8 @@ dslide_status dslide_get_last(dslide_ctx* ctx, int32_t which, void* host_dst, in
     case DSLIDE_LAST_ACT_LOGIT: src = c->act_z; break;
     case DSLIDE_LAST_ACT_PROB: src = c->act_p; break;
     case DSLIDE_LAST_ACT_ERR: src = c->act_g; break;
+    case DSLIDE_LAST_CODES1: src = c->codes1; break;
+    case DSLIDE_LAST_HIDDEN_MASK: src = c->hmask; break;
   }
   int64_t n = nbytes < size ? nbytes : size;
   if (n == 0 || !src) return DSLIDE_OK;

@@ -24,7 +24,7 @@ __host__ __device__ inline uint64_t ctr_rng(uint64_t seed, uint64_t stream, uint
   uint64_t b = sm64(a + g * (r + 1));
   return sm64(b + g * (ctr + 1));
 }
-enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2, RNG_PROBE = 3, RNG_SAMPLE = 4, RNG_FILL = 5 };
+enum : uint64_t { RNG_W1 = 0, RNG_W2 = 1, RNG_HASH = 2, RNG_PROBE = 3, RNG_SAMPLE = 4, RNG_FILL = 5, RNG_HASH1 = 6 };
 constexpr int DENSIFY_ATTEMPTS = 16;     // functions an all-zero DWTA bin of a query probes for a position to borrow
 
 // Device-resident step state (read and written by kernels only; the host reads it
@@ -121,6 +121,8 @@ struct LaunchScope {
 cudaError_t launch_init_gauss(Ctx* c, float* w, int64_t n, uint64_t stream_id);
 cudaError_t launch_draw_hash(Ctx* c, int64_t r);
 cudaError_t launch_build_tables(Ctx* c);
+cudaError_t launch_draw_proj1(Ctx* c, int64_t r);   // the hidden layer's projections of rebuild count r
+cudaError_t launch_build_tables1(Ctx* c);           // codes of the hidden neurons and their tables
 cudaError_t launch_order_buckets(Ctx* c, int min_n);
 cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
                                  const float* vals, const int32_t* label_ptr, const int32_t* labels, int inputs_ready);
@@ -148,6 +150,14 @@ struct Ctx {
   RowHdr *hdr1, *hdr2;             // per row of W1 / W2: touch count, slots and (W2) the bias b2 with its moments
   int32_t *hash_idx, *hash_sign;
   int32_t *bucket_off, *bucket_ids;
+  // LSH-sampled hidden layer (hidden_L > 0): projections over the input coordinates, tables over the hidden neurons,
+  // per-step codes and active masks, per row of W1 the hidden units some sample of the step touches it for
+  int K1, L1, KL1, cap1, Hw;       // Hw = 32-bit words of a mask over the hidden units
+  int8_t* proj1;                   // [D][KL1]
+  int32_t *bucket1_off, *bucket1_ids;
+  uint32_t *codes1n;               // [L1][H] codes of the hidden neurons (table build)
+  uint32_t *codes1, *hmask;        // [B][L1], [B][Hw]
+  uint32_t* cmask1;                // [D][Hw]
 
   // per-step work space
   float *h, *dh, *loss;

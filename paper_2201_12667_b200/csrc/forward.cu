@@ -62,6 +62,11 @@ struct FwdParams {
   int hash_sm_off;     // where in the staging region the hash functions' index tables are mirrored (-1: read from global memory)
   int hash_sm_bytes;
   int sort_small;      // candidate sets up to this size are deduplicated by sorting even when a bitmap is available
+  // LSH-sampled hidden layer (L1 > 0): projections over the input coordinates, tables over the hidden neurons
+  const int8_t* proj1;
+  const int32_t *bucket1_off, *bucket1_ids;
+  uint32_t *codes1, *hmask, *cmask1;
+  int K1, L1, KL1, cap1, Hw, off_h1;
   int inputs_ready;    // the batch arrays were complete before the launch: they may be read before griddep_wait()
   int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_tbeg, off_topk, off_ids, off_z, off_col, off_val,
       off_dedup;
@@ -465,6 +470,10 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   float* sh_g = reinterpret_cast<float*>(smem + p.off_topk);         // [ACT_SM] training: errors of a small set (predict: its best-k lists)
   int* sh_col = reinterpret_cast<int*>(smem + p.off_col);            // [hid_rows]
   float* sh_val = reinterpret_cast<float*>(smem + p.off_val);        // [hid_rows]
+  unsigned char* sh_b1 = smem + p.off_h1;                            // [256] bits of the hidden layer's projections
+  int* sh_c1beg = reinterpret_cast<int*>(smem + p.off_h1 + 256);     // [64] start of the slice of every hidden-layer table
+  int* sh_c1cnt = sh_c1beg + 64;                                     // [64] and its length
+  uint32_t* sh_hmask = reinterpret_cast<uint32_t*>(sh_c1cnt + 64);   // [32] active hidden neurons of the sample
   uint32_t* sh_dd = reinterpret_cast<uint32_t*>(smem + p.off_dedup);
   float* stage = reinterpret_cast<float*>(smem + p.off_dedup);       // overlays the dedup work space
 
@@ -516,6 +525,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   //      Up to here, and through the first chunk's column ids and values, only the caller's batch is read: with
   //      inputs_ready the kernel runs that far while the previous step's update kernel is still finishing.
   float acc[KPT];
+  float s1 = 0.f;                    // sampled hidden layer: the input's sum under projection `tid`
   int c1 = 0, line1 = -1;            // this thread's nonzero (tid-th of the sample), kept for the hand-off to the update kernel
   float x1 = 0.f;
   const int R = p.hid_rows;
@@ -554,6 +564,19 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         acc[u] = k < H ? p.b1[k] : 0.f;
       }
     }
+    if (p.L1 > 0 && tid < p.KL1) {
+      // sampled hidden layer: the input's sum under projection `tid`, nonzeros in stored order (coordinates that the
+      // projection does not select add nothing)
+      const int8_t* pj = p.proj1 + tid;
+      for (int i0 = 0; i0 < nr; i0 += 16) {
+        int e[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) e[j] = i0 + j < nr ? (int)__ldg(pj + (size_t)sh_col[i0 + j] * p.KL1) : 0;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (e[j] != 0) s1 = __fadd_rn(s1, e[j] > 0 ? sh_val[i0 + j] : -sh_val[i0 + j]);
+      }
+    }
     cp_async_wait_all();
     __syncthreads();
 #pragma unroll
@@ -582,11 +605,38 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     skip_sample<MODE>(p, s, (!bad && too_many_labels) ? DSLIDE_ERR_OVERFLOW : DSLIDE_ERR_BAD_INDEX);
     return;
   }
+  if (p.L1 > 0) {
+    // ---- sampled hidden layer (Algorithm 1: retrieve the layer's active neurons with the layer's input): codes of
+    //      the input, one bucket slice per table, union as a bit mask over the hidden neurons.  A neuron that is
+    //      not retrieved is a NoOp: activation 0 (Section 2.1) ----
+    if (tid < p.KL1) sh_b1[tid] = s1 >= 0.f ? 1 : 0;
+    if (tid < 32) sh_hmask[tid] = 0u;
+    __syncthreads();
+    if (tid < p.L1) {
+      uint32_t code = 0;
+      for (int k = 0; k < p.K1; ++k) code |= (uint32_t)sh_b1[tid * p.K1 + k] << k;
+      if (MODE == 0) p.codes1[(size_t)s * p.L1 + tid] = code;
+      const int32_t* off = p.bucket1_off + (size_t)tid * ((1 << p.K1) + 1) + code;
+      const int beg = __ldg(off);
+      int cnt = __ldg(off + 1) - beg;
+      sh_c1beg[tid] = beg;
+      sh_c1cnt[tid] = cnt < p.cap1 ? cnt : p.cap1;
+    }
+    __syncthreads();
+    for (int t = warp; t < p.L1; t += FWD_WARPS)
+      for (int i = lane; i < sh_c1cnt[t]; i += 32) {
+        const int k = __ldg(p.bucket1_ids + (size_t)t * H + sh_c1beg[t] + i);
+        atomicOr(&sh_hmask[k >> 5], 1u << (k & 31));
+      }
+    __syncthreads();
+    if (MODE == 0 && tid < p.Hw) p.hmask[(size_t)s * p.Hw + tid] = sh_hmask[tid];
+  }
 #pragma unroll
   for (int u = 0; u < KPT; ++u) {
     const int k = tid + u * FWD_THREADS;
     if (k < H) {
-      const float hv = acc[u] > 0.f ? acc[u] : 0.f;
+      const bool on = p.L1 == 0 || ((sh_hmask[k >> 5] >> (k & 31)) & 1u);
+      const float hv = (on && acc[u] > 0.f) ? acc[u] : 0.f;
       sh_h[k] = hv;
       if (MODE == 0 || p.dense) p.h[(size_t)s * H + k] = hv;
     }
@@ -1210,6 +1260,12 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   //      entries of both lists of distinct rows, and whatever did not fit the registers above ----
   own_store(tid < nnz && nth1 == 0u, base1, p.own1, c1, s);
   if (tid < nnz) list_row(p, &p.hdr1[c1].cnt, ~c1, nth1);
+  if (p.L1 > 0)          // sampled hidden layer: of the rows of W1 the sample touches, only its active neurons' weights
+    for (int i = tid; i < nnz; i += FWD_THREADS) {
+      const int c = i == tid ? c1 : __ldg(p.col_idx + rbeg + i);
+      for (int w = 0; w < p.Hw; ++w)
+        if (sh_hmask[w]) atomicOr(&p.cmask1[(size_t)c * p.Hw + w], sh_hmask[w]);
+    }
   for (int i0 = FWD_THREADS; i0 < nnz; i0 += FWD_THREADS) {
     const int i = i0 + tid;
     const bool live = i < nnz;
@@ -1433,7 +1489,7 @@ static int align128(int x) { return (x + 127) & ~127; }
 
 struct FwdLayout {
   int off_dh, off_code, off_part, off_misc, off_lab, off_tbase, off_tbeg, off_topk, off_ids, off_z, off_col, off_val,
-      off_dedup, fixed_bytes, hid_rows;
+      off_h1, off_dedup, fixed_bytes, hid_rows;
 };
 
 static FwdLayout fwd_layout(const Ctx* c) {
@@ -1456,6 +1512,7 @@ static FwdLayout fwd_layout(const Ctx* c) {
   l.off_z = o;       o = align16(o + ACT_SM * 4);
   l.off_col = o;     o = align16(o + hid_rows * 4);
   l.off_val = o;     o = align16(o + hid_rows * 4);
+  l.off_h1 = o;      o = align16(o + 256 + 64 * 4 * 2 + 32 * 4);     // sampled hidden layer: bits, slice starts and lengths, active mask
   o = align128(o);
   l.off_dedup = o;
   l.fixed_bytes = o;
@@ -1552,6 +1609,10 @@ static FwdParams make_params(Ctx* c, int batch, const int32_t* row_ptr, const in
   p.off_dh = l.off_dh; p.off_code = l.off_code; p.off_part = l.off_part; p.off_misc = l.off_misc;
   p.off_lab = l.off_lab; p.off_tbase = l.off_tbase; p.off_tbeg = l.off_tbeg; p.off_topk = l.off_topk;
   p.off_ids = l.off_ids; p.off_z = l.off_z; p.off_col = l.off_col; p.off_val = l.off_val; p.off_dedup = l.off_dedup;
+  p.off_h1 = l.off_h1;
+  p.proj1 = c->proj1; p.bucket1_off = c->bucket1_off; p.bucket1_ids = c->bucket1_ids;
+  p.codes1 = c->codes1; p.hmask = c->hmask; p.cmask1 = c->cmask1;
+  p.K1 = c->K1; p.L1 = c->L1; p.KL1 = c->KL1; p.cap1 = c->cap1; p.Hw = c->Hw;
   return p;
 }
 

@@ -102,6 +102,114 @@ cudaError_t launch_draw_hash(Ctx* c, int64_t r) {
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ LSH-sampled hidden layer
+// Projections over the D input coordinates (Section 3.6: the hidden layer as a sparse layer; Algorithm 1 retrieves
+// active neurons for every layer): entry (c, p) is +1, -1 or 0 with probability 1/6, 1/6, 2/3, drawn by itself from
+// the counter-based generator.
+__global__ void k_draw_proj1(int8_t* proj, long long n, uint64_t seed, uint64_t r) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long step = (long long)gridDim.x * blockDim.x;
+  for (; i < n; i += step) {
+    const uint64_t u = ctr_rng(seed, RNG_HASH1, r, (uint64_t)i) % 6ull;
+    proj[i] = u == 0 ? 1 : (u == 1 ? -1 : 0);
+  }
+}
+
+cudaError_t launch_draw_proj1(Ctx* c, int64_t r) {
+  if (c->L1 <= 0) return cudaSuccess;
+  LaunchScope ls(c, KID_DRAW_HASH);
+  k_draw_proj1<<<c->num_sms * 8, 256, 0, c->stream>>>(c->proj1, (long long)c->D * c->KL1, c->cfg.seed, (uint64_t)r);
+  return cudaGetLastError();
+}
+
+// Codes of the hidden neurons: neuron k's weight vector is column k of W1.  A thread owns one neuron and H1_PT
+// projections and walks the input coordinates in ascending order (the sums are sequential, like the oracle's): the
+// row of W1 is read coalesced over the neurons, the projections' entries of the coordinate as one broadcast word.
+constexpr int H1_THREADS = 128;
+constexpr int H1_PT = 4;
+__global__ void __launch_bounds__(H1_THREADS)
+k_hash_hidden(const float* __restrict__ W1, const int8_t* __restrict__ proj, unsigned char* bits, int D, int H, int KL1) {
+  const int k = blockIdx.x * H1_THREADS + threadIdx.x;
+  const int p0 = blockIdx.y * H1_PT;
+  float s[H1_PT];
+#pragma unroll
+  for (int q = 0; q < H1_PT; ++q) s[q] = 0.f;
+  const bool live = k < H;
+  const bool vec = (KL1 & 3) == 0;          // p0 is a multiple of 4: the four entries are one aligned word
+  for (int c = 0; c < D; ++c) {
+    const float w = live ? __ldg(W1 + (size_t)c * H + k) : 0.f;
+    int e[H1_PT];
+    if (vec) {
+      const int word = __ldg(reinterpret_cast<const int*>(proj + (size_t)c * KL1 + p0));
+#pragma unroll
+      for (int q = 0; q < H1_PT; ++q) e[q] = (int)(signed char)((word >> (8 * q)) & 0xff);
+    } else {
+#pragma unroll
+      for (int q = 0; q < H1_PT; ++q) e[q] = p0 + q < KL1 ? (int)__ldg(proj + (size_t)c * KL1 + p0 + q) : 0;
+    }
+#pragma unroll
+    for (int q = 0; q < H1_PT; ++q)
+      if (e[q] != 0) s[q] = __fadd_rn(s[q], e[q] > 0 ? w : -w);
+  }
+  if (live)
+#pragma unroll
+    for (int q = 0; q < H1_PT; ++q)
+      if (p0 + q < KL1) bits[(size_t)(p0 + q) * H + k] = s[q] >= 0.f ? 1 : 0;
+}
+
+// One block per table: codes from the bits, bucket sizes, offsets, and every neuron to its bucket's start plus the
+// number of lower-numbered neurons with the same code (ascending ids inside a bucket).  H <= 1024.
+__global__ void __launch_bounds__(1024)
+k_tables1(const unsigned char* bits, uint32_t* codes, int32_t* off, int32_t* ids, int H, int K1) {
+  extern __shared__ int t1_smem[];          // [H] codes, [2^K1 + 1] offsets
+  int* scode = t1_smem;
+  int* soff = t1_smem + H;
+  const int t = blockIdx.x, nb = 1 << K1, tid = threadIdx.x;
+  for (int b = tid; b <= nb; b += blockDim.x) soff[b] = 0;
+  __syncthreads();
+  for (int k = tid; k < H; k += blockDim.x) {
+    int code = 0;
+    for (int q = 0; q < K1; ++q) code |= (int)bits[(size_t)(t * K1 + q) * H + k] << q;
+    scode[k] = code;
+    codes[(size_t)t * H + k] = (uint32_t)code;
+    atomicAdd(&soff[code + 1], 1);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int b = 0; b <= nb; ++b) { run += soff[b]; soff[b] = run; }
+  }
+  __syncthreads();
+  int32_t* o = off + (size_t)t * (nb + 1);
+  for (int b = tid; b <= nb; b += blockDim.x) o[b] = soff[b];
+  for (int k = tid; k < H; k += blockDim.x) {
+    const int code = scode[k];
+    int before = 0;
+    for (int j = 0; j < k; ++j) before += scode[j] == code ? 1 : 0;
+    ids[(size_t)t * H + soff[code] + before] = k;
+  }
+}
+
+cudaError_t launch_build_tables1(Ctx* c) {
+  if (c->L1 <= 0) return cudaSuccess;
+  unsigned char* bits = reinterpret_cast<unsigned char*>(c->codes1n + (size_t)c->L1 * c->H);     // [KL1][H] after the codes
+  {
+    LaunchScope ls(c, KID_HASH_NEURONS);
+    dim3 grid((c->H + H1_THREADS - 1) / H1_THREADS, (c->KL1 + H1_PT - 1) / H1_PT);
+    k_hash_hidden<<<grid, H1_THREADS, 0, c->stream>>>(c->W1, c->proj1, bits, c->D, c->H, c->KL1);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int smem = (c->H + (1 << c->K1) + 1) * (int)sizeof(int);
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(k_tables1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+  }
+  LaunchScope ls(c, KID_BUCKET_SCAN);
+  k_tables1<<<c->L1, 1024, smem, c->stream>>>(bits, c->codes1n, c->bucket1_off, c->bucket1_ids, c->H, c->K1);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ codes of all neurons
 constexpr int HN_ROWS = 32;
 constexpr int HN_THREADS = 256;

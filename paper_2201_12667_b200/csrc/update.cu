@@ -59,6 +59,10 @@ struct UpdParams {
   unsigned int host_seq;
   int B, H, N, D, Wd, act_stride, dense, parity;
   float lr, beta1, beta2, eps, rb1, rb2;
+  // LSH-sampled hidden layer (L1 > 0): per row of W1 the hidden units some sample touches it for; per sample its active units
+  uint32_t* cmask1;
+  const uint32_t* hmask;
+  int L1, Hw;
 };
 
 // One element of Adam.  rb1 = 1 / (1 - beta1^t), rb2 = 1 / (1 - beta2^t).  The square root and the final
@@ -256,21 +260,33 @@ __device__ __forceinline__ void load_row(const float* base, size_t row, int H, i
   }
 }
 
-template <int NCH>
+template <int NCH, bool UMASK = false>      // UMASK: rows of W1 carry a mask of the hidden units to update (sampled hidden layer)
 __device__ __forceinline__ void adam_store(const UpdParams& p, const Side& sd, size_t row, float4 (&w)[NCH],
                                            float4 (&m)[NCH], float4 (&v)[NCH], const float4 (&g)[NCH], int H, int H4,
                                            int lane) {
   float4* w4 = reinterpret_cast<float4*>(sd.W + row * H);
   float4* m4 = reinterpret_cast<float4*>(sd.M + row * H);
   float4* v4 = reinterpret_cast<float4*>(sd.V + row * H);
+  // a row of W1 under a sampled hidden layer: only the units some sample touched the row for are updated (the
+  // others keep weight and moments bit for bit); the row's unit mask is cleared by finish_hdr
+  const uint32_t* um = (UMASK && !sd.is_w2) ? p.cmask1 + row * (size_t)p.Hw : nullptr;
 #pragma unroll
   for (int q = 0; q < NCH; ++q) {
     int c = lane + q * 32;
     if (c < H4) {
-      adam1(w[q].x, m[q].x, v[q].x, g[q].x, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
-      adam1(w[q].y, m[q].y, v[q].y, g[q].y, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
-      adam1(w[q].z, m[q].z, v[q].z, g[q].z, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
-      adam1(w[q].w, m[q].w, v[q].w, g[q].w, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      if (UMASK) {
+        unsigned on = 0xfu;
+        if (um) on = (um[(4 * c) >> 5] >> ((4 * c) & 31)) & 0xfu;
+        if (on & 1u) adam1(w[q].x, m[q].x, v[q].x, g[q].x, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+        if (on & 2u) adam1(w[q].y, m[q].y, v[q].y, g[q].y, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+        if (on & 4u) adam1(w[q].z, m[q].z, v[q].z, g[q].z, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+        if (on & 8u) adam1(w[q].w, m[q].w, v[q].w, g[q].w, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      } else {
+        adam1(w[q].x, m[q].x, v[q].x, g[q].x, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+        adam1(w[q].y, m[q].y, v[q].y, g[q].y, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+        adam1(w[q].z, m[q].z, v[q].z, g[q].z, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+        adam1(w[q].w, m[q].w, v[q].w, g[q].w, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      }
       w4[c] = w[q];
       __stcs(m4 + c, m[q]);      // the moments are not read again before the next update of this row
       __stcs(v4 + c, v[q]);
@@ -299,20 +315,24 @@ __device__ __forceinline__ void finish_hdr(const UpdParams& p, RowHdr* hd, bool 
     adam1(b, mb, vb, g, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
     if (lane == 0) reinterpret_cast<int2*>(hd)[0] = make_int2(0, __float_as_int(b));
     if (lane == 1) reinterpret_cast<int2*>(hd)[1] = make_int2(__float_as_int(mb), __float_as_int(vb));
-  } else if (lane == 0) {
-    hd->cnt = 0u;
+  } else {
+    if (lane == 0) hd->cnt = 0u;
+    if (p.L1 > 0 && lane < p.Hw) p.cmask1[(size_t)(hd - p.hdr1) * p.Hw + lane] = 0u;     // the row's unit mask, for the next step
   }
 }
 
 // The hidden bias (dense gradient, summed over the samples in eight fixed slices) and, in the first
 // of these blocks, the mean loss and the step statistics.
-__device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
+__device__ void aux_block(const UpdParams& p, int a, float* sm_part, unsigned* sm_on) {     // sm_on: UPD_WARPS * 32 words
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = p.H, B = p.B;
   const int k = a * 32 + lane;
   const int per = (B + UPD_WARPS - 1) / UPD_WARPS;
   const int s0 = warp * per, s1 = min(B, s0 + per);
   float g = 0.f;
+  unsigned any_on = p.L1 > 0 ? 0u : 1u;        // sampled hidden layer: was unit k active for any sample?
+  if (k < H && p.L1 > 0)
+    for (int s = s0; s < s1; ++s) any_on |= (p.hmask[(size_t)s * p.Hw + (k >> 5)] >> (k & 31)) & 1u;
   if (k < H) {
     int s = s0;
     for (; s + 8 <= s1; s += 8) {
@@ -325,13 +345,17 @@ __device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
     for (; s < s1; ++s) g += p.dh[(size_t)s * H + k];
   }
   sm_part[warp * 32 + lane] = g;
+  sm_on[warp * 32 + lane] = any_on;
   __syncthreads();
   if (warp == 0 && k < H) {
     float tot = 0.f;
-    for (int w = 0; w < UPD_WARPS; ++w) tot += sm_part[w * 32 + lane];
-    float w = p.b1[k], m = p.mb1[k], v = p.vb1[k];
-    adam1(w, m, v, tot, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
-    p.b1[k] = w; p.mb1[k] = m; p.vb1[k] = v;
+    unsigned on = 0u;
+    for (int w = 0; w < UPD_WARPS; ++w) { tot += sm_part[w * 32 + lane]; on |= sm_on[w * 32 + lane]; }
+    if (on) {
+      float w = p.b1[k], m = p.mb1[k], v = p.vb1[k];
+      adam1(w, m, v, tot, p.beta1, p.beta2, p.lr, p.eps, p.rb1, p.rb2);
+      p.b1[k] = w; p.mb1[k] = m; p.vb1[k] = v;
+    }
   }
   if (a != 0) return;
   __syncthreads();
@@ -368,7 +392,7 @@ __device__ void aux_block(const UpdParams& p, int a, float* sm_part) {
 // One slice of a row touched by many samples: the samples of HOT_SLICES-th of the row's mask words.  The slice
 // sum goes to scratch memory; the warp that completes the row's last slice adds the slices in slice
 // order (so the result does not depend on which warp that is), applies Adam and resets the row's state.
-template <int NCH>
+template <int NCH, bool UMASK>
 __device__ __forceinline__ void hot_item(const UpdParams& p, const int* rowptr, int item, int nwB, int* scr, int H,
                                          int H4, int lane) {
   const int hrow = item / HOT_SLICES, slice = item - hrow * HOT_SLICES;
@@ -423,7 +447,7 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* rowptr, 
     }
     csum += __ldcg(part + (size_t)sl * ld + H);
   }
-  adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
+  adam_store<NCH, UMASK>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
   finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
   if (lane == 0) {
     p.hot_done[hrow] = 0;
@@ -437,7 +461,7 @@ __device__ __forceinline__ void hot_item(const UpdParams& p, const int* rowptr, 
 // A row touched by more than ROW_SLOTS samples that the forward kernel listed: one warp sums it from slots and
 // mask (ascending samples), applies Adam and resets the row's state.  Rows that went on to the hot list are
 // summed in slices instead and skipped here.
-template <int NCH>
+template <int NCH, bool UMASK>
 __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowptr, int idx, int nwB, int* scr, int H,
                                             int H4, int lane) {
   const int code = p.med_rows[idx];
@@ -478,7 +502,7 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowpt
   } else {
     sum_masked<NCH>(p, sd, rowptr, row, sl.x, 0, nwB, scr, acc, csum, H, H4, lane);
   }
-  adam_store<NCH>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
+  adam_store<NCH, UMASK>(p, sd, (size_t)row, w, m, v, acc, H, H4, lane);
   finish_hdr(p, sd.hdr + row, w2, hv, csum, lane);
 }
 
@@ -486,7 +510,7 @@ __device__ __forceinline__ void medium_item(const UpdParams& p, const int* rowpt
 // the listed rows with more than ROW_SLOTS touches, then the ordinary rows, UPD_TROWS per ticket (small tickets keep the tail of the kernel short).
 constexpr int UPD_TROWS = 4;
 
-template <int NCH, int G>
+template <int NCH, int G, bool UMASK>
 __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1))) k_update(const UpdParams p) {
   extern __shared__ __align__(16) unsigned char upd_smem[];
   const int* rowptr = p.row_ptr;      // the batch's row offsets (read through the read-only path where needed)
@@ -500,7 +524,7 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
   // written by the forward kernel before it
   griddep_launch_dependents();
   griddep_wait();
-  if ((int)blockIdx.x < naux) { aux_block(p, (int)blockIdx.x, sm_part); return; }
+  if ((int)blockIdx.x < naux) { aux_block(p, (int)blockIdx.x, sm_part, reinterpret_cast<unsigned*>(&scratch[0][0])); return; }
 
 
   const int n2 = p.dense ? 0 : (int)p.st->n_own[p.parity][0];
@@ -530,8 +554,8 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
   for (;; cur = nxt, nxt = __shfl_sync(FULL, fut, 0), fut = (lane == 0 && nxt < n_tickets) ? 2 * nwarps + (int)atomicAdd(ticket, 1u) : fut) {
     const int t = cur;
     if (t >= n_tickets) break;
-    if (t < n_hot_items) { hot_item<NCH>(p, rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
-    if (t < n_hot_items + n_med) { medium_item<NCH>(p, rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
+    if (t < n_hot_items) { hot_item<NCH, UMASK>(p, rowptr, t, nwB, scratch[warp], H, H4, lane); continue; }
+    if (t < n_hot_items + n_med) { medium_item<NCH, UMASK>(p, rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
 
     // ---- ordinary rows: consecutive entries of the concatenated lists (rows of W2, then rows of W1) ----
     const int k = t - n_hot_items - n_med;
@@ -594,7 +618,7 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
           } else {      // more touches than slots, yet not listed (the list was full)
             sum_masked<NCH>(p, sd, rowptr, rr[q], sl[q].x, 0, nwB, scratch[warp], acc, csum, H, H4, lane);
           }
-          adam_store<NCH>(p, sd, (size_t)rr[q], w[q], m[q], v[q], acc, H, H4, lane);
+          adam_store<NCH, UMASK>(p, sd, (size_t)rr[q], w[q], m[q], v[q], acc, H, H4, lane);
           finish_hdr(p, sd.hdr + rr[q], w2[q], hv[q], csum, lane);
         }
     }
@@ -628,25 +652,25 @@ __global__ void __launch_bounds__(UPD_THREADS) k_adam_dense(const UpdParams p) {
   }
 }
 
-template <int NCH, int G>
+template <int NCH, int G, bool UMASK>
 static cudaError_t launch_k_update(Ctx* c, const UpdParams& p, int smem) {
   cudaError_t e = cudaSuccess;
   if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(k_update<NCH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(k_update<NCH, G, UMASK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
   // the kernel needs little shared memory: the rest of the unified store serves as cache for the h / dh rows
-  e = cudaFuncSetAttribute(k_update<NCH, G>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxL1);
+  e = cudaFuncSetAttribute(k_update<NCH, G, UMASK>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxL1);
   if (e != cudaSuccess) return e;
   // one wave: the blocks for the hidden bias come first, the rest fill the remaining block slots of the device
   const int naux = (c->H + 31) / 32;
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_update<NCH, G>, UPD_THREADS, smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_update<NCH, G, UMASK>, UPD_THREADS, smem);
   if (e != cudaSuccess) return e;
   int nblocks = c->num_sms * (per_sm > 0 ? per_sm : 1);
   if (nblocks < naux + 1) nblocks = naux + 1;
   LaunchScope ls(c, KID_ADAM);
-  e = launch_dependent(k_update<NCH, G>, dim3(nblocks), dim3(UPD_THREADS), (size_t)smem, c->stream, p);
+  e = launch_dependent(k_update<NCH, G, UMASK>, dim3(nblocks), dim3(UPD_THREADS), (size_t)smem, c->stream, p);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
@@ -665,6 +689,7 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   p.st = c->dstate; p.loss_out = loss_out; p.host_res = host_res; p.host_seq = host_seq;
   p.B = batch; p.H = c->H; p.N = c->N; p.D = c->D; p.Wd = c->Wd; p.act_stride = c->act_stride; p.dense = c->dense;
   p.parity = (int)(c->t_host & 1);
+  p.cmask1 = c->cmask1; p.hmask = c->hmask; p.L1 = c->L1; p.Hw = c->Hw;
   p.lr = c->cfg.lr; p.beta1 = c->cfg.beta1; p.beta2 = c->cfg.beta2; p.eps = c->cfg.eps;
   // reciprocal bias corrections of Adam with the global step count (the step being taken is t + 1)
   const double t = (double)(c->t_host + 1);
@@ -679,10 +704,16 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
   }
   const int smem = UPD_WARPS * 32 * 4;
   const int nch = (c->H / 4 + 31) / 32;
-  if (nch <= 1) return launch_k_update<1, 2>(c, p, smem);
-  if (nch <= 2) return launch_k_update<2, 2>(c, p, smem);
-  if (nch <= 4) return launch_k_update<4, 1>(c, p, smem);
-  return launch_k_update<8, 1>(c, p, smem);
+  if (c->L1 > 0) {        // sampled hidden layer: rows of W1 are updated under their unit masks
+    if (nch <= 1) return launch_k_update<1, 2, true>(c, p, smem);
+    if (nch <= 2) return launch_k_update<2, 2, true>(c, p, smem);
+    if (nch <= 4) return launch_k_update<4, 1, true>(c, p, smem);
+    return launch_k_update<8, 1, true>(c, p, smem);
+  }
+  if (nch <= 1) return launch_k_update<1, 2, false>(c, p, smem);
+  if (nch <= 2) return launch_k_update<2, 2, false>(c, p, smem);
+  if (nch <= 4) return launch_k_update<4, 1, false>(c, p, smem);
+  return launch_k_update<8, 1, false>(c, p, smem);
 }
 
 }  // namespace dslide

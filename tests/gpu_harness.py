@@ -19,18 +19,19 @@ class Pair:
     def __init__(self, D, H, N, family, K, L, bucket_cap, max_batch, bin_size=8, srp_nnz=0, max_labels=16,
                  rebuild_period0=0, rebuild_lambda=0.0, redraw=1, force_dense=0, max_active=0, lr=1e-3,
                  init_std=0.05, seed=0, dedup_mode=0, sync_weights=True, densify=0, budget=0, budget_fill=0,
-                 inputs_ready=0, oracle_build="float"):
+                 inputs_ready=0, oracle_build="float", hidden_K=0, hidden_L=0, hidden_cap=0):
         self.o = Oracle(oracle_build, D=D, H=H, N=N, family=family, K=K, L=L, bin_size=bin_size, srp_nnz=srp_nnz,
                         bucket_cap=bucket_cap, rebuild_period0=rebuild_period0, rebuild_lambda=rebuild_lambda,
                         redraw=redraw, force_dense=force_dense, max_active=max_active, lr=lr, init_std=init_std,
-                        seed=seed, densify=densify, budget=budget, budget_fill=budget_fill)
+                        seed=seed, densify=densify, budget=budget, budget_fill=budget_fill, hidden_K=hidden_K,
+                        hidden_L=hidden_L, hidden_cap=hidden_cap)
         self.cfg = ds.make_config(input_dim=D, hidden_dim=H, output_dim=N, hash_family=family, K=K, L=L,
                                   dwta_bin_size=bin_size, srp_nnz=srp_nnz, bucket_cap=bucket_cap,
                                   rebuild_period0=rebuild_period0, rebuild_growth_lambda=rebuild_lambda,
                                   redraw_hash_fns=redraw, force_dense=force_dense, max_batch=max_batch,
                                   max_labels=max_labels, max_active_per_sample=max_active, lr=lr, init_std=init_std,
                                   seed=seed, dedup_mode=dedup_mode, dwta_densify=densify, sample_budget=budget, budget_fill=budget_fill,
-                                  inputs_ready=inputs_ready)
+                                  inputs_ready=inputs_ready, hidden_K=hidden_K, hidden_L=hidden_L, hidden_cap=hidden_cap)
         self.ctx = ds.dslide_init(self.cfg)
         self.D, self.H, self.N, self.L, self.K = D, H, N, L, K
         self.dense = bool(force_dense)
@@ -52,6 +53,8 @@ class Pair:
             ds.dslide_set_tensor(self.ctx, "hash_idx", self.o.view("hash_idx"))
             if len(self.o.view("hash_sign")):
                 ds.dslide_set_tensor(self.ctx, "hash_sign", self.o.view("hash_sign"))
+        if len(self.o.view("proj1")):
+            ds.dslide_set_tensor(self.ctx, "proj1", self.o.view("proj1"))
         if counters:
             ds.dslide_set_tensor(self.ctx, "counters", np.array([self.o.t, self.o.r, self.o.next_rebuild], dtype=np.int64))
         ds.dslide_build_tables(self.ctx)
