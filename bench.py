@@ -81,6 +81,7 @@ def parse_args(argv=None):
     ap.add_argument("--rebuild-period", type=int, default=REBUILD_PERIOD)
     ap.add_argument("--rebuild-lambda", type=float, default=0.0, help="later gaps grow by exp(lambda * rebuilds)")
     ap.add_argument("--budget", type=int, default=0, help="sampling budget per sample (Section 3.7); 0 = none, as in the headline")
+    ap.add_argument("--hidden-lsh", default="", help="K,L,cap: sample the hidden layer too (tables over the hidden neurons); default dense")
     ap.add_argument("--sweep", action="store_true",
                     help="batch 64..2048 x active fraction 0.05%%..100%% on the 670K shape: one JSON line per cell")
     ap.add_argument("--sweep-batches", default="", help="comma-separated subset of the sweep's batch sizes")
@@ -294,6 +295,7 @@ def shard_seed(rank):
 def oracle_kwargs(c, **kw):
     d = dict(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"], L=c["L"], bin_size=c["bin_size"],
              bucket_cap=c["bucket_cap"], lr=c["lr"], seed=0, init_std=0.01, force_dense=int(bool(c.get("force_dense"))))
+    d.update(c.get("hidden_lsh", {}))
     d.update(kw)
     return d
 
@@ -335,7 +337,7 @@ def workload_config(c, B, args, nb):
     return {"workload": "%s-class shape: D %d, H %d, N %d, %s, batch %d, ~%d nnz/row Zipf(1.1), "
                         "~%d labels/sample" % (c["name"], c["D"], c["H"], c["N"], what, B, c["mean_nnz"], c["mean_labels"]),
             "batch": B, "rebuild_every": args.rebuild_period, "rebuild_lambda": args.rebuild_lambda,
-            "distinct_batches": nb, "sampling_budget": args.budget,
+            "distinct_batches": nb, "sampling_budget": args.budget, "hidden_lsh": args.hidden_lsh or "dense hidden layer",
             "l2": "inputs larger than L2: the model state is far larger than L2 and every step reads a different batch "
                   "(different rows)"}
 
@@ -380,8 +382,15 @@ def cpu_baseline(c, args, B):
     return out
 
 
+def hidden_lsh(args):
+    if not args.hidden_lsh:
+        return {}
+    k, l, cap = (int(x) for x in args.hidden_lsh.split(","))
+    return dict(hidden_K=k, hidden_L=l, hidden_cap=cap)
+
+
 def make_ctx_config(ds, c, args, B, local):
-    return ds.make_config(input_dim=c["D"], hidden_dim=c["H"], output_dim=c["N"], hash_family=c["family"], K=c["K"],
+    return ds.make_config(**hidden_lsh(args), input_dim=c["D"], hidden_dim=c["H"], output_dim=c["N"], hash_family=c["family"], K=c["K"],
                           L=c["L"], dwta_bin_size=c["bin_size"], bucket_cap=c["bucket_cap"],
                           rebuild_period0=args.rebuild_period, rebuild_growth_lambda=args.rebuild_lambda, redraw_hash_fns=1,
                           force_dense=int(bool(c.get("force_dense"))),
@@ -574,6 +583,7 @@ def run_dslide(args):
             run_sweep(args, world, rank, local)
         else:
             c = workloads.config(args.config)
+            c["hidden_lsh"] = hidden_lsh(args)
             B = args.batch_size or c["batch"]
             out = measure(args, c, B, world, rank, local, max(1, args.windows), not args.no_e2e,
                           world == 1 and not args.no_cpu_baseline, sampler)

@@ -122,39 +122,72 @@ cudaError_t launch_draw_proj1(Ctx* c, int64_t r) {
   return cudaGetLastError();
 }
 
-// Codes of the hidden neurons: neuron k's weight vector is column k of W1.  A thread owns one neuron and H1_PT
-// projections and walks the input coordinates in ascending order (the sums are sequential, like the oracle's): the
-// row of W1 is read coalesced over the neurons, the projections' entries of the coordinate as one broadcast word.
+// Codes of the hidden neurons: neuron k's weight vector is column k of W1.  A block owns 32 neurons (the lanes) and
+// 16 projections (four per warp) and walks the input coordinates in ascending order, because the sums are sequential
+// like the oracle's.  Tiles of H1_CT coordinates pass through shared memory: the 128-byte pieces of the rows of W1
+// by cp.async, two tiles deep; the projections' entries as floats (+1, -1, 0), so that one fused multiply-add per
+// (coordinate, projection) adds +w, -w or nothing -- fma(+-1, w, s) rounds like s +- w, and fma(0, w, s) is s.
 constexpr int H1_THREADS = 128;
-constexpr int H1_PT = 4;
+constexpr int H1_CT = 128;        // coordinates per tile
+constexpr int H1_PB = 16;         // projections per block
 __global__ void __launch_bounds__(H1_THREADS)
 k_hash_hidden(const float* __restrict__ W1, const int8_t* __restrict__ proj, unsigned char* bits, int D, int H, int KL1) {
-  const int k = blockIdx.x * H1_THREADS + threadIdx.x;
-  const int p0 = blockIdx.y * H1_PT;
-  float s[H1_PT];
-#pragma unroll
-  for (int q = 0; q < H1_PT; ++q) s[q] = 0.f;
-  const bool live = k < H;
-  const bool vec = (KL1 & 3) == 0;          // p0 is a multiple of 4: the four entries are one aligned word
-  for (int c = 0; c < D; ++c) {
-    const float w = live ? __ldg(W1 + (size_t)c * H + k) : 0.f;
-    int e[H1_PT];
-    if (vec) {
-      const int word = __ldg(reinterpret_cast<const int*>(proj + (size_t)c * KL1 + p0));
-#pragma unroll
-      for (int q = 0; q < H1_PT; ++q) e[q] = (int)(signed char)((word >> (8 * q)) & 0xff);
-    } else {
-#pragma unroll
-      for (int q = 0; q < H1_PT; ++q) e[q] = p0 + q < KL1 ? (int)__ldg(proj + (size_t)c * KL1 + p0 + q) : 0;
+  __shared__ __align__(16) float tw[2][H1_CT][32];
+  __shared__ __align__(16) float tf[2][H1_CT][H1_PB];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int k0 = blockIdx.x * 32, p0 = blockIdx.y * H1_PB;
+  const int ntiles = (D + H1_CT - 1) / H1_CT;
+  auto load_w = [&](int stage, int t) {        // 128 rows x 8 pieces of 16 bytes
+    const int c0 = t * H1_CT;
+    for (int e = tid; e < H1_CT * 8; e += H1_THREADS) {
+      const int row = e >> 3, piece = e & 7;
+      if (c0 + row < D && k0 + 4 * piece < H)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(&tw[stage][row][4 * piece])),
+                     "l"(W1 + (size_t)(c0 + row) * H + k0 + 4 * piece) : "memory");
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  // the projections' entries of a tile: thread = coordinate, 16 bytes each, held in registers until the tile's turn
+  signed char pe[H1_PB];
+  auto load_p = [&](int t) {
+    const int c = t * H1_CT + tid;
 #pragma unroll
-    for (int q = 0; q < H1_PT; ++q)
-      if (e[q] != 0) s[q] = __fadd_rn(s[q], e[q] > 0 ? w : -w);
+    for (int q = 0; q < H1_PB; ++q) pe[q] = (c < D && p0 + q < KL1) ? (signed char)__ldg(proj + (size_t)c * KL1 + p0 + q) : (signed char)0;
+  };
+  float s[4] = {0.f, 0.f, 0.f, 0.f};
+  load_w(0, 0);
+  load_p(0);
+  for (int t = 0; t < ntiles; ++t) {
+    const int st = t & 1;
+#pragma unroll
+    for (int q = 0; q < H1_PB; ++q) tf[st][tid][q] = (float)pe[q];
+    if (t + 1 < ntiles) {
+      load_w(st ^ 1, t + 1);
+      load_p(t + 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    const int nc = min(H1_CT, D - t * H1_CT);
+#pragma unroll 8
+    for (int c = 0; c < nc; ++c) {
+      const float w = tw[st][c][lane];
+      const float4 e = *reinterpret_cast<const float4*>(&tf[st][c][4 * warp]);
+      s[0] = __fmaf_rn(e.x, w, s[0]);
+      s[1] = __fmaf_rn(e.y, w, s[1]);
+      s[2] = __fmaf_rn(e.z, w, s[2]);
+      s[3] = __fmaf_rn(e.w, w, s[3]);
+    }
+    __syncthreads();
   }
-  if (live)
+  const int k = k0 + lane;
+  if (k < H)
 #pragma unroll
-    for (int q = 0; q < H1_PT; ++q)
-      if (p0 + q < KL1) bits[(size_t)(p0 + q) * H + k] = s[q] >= 0.f ? 1 : 0;
+    for (int q = 0; q < 4; ++q) {
+      const int p = p0 + 4 * warp + q;
+      if (p < KL1) bits[(size_t)p * H + k] = s[q] >= 0.f ? 1 : 0;
+    }
 }
 
 // One block per table: codes from the bits, bucket sizes, offsets, and every neuron to its bucket's start plus the
@@ -195,7 +228,7 @@ cudaError_t launch_build_tables1(Ctx* c) {
   unsigned char* bits = reinterpret_cast<unsigned char*>(c->codes1n + (size_t)c->L1 * c->H);     // [KL1][H] after the codes
   {
     LaunchScope ls(c, KID_HASH_NEURONS);
-    dim3 grid((c->H + H1_THREADS - 1) / H1_THREADS, (c->KL1 + H1_PT - 1) / H1_PT);
+    dim3 grid((c->H + 31) / 32, (c->KL1 + H1_PB - 1) / H1_PB);
     k_hash_hidden<<<grid, H1_THREADS, 0, c->stream>>>(c->W1, c->proj1, bits, c->D, c->H, c->KL1);
   }
   cudaError_t e = cudaGetLastError();

@@ -41,14 +41,16 @@ def precision_at_1(ctx, batch, dense):
     return float((ids.cpu().numpy() == batch[4]).mean())
 
 
-@pytest.mark.parametrize("family,K,L", [(ds.DWTA if torch.cuda.is_available() else 1, 2, 24), (0, 4, 24)])
-def test_precision_rises_on_planted_data(family, K, L):
+@pytest.mark.parametrize("family,K,L,hidden", [(1, 2, 24, None), (0, 4, 24, None),
+                                                (1, 2, 24, dict(hidden_K=2, hidden_L=10, hidden_cap=32))])
+def test_precision_rises_on_planted_data(family, K, L, hidden):
+    """The third case samples the hidden layer too (tables over the hidden neurons, queried with the sparse input)."""
     D, H, N, B = 1000, 64, 1000, 128
     rng = np.random.default_rng(0)
     proto = [rng.choice(D, size=6, replace=False) for _ in range(N)]
     cfg = ds.make_config(input_dim=D, hidden_dim=H, output_dim=N, hash_family=family, K=K, L=L, bucket_cap=64,
                          rebuild_period0=25, rebuild_growth_lambda=0.05, redraw_hash_fns=1, max_batch=B, max_labels=2,
-                         lr=5e-3, init_std=0.05, seed=3)
+                         lr=5e-3, init_std=0.05, seed=3, **(hidden or {}))
     ctx = ds.dslide_init(cfg)
     try:
         test = planted_batch(np.random.default_rng(1), B, D, N, proto)
@@ -61,7 +63,7 @@ def test_precision_rises_on_planted_data(family, K, L):
         assert ds.dslide_get_tensor(ctx, "counters")[1] >= 8            # the schedule rebuilt the tables many times
         assert before < 0.03                                             # chance is 1 / 1000
         assert np.mean(losses[-20:]) < 0.7 * np.mean(losses[:20]), (np.mean(losses[:20]), np.mean(losses[-20:]))
-        assert after_dense > 0.5, (before, after_dense, after_lsh)
-        assert after_lsh > 0.3, (before, after_dense, after_lsh)        # retrieval through the tables finds the class too
+        assert after_dense > (0.5 if hidden is None else 0.3), (before, after_dense, after_lsh)
+        assert after_lsh > (0.3 if hidden is None else 0.2), (before, after_dense, after_lsh)   # retrieval through the tables finds the class too
     finally:
         ds.dslide_destroy(ctx)
