@@ -248,6 +248,7 @@ constexpr int HN_ROWS = 32;
 constexpr int HN_THREADS = 256;
 constexpr int HN_WARPS = HN_THREADS / 32;
 constexpr int HN_FN_SMEM_MAX = 96 * 1024;    // hash-function tables larger than this stay in global memory
+constexpr size_t COUNT_SPLIT_BYTES = (size_t)64 << 20;   // bucket counters beyond this are counted table by table
 
 // A block stages HN_ROWS rows of W2 in shared memory (padded, so that 32 threads reading the same
 // column of 32 different rows hit 32 banks) and evaluates the L codes of each row: lane = row, the
@@ -259,7 +260,7 @@ template <bool FN_SMEM>
 __global__ void __launch_bounds__(HN_THREADS)
 k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, const int32_t* __restrict__ hsign,
                uint32_t* keys, uint32_t* ranks, int32_t* counts, int N, int H, int K, int L, int family, int lg_bin,
-               int fn_len, long long nb) {
+               int fn_len, long long nb) {      // counts == nullptr: codes only (k_count_ranks counts afterwards)
   extern __shared__ __align__(16) unsigned char hn_smem[];
   float* tile = reinterpret_cast<float*>(hn_smem);                    // [HN_ROWS][H + 1]
   const int ld = H + 1;
@@ -349,9 +350,11 @@ k_hash_neurons(const float* __restrict__ W2, const int32_t* __restrict__ hidx, c
           }
         }
         keys[(size_t)t * N + j0 + lane] = code;
-        int32_t* cnt = counts + (size_t)t * (size_t)(nb + 1) + code + 1;
-        if (ranks) ranks[(size_t)t * N + j0 + lane] = (uint32_t)atomicAdd(cnt, 1);
-        else atomicAdd(cnt, 1);
+        if (counts) {
+          int32_t* cnt = counts + (size_t)t * (size_t)(nb + 1) + code + 1;
+          if (ranks) ranks[(size_t)t * N + j0 + lane] = (uint32_t)atomicAdd(cnt, 1);
+          else atomicAdd(cnt, 1);
+        }
       }
     }
   }
@@ -430,6 +433,10 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
           if (pend1) ranks[pidx + 32] = pr1;
         }
         keys[(size_t)t * N + j0 + lane] = code0;
+        if (!counts) {                       // codes only: k_count_ranks counts afterwards, table by table
+          if (live1) keys[(size_t)t * N + j0 + 32 + lane] = code1;
+          continue;
+        }
         int32_t* cnt = counts + (size_t)t * (size_t)(nb + 1) + 1;
         if (ranks) {
           pr0 = (uint32_t)atomicAdd(cnt + code0, 1);
@@ -450,6 +457,20 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
         if (pend1) ranks[pidx + 32] = pr1;
       }
     }
+  }
+}
+
+// Counting as a pass of its own, for tables whose counters do not fit the L2 cache together (2^21 buckets x 64 tables
+// are half a gigabyte): the blocks walk table after table, so that the counters being incremented at any moment are
+// those of one or two tables and the atomics stay in L2.  ranks[t][j] = arrivals before j in its bucket.
+__global__ void __launch_bounds__(256) k_count_ranks(const uint32_t* keys, uint32_t* ranks, int32_t* counts, int N, long long nb) {
+  const int t = blockIdx.y;
+  const uint32_t* k = keys + (size_t)t * N;
+  uint32_t* r = ranks ? ranks + (size_t)t * N : nullptr;
+  int32_t* cnt = counts + (size_t)t * (size_t)(nb + 1) + 1;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < N; j += gridDim.x * blockDim.x) {
+    const uint32_t v = (uint32_t)atomicAdd(cnt + k[j], 1);
+    if (r) r[j] = v;
   }
 }
 
@@ -841,6 +862,10 @@ cudaError_t launch_build_tables(Ctx* c) {
   const size_t off_bytes = (size_t)c->L * (size_t)(c->nb + 1) * sizeof(int32_t);
   cudaError_t e = cudaMemsetAsync(c->bucket_off, 0, off_bytes, c->stream);
   if (e != cudaSuccess) return e;
+  // the counting atomics ride with the hashing while all the tables' counters fit the L2 cache together; beyond that
+  // every atomic would be a read-modify-write in DRAM, and the counting becomes a pass of its own, table by table
+  const bool split_count = off_bytes > COUNT_SPLIT_BYTES;
+  int32_t* hash_counts = split_count ? nullptr : c->bucket_off;
   const int tile_bytes = (HN_ROWS * (c->H + 1) * (int)sizeof(float) + 15) & ~15;
   const long long fn_bytes = (long long)c->KL * c->fn_len * 2;
   const bool fn_smem = fn_bytes <= HN_FN_SMEM_MAX && c->H <= 0x7fff;
@@ -858,7 +883,7 @@ cudaError_t launch_build_tables(Ctx* c) {
     if (per_sm < 1) per_sm = 1;
     LaunchScope ls(c, KID_HASH_NEURONS);
     k_hash_neurons_dwta8<<<c->num_sms * per_sm, HN_THREADS, smem2, c->stream>>>(c->W2, c->hash_idx, c->keysA, c->place_path ? c->keysB : nullptr,
-                                                                              c->bucket_off, c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
+                                                                              hash_counts, c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
   } else {
     auto kern = fn_smem ? k_hash_neurons<true> : k_hash_neurons<false>;
     if (smem > 48 * 1024) {
@@ -871,10 +896,16 @@ cudaError_t launch_build_tables(Ctx* c) {
     if (per_sm < 1) per_sm = 1;
     LaunchScope ls(c, KID_HASH_NEURONS);
     kern<<<c->num_sms * per_sm, HN_THREADS, smem, c->stream>>>(c->W2, c->hash_idx, c->hash_sign, c->keysA,
-                                                             c->place_path ? c->keysB : nullptr, c->bucket_off, c->N, c->H, c->K, c->L,
+                                                             c->place_path ? c->keysB : nullptr, hash_counts, c->N, c->H, c->K, c->L,
                                                              c->cfg.hash_family, c->lg_bin, c->fn_len, c->nb);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  if (split_count) {
+    LaunchScope ls(c, KID_HASH_NEURONS);
+    dim3 grid((unsigned)min((long long)(c->N + 255) / 256, 2048LL), c->L);
+    k_count_ranks<<<grid, 256, 0, c->stream>>>(c->keysA, c->place_path ? c->keysB : nullptr, c->bucket_off, c->N, c->nb);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
   const bool list_in_scan = c->place_path && c->cap >= ORD_SMALL;
   {
     const int nchunks = (int)((c->nb + 1 + BS_CHUNK - 1) / BS_CHUNK);

@@ -317,3 +317,18 @@ def test_paper_shapes_with_batch_2048_at_reduced_vocabulary(name):
         one_and_two_steps(pr, [wl.batch(i) for i in range(2)])
     finally:
         pr.close()
+
+
+def test_tables_whose_counters_exceed_the_cache_are_counted_table_by_table():
+    """21-bit codes x 9 tables: 75 MB of bucket counters, beyond what the table build counts while it hashes; the
+    counting then runs as a pass of its own.  Tables must not change by a bit, two rebuilds in a row."""
+    pr = Pair(D=64, H=64, N=30011, family=DWTA, K=7, L=9, bucket_cap=16, max_batch=8)
+    try:
+        for trial in range(2):
+            assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_off"), pr.o.view("bucket_off"))
+            assert np.array_equal(ds.dslide_get_tensor(pr.ctx, "bucket_ids"), pr.o.view("bucket_ids"))
+            ds.dslide_rebuild_tables(pr.ctx)
+            ds.dslide_sync(pr.ctx)
+            pr.o.rebuild_tables()
+    finally:
+        pr.close()
