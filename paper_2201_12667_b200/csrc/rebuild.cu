@@ -369,6 +369,7 @@ __device__ __forceinline__ void wta_step(float x, int i, float& bv, int& best) {
   if (x > bv) { bv = x; best = i; }          // strict: the lowest position wins ties
 }
 
+template <bool COUNT>      // COUNT = false: codes only, the counting is a pass of its own
 __global__ void __launch_bounds__(HN_THREADS)
 k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ hidx, uint32_t* keys, uint32_t* ranks,
                      int32_t* counts, int N, int H, int K, int L, int lg_bin, long long nb) {
@@ -433,7 +434,7 @@ k_hash_neurons_dwta8(const float* __restrict__ W2, const int32_t* __restrict__ h
           if (pend1) ranks[pidx + 32] = pr1;
         }
         keys[(size_t)t * N + j0 + lane] = code0;
-        if (!counts) {                       // codes only: k_count_ranks counts afterwards, table by table
+        if (!COUNT) {                        // codes only: k_count_ranks counts afterwards, table by table
           if (live1) keys[(size_t)t * N + j0 + 32 + lane] = code1;
           continue;
         }
@@ -874,16 +875,19 @@ cudaError_t launch_build_tables(Ctx* c) {
   if (fn_smem && c->cfg.hash_family == DSLIDE_DWTA && c->fn_len == 8 && smem2_ll <= 100 * 1024) {
     const int smem2 = (int)smem2_ll;
     if (smem2 > 48 * 1024) {
-      e = cudaFuncSetAttribute(k_hash_neurons_dwta8, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2);
+      e = cudaFuncSetAttribute(split_count ? k_hash_neurons_dwta8<false> : k_hash_neurons_dwta8<true>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, smem2);
       if (e != cudaSuccess) return e;
     }
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_hash_neurons_dwta8, HN_THREADS, smem2);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, split_count ? k_hash_neurons_dwta8<false> : k_hash_neurons_dwta8<true>,
+                                                      HN_THREADS, smem2);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     LaunchScope ls(c, KID_HASH_NEURONS);
-    k_hash_neurons_dwta8<<<c->num_sms * per_sm, HN_THREADS, smem2, c->stream>>>(c->W2, c->hash_idx, c->keysA, c->place_path ? c->keysB : nullptr,
-                                                                              hash_counts, c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
+    auto kern8 = split_count ? k_hash_neurons_dwta8<false> : k_hash_neurons_dwta8<true>;
+    kern8<<<c->num_sms * per_sm, HN_THREADS, smem2, c->stream>>>(c->W2, c->hash_idx, c->keysA, c->place_path ? c->keysB : nullptr,
+                                                               hash_counts, c->N, c->H, c->K, c->L, c->lg_bin, c->nb);
   } else {
     auto kern = fn_smem ? k_hash_neurons<true> : k_hash_neurons<false>;
     if (smem > 48 * 1024) {
