@@ -87,6 +87,7 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -844,6 +845,17 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       __syncthreads();
       uint32_t* srt = sh_dd + RANK_MAX;
       const int per = (n + FWD_THREADS - 1) / FWD_THREADS;
+      if (packed && n <= FWD_THREADS - 64) {
+        // the warps the counting below leaves idle ask L2 for the candidates' rows of W2 meanwhile (the staging after
+        // the dedup then finds most of them there); a hint only: duplicates are asked twice, nothing waits for it
+        const int idle0 = (n + 31) & ~31;                          // first thread without a value to rank
+        const int lines = (H * 4 + 127) >> 7;
+        for (int e = tid - idle0; e >= 0 && e < n * (lines + 1); e += FWD_THREADS - idle0) {
+          const int c = e / (lines + 1), q = e - c * (lines + 1);
+          const int j = (int)(sh_dd[c] >> RANK_BITS);
+          prefetch_l2(q < lines ? static_cast<const void*>(p.W2 + (size_t)j * H + 32 * q) : static_cast<const void*>(p.hdr2 + j));
+        }
+      }
       if (packed) {
         if (per <= 1) rank_sort<1, true>(sh_dd, srt, n);
         else if (per == 2) rank_sort<2, true>(sh_dd, srt, n);
