@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["api.cu", "forward.cu", "update.cu", "rebuild.cu", "static_sort.cu"]
+SOURCES = ["api.cu", "forward.cu", "update.cu", "rebuild.cu", "static_sort.cu", "dense_tc.cu"]
 LIB = os.path.join(HERE, "libdslide.so")
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

@@ -130,6 +130,8 @@ cudaError_t launch_update(Ctx* c, int batch, const int32_t* row_ptr, const int32
                           float* loss_out, HostResult* host_res, unsigned int host_seq);
 cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int32_t* col_idx,
                            const float* vals, int k, int dense, int32_t* out_ids, float* out_scores);
+bool dense_tc_usable(const Ctx* c, int k);           // inference over all neurons on the tensor pipe: shapes it covers
+cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* out_scores);
 cudaError_t setup_forward(Ctx* c);   // chooses the dedup path and the shared-memory layout
 
 struct Ctx {

@@ -1,0 +1,561 @@
+// Inference over all N neurons on the tensor pipe (dslide_predict_topk with dense = 1, k <= TC_K_MAX).
+//
+// The logits of a batch against every output neuron are one contraction, Z[B][N] = h[B][H] . W2[N][H]^T + b2
+// (Section 3.6: "layer sparsity is 1"), so this path runs it on the fifth-generation tensor cores: tiles of W2 and
+// the batch's hidden activations arrive in shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), a single
+// thread issues tcgen05.mma (kind::tf32, accumulators in tensor memory), and four warps read the accumulators back
+// (tcgen05.ld) and keep, per sample, the best candidates of the block's slice of neurons.  W2 is streamed once per
+// 128 samples.
+//
+// TF32 rounds both operands to 10 mantissa bits, far from the 1e-4 the scores must meet.  The tensor pass is
+// therefore a FILTER: it keeps the 2k + TC_EXTRA best neurons per sample by approximate score; k_tc_refine recomputes
+// those few exactly in fp32 and orders them (logit descending, id ascending).  The filter is exact when the k-th
+// exact score clears every discarded neuron's approximate score by more than the approximation's error bound,
+// 2^-9 |h| |w|_max (plus accumulation); a sample for which that cannot be shown is flagged and k_tc_fixup scores
+// all N neurons for it in fp32.  Results are therefore those of the exact path.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace dslide {
+
+constexpr int TC_M = 128;          // samples per block = lanes of the accumulator
+constexpr int TC_N = 128;          // neurons per tile = columns of the accumulator
+constexpr int TC_KB = 32;          // hidden units per 128-byte swizzled row
+constexpr int TC_STAGES = 2;       // tiles of W2 in flight
+constexpr int TC_SPLIT = 1;        // read-back warps per quarter of tensor memory (each takes 1 / TC_SPLIT of a tile's columns)
+constexpr int TC_EPI = 128 * TC_SPLIT;                 // read-back threads
+constexpr int TC_THREADS = 64 + TC_EPI;                // warp 0: TMA producer; warp 1: tensor memory + MMA issue; then the read-back warps
+constexpr int TC_EXTRA = 8;        // candidates kept beyond k: TC_EXTRA + k (the wider the margin, the rarer the exact fall-back)
+constexpr int TC_K_MAX = 8;
+constexpr int TC_CAP = 2 * TC_K_MAX + TC_EXTRA;
+constexpr int TC_SUB_BYTES = TC_M * 128;               // one 32-unit slab of 128 rows
+constexpr float TC_ERR = 2.2e-3f;  // |approximate - exact| <= TC_ERR * |h| * |w|: two operands cut to 10 mantissa bits, fp32 sums
+
+struct TcParams {
+  const RowHdr* hdr2;
+  int2* cand;                      // [TC_SPLIT * slices][Bpad][TC_GBUF] (score bits, id): the first cand_cnt entries are the slice's best, best first
+  int* cand_cnt;                   // [TC_SPLIT * slices][Bpad]
+  DevState* st;
+  int B, Bpad, H, N, cap, nslices, ntiles;
+};
+
+__device__ __forceinline__ uint32_t tc_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void tc_bar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(tc_smem(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void tc_bar_expect(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tc_smem(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tc_bar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc_smem(bar)) : "memory");
+}
+// Bounded wait; once any wait of the block has run out, *abort is set and every later wait returns at once, so that
+// all the roles run through their loops, tensor memory is released and the kernel ends (its results are flagged).
+__device__ __forceinline__ void tc_bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  const uint32_t a = tc_smem(bar);
+  for (int it = 0; it < (1 << 22); ++it) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    if (ok) return;
+    if ((it & 1023) == 1023 && *abort) return;
+  }
+  *abort = 1;
+}
+__device__ __forceinline__ void tc_tma_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(tc_smem(dst)), "l"(map), "r"(x), "r"(y), "r"(tc_smem(bar)) : "memory");
+}
+// Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t tc_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);            // start address
+  d |= (uint64_t)1 << 16;                              // leading-dimension offset: unused with swizzled K-major rows
+  d |= (uint64_t)(1024 >> 4) << 32;                    // stride between groups of eight rows
+  d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                              // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, N x M tile.
+__host__ __device__ constexpr uint32_t tc_idesc(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, "
+      "%19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ bool tc_better(float za, int ia, float zb, int ib) { return za > zb || (za == zb && ia < ib); }
+
+// Candidate buffers live in global memory (they stay in L2): TC_GBUF (score, id) pairs per sample and slice.  A
+// thread appends the scores of its sample that pass its threshold; when a buffer is nearly full the whole warp
+// selects its best `cap` entries (tc_select: `cap` rounds of a warp-wide maximum over the lanes' entries), moves
+// them to the front, best first, and the sample's threshold becomes the cap-th.  With the threshold rising that
+// happens about three times per sample and slice.  Kept out of line (the read-back loop around it is unrolled).
+constexpr int TC_GBUF = 256;
+constexpr int TC_PER = TC_GBUF / 32;
+struct TcLane { int cnt; float tau; int tau_id; };      // a sample's buffer fill and threshold, held by its thread
+__device__ __noinline__ TcLane tc_select(int2* buf, int l, int cap, TcLane me) {
+  const int lane = threadIdx.x & 31;
+  __syncwarp();                                  // the owner's appends are visible to the other lanes
+  const int n = __shfl_sync(0xffffffffu, me.cnt, l);
+  float z[TC_PER];
+  int id[TC_PER];
+#pragma unroll
+  for (int u = 0; u < TC_PER; ++u) {
+    const int e = lane + 32 * u;
+    const int2 v = e < n ? __ldcg(buf + e) : make_int2(__float_as_int(-INFINITY), 0x7fffffff);
+    z[u] = __int_as_float(v.x);
+    id[u] = v.y;
+  }
+  __syncwarp();
+  const int kept = n < cap ? n : cap;
+  float lastz = -INFINITY;
+  int lasti = 0x7fffffff;
+  for (int r = 0; r < kept; ++r) {
+    // the lane's best remaining entry, then the warp's
+    float bz = z[0];
+    int bi = id[0], bu = 0;
+#pragma unroll
+    for (int u = 1; u < TC_PER; ++u)
+      if (tc_better(z[u], id[u], bz, bi)) { bz = z[u]; bi = id[u]; bu = u; }
+    float wz = bz;
+    int wi = bi;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const float oz = __shfl_xor_sync(0xffffffffu, wz, d);
+      const int oi = __shfl_xor_sync(0xffffffffu, wi, d);
+      if (tc_better(oz, oi, wz, wi)) { wz = oz; wi = oi; }
+    }
+    if (wi == bi && wz == bz) {                   // ids are distinct: exactly one lane owns the winner
+#pragma unroll
+      for (int u = 0; u < TC_PER; ++u)
+        if (u == bu) { z[u] = -INFINITY; id[u] = 0x7fffffff; }
+      __stcg(buf + r, make_int2(__float_as_int(wz), wi));
+    }
+    lastz = wz; lasti = wi;
+  }
+  __syncwarp();
+  if (lane == l) {
+    me.cnt = kept;
+    if (n >= cap) { me.tau = lastz; me.tau_id = lasti; }
+  }
+  return me;
+}
+
+// Grid: (slices of the neurons, groups of 128 samples).  Dynamic shared memory (1024-byte aligned):
+// activations [H/32][128 rows][128 B], then TC_STAGES tiles of W2 in the same form, then
+// the tiles' biases, the barriers.  (The samples' candidate buffers are in global memory.)
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, const TcParams p) {
+  extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int ksub = p.H / TC_KB;
+  const uint32_t tile_bytes = (uint32_t)ksub * TC_SUB_BYTES;
+  unsigned char* smA = sm;
+  unsigned char* smB = sm + tile_bytes;
+  float* sb = reinterpret_cast<float*>(smB + (size_t)TC_STAGES * tile_bytes);                         // [2][128] biases of the tile
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sb + 2 * TC_N);
+  uint64_t* bar_a = bars;                      // activations have arrived
+  uint64_t* bar_full = bars + 1;               // [TC_STAGES] tile of W2 has arrived
+  uint64_t* bar_empty = bars + 1 + TC_STAGES;  // [TC_STAGES] tile of W2 has been consumed
+  uint64_t* bar_accfull = bars + 1 + 2 * TC_STAGES;   // [2] accumulator written
+  uint64_t* bar_accempty = bars + 3 + 2 * TC_STAGES;  // [2] accumulator read back
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5 + 2 * TC_STAGES);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int slice = blockIdx.x, s0 = blockIdx.y * TC_M;
+  // tiles of this slice: slice, slice + nslices, ... (both sample groups walk the same tiles at the same time: the
+  // second read of a tile is served by L2)
+  const int my_tiles = slice < p.ntiles ? (p.ntiles - slice + p.nslices - 1) / p.nslices : 0;
+
+  if (tid == 0) {
+    tc_bar_init(bar_a, 1);
+    for (int i = 0; i < TC_STAGES; ++i) { tc_bar_init(bar_full + i, 1); tc_bar_init(bar_empty + i, 1); }
+    for (int i = 0; i < 2; ++i) { tc_bar_init(bar_accfull + i, 1); tc_bar_init(bar_accempty + i, TC_EPI); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {      // tensor memory: two accumulators of 128 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem(tmem_slot)), "r"(2 * TC_N) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- producer: one thread feeds the TMA ----------------
+    if (lane == 0) {
+      tc_bar_expect(bar_a, tile_bytes);
+      for (int ks = 0; ks < ksub; ++ks) tc_tma_2d(smA + (size_t)ks * TC_SUB_BYTES, &tmH, ks * TC_KB, s0, bar_a);
+      for (int i = 0; i < my_tiles; ++i) {
+        const int st = i % TC_STAGES;
+        if (i >= TC_STAGES) tc_bar_wait(bar_empty + st, ((i / TC_STAGES) - 1) & 1, abort_flag);
+        const int row0 = (slice + i * p.nslices) * TC_N;
+        tc_bar_expect(bar_full + st, tile_bytes);
+        for (int ks = 0; ks < ksub; ++ks)
+          tc_tma_2d(smB + (size_t)st * tile_bytes + (size_t)ks * TC_SUB_BYTES, &tmW, ks * TC_KB, row0, bar_full + st);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issue: one thread ----------------
+    if (lane == 0) {
+      const uint32_t idesc = tc_idesc(TC_M, TC_N);
+      tc_bar_wait(bar_a, 0, abort_flag);
+      for (int i = 0; i < my_tiles; ++i) {
+        const int st = i % TC_STAGES, acc = i & 1;
+        tc_bar_wait(bar_full + st, (i / TC_STAGES) & 1, abort_flag);
+        if (i >= 2) tc_bar_wait(bar_accempty + acc, ((i >> 1) - 1) & 1, abort_flag);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d = tmem_base + (uint32_t)(acc * TC_N);
+        for (int ks = 0; ks < ksub; ++ks)
+          for (int kk = 0; kk < TC_KB / 8; ++kk) {            // eight tf32 = 32 bytes per instruction
+            const uint64_t a = tc_desc(tc_smem(smA + (size_t)ks * TC_SUB_BYTES) + (uint32_t)kk * 32u);
+            const uint64_t b = tc_desc(tc_smem(smB + (size_t)st * tile_bytes + (size_t)ks * TC_SUB_BYTES) + (uint32_t)kk * 32u);
+            tc_mma(d, a, b, idesc, (ks | kk) != 0 ? 1u : 0u);
+          }
+        tc_commit(bar_empty + st);          // the tile's shared memory is free once these instructions have read it
+        tc_commit(bar_accfull + acc);       // and the accumulator is complete
+      }
+    }
+  } else {
+    // ---------------- read-back: thread = (sample, half of a tile's columns); the best `cap` neurons it sees ----------------
+    // Per 32 columns: first which of them reach the sample's threshold (32 independent comparisons, a bit each), then
+    // the appends of those that do.  The threshold is brought up to date only when the buffer runs full, and a score
+    // equal to it passes too: a stale or loose threshold lets a few more candidates through, it never loses one.
+    const int q = warp & 3;                 // a warp reaches the 32 lanes of tensor memory of its number modulo four
+    const int half = (warp - 2) >> 2;       // which share of a tile's 128 columns
+    const int row = 32 * q + lane;          // sample inside the block
+    const int et = tid - 64;                // the first 128 read-back threads fetch the tile's biases
+    const int cap = p.cap;
+    const int vslice = slice * TC_SPLIT + half;    // buffers are kept per (slice, share of the columns)
+    int2* wbuf = p.cand + ((size_t)vslice * p.Bpad + s0 + 32 * q) * TC_GBUF;      // the warp's 32 buffers
+    int2* mybuf = wbuf + (size_t)lane * TC_GBUF;
+    TcLane me;
+    me.cnt = 0; me.tau = -INFINITY; me.tau_id = 0x7fffffff;
+    for (int i = 0; i < my_tiles; ++i) {
+      const int acc = i & 1;
+      const int j0 = (slice + i * p.nslices) * TC_N;
+      if (et < TC_N) sb[acc * TC_N + et] = j0 + et < p.N ? __ldg(&p.hdr2[j0 + et].b) : 0.f;
+      tc_bar_wait(bar_accfull + acc, (i >> 1) & 1, abort_flag);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      asm volatile("bar.sync 1, %0;" ::"n"(TC_EPI) : "memory");          // the tile's biases are in place
+      for (int c0 = (TC_N / TC_SPLIT) * half; c0 < (TC_N / TC_SPLIT) * (half + 1); c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * TC_N + c0), r);
+        unsigned full = __ballot_sync(0xffffffffu, me.cnt > TC_GBUF - 32);      // room for a whole group of columns?
+        while (full) {
+          const int l = __ffs(full) - 1;
+          full &= full - 1;
+          me = tc_select(wbuf + (size_t)l * TC_GBUF, l, cap, me);
+        }
+        const int jb = j0 + c0;
+        const float4* sb4 = reinterpret_cast<const float4*>(sb + acc * TC_N + c0);
+        unsigned hm = 0u;
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 bq = sb4[c4];
+          const float z0 = __uint_as_float(r[4 * c4]) + bq.x, z1 = __uint_as_float(r[4 * c4 + 1]) + bq.y;
+          const float z2 = __uint_as_float(r[4 * c4 + 2]) + bq.z, z3 = __uint_as_float(r[4 * c4 + 3]) + bq.w;
+          r[4 * c4] = __float_as_uint(z0); r[4 * c4 + 1] = __float_as_uint(z1);
+          r[4 * c4 + 2] = __float_as_uint(z2); r[4 * c4 + 3] = __float_as_uint(z3);
+          if (z0 >= me.tau) hm |= 1u << (4 * c4);
+          if (z1 >= me.tau) hm |= 2u << (4 * c4);
+          if (z2 >= me.tau) hm |= 4u << (4 * c4);
+          if (z3 >= me.tau) hm |= 8u << (4 * c4);
+        }
+        if (p.N - jb < 32) hm &= p.N > jb ? (1u << (p.N - jb)) - 1u : 0u;      // neurons past the end (last tile only)
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          if ((hm >> (8 * g)) & 0xffu) {
+#pragma unroll
+            for (int c = 8 * g; c < 8 * g + 8; ++c)
+              if ((hm >> c) & 1u) { __stcg(mybuf + me.cnt, make_int2((int)r[c], jb + c)); ++me.cnt; }
+          }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      tc_bar_arrive(bar_accempty + acc);
+    }
+    __syncwarp();
+    for (int l = 0; l < 32; ++l) me = tc_select(wbuf + (size_t)l * TC_GBUF, l, cap, me);
+    if (s0 + row < p.B) p.cand_cnt[(size_t)vslice * p.Bpad + s0 + row] = me.cnt;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * TC_N) : "memory");
+  }
+  if (tid == 0 && *abort_flag) atomicCAS(&p.st->status, 0, (int)DSLIDE_ERR_TIMEOUT);
+}
+
+// Largest squared norm of a row of W2 (for the filter's error bound).  Non-negative floats order like their bits.
+__global__ void __launch_bounds__(256) k_row_norm_max(const float* W2, int N, int H, unsigned int* out) {
+  const int lane = threadIdx.x & 31;
+  const int H4 = H >> 2;
+  float best = 0.f;
+  for (int j = blockIdx.x * 8 + (threadIdx.x >> 5); j < N; j += gridDim.x * 8) {
+    const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
+    float s = 0.f;
+    for (int c = lane; c < H4; c += 32) { const float4 w = __ldg(r + c); s += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w; }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+    best = fmaxf(best, s);
+  }
+  if (lane == 0) atomicMax(out, __float_as_uint(best));
+}
+
+// One block per sample: the slices' candidates -> the cap best by approximate score -> their exact fp32 logits ->
+// the k best by (logit descending, id ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
+constexpr int RF_THREADS = 128;
+constexpr int RF_MAXC = 4096;
+__global__ void __launch_bounds__(RF_THREADS)
+k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, int Bpad, const unsigned int* norm2max,
+            int B, int H, int N, int cap, int nslices, int k, int32_t* out_ids, float* out_scores, int* need_fix) {
+  __shared__ float cz[RF_MAXC];
+  __shared__ int ci[RF_MAXC];
+  __shared__ float ez[TC_CAP];
+  __shared__ int ei[TC_CAP];
+  __shared__ float red[RF_THREADS / 32];
+  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int total = nslices * cap;
+  int n2 = 1;
+  while (n2 < total) n2 <<= 1;
+  for (int e = tid; e < n2; e += RF_THREADS) {
+    if (e < total) {
+      const int sl = e / cap, q = e - sl * cap;
+      const bool have = q < cand_cnt[(size_t)sl * Bpad + s];
+      const int2 v = have ? cand[((size_t)sl * Bpad + s) * TC_GBUF + q] : make_int2(0, -1);
+      ci[e] = v.y;
+      cz[e] = have ? __int_as_float(v.x) : -INFINITY;
+    } else { ci[e] = -1; cz[e] = -INFINITY; }
+    if (ci[e] < 0) ci[e] = 0x7fffffff;
+  }
+  __syncthreads();
+  // bitonic sort, best first: (score descending, id ascending)
+  for (int kk = 2; kk <= n2; kk <<= 1)
+    for (int j = kk >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < n2; i += RF_THREADS) {
+        const int x = i ^ j;
+        if (x > i) {
+          const bool up = (i & kk) == 0;
+          const bool i_first = tc_better(cz[i], ci[i], cz[x], ci[x]);
+          if (i_first != up) { const float tz = cz[i]; cz[i] = cz[x]; cz[x] = tz; const int ti = ci[i]; ci[i] = ci[x]; ci[x] = ti; }
+        }
+      }
+      __syncthreads();
+    }
+  int nc = 0;                                   // candidates that exist, at most cap
+  for (int e = 0; e < cap && e < n2; ++e) nc += ci[e] != 0x7fffffff ? 1 : 0;
+  // exact logits of the kept candidates: a warp per candidate, four partial sums per lane as in the exact path
+  const float4* h4 = reinterpret_cast<const float4*>(h + (size_t)s * H);
+  const int H4 = H >> 2;
+  for (int e = warp; e < nc; e += RF_THREADS / 32) {
+    const int j = ci[e];
+    const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
+    float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+    for (int c = lane; c < H4; c += 32) {
+      const float4 w = __ldg(r + c), x = h4[c];
+      d0 = fmaf(w.x, x.x, d0); d1 = fmaf(w.y, x.y, d1); d2 = fmaf(w.z, x.z, d2); d3 = fmaf(w.w, x.w, d3);
+    }
+    float d = (d0 + d1) + (d2 + d3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+    if (lane == 0) { ez[e] = __ldg(&hdr2[j].b) + d; ei[e] = j; }
+  }
+  // |h|^2 of the sample
+  float hs = 0.f;
+  for (int c = tid; c < H; c += RF_THREADS) { const float x = h[(size_t)s * H + c]; hs += x * x; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
+  if (lane == 0) red[warp] = hs;
+  __syncthreads();
+  if (tid == 0) {
+    float hn = 0.f;
+    for (int w = 0; w < RF_THREADS / 32; ++w) hn += red[w];
+    // order the exact scores (insertion sort of at most cap entries)
+    for (int a = 1; a < nc; ++a) {
+      const float z = ez[a]; const int j = ei[a];
+      int b = a;
+      while (b > 0 && tc_better(z, j, ez[b - 1], ei[b - 1])) { ez[b] = ez[b - 1]; ei[b] = ei[b - 1]; --b; }
+      ez[b] = z; ei[b] = j;
+    }
+    for (int qk = 0; qk < k; ++qk) {
+      out_ids[(size_t)s * k + qk] = qk < nc ? ei[qk] : -1;
+      out_scores[(size_t)s * k + qk] = qk < nc ? ez[qk] : -INFINITY;
+    }
+    // Everything that was discarded (inside a slice or here) has an approximate score of at most the last kept
+    // one's, hence an exact score of at most that plus the error bound.  The k best are certain when the k-th exact
+    // score lies above that; nothing was discarded when fewer than cap candidates exist.
+    int fix = 0;
+    if (nc == cap && total > cap) {
+      const float bound = cz[cap - 1] + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
+      const int kth = (k < nc ? k : nc) - 1;
+      if (!(ez[kth] > bound)) fix = 1;
+    }
+    need_fix[s] = fix;
+  }
+}
+
+// A flagged sample: every neuron scored exactly (rare; one block walks all of W2).
+constexpr int FX_THREADS = 256;
+__global__ void __launch_bounds__(FX_THREADS)
+k_tc_fixup(const float* W2, const RowHdr* hdr2, const float* h, const int* need_fix, int H, int N, int k, int32_t* out_ids,
+           float* out_scores) {
+  const int s = blockIdx.x;
+  if (!need_fix[s]) return;
+  extern __shared__ float fx_smem[];            // [H] activation, then [warps][k] lists
+  float* hs = fx_smem;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = FX_THREADS / 32;
+  float* wz = hs + H + warp * k;
+  int* wi = reinterpret_cast<int*>(hs + H + nw * k) + warp * k;
+  for (int c = tid; c < H; c += FX_THREADS) hs[c] = h[(size_t)s * H + c];
+  __syncthreads();
+  const int H4 = H >> 2;
+  const float4* h4 = reinterpret_cast<const float4*>(hs);
+  int cnt = 0;                                  // lane 0: entries of the warp's list
+  for (int j = warp; j < N; j += nw) {
+    const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
+    float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+    for (int c = lane; c < H4; c += 32) {
+      const float4 w = __ldg(r + c), x = h4[c];
+      d0 = fmaf(w.x, x.x, d0); d1 = fmaf(w.y, x.y, d1); d2 = fmaf(w.z, x.z, d2); d3 = fmaf(w.w, x.w, d3);
+    }
+    float d = (d0 + d1) + (d2 + d3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+    if (lane == 0) {
+      const float z = __ldg(&hdr2[j].b) + d;
+      if (cnt < k || tc_better(z, j, wz[cnt - 1], wi[cnt - 1])) {
+        int at = cnt < k ? cnt++ : k - 1;
+        while (at > 0 && tc_better(z, j, wz[at - 1], wi[at - 1])) { wz[at] = wz[at - 1]; wi[at] = wi[at - 1]; --at; }
+        wz[at] = z; wi[at] = j;
+      }
+    }
+  }
+  int* cnts = reinterpret_cast<int*>(hs + H + 2 * nw * k);
+  if (lane == 0) cnts[warp] = cnt;
+  __syncthreads();
+  if (tid == 0) {
+    int head[FX_THREADS / 32];
+    for (int w = 0; w < nw; ++w) head[w] = 0;
+    float* az = hs + H;
+    int* ai = reinterpret_cast<int*>(hs + H + nw * k);
+    for (int qk = 0; qk < k; ++qk) {
+      int bw = -1;
+      for (int w = 0; w < nw; ++w) {
+        if (head[w] >= cnts[w]) continue;
+        if (bw < 0 || tc_better(az[w * k + head[w]], ai[w * k + head[w]], az[bw * k + head[bw]], ai[bw * k + head[bw]])) bw = w;
+      }
+      out_ids[(size_t)s * k + qk] = bw >= 0 ? ai[bw * k + head[bw]] : -1;
+      out_scores[(size_t)s * k + qk] = bw >= 0 ? az[bw * k + head[bw]] : -INFINITY;
+      if (bw >= 0) head[bw]++;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// rows x H fp32, row-major; boxes of 128 rows x 32 units, 128-byte swizzle; rows past the end read as zero
+static bool make_map(CUtensorMap* m, const float* base, int rows, int H) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)H, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)H * 4};
+  const cuuint32_t box[2] = {(cuuint32_t)TC_KB, (cuuint32_t)TC_M};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool dense_tc_usable(const Ctx* c, int k) {
+  return k >= 1 && k <= TC_K_MAX && c->H % TC_KB == 0 && c->H >= TC_KB && c->H <= 256 && c->N >= TC_N && encode_fn() != nullptr;
+}
+
+// The hidden activations of the batch are in c->h (left there by the forward kernel in predict mode).
+cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* out_scores) {
+  const int cap = 2 * k + TC_EXTRA;
+  const int groups = (batch + TC_M - 1) / TC_M;
+  const int ntiles = (c->N + TC_N - 1) / TC_N;
+  int nslices = c->num_sms / groups;
+  if (nslices < 1) nslices = 1;
+  if (nslices > ntiles) nslices = ntiles;
+  if (TC_SPLIT * nslices * cap > RF_MAXC) nslices = RF_MAXC / (TC_SPLIT * cap);
+  // work space: the norm bound, the flags, the candidate buffers of every slice and their fill
+  const int Bpad = groups * TC_M;
+  const size_t off_fix = 256, off_cnt = off_fix + (((size_t)batch * 4 + 255) & ~(size_t)255);
+  const size_t off_cand = off_cnt + (((size_t)TC_SPLIT * nslices * Bpad * 4 + 255) & ~(size_t)255);
+  const size_t need = off_cand + (size_t)TC_SPLIT * nslices * Bpad * TC_GBUF * sizeof(int2);
+  cudaError_t e;
+  if (need > c->pd_cap) {
+    if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) return e;
+    if (c->pd_part) cudaFree(c->pd_part);
+    c->pd_part = nullptr; c->pd_cap = 0;
+    if ((e = cudaMalloc(&c->pd_part, need)) != cudaSuccess) return e;
+    c->pd_cap = need;
+  }
+  unsigned char* ws = reinterpret_cast<unsigned char*>(c->pd_part);
+  unsigned int* norm2 = reinterpret_cast<unsigned int*>(ws);
+  int* need_fix = reinterpret_cast<int*>(ws + off_fix);
+  int* cand_cnt = reinterpret_cast<int*>(ws + off_cnt);
+  int2* cand = reinterpret_cast<int2*>(ws + off_cand);
+
+  CUtensorMap tmH, tmW;
+  if (!make_map(&tmH, c->h, c->cfg.max_batch, c->H) || !make_map(&tmW, c->W2, c->N, c->H)) return cudaErrorInvalidValue;
+
+  if ((e = cudaMemsetAsync(norm2, 0, sizeof(unsigned int), c->stream)) != cudaSuccess) return e;
+  k_row_norm_max<<<c->num_sms * 8, 256, 0, c->stream>>>(c->W2, c->N, c->H, norm2);
+
+  TcParams p;
+  p.hdr2 = c->hdr2; p.cand = cand; p.cand_cnt = cand_cnt; p.st = c->dstate;
+  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.nslices = nslices; p.ntiles = ntiles;
+  const size_t tile_bytes = (size_t)(c->H / TC_KB) * TC_SUB_BYTES;
+  const size_t smem = 1024 + tile_bytes * (1 + TC_STAGES) + 2 * TC_N * 4 + 16 * 8 + 64;
+  if ((e = cudaFuncSetAttribute(k_dense_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  {
+    LaunchScope ls(c, KID_PREDICT);
+    k_dense_tc<<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmH, tmW, p);
+  }
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  k_tc_refine<<<batch, RF_THREADS, 0, c->stream>>>(c->W2, c->hdr2, c->h, cand, cand_cnt, Bpad, norm2, batch, c->H, c->N, cap, TC_SPLIT * nslices, k,
+                                                   out_ids, out_scores, need_fix);
+  const size_t fx_smem = ((size_t)c->H + 2 * (FX_THREADS / 32) * k + FX_THREADS / 32) * 4;
+  k_tc_fixup<<<batch, FX_THREADS, fx_smem, c->stream>>>(c->W2, c->hdr2, c->h, need_fix, c->H, c->N, k, out_ids, out_scores);
+  return cudaGetLastError();
+}
+
+}  // namespace dslide

@@ -1655,7 +1655,9 @@ cudaError_t launch_predict(Ctx* c, int batch, const int32_t* row_ptr, const int3
   else k_forward<1, MAX_KPT><<<batch, FWD_THREADS, c->fwd_smem, c->stream>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || !dense) return e;
-  // over all neurons: the kernel above has left the hidden activations; groups of sg samples x slices of W2
+  // over all neurons: the kernel above has left the hidden activations.  Small k on supported shapes: the tensor pipe
+  // filters the candidates and an exact pass orders them; otherwise groups of sg samples x slices of W2 on the ALUs
+  if (dense_tc_usable(c, k)) return launch_dense_tc(c, batch, k, out_ids, out_scores);
   const int sg = k <= 8 ? 32 : (k <= 16 ? 16 : 8);
   const int ngroups = (batch + sg - 1) / sg;
   int nslices = (2 * c->num_sms + ngroups - 1) / ngroups;

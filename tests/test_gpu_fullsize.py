@@ -73,3 +73,31 @@ def test_full_size_325k_step_against_oracle():
 def test_full_size_1b_step_against_oracle():
     sizes, distinct = full_size_step("1b", 997)
     assert 20 < sizes.mean() < 2000 and distinct > 2 ** 14
+
+
+@pytest.mark.parametrize("k", [1, 5])
+def test_full_size_670k_dense_inference_against_oracle(k):
+    """Inference over all 670,091 neurons (the tensor-pipe filter, then exact logits of the kept candidates): ids equal
+    to the oracle's exact top-k wherever its scores are separated, scores at the usual bar."""
+    c = workloads.config("670k")
+    B = 96
+    pr = Pair(D=c["D"], H=c["H"], N=c["N"], family=c["family"], K=c["K"], L=c["L"], bucket_cap=c["bucket_cap"],
+              max_batch=B, max_labels=c["max_labels"], lr=c["lr"], init_std=0.01, seed=0, oracle_build="float_omp")
+    try:
+        pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.002)
+        pr.push_state()
+        batch = workloads.Workload(c, seed=0).batch(3, batch_size=B)
+        ids_o, sc_o = pr.o.predict_topk(batch[0], batch[1], batch[2], k, dense=True)
+        dev = [torch.from_numpy(a).cuda() for a in batch[:3]]
+        ids_g = torch.empty(B * k, dtype=torch.int32, device="cuda")
+        sc_g = torch.empty(B * k, dtype=torch.float32, device="cuda")
+        ds.dslide_predict_topk(pr.ctx, B, *dev, k, 1, ids_g, sc_g)
+        ds.dslide_sync(pr.ctx)
+        ids_g, sc_g = ids_g.cpu().numpy().reshape(B, k), sc_g.cpu().numpy().reshape(B, k)
+        for s in range(B):
+            assert max_rel_err(sc_g[s], sc_o[s], 1e-2) < ACT_TOL, s
+            for q in range(k):
+                near = np.abs(sc_o[s] - sc_o[s][q]) <= 2 * ACT_TOL * np.abs(sc_o[s][q])
+                assert ids_g[s][q] == ids_o[s][q] if near.sum() == 1 else ids_g[s][q] in ids_o[s][near], (s, q)
+    finally:
+        pr.close()
