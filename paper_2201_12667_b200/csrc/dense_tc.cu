@@ -8,11 +8,15 @@
 // 128 samples.
 //
 // TF32 rounds both operands to 10 mantissa bits, far from the 1e-4 the scores must meet.  The tensor pass is
-// therefore a FILTER: it keeps the 2k + TC_EXTRA best neurons per sample by approximate score; k_tc_refine recomputes
-// those few exactly in fp32 and orders them (logit descending, id ascending).  The filter is exact when the k-th
-// exact score clears every discarded neuron's approximate score by more than the approximation's error bound,
-// 2^-9 |h| |w|_max (plus accumulation); a sample for which that cannot be shown is flagged and k_tc_fixup scores
-// all N neurons for it in fp32.  Results are therefore those of the exact path.
+// therefore a FILTER, in two launches of the same kernel.  The first scores every TC_SUBSET-th tile of neurons and
+// writes the scores out; k_tc_tau takes, per sample, the cap-th best of them (cap = 2k + TC_EXTRA) as the sample's
+// threshold -- at least cap neurons reach it, and about cap * TC_SUBSET do over all N.  The second launch scores all
+// tiles and a thread appends the few scores of its sample that reach the threshold to the sample's candidate buffer.
+// k_tc_refine recomputes the cap best candidates exactly in fp32 and orders them (logit descending, id ascending).
+// The filter is exact when the k-th exact score clears every discarded neuron's approximate score by more than the
+// approximation's error bound, 2^-9 |h| |w|_max (plus accumulation); a sample for which that cannot be shown (or
+// whose buffers ran over) is flagged and k_tc_fixup scores all N neurons for it in fp32.  Results are therefore
+// those of the exact path.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -28,16 +32,23 @@ constexpr int TC_EPI = 128 * TC_SPLIT;                 // read-back threads
 constexpr int TC_THREADS = 64 + TC_EPI;                // warp 0: TMA producer; warp 1: tensor memory + MMA issue; then the read-back warps
 constexpr int TC_EXTRA = 8;        // candidates kept beyond k: TC_EXTRA + k (the wider the margin, the rarer the exact fall-back)
 constexpr int TC_K_MAX = 8;
+constexpr int TC_GBUF = 64;        // candidate slots per (slice, sample); a buffer that runs over sends the sample to the exact scan
+constexpr int TC_SUBSET = 64;      // the threshold pass scores every TC_SUBSET-th tile
 constexpr int TC_CAP = 2 * TC_K_MAX + TC_EXTRA;
 constexpr int TC_SUB_BYTES = TC_M * 128;               // one 32-unit slab of 128 rows
 constexpr float TC_ERR = 2.2e-3f;  // |approximate - exact| <= TC_ERR * |h| * |w|: two operands cut to 10 mantissa bits, fp32 sums
 
 struct TcParams {
   const RowHdr* hdr2;
-  int2* cand;                      // [TC_SPLIT * slices][Bpad][TC_GBUF] (score bits, id): the first cand_cnt entries are the slice's best, best first
+  int2* cand;                      // [TC_SPLIT * slices][Bpad][TC_GBUF] (score bits, id), cand_cnt of them valid, no order
   int* cand_cnt;                   // [TC_SPLIT * slices][Bpad]
+  float* dump;                     // DUMP launch: [Bpad][dump_cols] scores of the subset's tiles
+  const float* tau;                // filter launch: [Bpad] thresholds
+  int* need_fix;                   // [B] set when a sample's buffer ran over
   DevState* st;
-  int B, Bpad, H, N, cap, nslices, ntiles;
+  int B, Bpad, H, N, cap, nslices, ntiles;     // ntiles: tiles this launch walks
+  int tile_stride;                 // tile i of the launch is tile i * tile_stride of W2
+  int dump_cols;
 };
 
 __device__ __forceinline__ uint32_t tc_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -102,65 +113,10 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 
 __device__ __forceinline__ bool tc_better(float za, int ia, float zb, int ib) { return za > zb || (za == zb && ia < ib); }
 
-// Candidate buffers live in global memory (they stay in L2): TC_GBUF (score, id) pairs per sample and slice.  A
-// thread appends the scores of its sample that pass its threshold; when a buffer is nearly full the whole warp
-// selects its best `cap` entries (tc_select: `cap` rounds of a warp-wide maximum over the lanes' entries), moves
-// them to the front, best first, and the sample's threshold becomes the cap-th.  With the threshold rising that
-// happens about three times per sample and slice.  Kept out of line (the read-back loop around it is unrolled).
-constexpr int TC_GBUF = 256;
-constexpr int TC_PER = TC_GBUF / 32;
-struct TcLane { int cnt; float tau; int tau_id; };      // a sample's buffer fill and threshold, held by its thread
-__device__ __noinline__ TcLane tc_select(int2* buf, int l, int cap, TcLane me) {
-  const int lane = threadIdx.x & 31;
-  __syncwarp();                                  // the owner's appends are visible to the other lanes
-  const int n = __shfl_sync(0xffffffffu, me.cnt, l);
-  float z[TC_PER];
-  int id[TC_PER];
-#pragma unroll
-  for (int u = 0; u < TC_PER; ++u) {
-    const int e = lane + 32 * u;
-    const int2 v = e < n ? __ldcg(buf + e) : make_int2(__float_as_int(-INFINITY), 0x7fffffff);
-    z[u] = __int_as_float(v.x);
-    id[u] = v.y;
-  }
-  __syncwarp();
-  const int kept = n < cap ? n : cap;
-  float lastz = -INFINITY;
-  int lasti = 0x7fffffff;
-  for (int r = 0; r < kept; ++r) {
-    // the lane's best remaining entry, then the warp's
-    float bz = z[0];
-    int bi = id[0], bu = 0;
-#pragma unroll
-    for (int u = 1; u < TC_PER; ++u)
-      if (tc_better(z[u], id[u], bz, bi)) { bz = z[u]; bi = id[u]; bu = u; }
-    float wz = bz;
-    int wi = bi;
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-      const float oz = __shfl_xor_sync(0xffffffffu, wz, d);
-      const int oi = __shfl_xor_sync(0xffffffffu, wi, d);
-      if (tc_better(oz, oi, wz, wi)) { wz = oz; wi = oi; }
-    }
-    if (wi == bi && wz == bz) {                   // ids are distinct: exactly one lane owns the winner
-#pragma unroll
-      for (int u = 0; u < TC_PER; ++u)
-        if (u == bu) { z[u] = -INFINITY; id[u] = 0x7fffffff; }
-      __stcg(buf + r, make_int2(__float_as_int(wz), wi));
-    }
-    lastz = wz; lasti = wi;
-  }
-  __syncwarp();
-  if (lane == l) {
-    me.cnt = kept;
-    if (n >= cap) { me.tau = lastz; me.tau_id = lasti; }
-  }
-  return me;
-}
-
 // Grid: (slices of the neurons, groups of 128 samples).  Dynamic shared memory (1024-byte aligned):
 // activations [H/32][128 rows][128 B], then TC_STAGES tiles of W2 in the same form, then
 // the tiles' biases, the barriers.  (The samples' candidate buffers are in global memory.)
+template <bool DUMP>      // DUMP: write every score out (threshold pass); else append the scores that reach the sample's threshold
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, const TcParams p) {
   extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
@@ -209,7 +165,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
       for (int i = 0; i < my_tiles; ++i) {
         const int st = i % TC_STAGES;
         if (i >= TC_STAGES) tc_bar_wait(bar_empty + st, ((i / TC_STAGES) - 1) & 1, abort_flag);
-        const int row0 = (slice + i * p.nslices) * TC_N;
+        const int row0 = (slice + i * p.nslices) * p.tile_stride * TC_N;
         tc_bar_expect(bar_full + st, tile_bytes);
         for (int ks = 0; ks < ksub; ++ks)
           tc_tma_2d(smB + (size_t)st * tile_bytes + (size_t)ks * TC_SUB_BYTES, &tmW, ks * TC_KB, row0, bar_full + st);
@@ -237,23 +193,21 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
       }
     }
   } else {
-    // ---------------- read-back: thread = (sample, half of a tile's columns); the best `cap` neurons it sees ----------------
-    // Per 32 columns: first which of them reach the sample's threshold (32 independent comparisons, a bit each), then
-    // the appends of those that do.  The threshold is brought up to date only when the buffer runs full, and a score
-    // equal to it passes too: a stale or loose threshold lets a few more candidates through, it never loses one.
+    // ---------------- read-back: thread = (sample, share of a tile's columns) ----------------
+    // Per 32 columns the bias is added; then, threshold pass: the scores are written out; filter pass: which of them
+    // reach the sample's threshold (32 independent comparisons, a bit each), then the appends of those that do.
     const int q = warp & 3;                 // a warp reaches the 32 lanes of tensor memory of its number modulo four
     const int half = (warp - 2) >> 2;       // which share of a tile's 128 columns
     const int row = 32 * q + lane;          // sample inside the block
     const int et = tid - 64;                // the first 128 read-back threads fetch the tile's biases
-    const int cap = p.cap;
     const int vslice = slice * TC_SPLIT + half;    // buffers are kept per (slice, share of the columns)
-    int2* wbuf = p.cand + ((size_t)vslice * p.Bpad + s0 + 32 * q) * TC_GBUF;      // the warp's 32 buffers
-    int2* mybuf = wbuf + (size_t)lane * TC_GBUF;
-    TcLane me;
-    me.cnt = 0; me.tau = -INFINITY; me.tau_id = 0x7fffffff;
+    int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * TC_GBUF;
+    const float tau = DUMP ? 0.f : p.tau[s0 + row];
+    int cnt = 0;
     for (int i = 0; i < my_tiles; ++i) {
       const int acc = i & 1;
-      const int j0 = (slice + i * p.nslices) * TC_N;
+      const int tile = slice + i * p.nslices;
+      const int j0 = tile * p.tile_stride * TC_N;
       if (et < TC_N) sb[acc * TC_N + et] = j0 + et < p.N ? __ldg(&p.hdr2[j0 + et].b) : 0.f;
       tc_bar_wait(bar_accfull + acc, (i >> 1) & 1, abort_flag);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -261,12 +215,6 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
       for (int c0 = (TC_N / TC_SPLIT) * half; c0 < (TC_N / TC_SPLIT) * (half + 1); c0 += 32) {
         uint32_t r[32];
         tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * TC_N + c0), r);
-        unsigned full = __ballot_sync(0xffffffffu, me.cnt > TC_GBUF - 32);      // room for a whole group of columns?
-        while (full) {
-          const int l = __ffs(full) - 1;
-          full &= full - 1;
-          me = tc_select(wbuf + (size_t)l * TC_GBUF, l, cap, me);
-        }
         const int jb = j0 + c0;
         const float4* sb4 = reinterpret_cast<const float4*>(sb + acc * TC_N + c0);
         unsigned hm = 0u;
@@ -277,26 +225,46 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
           const float z2 = __uint_as_float(r[4 * c4 + 2]) + bq.z, z3 = __uint_as_float(r[4 * c4 + 3]) + bq.w;
           r[4 * c4] = __float_as_uint(z0); r[4 * c4 + 1] = __float_as_uint(z1);
           r[4 * c4 + 2] = __float_as_uint(z2); r[4 * c4 + 3] = __float_as_uint(z3);
-          if (z0 >= me.tau) hm |= 1u << (4 * c4);
-          if (z1 >= me.tau) hm |= 2u << (4 * c4);
-          if (z2 >= me.tau) hm |= 4u << (4 * c4);
-          if (z3 >= me.tau) hm |= 8u << (4 * c4);
-        }
-        if (p.N - jb < 32) hm &= p.N > jb ? (1u << (p.N - jb)) - 1u : 0u;      // neurons past the end (last tile only)
-#pragma unroll
-        for (int g = 0; g < 4; ++g)
-          if ((hm >> (8 * g)) & 0xffu) {
-#pragma unroll
-            for (int c = 8 * g; c < 8 * g + 8; ++c)
-              if ((hm >> c) & 1u) { __stcg(mybuf + me.cnt, make_int2((int)r[c], jb + c)); ++me.cnt; }
+          if (!DUMP) {
+            if (z0 >= tau) hm |= 1u << (4 * c4);
+            if (z1 >= tau) hm |= 2u << (4 * c4);
+            if (z2 >= tau) hm |= 4u << (4 * c4);
+            if (z3 >= tau) hm |= 8u << (4 * c4);
           }
+        }
+        if (DUMP) {
+          // neurons past the end score -infinity; a thread's 32 scores are 128 contiguous bytes
+          float4* out = reinterpret_cast<float4*>(p.dump + (size_t)(s0 + row) * p.dump_cols + (size_t)tile * TC_N + c0);
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            float4 v;
+            v.x = jb + 4 * c4 < p.N ? __uint_as_float(r[4 * c4]) : -INFINITY;
+            v.y = jb + 4 * c4 + 1 < p.N ? __uint_as_float(r[4 * c4 + 1]) : -INFINITY;
+            v.z = jb + 4 * c4 + 2 < p.N ? __uint_as_float(r[4 * c4 + 2]) : -INFINITY;
+            v.w = jb + 4 * c4 + 3 < p.N ? __uint_as_float(r[4 * c4 + 3]) : -INFINITY;
+            __stcg(out + c4, v);
+          }
+        } else {
+          if (p.N - jb < 32) hm &= p.N > jb ? (1u << (p.N - jb)) - 1u : 0u;      // neurons past the end (last tile only)
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            if ((hm >> (8 * g)) & 0xffu) {
+#pragma unroll
+              for (int c = 8 * g; c < 8 * g + 8; ++c)
+                if ((hm >> c) & 1u) {
+                  if (cnt < TC_GBUF) __stcg(mybuf + cnt, make_int2((int)r[c], jb + c));
+                  ++cnt;
+                }
+            }
+        }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       tc_bar_arrive(bar_accempty + acc);
     }
-    __syncwarp();
-    for (int l = 0; l < 32; ++l) me = tc_select(wbuf + (size_t)l * TC_GBUF, l, cap, me);
-    if (s0 + row < p.B) p.cand_cnt[(size_t)vslice * p.Bpad + s0 + row] = me.cnt;
+    if (!DUMP && s0 + row < p.B) {
+      p.cand_cnt[(size_t)vslice * p.Bpad + s0 + row] = cnt < TC_GBUF ? cnt : TC_GBUF;
+      if (cnt > TC_GBUF) p.need_fix[s0 + row] = 1;          // candidates were dropped: the sample is scored exactly
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -323,32 +291,79 @@ __global__ void __launch_bounds__(256) k_row_norm_max(const float* W2, int N, in
   if (lane == 0) atomicMax(out, __float_as_uint(best));
 }
 
+// One block per sample: the cap-th largest of the sample's scores of the subset (found bit by bit on a key that
+// orders like the floats) is the sample's threshold; -infinity when the subset holds fewer than cap neurons.
+constexpr int TAU_THREADS = 256;
+__device__ __forceinline__ uint32_t tc_key(float z) {
+  const uint32_t b = __float_as_uint(z);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int cols, int cap, float* tau) {
+  extern __shared__ uint32_t tau_keys[];        // [cols]
+  __shared__ int wsum[TAU_THREADS / 32];
+  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < cols; e += TAU_THREADS) tau_keys[e] = tc_key(__ldcg(dump + (size_t)s * cols + e));
+  __syncthreads();
+  uint32_t K = 0u;
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t trial = K | (1u << bit);
+    int cnt = 0;
+    for (int e = tid; e < cols; e += TAU_THREADS) cnt += tau_keys[e] >= trial ? 1 : 0;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+    if (lane == 0) wsum[warp] = cnt;
+    __syncthreads();
+    int total = 0;
+    for (int w = 0; w < TAU_THREADS / 32; ++w) total += wsum[w];
+    if (total >= cap) K = trial;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const uint32_t b = (K & 0x80000000u) ? (K & 0x7fffffffu) : ~K;
+    float t = __uint_as_float(b);
+    if (K == 0u || !(t == t)) t = -INFINITY;      // fewer than cap scores: everything passes
+    tau[s] = t;
+  }
+}
+
 // One block per sample: the slices' candidates -> the cap best by approximate score -> their exact fp32 logits ->
 // the k best by (logit descending, id ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
 constexpr int RF_THREADS = 128;
 constexpr int RF_MAXC = 4096;
 __global__ void __launch_bounds__(RF_THREADS)
-k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, int Bpad, const unsigned int* norm2max,
-            int B, int H, int N, int cap, int nslices, int k, int32_t* out_ids, float* out_scores, int* need_fix) {
+k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, const float* tau, int Bpad,
+            const unsigned int* norm2max, int B, int H, int N, int cap, int nvs, int k, int32_t* out_ids, float* out_scores,
+            int* need_fix) {
   __shared__ float cz[RF_MAXC];
   __shared__ int ci[RF_MAXC];
+  __shared__ int offs[512];
   __shared__ float ez[TC_CAP];
   __shared__ int ei[TC_CAP];
   __shared__ float red[RF_THREADS / 32];
+  __shared__ int sh_total;
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int total = nslices * cap;
+  if (tid == 0) {
+    int run = 0;
+    for (int v = 0; v < nvs; ++v) { offs[v] = run; run += cand_cnt[(size_t)v * Bpad + s]; }
+    sh_total = run;
+  }
+  __syncthreads();
+  const int total = sh_total;
+  if (total > RF_MAXC) {                          // more candidates than this pass handles: the sample is scored exactly
+    if (tid == 0) need_fix[s] = 1;
+    return;
+  }
   int n2 = 1;
   while (n2 < total) n2 <<= 1;
-  for (int e = tid; e < n2; e += RF_THREADS) {
-    if (e < total) {
-      const int sl = e / cap, q = e - sl * cap;
-      const bool have = q < cand_cnt[(size_t)sl * Bpad + s];
-      const int2 v = have ? cand[((size_t)sl * Bpad + s) * TC_GBUF + q] : make_int2(0, -1);
-      ci[e] = v.y;
-      cz[e] = have ? __int_as_float(v.x) : -INFINITY;
-    } else { ci[e] = -1; cz[e] = -INFINITY; }
-    if (ci[e] < 0) ci[e] = 0x7fffffff;
+  for (int v = warp; v < nvs; v += RF_THREADS / 32) {
+    const int n = cand_cnt[(size_t)v * Bpad + s];
+    for (int e = lane; e < n; e += 32) {
+      const int2 x = __ldcg(cand + ((size_t)v * Bpad + s) * TC_GBUF + e);
+      cz[offs[v] + e] = __int_as_float(x.x);
+      ci[offs[v] + e] = x.y;
+    }
   }
+  for (int e = total + tid; e < n2; e += RF_THREADS) { cz[e] = -INFINITY; ci[e] = 0x7fffffff; }
   __syncthreads();
   // bitonic sort, best first: (score descending, id ascending)
   for (int kk = 2; kk <= n2; kk <<= 1)
@@ -363,8 +378,7 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
       }
       __syncthreads();
     }
-  int nc = 0;                                   // candidates that exist, at most cap
-  for (int e = 0; e < cap && e < n2; ++e) nc += ci[e] != 0x7fffffff ? 1 : 0;
+  const int nc = total < cap ? total : cap;     // candidates that go on to the exact pass
   // exact logits of the kept candidates: a warp per candidate, four partial sums per lane as in the exact path
   const float4* h4 = reinterpret_cast<const float4*>(h + (size_t)s * H);
   const int H4 = H >> 2;
@@ -402,16 +416,15 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
       out_ids[(size_t)s * k + qk] = qk < nc ? ei[qk] : -1;
       out_scores[(size_t)s * k + qk] = qk < nc ? ez[qk] : -INFINITY;
     }
-    // Everything that was discarded (inside a slice or here) has an approximate score of at most the last kept
-    // one's, hence an exact score of at most that plus the error bound.  The k best are certain when the k-th exact
-    // score lies above that; nothing was discarded when fewer than cap candidates exist.
-    int fix = 0;
-    if (nc == cap && total > cap) {
-      const float bound = cz[cap - 1] + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
+    // Every neuron that did not go on to the exact pass has an approximate score of at most T: the last kept one's
+    // when candidates were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its
+    // exact score is at most T plus the error bound; the k best are certain when the k-th exact score lies above.
+    const float T = total > cap ? cz[cap - 1] : tau[s];
+    if (nc > 0 && T > -INFINITY) {
+      const float bound = T + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
       const int kth = (k < nc ? k : nc) - 1;
-      if (!(ez[kth] > bound)) fix = 1;
+      if (nc < k || !(ez[kth] > bound)) need_fix[s] = 1;
     }
-    need_fix[s] = fix;
   }
 }
 
@@ -514,12 +527,23 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   int nslices = c->num_sms / groups;
   if (nslices < 1) nslices = 1;
   if (nslices > ntiles) nslices = ntiles;
-  if (TC_SPLIT * nslices * cap > RF_MAXC) nslices = RF_MAXC / (TC_SPLIT * cap);
-  // work space: the norm bound, the flags, the candidate buffers of every slice and their fill
+  if (TC_SPLIT * nslices > 512) nslices = 512 / TC_SPLIT;       // k_tc_refine's table of buffer offsets
+  // threshold pass: every `stride`-th tile, at most TAU_MAX_TILES of them
+  constexpr int TAU_MAX_TILES = 128;
+  int stride = TC_SUBSET;
+  if ((ntiles + stride - 1) / stride > TAU_MAX_TILES) stride = (ntiles + TAU_MAX_TILES - 1) / TAU_MAX_TILES;
+  const int nsub = (ntiles + stride - 1) / stride;
+  const int dump_cols = nsub * TC_N;
+  int nslices_sub = nslices < nsub ? nslices : nsub;
+  // work space: the norm bound, the flags, the thresholds, the candidate buffers of every slice and their fill, the
+  // threshold pass's scores
   const int Bpad = groups * TC_M;
-  const size_t off_fix = 256, off_cnt = off_fix + (((size_t)batch * 4 + 255) & ~(size_t)255);
-  const size_t off_cand = off_cnt + (((size_t)TC_SPLIT * nslices * Bpad * 4 + 255) & ~(size_t)255);
-  const size_t need = off_cand + (size_t)TC_SPLIT * nslices * Bpad * TC_GBUF * sizeof(int2);
+  const int nvs = TC_SPLIT * nslices;
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  const size_t off_fix = 256, off_tau = off_fix + up((size_t)Bpad * 4), off_cnt = off_tau + up((size_t)Bpad * 4);
+  const size_t off_cand = off_cnt + up((size_t)nvs * Bpad * 4);
+  const size_t off_dump = off_cand + up((size_t)nvs * Bpad * TC_GBUF * sizeof(int2));
+  const size_t need = off_dump + (size_t)Bpad * dump_cols * 4;
   cudaError_t e;
   if (need > c->pd_cap) {
     if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) return e;
@@ -531,27 +555,37 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   unsigned char* ws = reinterpret_cast<unsigned char*>(c->pd_part);
   unsigned int* norm2 = reinterpret_cast<unsigned int*>(ws);
   int* need_fix = reinterpret_cast<int*>(ws + off_fix);
+  float* tau = reinterpret_cast<float*>(ws + off_tau);
   int* cand_cnt = reinterpret_cast<int*>(ws + off_cnt);
   int2* cand = reinterpret_cast<int2*>(ws + off_cand);
+  float* dump = reinterpret_cast<float*>(ws + off_dump);
 
   CUtensorMap tmH, tmW;
   if (!make_map(&tmH, c->h, c->cfg.max_batch, c->H) || !make_map(&tmW, c->W2, c->N, c->H)) return cudaErrorInvalidValue;
 
-  if ((e = cudaMemsetAsync(norm2, 0, sizeof(unsigned int), c->stream)) != cudaSuccess) return e;
+  // the norm bound and the flags start at zero (one clear: they are neighbours)
+  if ((e = cudaMemsetAsync(ws, 0, off_tau, c->stream)) != cudaSuccess) return e;
   k_row_norm_max<<<c->num_sms * 8, 256, 0, c->stream>>>(c->W2, c->N, c->H, norm2);
 
   TcParams p;
-  p.hdr2 = c->hdr2; p.cand = cand; p.cand_cnt = cand_cnt; p.st = c->dstate;
-  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.nslices = nslices; p.ntiles = ntiles;
+  p.hdr2 = c->hdr2; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.st = c->dstate;
+  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.dump_cols = dump_cols;
   const size_t tile_bytes = (size_t)(c->H / TC_KB) * TC_SUB_BYTES;
   const size_t smem = 1024 + tile_bytes * (1 + TC_STAGES) + 2 * TC_N * 4 + 16 * 8 + 64;
-  if ((e = cudaFuncSetAttribute(k_dense_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(k_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(k_dense_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  const size_t tau_smem = (size_t)dump_cols * 4;
+  if ((e = cudaFuncSetAttribute(k_tc_tau, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tau_smem)) != cudaSuccess) return e;
   {
     LaunchScope ls(c, KID_PREDICT);
-    k_dense_tc<<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmH, tmW, p);
+    p.nslices = nslices_sub; p.ntiles = nsub; p.tile_stride = stride;
+    k_dense_tc<true><<<dim3(nslices_sub, groups), TC_THREADS, smem, c->stream>>>(tmH, tmW, p);
+    k_tc_tau<<<Bpad, TAU_THREADS, tau_smem, c->stream>>>(dump, dump_cols, cap, tau);
+    p.nslices = nslices; p.ntiles = ntiles; p.tile_stride = 1;
+    k_dense_tc<false><<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmH, tmW, p);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  k_tc_refine<<<batch, RF_THREADS, 0, c->stream>>>(c->W2, c->hdr2, c->h, cand, cand_cnt, Bpad, norm2, batch, c->H, c->N, cap, TC_SPLIT * nslices, k,
+  k_tc_refine<<<batch, RF_THREADS, 0, c->stream>>>(c->W2, c->hdr2, c->h, cand, cand_cnt, tau, Bpad, norm2, batch, c->H, c->N, cap, nvs, k,
                                                    out_ids, out_scores, need_fix);
   const size_t fx_smem = ((size_t)c->H + 2 * (FX_THREADS / 32) * k + FX_THREADS / 32) * 4;
   k_tc_fixup<<<batch, FX_THREADS, fx_smem, c->stream>>>(c->W2, c->hdr2, c->h, need_fix, c->H, c->N, k, out_ids, out_scores);
