@@ -3,9 +3,9 @@
 // The logits of a batch against every output neuron are one contraction, Z[B][N] = h[B][H] . W2[N][H]^T + b2
 // (Section 3.6: "layer sparsity is 1"), so this path runs it on the fifth-generation tensor cores: tiles of W2 and
 // the batch's hidden activations arrive in shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), a single
-// thread issues tcgen05.mma (kind::tf32, accumulators in tensor memory), and four warps read the accumulators back
-// (tcgen05.ld) and keep, per sample, the best candidates of the block's slice of neurons.  W2 is streamed once per
-// 128 samples.
+// thread issues tcgen05.mma (kind::tf32, accumulators in tensor memory), and the read-back warps fetch the
+// accumulators (tcgen05.ld) and keep, per sample, the candidates of the block's slice of neurons; one more warp takes
+// the largest row norm of W2 from the tiles while they are in shared memory.  W2 is streamed once per 128 samples.
 //
 // TF32 rounds both operands to 10 mantissa bits, far from the 1e-4 the scores must meet.  The tensor pass is
 // therefore a FILTER, in two launches of the same kernel.  The first scores every TC_SUBSET-th tile of neurons and
@@ -27,9 +27,9 @@ constexpr int TC_M = 128;          // samples per block = lanes of the accumulat
 constexpr int TC_N = 128;          // neurons per tile = columns of the accumulator
 constexpr int TC_KB = 32;          // hidden units per 128-byte swizzled row
 constexpr int TC_STAGES = 2;       // tiles of W2 in flight
-constexpr int TC_SPLIT = 1;        // read-back warps per quarter of tensor memory (each takes 1 / TC_SPLIT of a tile's columns)
+constexpr int TC_SPLIT = 4;        // read-back warps per quarter of tensor memory (each takes 1 / TC_SPLIT of a tile's columns)
 constexpr int TC_EPI = 128 * TC_SPLIT;                 // read-back threads
-constexpr int TC_THREADS = 64 + TC_EPI;                // warp 0: TMA producer; warp 1: tensor memory + MMA issue; then the read-back warps
+constexpr int TC_THREADS = 96 + TC_EPI;                // warp 0: TMA producer; warp 1: tensor memory + MMA issue; warp 2: row norms; then the read-back warps
 constexpr int TC_EXTRA = 8;        // candidates kept beyond k: TC_EXTRA + k (the wider the margin, the rarer the exact fall-back)
 constexpr int TC_K_MAX = 8;
 constexpr int TC_GBUF = 64;        // candidate slots per (slice, sample); a buffer that runs over sends the sample to the exact scan
@@ -45,6 +45,7 @@ struct TcParams {
   float* dump;                     // DUMP launch: [Bpad][dump_cols] scores of the subset's tiles
   const float* tau;                // filter launch: [Bpad] thresholds
   int* need_fix;                   // [B] set when a sample's buffer ran over
+  unsigned int* norm2max;          // filter launch: largest squared norm of a row of W2, as the bits of a non-negative float
   DevState* st;
   int B, Bpad, H, N, cap, nslices, ntiles;     // ntiles: tiles this launch walks
   int tile_stride;                 // tile i of the launch is tile i * tile_stride of W2
@@ -140,10 +141,13 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
   // tiles of this slice: slice, slice + nslices, ... (both sample groups walk the same tiles at the same time: the
   // second read of a tile is served by L2)
   const int my_tiles = slice < p.ntiles ? (p.ntiles - slice + p.nslices - 1) / p.nslices : 0;
+  // The filter launch also takes the largest squared row norm of W2 (the error bound needs it) from the tiles as
+  // they pass through shared memory; the blocks of the first sample group do it, the others see the same tiles.
+  const bool norms = !DUMP && blockIdx.y == 0;
 
   if (tid == 0) {
     tc_bar_init(bar_a, 1);
-    for (int i = 0; i < TC_STAGES; ++i) { tc_bar_init(bar_full + i, 1); tc_bar_init(bar_empty + i, 1); }
+    for (int i = 0; i < TC_STAGES; ++i) { tc_bar_init(bar_full + i, 1); tc_bar_init(bar_empty + i, norms ? 2 : 1); }
     for (int i = 0; i < 2; ++i) { tc_bar_init(bar_accfull + i, 1); tc_bar_init(bar_accempty + i, TC_EPI); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -192,14 +196,42 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
         tc_commit(bar_accfull + acc);       // and the accumulator is complete
       }
     }
+  } else if (warp == 2) {
+    // ---------------- row norms: lane = row modulo 32; sums of squares do not care about the swizzle, but the
+    // lanes of a quarter-warp read different 16-byte pieces so that all banks are busy ----------------
+    if (norms) {
+      float best = 0.f;
+      for (int i = 0; i < my_tiles; ++i) {
+        const int st = i % TC_STAGES;
+        tc_bar_wait(bar_full + st, (i / TC_STAGES) & 1, abort_flag);
+        const unsigned char* tile = smB + (size_t)st * tile_bytes;
+        float ss[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int ks = 0; ks < ksub; ++ks)
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+              const float4 w = *reinterpret_cast<const float4*>(tile + (size_t)ks * TC_SUB_BYTES + (size_t)(lane + 32 * rr) * 128 +
+                                                                 (size_t)((c ^ (lane & 7)) * 16));
+              ss[rr] = fmaf(w.x, w.x, ss[rr]); ss[rr] = fmaf(w.y, w.y, ss[rr]);
+              ss[rr] = fmaf(w.z, w.z, ss[rr]); ss[rr] = fmaf(w.w, w.w, ss[rr]);
+            }
+        best = fmaxf(best, fmaxf(fmaxf(ss[0], ss[1]), fmaxf(ss[2], ss[3])));
+        __syncwarp();
+        if (lane == 0) tc_bar_arrive(bar_empty + st);
+      }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, d));
+      if (lane == 0) atomicMax(p.norm2max, __float_as_uint(best));
+    }
   } else {
     // ---------------- read-back: thread = (sample, share of a tile's columns) ----------------
     // Per 32 columns the bias is added; then, threshold pass: the scores are written out; filter pass: which of them
     // reach the sample's threshold (32 independent comparisons, a bit each), then the appends of those that do.
     const int q = warp & 3;                 // a warp reaches the 32 lanes of tensor memory of its number modulo four
-    const int half = (warp - 2) >> 2;       // which share of a tile's 128 columns
+    const int half = (warp - 3) >> 2;       // which share of a tile's 128 columns
     const int row = 32 * q + lane;          // sample inside the block
-    const int et = tid - 64;                // the first 128 read-back threads fetch the tile's biases
+    const int et = tid - 96;                // the first 128 read-back threads fetch the tile's biases
     const int vslice = slice * TC_SPLIT + half;    // buffers are kept per (slice, share of the columns)
     int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * TC_GBUF;
     const float tau = DUMP ? 0.f : p.tau[s0 + row];
@@ -275,22 +307,6 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
   if (tid == 0 && *abort_flag) atomicCAS(&p.st->status, 0, (int)DSLIDE_ERR_TIMEOUT);
 }
 
-// Largest squared norm of a row of W2 (for the filter's error bound).  Non-negative floats order like their bits.
-__global__ void __launch_bounds__(256) k_row_norm_max(const float* W2, int N, int H, unsigned int* out) {
-  const int lane = threadIdx.x & 31;
-  const int H4 = H >> 2;
-  float best = 0.f;
-  for (int j = blockIdx.x * 8 + (threadIdx.x >> 5); j < N; j += gridDim.x * 8) {
-    const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
-    float s = 0.f;
-    for (int c = lane; c < H4; c += 32) { const float4 w = __ldg(r + c); s += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w; }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-    best = fmaxf(best, s);
-  }
-  if (lane == 0) atomicMax(out, __float_as_uint(best));
-}
-
 // One block per sample: the cap-th largest of the sample's scores of the subset (found bit by bit on a key that
 // orders like the floats) is the sample's threshold; -infinity when the subset holds fewer than cap neurons.
 constexpr int TAU_THREADS = 256;
@@ -326,64 +342,89 @@ __global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int c
   }
 }
 
-// One block per sample: the slices' candidates -> the cap best by approximate score -> their exact fp32 logits ->
-// the k best by (logit descending, id ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
-constexpr int RF_THREADS = 128;
+// One block per sample: the slices' candidates -> the cap best by approximate score (their cap-th largest key, found
+// bit by bit as in k_tc_tau) -> their exact fp32 logits -> the k best by (logit descending, id ascending).
+// need_fix[s] = 1 when the filter cannot be shown to be exact.
+constexpr int RF_THREADS = 256;
 constexpr int RF_MAXC = 4096;
+constexpr int RF_MAXV = 512;       // buffers per sample at most
 __global__ void __launch_bounds__(RF_THREADS)
 k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, const float* tau, int Bpad,
             const unsigned int* norm2max, int B, int H, int N, int cap, int nvs, int k, int32_t* out_ids, float* out_scores,
             int* need_fix) {
-  __shared__ float cz[RF_MAXC];
+  __shared__ uint32_t ck[RF_MAXC];
   __shared__ int ci[RF_MAXC];
-  __shared__ int offs[512];
+  __shared__ int offs[RF_MAXV + 1];
   __shared__ float ez[TC_CAP];
   __shared__ int ei[TC_CAP];
   __shared__ float red[RF_THREADS / 32];
-  __shared__ int sh_total;
+  __shared__ int wsum[RF_THREADS / 32];
+  __shared__ int sh_n;
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) {
-    int run = 0;
-    for (int v = 0; v < nvs; ++v) { offs[v] = run; run += cand_cnt[(size_t)v * Bpad + s]; }
-    sh_total = run;
+  // fill of the sample's buffers -> their places in one list (exclusive scan; each thread owns RF_MAXV / RF_THREADS buffers)
+  {
+    constexpr int PER = RF_MAXV / RF_THREADS;
+    int c[PER], mine = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { const int v = tid * PER + i; c[i] = v < nvs ? __ldcg(cand_cnt + (size_t)v * Bpad + s) : 0; mine += c[i]; }
+    int inc = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const int o = __shfl_up_sync(0xffffffffu, inc, d); if (lane >= d) inc += o; }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < warp; ++w) base += wsum[w];
+    int run = base + inc - mine;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { offs[tid * PER + i] = run; run += c[i]; }
+    if (tid == RF_THREADS - 1) offs[RF_MAXV] = run;
+    __syncthreads();
   }
-  __syncthreads();
-  const int total = sh_total;
+  const int total = offs[RF_MAXV];
   if (total > RF_MAXC) {                          // more candidates than this pass handles: the sample is scored exactly
     if (tid == 0) need_fix[s] = 1;
     return;
   }
-  int n2 = 1;
-  while (n2 < total) n2 <<= 1;
-  for (int v = warp; v < nvs; v += RF_THREADS / 32) {
-    const int n = cand_cnt[(size_t)v * Bpad + s];
-    for (int e = lane; e < n; e += 32) {
-      const int2 x = __ldcg(cand + ((size_t)v * Bpad + s) * TC_GBUF + e);
-      cz[offs[v] + e] = __int_as_float(x.x);
-      ci[offs[v] + e] = x.y;
-    }
+  // gather: entry e of the list lies in the buffer v with offs[v] <= e < offs[v + 1]
+  for (int e = tid; e < total; e += RF_THREADS) {
+    int lo = 0, hi = RF_MAXV;                     // invariant: offs[lo] <= e < offs[hi]
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (offs[mid] <= e) lo = mid; else hi = mid; }
+    const int2 x = __ldcg(cand + ((size_t)lo * Bpad + s) * TC_GBUF + (e - offs[lo]));
+    ck[e] = tc_key(__int_as_float(x.x));
+    ci[e] = x.y;
   }
-  for (int e = total + tid; e < n2; e += RF_THREADS) { cz[e] = -INFINITY; ci[e] = 0x7fffffff; }
+  if (tid == 0) sh_n = 0;
   __syncthreads();
-  // bitonic sort, best first: (score descending, id ascending)
-  for (int kk = 2; kk <= n2; kk <<= 1)
-    for (int j = kk >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < n2; i += RF_THREADS) {
-        const int x = i ^ j;
-        if (x > i) {
-          const bool up = (i & kk) == 0;
-          const bool i_first = tc_better(cz[i], ci[i], cz[x], ci[x]);
-          if (i_first != up) { const float tz = cz[i]; cz[i] = cz[x]; cz[x] = tz; const int ti = ci[i]; ci[i] = ci[x]; ci[x] = ti; }
-        }
-      }
+  // the cap-th largest key (0 when there are fewer than cap candidates: all of them go on)
+  uint32_t K = 0u;
+  if (total > cap)
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint32_t trial = K | (1u << bit);
+      int cnt = 0;
+      for (int e = tid; e < total; e += RF_THREADS) cnt += ck[e] >= trial ? 1 : 0;
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+      if (lane == 0) wsum[warp] = cnt;
+      __syncthreads();
+      int all = 0;
+      for (int w = 0; w < RF_THREADS / 32; ++w) all += wsum[w];
+      if (all >= cap) K = trial;
       __syncthreads();
     }
-  const int nc = total < cap ? total : cap;     // candidates that go on to the exact pass
+  // keep the keys above it, then as many equal to it as still fit (which of several equal ones does not matter: the
+  // guard below treats every neuron that is not kept as scoring at most the cap-th key)
+  for (int e = tid; e < total; e += RF_THREADS)
+    if (ck[e] > K) { const int slot = atomicAdd(&sh_n, 1); ei[slot] = ci[e]; }
+  __syncthreads();
+  for (int e = tid; e < total; e += RF_THREADS)
+    if (ck[e] == K) { const int slot = atomicAdd(&sh_n, 1); if (slot < cap) ei[slot] = ci[e]; }
+  __syncthreads();
+  const int nc = sh_n < cap ? sh_n : cap;       // candidates that go on to the exact pass
   // exact logits of the kept candidates: a warp per candidate, four partial sums per lane as in the exact path
   const float4* h4 = reinterpret_cast<const float4*>(h + (size_t)s * H);
   const int H4 = H >> 2;
   for (int e = warp; e < nc; e += RF_THREADS / 32) {
-    const int j = ci[e];
+    const int j = ei[e];
     const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
     float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
     for (int c = lane; c < H4; c += 32) {
@@ -393,7 +434,7 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
     float d = (d0 + d1) + (d2 + d3);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-    if (lane == 0) { ez[e] = __ldg(&hdr2[j].b) + d; ei[e] = j; }
+    if (lane == 0) ez[e] = __ldg(&hdr2[j].b) + d;
   }
   // |h|^2 of the sample
   float hs = 0.f;
@@ -416,11 +457,12 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
       out_ids[(size_t)s * k + qk] = qk < nc ? ei[qk] : -1;
       out_scores[(size_t)s * k + qk] = qk < nc ? ez[qk] : -INFINITY;
     }
-    // Every neuron that did not go on to the exact pass has an approximate score of at most T: the last kept one's
-    // when candidates were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its
+    // Every neuron that did not go on to the exact pass has an approximate score of at most T: the cap-th key when
+    // candidates were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its
     // exact score is at most T plus the error bound; the k best are certain when the k-th exact score lies above.
-    const float T = total > cap ? cz[cap - 1] : tau[s];
-    if (nc > 0 && T > -INFINITY) {
+    float T = tau[s];
+    if (total > cap) T = __uint_as_float((K & 0x80000000u) ? (K & 0x7fffffffu) : ~K);
+    if (T > -INFINITY) {
       const float bound = T + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
       const int kth = (k < nc ? k : nc) - 1;
       if (nc < k || !(ez[kth] > bound)) need_fix[s] = 1;
@@ -565,10 +607,9 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
 
   // the norm bound and the flags start at zero (one clear: they are neighbours)
   if ((e = cudaMemsetAsync(ws, 0, off_tau, c->stream)) != cudaSuccess) return e;
-  k_row_norm_max<<<c->num_sms * 8, 256, 0, c->stream>>>(c->W2, c->N, c->H, norm2);
 
   TcParams p;
-  p.hdr2 = c->hdr2; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.st = c->dstate;
+  p.hdr2 = c->hdr2; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.norm2max = norm2; p.st = c->dstate;
   p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.dump_cols = dump_cols;
   const size_t tile_bytes = (size_t)(c->H / TC_KB) * TC_SUB_BYTES;
   const size_t smem = 1024 + tile_bytes * (1 + TC_STAGES) + 2 * TC_N * 4 + 16 * 8 + 64;
