@@ -142,8 +142,9 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
   // second read of a tile is served by L2)
   const int my_tiles = slice < p.ntiles ? (p.ntiles - slice + p.nslices - 1) / p.nslices : 0;
   // The filter launch also takes the largest squared row norm of W2 (the error bound needs it) from the tiles as
-  // they pass through shared memory; the blocks of the first sample group do it, the others see the same tiles.
-  const bool norms = !DUMP && blockIdx.y == 0;
+  // they pass through shared memory; up to four sample groups share a tile's rows (they all see the same tiles).
+  const int nshare = gridDim.y >= 4 ? 4 : (gridDim.y >= 2 ? 2 : 1);      // blocks that share a tile's 128 rows
+  const bool norms = !DUMP && (int)blockIdx.y < nshare;
 
   if (tid == 0) {
     tc_bar_init(bar_a, 1);
@@ -205,18 +206,21 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
         const int st = i % TC_STAGES;
         tc_bar_wait(bar_full + st, (i / TC_STAGES) & 1, abort_flag);
         const unsigned char* tile = smB + (size_t)st * tile_bytes;
-        float ss[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int ks = 0; ks < ksub; ++ks)
+        const int nrr = 4 / nshare;                    // rows of this block: nrr per lane
+        for (int rr = 0; rr < nrr; ++rr) {
+          const unsigned char* rowp = tile + (size_t)(32 * (nrr * (int)blockIdx.y + rr) + lane) * 128;
+          unsigned long long s0 = 0ull, s1 = 0ull;    // two pairs of partial sums (packed fp32 fused multiply-adds)
+          for (int ks = 0; ks < ksub; ++ks)
 #pragma unroll
-          for (int c = 0; c < 8; ++c)
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-              const float4 w = *reinterpret_cast<const float4*>(tile + (size_t)ks * TC_SUB_BYTES + (size_t)(lane + 32 * rr) * 128 +
-                                                                 (size_t)((c ^ (lane & 7)) * 16));
-              ss[rr] = fmaf(w.x, w.x, ss[rr]); ss[rr] = fmaf(w.y, w.y, ss[rr]);
-              ss[rr] = fmaf(w.z, w.z, ss[rr]); ss[rr] = fmaf(w.w, w.w, ss[rr]);
+            for (int c = 0; c < 8; ++c) {
+              const ulonglong2 w = *reinterpret_cast<const ulonglong2*>(rowp + (size_t)ks * TC_SUB_BYTES + (size_t)((c ^ (lane & 7)) * 16));
+              asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(s0) : "l"(w.x));
+              asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(s1) : "l"(w.y));
             }
-        best = fmaxf(best, fmaxf(fmaxf(ss[0], ss[1]), fmaxf(ss[2], ss[3])));
+          const float ssum = (__uint_as_float((unsigned)s0) + __uint_as_float((unsigned)(s0 >> 32))) +
+                             (__uint_as_float((unsigned)s1) + __uint_as_float((unsigned)(s1 >> 32)));
+          best = fmaxf(best, ssum);
+        }
         __syncwarp();
         if (lane == 0) tc_bar_arrive(bar_empty + st);
       }
@@ -236,11 +240,18 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
     int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * TC_GBUF;
     const float tau = DUMP ? 0.f : p.tau[s0 + row];
     int cnt = 0;
+    // a tile's biases are asked for one tile ahead, so that their latency is not part of the tile's read-back
+    auto bias_of = [&](int i) {
+      const int j = (slice + i * p.nslices) * p.tile_stride * TC_N + et;
+      return et < TC_N && i < my_tiles && j < p.N ? __ldg(&p.hdr2[j].b) : 0.f;
+    };
+    float bias_next = bias_of(0);
     for (int i = 0; i < my_tiles; ++i) {
       const int acc = i & 1;
       const int tile = slice + i * p.nslices;
       const int j0 = tile * p.tile_stride * TC_N;
-      if (et < TC_N) sb[acc * TC_N + et] = j0 + et < p.N ? __ldg(&p.hdr2[j0 + et].b) : 0.f;
+      if (et < TC_N) sb[acc * TC_N + et] = bias_next;
+      bias_next = bias_of(i + 1);
       tc_bar_wait(bar_accfull + acc, (i >> 1) & 1, abort_flag);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       asm volatile("bar.sync 1, %0;" ::"n"(TC_EPI) : "memory");          // the tile's biases are in place
@@ -278,16 +289,20 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
           }
         } else {
           if (p.N - jb < 32) hm &= p.N > jb ? (1u << (p.N - jb)) - 1u : 0u;      // neurons past the end (last tile only)
-#pragma unroll
-          for (int g = 0; g < 4; ++g)
-            if ((hm >> (8 * g)) & 0xffu) {
-#pragma unroll
-              for (int c = 8 * g; c < 8 * g + 8; ++c)
-                if ((hm >> c) & 1u) {
-                  if (cnt < TC_GBUF) __stcg(mybuf + cnt, make_int2((int)r[c], jb + c));
-                  ++cnt;
-                }
+          // the columns that some sample of the warp keeps (few): one more read of that column, same sum as above
+          unsigned any = __reduce_or_sync(0xffffffffu, hm);
+          while (any) {
+            const int c = __ffs(any) - 1;
+            any &= any - 1;
+            uint32_t raw;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\n\ttcgen05.wait::ld.sync.aligned;"
+                         : "=r"(raw) : "r"(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * TC_N + c0 + c)) : "memory");
+            if ((hm >> c) & 1u) {
+              const float z = __uint_as_float(raw) + sb[acc * TC_N + c0 + c];
+              if (cnt < TC_GBUF) __stcg(mybuf + cnt, make_int2(__float_as_int(z), jb + c));
+              ++cnt;
             }
+          }
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
