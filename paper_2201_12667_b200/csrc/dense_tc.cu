@@ -26,7 +26,9 @@ namespace dslide {
 constexpr int TC_M = 128;          // samples per block = lanes of the accumulator
 constexpr int TC_N = 128;          // neurons per tile = columns of the accumulator
 constexpr int TC_KB = 32;          // hidden units per 128-byte swizzled row
-constexpr int TC_STAGES = 2;       // tiles of W2 in flight
+constexpr int TC_STAGES = 3;       // tiles of W2 in flight at most (as many as fit in shared memory)
+constexpr int TC_NACC = 3;         // tensor memory: up to three accumulators of TC_N columns (two when H > TC_N), then the activations (H columns)
+constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_SPLIT = 4;        // read-back warps per quarter of tensor memory (each takes 1 / TC_SPLIT of a tile's columns)
 constexpr int TC_EPI = 128 * TC_SPLIT;                 // read-back threads
 constexpr int TC_THREADS = 96 + TC_EPI;                // warp 0: TMA producer; warp 1: tensor memory + MMA issue; warp 2: row norms; then the read-back warps
@@ -40,6 +42,7 @@ constexpr float TC_ERR = 2.2e-3f;  // |approximate - exact| <= TC_ERR * |h| * |w
 
 struct TcParams {
   const RowHdr* hdr2;
+  const float* h;                  // [>= B][H] hidden activations of the batch
   int2* cand;                      // [TC_SPLIT * slices][Bpad][TC_GBUF] (score bits, id), cand_cnt of them valid, no order
   int* cand_cnt;                   // [TC_SPLIT * slices][Bpad]
   float* dump;                     // DUMP launch: [Bpad][dump_cols] scores of the subset's tiles
@@ -49,6 +52,7 @@ struct TcParams {
   DevState* st;
   int B, Bpad, H, N, cap, nslices, ntiles;     // ntiles: tiles this launch walks
   int tile_stride;                 // tile i of the launch is tile i * tile_stride of W2
+  int stages;                      // tiles of W2 in flight, 1 .. TC_STAGES
   int dump_cols;
 };
 
@@ -66,10 +70,10 @@ __device__ __forceinline__ void tc_bar_arrive(uint64_t* bar) {
 // all the roles run through their loops, tensor memory is released and the kernel ends (its results are flagged).
 __device__ __forceinline__ void tc_bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
   const uint32_t a = tc_smem(bar);
-  for (int it = 0; it < (1 << 22); ++it) {
+  for (int it = 0; it < (1 << 20); ++it) {
     uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity), "r"(2000u) : "memory");      // may sleep up to 2 us per try: a waiting warp issues little
     if (ok) return;
     if ((it & 1023) == 1023 && *abort) return;
   }
@@ -93,9 +97,20 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr) {
 __host__ __device__ constexpr uint32_t tc_idesc(int M, int N) {
   return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+// D[tmem] (+)= A[tmem] . B[smem]^T: the first operand is read from tensor memory, so shared memory serves one operand only
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, "
+      "%19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem(bar)) : "memory");
@@ -115,25 +130,25 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ bool tc_better(float za, int ia, float zb, int ib) { return za > zb || (za == zb && ia < ib); }
 
 // Grid: (slices of the neurons, groups of 128 samples).  Dynamic shared memory (1024-byte aligned):
-// activations [H/32][128 rows][128 B], then TC_STAGES tiles of W2 in the same form, then
+// TC_STAGES tiles of W2 as [H/32][128 rows][128 B], then
 // the tiles' biases, the barriers.  (The samples' candidate buffers are in global memory.)
 template <bool DUMP>      // DUMP: write every score out (threshold pass); else append the scores that reach the sample's threshold
 __global__ void __launch_bounds__(TC_THREADS, 1)
-k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, const TcParams p) {
+k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
   extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
   const int ksub = p.H / TC_KB;
   const uint32_t tile_bytes = (uint32_t)ksub * TC_SUB_BYTES;
-  unsigned char* smA = sm;
-  unsigned char* smB = sm + tile_bytes;
-  float* sb = reinterpret_cast<float*>(smB + (size_t)TC_STAGES * tile_bytes);                         // [2][128] biases of the tile
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sb + 2 * TC_N);
-  uint64_t* bar_a = bars;                      // activations have arrived
+  unsigned char* smB = sm;
+  const int nst = p.stages;
+  float* sb = reinterpret_cast<float*>(smB + (size_t)nst * tile_bytes);                         // [accumulator][128] biases of its tile
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sb + TC_NACC * TC_N);
+  uint64_t* bar_a = bars;                      // activations are in tensor memory
   uint64_t* bar_full = bars + 1;               // [TC_STAGES] tile of W2 has arrived
   uint64_t* bar_empty = bars + 1 + TC_STAGES;  // [TC_STAGES] tile of W2 has been consumed
-  uint64_t* bar_accfull = bars + 1 + 2 * TC_STAGES;   // [2] accumulator written
-  uint64_t* bar_accempty = bars + 3 + 2 * TC_STAGES;  // [2] accumulator read back
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5 + 2 * TC_STAGES);
+  uint64_t* bar_accfull = bars + 1 + 2 * TC_STAGES;              // [TC_NACC] accumulator written
+  uint64_t* bar_accempty = bars + 1 + 2 * TC_STAGES + TC_NACC;   // [TC_NACC] accumulator read back
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 1 + 2 * TC_STAGES + 2 * TC_NACC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -145,16 +160,18 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
   // they pass through shared memory; up to four sample groups share a tile's rows (they all see the same tiles).
   const int nshare = gridDim.y >= 4 ? 4 : (gridDim.y >= 2 ? 2 : 1);      // blocks that share a tile's 128 rows
   const bool norms = !DUMP && (int)blockIdx.y < nshare;
+  const int nacc = p.H <= TC_N ? TC_NACC : 2;      // accumulators in use; the activations follow them
+  const uint32_t acol = (uint32_t)(nacc * TC_N);
 
   if (tid == 0) {
-    tc_bar_init(bar_a, 1);
+    tc_bar_init(bar_a, 128);
     for (int i = 0; i < TC_STAGES; ++i) { tc_bar_init(bar_full + i, 1); tc_bar_init(bar_empty + i, norms ? 2 : 1); }
-    for (int i = 0; i < 2; ++i) { tc_bar_init(bar_accfull + i, 1); tc_bar_init(bar_accempty + i, TC_EPI); }
+    for (int i = 0; i < TC_NACC; ++i) { tc_bar_init(bar_accfull + i, 1); tc_bar_init(bar_accempty + i, TC_EPI); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {      // tensor memory: two accumulators of 128 columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem(tmem_slot)), "r"(2 * TC_N) : "memory");
+  if (warp == 1) {      // tensor memory: all of it (one block per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem(tmem_slot)), "r"(TC_TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -165,15 +182,14 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
   if (warp == 0) {
     // ---------------- producer: one thread feeds the TMA ----------------
     if (lane == 0) {
-      tc_bar_expect(bar_a, tile_bytes);
-      for (int ks = 0; ks < ksub; ++ks) tc_tma_2d(smA + (size_t)ks * TC_SUB_BYTES, &tmH, ks * TC_KB, s0, bar_a);
+      int st = 0, stround = 0;
       for (int i = 0; i < my_tiles; ++i) {
-        const int st = i % TC_STAGES;
-        if (i >= TC_STAGES) tc_bar_wait(bar_empty + st, ((i / TC_STAGES) - 1) & 1, abort_flag);
+        if (stround > 0) tc_bar_wait(bar_empty + st, (stround - 1) & 1, abort_flag);
         const int row0 = (slice + i * p.nslices) * p.tile_stride * TC_N;
         tc_bar_expect(bar_full + st, tile_bytes);
         for (int ks = 0; ks < ksub; ++ks)
           tc_tma_2d(smB + (size_t)st * tile_bytes + (size_t)ks * TC_SUB_BYTES, &tmW, ks * TC_KB, row0, bar_full + st);
+        if (++st == nst) { st = 0; ++stround; }
       }
     }
   } else if (warp == 1) {
@@ -181,20 +197,25 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
     if (lane == 0) {
       const uint32_t idesc = tc_idesc(TC_M, TC_N);
       tc_bar_wait(bar_a, 0, abort_flag);
+      const uint64_t b_base = tc_desc(tc_smem(smB));      // a descriptor's address field counts 16-byte units
+      int st = 0, stround = 0, acc = 0, accround = 0;
       for (int i = 0; i < my_tiles; ++i) {
-        const int st = i % TC_STAGES, acc = i & 1;
-        tc_bar_wait(bar_full + st, (i / TC_STAGES) & 1, abort_flag);
-        if (i >= 2) tc_bar_wait(bar_accempty + acc, ((i >> 1) - 1) & 1, abort_flag);
+        tc_bar_wait(bar_full + st, stround & 1, abort_flag);
+        if (accround > 0) tc_bar_wait(bar_accempty + acc, (accround - 1) & 1, abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d = tmem_base + (uint32_t)(acc * TC_N);
-        for (int ks = 0; ks < ksub; ++ks)
-          for (int kk = 0; kk < TC_KB / 8; ++kk) {            // eight tf32 = 32 bytes per instruction
-            const uint64_t a = tc_desc(tc_smem(smA + (size_t)ks * TC_SUB_BYTES) + (uint32_t)kk * 32u);
-            const uint64_t b = tc_desc(tc_smem(smB + (size_t)st * tile_bytes + (size_t)ks * TC_SUB_BYTES) + (uint32_t)kk * 32u);
-            tc_mma(d, a, b, idesc, (ks | kk) != 0 ? 1u : 0u);
-          }
+        const uint64_t b_tile = b_base + (uint64_t)(((uint32_t)st * tile_bytes) >> 4);
+        for (int ks = 0; ks < ksub; ++ks) {
+          const uint32_t a = tmem_base + acol + (uint32_t)(ks * TC_KB);      // lanes = samples, columns = hidden units
+          const uint64_t b = b_tile + (uint64_t)((ks * TC_SUB_BYTES) >> 4);
+#pragma unroll
+          for (int kk = 0; kk < TC_KB / 8; ++kk)              // eight tf32 = 32 bytes per instruction
+            tc_mma(d, a + (uint32_t)(kk * 8), b + (uint64_t)(kk * 2), idesc, (ks | kk) != 0 ? 1u : 0u);
+        }
         tc_commit(bar_empty + st);          // the tile's shared memory is free once these instructions have read it
         tc_commit(bar_accfull + acc);       // and the accumulator is complete
+        if (++st == nst) { st = 0; ++stround; }
+        if (++acc == nacc) { acc = 0; ++accround; }
       }
     }
   } else if (warp == 2) {
@@ -202,9 +223,9 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
     // lanes of a quarter-warp read different 16-byte pieces so that all banks are busy ----------------
     if (norms) {
       float best = 0.f;
+      int st = 0, stround = 0;
       for (int i = 0; i < my_tiles; ++i) {
-        const int st = i % TC_STAGES;
-        tc_bar_wait(bar_full + st, (i / TC_STAGES) & 1, abort_flag);
+        tc_bar_wait(bar_full + st, stround & 1, abort_flag);
         const unsigned char* tile = smB + (size_t)st * tile_bytes;
         const int nrr = 4 / nshare;                    // rows of this block: nrr per lane
         for (int rr = 0; rr < nrr; ++rr) {
@@ -223,6 +244,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
         }
         __syncwarp();
         if (lane == 0) tc_bar_arrive(bar_empty + st);
+        if (++st == nst) { st = 0; ++stround; }
       }
 #pragma unroll
       for (int d = 16; d > 0; d >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, d));
@@ -240,21 +262,39 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
     int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * TC_GBUF;
     const float tau = DUMP ? 0.f : p.tau[s0 + row];
     int cnt = 0;
+    if (half == 0) {
+      // the block's activations -> tensor memory: lane = sample, column = hidden unit (samples past the batch: zeros)
+      const float4* hrow = reinterpret_cast<const float4*>(p.h + (size_t)(s0 + row) * p.H);
+      const bool live = s0 + row < p.B;
+      for (int c0 = 0; c0 < p.H; c0 += 32) {
+        uint32_t r[32];
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 v = live ? __ldg(hrow + (c0 >> 2) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          r[4 * c4] = __float_as_uint(v.x); r[4 * c4 + 1] = __float_as_uint(v.y);
+          r[4 * c4 + 2] = __float_as_uint(v.z); r[4 * c4 + 3] = __float_as_uint(v.w);
+        }
+        tc_st32(tmem_base + ((uint32_t)(32 * q) << 16) + acol + (uint32_t)c0, r);
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      tc_bar_arrive(bar_a);
+    }
     // a tile's biases are asked for one tile ahead, so that their latency is not part of the tile's read-back
     auto bias_of = [&](int i) {
       const int j = (slice + i * p.nslices) * p.tile_stride * TC_N + et;
       return et < TC_N && i < my_tiles && j < p.N ? __ldg(&p.hdr2[j].b) : 0.f;
     };
     float bias_next = bias_of(0);
+    int acc = 0, accround = 0;
     for (int i = 0; i < my_tiles; ++i) {
-      const int acc = i & 1;
       const int tile = slice + i * p.nslices;
       const int j0 = tile * p.tile_stride * TC_N;
       if (et < TC_N) sb[acc * TC_N + et] = bias_next;
       bias_next = bias_of(i + 1);
-      tc_bar_wait(bar_accfull + acc, (i >> 1) & 1, abort_flag);
+      if (warp == 3) tc_bar_wait(bar_accfull + acc, accround & 1, abort_flag);      // one warp polls, the others sleep in the barrier
+      asm volatile("bar.sync 1, %0;" ::"n"(TC_EPI) : "memory");          // the accumulator is complete, the tile's biases are in place
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      asm volatile("bar.sync 1, %0;" ::"n"(TC_EPI) : "memory");          // the tile's biases are in place
       for (int c0 = (TC_N / TC_SPLIT) * half; c0 < (TC_N / TC_SPLIT) * (half + 1); c0 += 32) {
         uint32_t r[32];
         tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * TC_N + c0), r);
@@ -307,6 +347,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       tc_bar_arrive(bar_accempty + acc);
+      if (++acc == nacc) { acc = 0; ++accround; }
     }
     if (!DUMP && s0 + row < p.B) {
       p.cand_cnt[(size_t)vslice * p.Bpad + s0 + row] = cnt < TC_GBUF ? cnt : TC_GBUF;
@@ -317,7 +358,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUte
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * TC_N) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicCAS(&p.st->status, 0, (int)DSLIDE_ERR_TIMEOUT);
 }
@@ -617,17 +658,20 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   int2* cand = reinterpret_cast<int2*>(ws + off_cand);
   float* dump = reinterpret_cast<float*>(ws + off_dump);
 
-  CUtensorMap tmH, tmW;
-  if (!make_map(&tmH, c->h, c->cfg.max_batch, c->H) || !make_map(&tmW, c->W2, c->N, c->H)) return cudaErrorInvalidValue;
+  CUtensorMap tmW;
+  if (!make_map(&tmW, c->W2, c->N, c->H)) return cudaErrorInvalidValue;
 
   // the norm bound and the flags start at zero (one clear: they are neighbours)
   if ((e = cudaMemsetAsync(ws, 0, off_tau, c->stream)) != cudaSuccess) return e;
 
   TcParams p;
-  p.hdr2 = c->hdr2; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.norm2max = norm2; p.st = c->dstate;
+  p.hdr2 = c->hdr2; p.h = c->h; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.norm2max = norm2; p.st = c->dstate;
   p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.dump_cols = dump_cols;
   const size_t tile_bytes = (size_t)(c->H / TC_KB) * TC_SUB_BYTES;
-  const size_t smem = 1024 + tile_bytes * (1 + TC_STAGES) + 2 * TC_N * 4 + 16 * 8 + 64;
+  int stages = (int)(((size_t)200 << 10) / tile_bytes);
+  if (stages > TC_STAGES) stages = TC_STAGES;
+  p.stages = stages;
+  const size_t smem = 1024 + tile_bytes * stages + TC_NACC * TC_N * 4 + 24 * 8 + 64;
   if ((e = cudaFuncSetAttribute(k_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k_dense_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   const size_t tau_smem = (size_t)dump_cols * 4;
@@ -635,10 +679,10 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   {
     LaunchScope ls(c, KID_PREDICT);
     p.nslices = nslices_sub; p.ntiles = nsub; p.tile_stride = stride;
-    k_dense_tc<true><<<dim3(nslices_sub, groups), TC_THREADS, smem, c->stream>>>(tmH, tmW, p);
+    k_dense_tc<true><<<dim3(nslices_sub, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
     k_tc_tau<<<Bpad, TAU_THREADS, tau_smem, c->stream>>>(dump, dump_cols, cap, tau);
     p.nslices = nslices; p.ntiles = ntiles; p.tile_stride = 1;
-    k_dense_tc<false><<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmH, tmW, p);
+    k_dense_tc<false><<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   k_tc_refine<<<batch, RF_THREADS, 0, c->stream>>>(c->W2, c->hdr2, c->h, cand, cand_cnt, tau, Bpad, norm2, batch, c->H, c->N, cap, nvs, k,

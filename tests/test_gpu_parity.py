@@ -318,9 +318,12 @@ def test_force_dense_matches_oracle_and_dense_softmax():
 
 
 # ------------------------------------------------------------------ inference
-@pytest.mark.parametrize("dense,k", [(0, 5), (1, 5), (1, 12), (1, 40)])   # over all neurons: 32, 16, 8 samples per block
-def test_predict_topk(dense, k):
-    pr = mid_pair()
+# over all neurons: k <= 8 runs on the tensor pipe when the hidden width allows it (32 .. 256 in steps of 32; one, two or
+# three tiles of W2 in flight), else the fp32 scan with 32, 16, 8 samples per block
+@pytest.mark.parametrize("dense,k,H", [(0, 5, 128), (1, 5, 128), (1, 12, 128), (1, 40, 128), (1, 3, 32), (1, 8, 96), (1, 5, 192),
+                                       (1, 5, 256), (1, 5, 104)])
+def test_predict_topk(dense, k, H):
+    pr = mid_pair(H=H)
     try:
         pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.05)
         pr.push_state()
