@@ -36,7 +36,6 @@ constexpr int TC_EXTRA = 8;        // candidates kept beyond k: TC_EXTRA + k (th
 constexpr int TC_K_MAX = 8;
 constexpr int TC_GBUF = 64;        // candidate slots per (slice, sample); a buffer that runs over sends the sample to the exact scan
 constexpr int TC_SUBSET = 64;      // the threshold pass scores every TC_SUBSET-th tile
-constexpr int TC_CAP = 2 * TC_K_MAX + TC_EXTRA;
 constexpr int TC_SUB_BYTES = TC_M * 128;               // one 32-unit slab of 128 rows
 constexpr float TC_ERR = 2.2e-3f;  // |approximate - exact| <= TC_ERR * |h| * |w|: two operands cut to 10 mantissa bits, fp32 sums
 
@@ -363,47 +362,50 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
   if (tid == 0 && *abort_flag) atomicCAS(&p.st->status, 0, (int)DSLIDE_ERR_TIMEOUT);
 }
 
-// One block per sample: the cap-th largest of the sample's scores of the subset (found bit by bit on a key that
-// orders like the floats) is the sample's threshold; -infinity when the subset holds fewer than cap neurons.
-constexpr int TAU_THREADS = 256;
+// Floats as keys that order like them (unsigned); no real score has key 0.
 __device__ __forceinline__ uint32_t tc_key(float z) {
   const uint32_t b = __float_as_uint(z);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
-__global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int cols, int cap, float* tau) {
-  extern __shared__ uint32_t tau_keys[];        // [cols]
-  __shared__ int wsum[TAU_THREADS / 32];
-  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int e = tid; e < cols; e += TAU_THREADS) tau_keys[e] = tc_key(__ldcg(dump + (size_t)s * cols + e));
-  __syncthreads();
+__device__ __forceinline__ float tc_unkey(uint32_t k) { return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k); }
+// The cap-th largest of the block's per-thread keys, found bit by bit (a block-wide count per bit); 0 when fewer than
+// cap threads hold a key.
+__device__ __forceinline__ uint32_t tc_select(uint32_t mine, int cap) {
   uint32_t K = 0u;
   for (int bit = 31; bit >= 0; --bit) {
     const uint32_t trial = K | (1u << bit);
-    int cnt = 0;
-    for (int e = tid; e < cols; e += TAU_THREADS) cnt += tau_keys[e] >= trial ? 1 : 0;
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
-    if (lane == 0) wsum[warp] = cnt;
-    __syncthreads();
-    int total = 0;
-    for (int w = 0; w < TAU_THREADS / 32; ++w) total += wsum[w];
-    if (total >= cap) K = trial;
-    __syncthreads();
+    if (__syncthreads_count(mine >= trial) >= cap) K = trial;
   }
+  return K;
+}
+
+// One block per sample.  Each thread takes the largest of its share of the sample's scores of the subset; the cap-th
+// largest of these maxima is the sample's threshold.  At least cap neurons of the subset reach it (exactly cap when
+// the cap best fell to different threads); -infinity when the subset is smaller than that.  Any threshold gives the
+// same results: it only decides how many candidates the filter pass hands on.
+constexpr int TAU_THREADS = 256;
+__global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int cols, int cap, float* tau) {
+  const int s = blockIdx.x, tid = threadIdx.x;
+  uint32_t mine = 0u;
+  for (int e = tid; e < cols; e += TAU_THREADS) {
+    const uint32_t key = tc_key(__ldcg(dump + (size_t)s * cols + e));
+    mine = key > mine ? key : mine;
+  }
+  const uint32_t K = tc_select(mine, cap);
   if (tid == 0) {
-    const uint32_t b = (K & 0x80000000u) ? (K & 0x7fffffffu) : ~K;
-    float t = __uint_as_float(b);
-    if (K == 0u || !(t == t)) t = -INFINITY;      // fewer than cap scores: everything passes
+    float t = tc_unkey(K);
+    if (K == 0u || !(t == t)) t = -INFINITY;      // everything passes
     tau[s] = t;
   }
 }
 
-// One block per sample: the slices' candidates -> the cap best by approximate score (their cap-th largest key, found
-// bit by bit as in k_tc_tau) -> their exact fp32 logits -> the k best by (logit descending, id ascending).
-// need_fix[s] = 1 when the filter cannot be shown to be exact.
+// One block per sample: the slices' candidates -> those whose approximate score reaches the cap-th largest of the
+// threads' maxima (cap of them, or a few more) -> their exact fp32 logits -> the k best by (logit descending, id
+// ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
 constexpr int RF_THREADS = 256;
-constexpr int RF_MAXC = 4096;
+constexpr int RF_MAXC = 4096;      // candidates per sample at most
 constexpr int RF_MAXV = 512;       // buffers per sample at most
+constexpr int RF_SLOTS = 64;       // candidates scored exactly at most
 __global__ void __launch_bounds__(RF_THREADS)
 k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, const float* tau, int Bpad,
             const unsigned int* norm2max, int B, int H, int N, int cap, int nvs, int k, int32_t* out_ids, float* out_scores,
@@ -411,8 +413,8 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
   __shared__ uint32_t ck[RF_MAXC];
   __shared__ int ci[RF_MAXC];
   __shared__ int offs[RF_MAXV + 1];
-  __shared__ float ez[TC_CAP];
-  __shared__ int ei[TC_CAP];
+  __shared__ float ez[RF_SLOTS], sz[RF_SLOTS];
+  __shared__ int ei[RF_SLOTS], si[RF_SLOTS];
   __shared__ float red[RF_THREADS / 32];
   __shared__ int wsum[RF_THREADS / 32];
   __shared__ int sh_n;
@@ -427,6 +429,7 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) { const int o = __shfl_up_sync(0xffffffffu, inc, d); if (lane >= d) inc += o; }
     if (lane == 31) wsum[warp] = inc;
+    if (tid == 0) sh_n = 0;
     __syncthreads();
     int base = 0;
     for (int w = 0; w < warp; ++w) base += wsum[w];
@@ -441,41 +444,27 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
     if (tid == 0) need_fix[s] = 1;
     return;
   }
-  // gather: entry e of the list lies in the buffer v with offs[v] <= e < offs[v + 1]
+  // gather: entry e of the list lies in the buffer v with offs[v] <= e < offs[v + 1]; a thread keeps its largest key
+  uint32_t mine = 0u;
   for (int e = tid; e < total; e += RF_THREADS) {
     int lo = 0, hi = RF_MAXV;                     // invariant: offs[lo] <= e < offs[hi]
     while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (offs[mid] <= e) lo = mid; else hi = mid; }
     const int2 x = __ldcg(cand + ((size_t)lo * Bpad + s) * TC_GBUF + (e - offs[lo]));
-    ck[e] = tc_key(__int_as_float(x.x));
+    const uint32_t key = tc_key(__int_as_float(x.x));
+    ck[e] = key;
     ci[e] = x.y;
+    mine = key > mine ? key : mine;
   }
-  if (tid == 0) sh_n = 0;
-  __syncthreads();
-  // the cap-th largest key (0 when there are fewer than cap candidates: all of them go on)
-  uint32_t K = 0u;
-  if (total > cap)
-    for (int bit = 31; bit >= 0; --bit) {
-      const uint32_t trial = K | (1u << bit);
-      int cnt = 0;
-      for (int e = tid; e < total; e += RF_THREADS) cnt += ck[e] >= trial ? 1 : 0;
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
-      if (lane == 0) wsum[warp] = cnt;
-      __syncthreads();
-      int all = 0;
-      for (int w = 0; w < RF_THREADS / 32; ++w) all += wsum[w];
-      if (all >= cap) K = trial;
-      __syncthreads();
-    }
-  // keep the keys above it, then as many equal to it as still fit (which of several equal ones does not matter: the
-  // guard below treats every neuron that is not kept as scoring at most the cap-th key)
+  // the candidates that reach the cap-th largest of the threads' maxima go on (all of them when there are no more than cap)
+  const uint32_t K = total > cap ? tc_select(mine, cap) : 0u;
   for (int e = tid; e < total; e += RF_THREADS)
-    if (ck[e] > K) { const int slot = atomicAdd(&sh_n, 1); ei[slot] = ci[e]; }
+    if (ck[e] >= K) { const int slot = atomicAdd(&sh_n, 1); if (slot < RF_SLOTS) ei[slot] = ci[e]; }
   __syncthreads();
-  for (int e = tid; e < total; e += RF_THREADS)
-    if (ck[e] == K) { const int slot = atomicAdd(&sh_n, 1); if (slot < cap) ei[slot] = ci[e]; }
-  __syncthreads();
-  const int nc = sh_n < cap ? sh_n : cap;       // candidates that go on to the exact pass
+  const int nc = sh_n;
+  if (nc > RF_SLOTS) {                            // many equal scores at the cut: the sample is scored exactly
+    if (tid == 0) need_fix[s] = 1;
+    return;
+  }
   // exact logits of the kept candidates: a warp per candidate, four partial sums per lane as in the exact path
   const float4* h4 = reinterpret_cast<const float4*>(h + (size_t)s * H);
   const int H4 = H >> 2;
@@ -499,29 +488,29 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
   for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
   if (lane == 0) red[warp] = hs;
   __syncthreads();
+  // order the exact scores: an entry's place is the number of better ones ((score, id) pairs are all different)
+  if (tid < nc) {
+    const float z = ez[tid]; const int j = ei[tid];
+    int rank = 0;
+    for (int u = 0; u < nc; ++u) rank += tc_better(ez[u], ei[u], z, j) ? 1 : 0;
+    sz[rank] = z; si[rank] = j;
+  }
+  __syncthreads();
+  if (tid < k) {
+    out_ids[(size_t)s * k + tid] = tid < nc ? si[tid] : -1;
+    out_scores[(size_t)s * k + tid] = tid < nc ? sz[tid] : -INFINITY;
+  }
   if (tid == 0) {
     float hn = 0.f;
     for (int w = 0; w < RF_THREADS / 32; ++w) hn += red[w];
-    // order the exact scores (insertion sort of at most cap entries)
-    for (int a = 1; a < nc; ++a) {
-      const float z = ez[a]; const int j = ei[a];
-      int b = a;
-      while (b > 0 && tc_better(z, j, ez[b - 1], ei[b - 1])) { ez[b] = ez[b - 1]; ei[b] = ei[b - 1]; --b; }
-      ez[b] = z; ei[b] = j;
-    }
-    for (int qk = 0; qk < k; ++qk) {
-      out_ids[(size_t)s * k + qk] = qk < nc ? ei[qk] : -1;
-      out_scores[(size_t)s * k + qk] = qk < nc ? ez[qk] : -INFINITY;
-    }
-    // Every neuron that did not go on to the exact pass has an approximate score of at most T: the cap-th key when
-    // candidates were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its
-    // exact score is at most T plus the error bound; the k best are certain when the k-th exact score lies above.
-    float T = tau[s];
-    if (total > cap) T = __uint_as_float((K & 0x80000000u) ? (K & 0x7fffffffu) : ~K);
+    // Every neuron that did not go on to the exact pass has an approximate score below T: the cut when candidates
+    // were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its exact score is
+    // at most T plus the error bound; the k best are certain when the k-th exact score lies above.
+    const float T = total > cap ? tc_unkey(K) : tau[s];
     if (T > -INFINITY) {
       const float bound = T + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
       const int kth = (k < nc ? k : nc) - 1;
-      if (nc < k || !(ez[kth] > bound)) need_fix[s] = 1;
+      if (nc < k || !(sz[kth] > bound)) need_fix[s] = 1;
     }
   }
 }
@@ -674,13 +663,11 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   const size_t smem = 1024 + tile_bytes * stages + TC_NACC * TC_N * 4 + 24 * 8 + 64;
   if ((e = cudaFuncSetAttribute(k_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k_dense_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-  const size_t tau_smem = (size_t)dump_cols * 4;
-  if ((e = cudaFuncSetAttribute(k_tc_tau, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tau_smem)) != cudaSuccess) return e;
   {
     LaunchScope ls(c, KID_PREDICT);
     p.nslices = nslices_sub; p.ntiles = nsub; p.tile_stride = stride;
     k_dense_tc<true><<<dim3(nslices_sub, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
-    k_tc_tau<<<Bpad, TAU_THREADS, tau_smem, c->stream>>>(dump, dump_cols, cap, tau);
+    k_tc_tau<<<Bpad, TAU_THREADS, 0, c->stream>>>(dump, dump_cols, cap, tau);
     p.nslices = nslices; p.ntiles = ntiles; p.tile_stride = 1;
     k_dense_tc<false><<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
   }
