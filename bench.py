@@ -84,6 +84,8 @@ def parse_args(argv=None):
     ap.add_argument("--rebuild-lambda", type=float, default=0.0, help="later gaps grow by exp(lambda * rebuilds)")
     ap.add_argument("--budget", type=int, default=0, help="sampling budget per sample (Section 3.7); 0 = none, as in the headline")
     ap.add_argument("--hidden-lsh", default="", help="K,L,cap: sample the hidden layer too (tables over the hidden neurons); default dense")
+    ap.add_argument("--predict", type=int, default=0, metavar="K",
+                    help="time top-K inference instead of training: over the retrieved neurons and over all neurons")
     ap.add_argument("--sweep", action="store_true",
                     help="batch 64..2048 x active fraction 0.05%%..100%% on the 670K shape: one JSON line per cell")
     ap.add_argument("--sweep-batches", default="", help="comma-separated subset of the sweep's batch sizes")
@@ -535,7 +537,7 @@ def measure(args, c, B, world, rank, local, windows, with_e2e, with_cpu, sampler
     achieved = booked / dur / 1e9
     step_gbs = model["total"] / (ms_step * 1e-3) / 1e9
     rebuild_us = 1e3 * rebuild_ms / args.rebuild_period if args.rebuild_period else 0.0
-    roofline = {"bound": "hbm", "kernel": "k_" + dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": {"adam": "k_update", "adam_dense": "k_adam_dense", "forward": "k_forward"}[dominant], "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": ncu_traffic(dominant, model_prof),
                 "algorithmic_bytes_per_launch": booked, "us_per_launch": dur * 1e6,
                 "peak_source": "MEASURED_PEAKS.json hbm_gbs (of %s)" % peak_kind,
@@ -583,6 +585,12 @@ def run_dslide(args):
     try:
         if args.sweep:
             run_sweep(args, world, rank, local)
+        elif args.predict:
+            out = run_predict(args, world, rank, local)
+            if out is not None:
+                sampler.stop()
+                out["clocks"] = sampler.summary()
+                print(json.dumps(out))
         else:
             c = workloads.config(args.config)
             c["hidden_lsh"] = hidden_lsh(args)
@@ -599,6 +607,60 @@ def run_dslide(args):
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_predict(args, world, rank, local):
+    """Top-k inference on batches resident in HBM, CUDA events on the library's stream: over the neurons the tables
+    retrieve (Algorithm 1's forward pass without labels) and over all neurons (Section 3.6: layer sparsity 1; on the
+    tensor pipe when k <= 8).  Weights are the random initialisation: the work per batch does not depend on them."""
+    import torch
+    from paper_2201_12667_b200 import binding as ds
+    c = workloads.config(args.config)
+    B = args.batch_size or c["batch"]
+    k, K, W = args.predict, args.steps, max(args.warmup, 3)
+    ctx = ds.dslide_init(make_ctx_config(ds, c, args, B, local))
+    wl = workloads.Workload(c, seed=shard_seed(rank))
+    nb = min(args.batches, 16)
+    dev = [[torch.from_numpy(a).cuda() for a in wl.batch(i, B)[:3]] for i in range(nb)]
+    ids = torch.zeros(B * k, dtype=torch.int32, device="cuda")
+    sc = torch.zeros(B * k, dtype=torch.float32, device="cuda")
+    res = {}
+    for name, dense in (("retrieved", 0), ("all_neurons", 1)):
+        n = K if not dense else max(3, K // 10)
+        for i in range(W):
+            ds.dslide_predict_topk(ctx, B, *dev[i % nb], k, dense, ids, sc)
+        ds.dslide_sync(ctx)
+        barrier = (lambda: None) if world == 1 else torch.distributed.barrier
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()           # the context enqueues on torch's current stream
+        for i in range(n):
+            ds.dslide_predict_topk(ctx, B, *dev[(W + i) % nb], k, dense, ids, sc)
+        e1.record()
+        ds.dslide_sync(ctx)
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda") / n
+        res[name] = {"value": world * B / (ms * 1e-3), "unit": "samples/s", "us_per_batch": 1e3 * ms, "calls": n}
+    status = ds.dslide_sync(ctx, check=False)
+    ds.dslide_destroy(ctx)
+    if rank != 0:
+        return None
+    peak, peak_kind = hbm_peak()
+    w2_bytes = c["N"] * (c["H"] * 4 + 16)                       # every row of W2 and its record, read once per call
+    d_us = res["all_neurons"]["us_per_batch"]
+    groups = (B + 127) // 128
+    res["all_neurons"]["roofline"] = {
+        "bound": "hbm", "kernel": "k_dense_tc" if k <= 8 and c["H"] % 32 == 0 and c["H"] <= 256 else "k_predict_dense",
+        "achieved": w2_bytes / (d_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s", "frac": w2_bytes / (d_us * 1e-6) / 1e9 / peak,
+        "traffic": None, "algorithmic_bytes_per_call": w2_bytes, "peak_source": "MEASURED_PEAKS.json hbm_gbs (of %s)" % peak_kind,
+        "tf32_tflops": 2.0 * groups * 128 * c["N"] * c["H"] / (d_us * 1e-6) / 1e12,
+        "note": "whole call (hidden layer, threshold pass, filter pass, exact pass), not one kernel"}
+    return {"metric": "top-%d inference samples/s at the %s shape on %d B200" % (k, args.config, world),
+            "value": res["retrieved"]["value"], "unit": "samples/s", "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": res["retrieved"]["us_per_batch"] * 1e-3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": dict(workload_config(c, B, args, nb), predict_k=k), "retrieved": res["retrieved"],
+            "all_neurons": res["all_neurons"], "device_status": int(status)}
 
 
 def run_sweep(args, world, rank, local):
