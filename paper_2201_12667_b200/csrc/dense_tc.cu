@@ -15,7 +15,7 @@
 // k_tc_refine recomputes the cap best candidates exactly in fp32 and orders them (logit descending, id ascending).
 // The filter is exact when the k-th exact score clears every discarded neuron's approximate score by more than the
 // approximation's error bound, 2^-9 |h| |w|_max (plus accumulation); a sample for which that cannot be shown (or
-// whose buffers ran over) is flagged and k_tc_fixup scores all N neurons for it in fp32.  Results are therefore
+// whose buffers ran over) is flagged and its block then scores all N neurons for it in fp32.  Results are therefore
 // those of the exact path.
 #include <cuda.h>
 
@@ -177,6 +177,8 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();       // the next kernel of the call may be placed as blocks of this one leave
+  griddep_wait();                    // the filter launch reads the thresholds of the kernel before it
 
   if (warp == 0) {
     // ---------------- producer: one thread feeds the TMA ----------------
@@ -386,6 +388,8 @@ __device__ __forceinline__ uint32_t tc_select(uint32_t mine, int cap) {
 constexpr int TAU_THREADS = 256;
 __global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int cols, int cap, float* tau) {
   const int s = blockIdx.x, tid = threadIdx.x;
+  griddep_launch_dependents();
+  griddep_wait();                    // the threshold pass has completed
   uint32_t mine = 0u;
   for (int e = tid; e < cols; e += TAU_THREADS) {
     const uint32_t key = tc_key(__ldcg(dump + (size_t)s * cols + e));
@@ -399,130 +403,11 @@ __global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int c
   }
 }
 
-// One block per sample: the slices' candidates -> those whose approximate score reaches the cap-th largest of the
-// threads' maxima (cap of them, or a few more) -> their exact fp32 logits -> the k best by (logit descending, id
-// ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
-constexpr int RF_THREADS = 256;
-constexpr int RF_MAXC = 4096;      // candidates per sample at most
-constexpr int RF_MAXV = 512;       // buffers per sample at most
-constexpr int RF_SLOTS = 64;       // candidates scored exactly at most
-__global__ void __launch_bounds__(RF_THREADS)
-k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, const float* tau, int Bpad,
-            const unsigned int* norm2max, int B, int H, int N, int cap, int nvs, int k, int32_t* out_ids, float* out_scores,
-            int* need_fix) {
-  __shared__ uint32_t ck[RF_MAXC];
-  __shared__ int ci[RF_MAXC];
-  __shared__ int offs[RF_MAXV + 1];
-  __shared__ float ez[RF_SLOTS], sz[RF_SLOTS];
-  __shared__ int ei[RF_SLOTS], si[RF_SLOTS];
-  __shared__ float red[RF_THREADS / 32];
-  __shared__ int wsum[RF_THREADS / 32];
-  __shared__ int sh_n;
-  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // fill of the sample's buffers -> their places in one list (exclusive scan; each thread owns RF_MAXV / RF_THREADS buffers)
-  {
-    constexpr int PER = RF_MAXV / RF_THREADS;
-    int c[PER], mine = 0;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) { const int v = tid * PER + i; c[i] = v < nvs ? __ldcg(cand_cnt + (size_t)v * Bpad + s) : 0; mine += c[i]; }
-    int inc = mine;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) { const int o = __shfl_up_sync(0xffffffffu, inc, d); if (lane >= d) inc += o; }
-    if (lane == 31) wsum[warp] = inc;
-    if (tid == 0) sh_n = 0;
-    __syncthreads();
-    int base = 0;
-    for (int w = 0; w < warp; ++w) base += wsum[w];
-    int run = base + inc - mine;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) { offs[tid * PER + i] = run; run += c[i]; }
-    if (tid == RF_THREADS - 1) offs[RF_MAXV] = run;
-    __syncthreads();
-  }
-  const int total = offs[RF_MAXV];
-  if (total > RF_MAXC) {                          // more candidates than this pass handles: the sample is scored exactly
-    if (tid == 0) need_fix[s] = 1;
-    return;
-  }
-  // gather: entry e of the list lies in the buffer v with offs[v] <= e < offs[v + 1]; a thread keeps its largest key
-  uint32_t mine = 0u;
-  for (int e = tid; e < total; e += RF_THREADS) {
-    int lo = 0, hi = RF_MAXV;                     // invariant: offs[lo] <= e < offs[hi]
-    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (offs[mid] <= e) lo = mid; else hi = mid; }
-    const int2 x = __ldcg(cand + ((size_t)lo * Bpad + s) * TC_GBUF + (e - offs[lo]));
-    const uint32_t key = tc_key(__int_as_float(x.x));
-    ck[e] = key;
-    ci[e] = x.y;
-    mine = key > mine ? key : mine;
-  }
-  // the candidates that reach the cap-th largest of the threads' maxima go on (all of them when there are no more than cap)
-  const uint32_t K = total > cap ? tc_select(mine, cap) : 0u;
-  for (int e = tid; e < total; e += RF_THREADS)
-    if (ck[e] >= K) { const int slot = atomicAdd(&sh_n, 1); if (slot < RF_SLOTS) ei[slot] = ci[e]; }
-  __syncthreads();
-  const int nc = sh_n;
-  if (nc > RF_SLOTS) {                            // many equal scores at the cut: the sample is scored exactly
-    if (tid == 0) need_fix[s] = 1;
-    return;
-  }
-  // exact logits of the kept candidates: a warp per candidate, four partial sums per lane as in the exact path
-  const float4* h4 = reinterpret_cast<const float4*>(h + (size_t)s * H);
-  const int H4 = H >> 2;
-  for (int e = warp; e < nc; e += RF_THREADS / 32) {
-    const int j = ei[e];
-    const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
-    float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-    for (int c = lane; c < H4; c += 32) {
-      const float4 w = __ldg(r + c), x = h4[c];
-      d0 = fmaf(w.x, x.x, d0); d1 = fmaf(w.y, x.y, d1); d2 = fmaf(w.z, x.z, d2); d3 = fmaf(w.w, x.w, d3);
-    }
-    float d = (d0 + d1) + (d2 + d3);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-    if (lane == 0) ez[e] = __ldg(&hdr2[j].b) + d;
-  }
-  // |h|^2 of the sample
-  float hs = 0.f;
-  for (int c = tid; c < H; c += RF_THREADS) { const float x = h[(size_t)s * H + c]; hs += x * x; }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
-  if (lane == 0) red[warp] = hs;
-  __syncthreads();
-  // order the exact scores: an entry's place is the number of better ones ((score, id) pairs are all different)
-  if (tid < nc) {
-    const float z = ez[tid]; const int j = ei[tid];
-    int rank = 0;
-    for (int u = 0; u < nc; ++u) rank += tc_better(ez[u], ei[u], z, j) ? 1 : 0;
-    sz[rank] = z; si[rank] = j;
-  }
-  __syncthreads();
-  if (tid < k) {
-    out_ids[(size_t)s * k + tid] = tid < nc ? si[tid] : -1;
-    out_scores[(size_t)s * k + tid] = tid < nc ? sz[tid] : -INFINITY;
-  }
-  if (tid == 0) {
-    float hn = 0.f;
-    for (int w = 0; w < RF_THREADS / 32; ++w) hn += red[w];
-    // Every neuron that did not go on to the exact pass has an approximate score below T: the cut when candidates
-    // were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its exact score is
-    // at most T plus the error bound; the k best are certain when the k-th exact score lies above.
-    const float T = total > cap ? tc_unkey(K) : tau[s];
-    if (T > -INFINITY) {
-      const float bound = T + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
-      const int kth = (k < nc ? k : nc) - 1;
-      if (nc < k || !(sz[kth] > bound)) need_fix[s] = 1;
-    }
-  }
-}
-
-// A flagged sample: every neuron scored exactly (rare; one block walks all of W2).
+// A flagged sample: every neuron scored exactly in fp32 by the sample's block (rare; the block walks all of W2).
+// fx_smem: [H] activation, then [warps][k] lists of scores and of ids, then the lists' lengths.
 constexpr int FX_THREADS = 256;
-__global__ void __launch_bounds__(FX_THREADS)
-k_tc_fixup(const float* W2, const RowHdr* hdr2, const float* h, const int* need_fix, int H, int N, int k, int32_t* out_ids,
-           float* out_scores) {
-  const int s = blockIdx.x;
-  if (!need_fix[s]) return;
-  extern __shared__ float fx_smem[];            // [H] activation, then [warps][k] lists
+__device__ void tc_exact_scan(float* fx_smem, int s, const float* W2, const RowHdr* hdr2, const float* h, int H, int N, int k,
+                              int32_t* out_ids, float* out_scores) {
   float* hs = fx_smem;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = FX_THREADS / 32;
   float* wz = hs + H + warp * k;
@@ -570,6 +455,125 @@ k_tc_fixup(const float* W2, const RowHdr* hdr2, const float* h, const int* need_
       if (bw >= 0) head[bw]++;
     }
   }
+}
+
+// One block per sample: the slices' candidates -> those whose approximate score reaches the cap-th largest of the
+// threads' maxima (cap of them, or a few more) -> their exact fp32 logits -> the k best by (logit descending, id
+// ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
+constexpr int RF_THREADS = FX_THREADS;
+constexpr int RF_MAXC = 4096;      // candidates per sample at most
+constexpr int RF_MAXV = 512;       // buffers per sample at most
+constexpr int RF_SLOTS = 64;       // candidates scored exactly at most
+__global__ void __launch_bounds__(RF_THREADS)
+k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, const float* tau, int Bpad,
+            const unsigned int* norm2max, int B, int H, int N, int cap, int nvs, int k, int32_t* out_ids, float* out_scores,
+            const int* need_fix) {
+  __shared__ uint32_t ck[RF_MAXC];
+  __shared__ int ci[RF_MAXC];
+  __shared__ int offs[RF_MAXV + 1];
+  __shared__ float ez[RF_SLOTS], sz[RF_SLOTS];
+  __shared__ int ei[RF_SLOTS], si[RF_SLOTS];
+  __shared__ float red[RF_THREADS / 32];
+  __shared__ int wsum[RF_THREADS / 32];
+  __shared__ int sh_n, sh_fix;
+  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  griddep_wait();                                // the filter pass has completed
+  // fill of the sample's buffers -> their places in one list (exclusive scan; each thread owns RF_MAXV / RF_THREADS buffers)
+  {
+    constexpr int PER = RF_MAXV / RF_THREADS;
+    int c[PER], mine = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { const int v = tid * PER + i; c[i] = v < nvs ? __ldcg(cand_cnt + (size_t)v * Bpad + s) : 0; mine += c[i]; }
+    int inc = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const int o = __shfl_up_sync(0xffffffffu, inc, d); if (lane >= d) inc += o; }
+    if (lane == 31) wsum[warp] = inc;
+    if (tid == 0) { sh_n = 0; sh_fix = need_fix[s]; }      // a buffer of the sample ran over in the filter pass
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < warp; ++w) base += wsum[w];
+    int run = base + inc - mine;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { offs[tid * PER + i] = run; run += c[i]; }
+    if (tid == RF_THREADS - 1) offs[RF_MAXV] = run;
+    __syncthreads();
+  }
+  const int total = offs[RF_MAXV];
+  int nc = 0;
+  uint32_t K = 0u;
+  bool fix = total > RF_MAXC;                     // more candidates than this pass handles: the sample is scored exactly
+  if (!fix) {
+  // gather: entry e of the list lies in the buffer v with offs[v] <= e < offs[v + 1]; a thread keeps its largest key
+  uint32_t mine = 0u;
+  for (int e = tid; e < total; e += RF_THREADS) {
+    int lo = 0, hi = RF_MAXV;                     // invariant: offs[lo] <= e < offs[hi]
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (offs[mid] <= e) lo = mid; else hi = mid; }
+    const int2 x = __ldcg(cand + ((size_t)lo * Bpad + s) * TC_GBUF + (e - offs[lo]));
+    const uint32_t key = tc_key(__int_as_float(x.x));
+    ck[e] = key;
+    ci[e] = x.y;
+    mine = key > mine ? key : mine;
+  }
+  // the candidates that reach the cap-th largest of the threads' maxima go on (all of them when there are no more than cap)
+  K = total > cap ? tc_select(mine, cap) : 0u;
+  for (int e = tid; e < total; e += RF_THREADS)
+    if (ck[e] >= K) { const int slot = atomicAdd(&sh_n, 1); if (slot < RF_SLOTS) ei[slot] = ci[e]; }
+  __syncthreads();
+  nc = sh_n;
+  fix = nc > RF_SLOTS;                            // many equal scores at the cut: the sample is scored exactly
+  }
+  if (!fix) {
+  // exact logits of the kept candidates: a warp per candidate, four partial sums per lane as in the exact path
+  const float4* h4 = reinterpret_cast<const float4*>(h + (size_t)s * H);
+  const int H4 = H >> 2;
+  for (int e = warp; e < nc; e += RF_THREADS / 32) {
+    const int j = ei[e];
+    const float4* r = reinterpret_cast<const float4*>(W2 + (size_t)j * H);
+    float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+    for (int c = lane; c < H4; c += 32) {
+      const float4 w = __ldg(r + c), x = h4[c];
+      d0 = fmaf(w.x, x.x, d0); d1 = fmaf(w.y, x.y, d1); d2 = fmaf(w.z, x.z, d2); d3 = fmaf(w.w, x.w, d3);
+    }
+    float d = (d0 + d1) + (d2 + d3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+    if (lane == 0) ez[e] = __ldg(&hdr2[j].b) + d;
+  }
+  // |h|^2 of the sample
+  float hs = 0.f;
+  for (int c = tid; c < H; c += RF_THREADS) { const float x = h[(size_t)s * H + c]; hs += x * x; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
+  if (lane == 0) red[warp] = hs;
+  __syncthreads();
+  // order the exact scores: an entry's place is the number of better ones ((score, id) pairs are all different)
+  if (tid < nc) {
+    const float z = ez[tid]; const int j = ei[tid];
+    int rank = 0;
+    for (int u = 0; u < nc; ++u) rank += tc_better(ez[u], ei[u], z, j) ? 1 : 0;
+    sz[rank] = z; si[rank] = j;
+  }
+  __syncthreads();
+  if (tid < k) {
+    out_ids[(size_t)s * k + tid] = tid < nc ? si[tid] : -1;
+    out_scores[(size_t)s * k + tid] = tid < nc ? sz[tid] : -INFINITY;
+  }
+  if (tid == 0) {
+    float hn = 0.f;
+    for (int w = 0; w < RF_THREADS / 32; ++w) hn += red[w];
+    // Every neuron that did not go on to the exact pass has an approximate score below T: the cut when candidates
+    // were dropped here, else the sample's threshold (a neuron below it was never a candidate).  Its exact score is
+    // at most T plus the error bound; the k best are certain when the k-th exact score lies above.
+    const float T = total > cap ? tc_unkey(K) : tau[s];
+    if (T > -INFINITY) {
+      const float bound = T + TC_ERR * sqrtf(hn) * sqrtf(__uint_as_float(*norm2max)) + 1e-30f;
+      const int kth = (k < nc ? k : nc) - 1;
+      if (nc < k || !(sz[kth] > bound)) sh_fix = 1;
+    }
+  }
+  }
+  __syncthreads();
+  if (fix || sh_fix) tc_exact_scan(reinterpret_cast<float*>(ck), s, W2, hdr2, h, H, N, k, out_ids, out_scores);
 }
 
 // ---------------------------------------------------------------------------
@@ -667,15 +671,17 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
     LaunchScope ls(c, KID_PREDICT);
     p.nslices = nslices_sub; p.ntiles = nsub; p.tile_stride = stride;
     k_dense_tc<true><<<dim3(nslices_sub, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
-    k_tc_tau<<<Bpad, TAU_THREADS, 0, c->stream>>>(dump, dump_cols, cap, tau);
+    // each of the next three may be placed while the kernel before it drains (they wait for it before they read)
+    if ((e = launch_dependent(k_tc_tau, dim3(Bpad), dim3(TAU_THREADS), 0, c->stream, (const float*)dump, dump_cols, cap, tau)) != cudaSuccess)
+      return e;
     p.nslices = nslices; p.ntiles = ntiles; p.tile_stride = 1;
-    k_dense_tc<false><<<dim3(nslices, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
+    if ((e = launch_dependent(k_dense_tc<false>, dim3(nslices, groups), dim3(TC_THREADS), smem, c->stream, tmW, p)) != cudaSuccess) return e;
+    if ((e = launch_dependent(k_tc_refine, dim3(batch), dim3(RF_THREADS), 0, c->stream, (const float*)c->W2, (const RowHdr*)c->hdr2,
+                              (const float*)c->h, (const int2*)cand, (const int*)cand_cnt, (const float*)tau, Bpad,
+                              (const unsigned int*)norm2, batch, c->H, c->N, cap, nvs, k, out_ids, out_scores, (const int*)need_fix)) !=
+        cudaSuccess)
+      return e;
   }
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  k_tc_refine<<<batch, RF_THREADS, 0, c->stream>>>(c->W2, c->hdr2, c->h, cand, cand_cnt, tau, Bpad, norm2, batch, c->H, c->N, cap, nvs, k,
-                                                   out_ids, out_scores, need_fix);
-  const size_t fx_smem = ((size_t)c->H + 2 * (FX_THREADS / 32) * k + FX_THREADS / 32) * 4;
-  k_tc_fixup<<<batch, FX_THREADS, fx_smem, c->stream>>>(c->W2, c->hdr2, c->h, need_fix, c->H, c->N, k, out_ids, out_scores);
   return cudaGetLastError();
 }
 
