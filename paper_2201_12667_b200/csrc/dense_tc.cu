@@ -263,6 +263,10 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
     int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * TC_GBUF;
     const float tau = DUMP ? 0.f : p.tau[s0 + row];
     int cnt = 0;
+    if (DUMP && slice == 0 && half == 0) {      // the threshold pass also clears what the filter pass accumulates into
+      if (s0 + row < p.B) p.need_fix[s0 + row] = 0;
+      if (tid == 96 && blockIdx.y == 0) *p.norm2max = 0u;
+    }
     if (half == 0) {
       // the block's activations -> tensor memory: lane = sample, column = hidden unit (samples past the batch: zeros)
       const float4* hrow = reinterpret_cast<const float4*>(p.h + (size_t)(s0 + row) * p.H);
@@ -654,8 +658,6 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   CUtensorMap tmW;
   if (!make_map(&tmW, c->W2, c->N, c->H)) return cudaErrorInvalidValue;
 
-  // the norm bound and the flags start at zero (one clear: they are neighbours)
-  if ((e = cudaMemsetAsync(ws, 0, off_tau, c->stream)) != cudaSuccess) return e;
 
   TcParams p;
   p.hdr2 = c->hdr2; p.h = c->h; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.norm2max = norm2; p.st = c->dstate;
@@ -670,8 +672,9 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   {
     LaunchScope ls(c, KID_PREDICT);
     p.nslices = nslices_sub; p.ntiles = nsub; p.tile_stride = stride;
-    k_dense_tc<true><<<dim3(nslices_sub, groups), TC_THREADS, smem, c->stream>>>(tmW, p);
-    // each of the next three may be placed while the kernel before it drains (they wait for it before they read)
+    // each kernel of the call may be placed while the kernel before it drains (they wait for it before they read or
+    // write anything); the first follows the hidden-layer kernel in the same way
+    if ((e = launch_dependent(k_dense_tc<true>, dim3(nslices_sub, groups), dim3(TC_THREADS), smem, c->stream, tmW, p)) != cudaSuccess) return e;
     if ((e = launch_dependent(k_tc_tau, dim3(Bpad), dim3(TAU_THREADS), 0, c->stream, (const float*)dump, dump_cols, cap, tau)) != cudaSuccess)
       return e;
     p.nslices = nslices; p.ntiles = ntiles; p.tile_stride = 1;
