@@ -34,7 +34,8 @@ constexpr int TC_EPI = 128 * TC_SPLIT;                 // read-back threads
 constexpr int TC_THREADS = 96 + TC_EPI;                // warp 0: TMA producer; warp 1: tensor memory + MMA issue; warp 2: row norms; then the read-back warps
 constexpr int TC_EXTRA = 8;        // candidates kept beyond k: TC_EXTRA + k (the wider the margin, the rarer the exact fall-back)
 constexpr int TC_K_MAX = 8;
-constexpr int TC_GBUF = 64;        // candidate slots per (slice, sample); a buffer that runs over sends the sample to the exact scan
+constexpr int TC_GBUF_MIN = 64;    // candidate slots per (buffer, sample) at least; a buffer that runs over sends the sample to the exact scan
+constexpr int TC_TARGET = 64;      // candidates aimed at per sample: TC_TARGET x cap
 constexpr int TC_SUBSET = 64;      // the threshold pass scores every TC_SUBSET-th tile
 constexpr int TC_SUB_BYTES = TC_M * 128;               // one 32-unit slab of 128 rows
 constexpr float TC_ERR = 2.2e-3f;  // |approximate - exact| <= TC_ERR * |h| * |w|: two operands cut to 10 mantissa bits, fp32 sums
@@ -42,7 +43,7 @@ constexpr float TC_ERR = 2.2e-3f;  // |approximate - exact| <= TC_ERR * |h| * |w
 struct TcParams {
   const RowHdr* hdr2;
   const float* h;                  // [>= B][H] hidden activations of the batch
-  int2* cand;                      // [TC_SPLIT * slices][Bpad][TC_GBUF] (score bits, id), cand_cnt of them valid, no order
+  int2* cand;                      // [TC_SPLIT * slices][Bpad][gbuf] (score bits, id), cand_cnt of them valid, no order
   int* cand_cnt;                   // [TC_SPLIT * slices][Bpad]
   float* dump;                     // DUMP launch: [Bpad][dump_cols] scores of the subset's tiles
   const float* tau;                // filter launch: [Bpad] thresholds
@@ -53,6 +54,7 @@ struct TcParams {
   int tile_stride;                 // tile i of the launch is tile i * tile_stride of W2
   int stages;                      // tiles of W2 in flight, 1 .. TC_STAGES
   int dump_cols;
+  int gbuf;                        // slots per candidate buffer
 };
 
 __device__ __forceinline__ uint32_t tc_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -260,7 +262,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
     const int row = 32 * q + lane;          // sample inside the block
     const int et = tid - 96;                // the first 128 read-back threads fetch the tile's biases
     const int vslice = slice * TC_SPLIT + half;    // buffers are kept per (slice, share of the columns)
-    int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * TC_GBUF;
+    int2* mybuf = p.cand + ((size_t)vslice * p.Bpad + s0 + row) * p.gbuf;
     const float tau = DUMP ? 0.f : p.tau[s0 + row];
     int cnt = 0;
     if (DUMP && slice == 0 && half == 0) {      // the threshold pass also clears what the filter pass accumulates into
@@ -344,7 +346,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
                          : "=r"(raw) : "r"(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * TC_N + c0 + c)) : "memory");
             if ((hm >> c) & 1u) {
               const float z = __uint_as_float(raw) + sb[acc * TC_N + c0 + c];
-              if (cnt < TC_GBUF) __stcg(mybuf + cnt, make_int2(__float_as_int(z), jb + c));
+              if (cnt < p.gbuf) __stcg(mybuf + cnt, make_int2(__float_as_int(z), jb + c));
               ++cnt;
             }
           }
@@ -355,8 +357,8 @@ k_dense_tc(const __grid_constant__ CUtensorMap tmW, const TcParams p) {
       if (++acc == nacc) { acc = 0; ++accround; }
     }
     if (!DUMP && s0 + row < p.B) {
-      p.cand_cnt[(size_t)vslice * p.Bpad + s0 + row] = cnt < TC_GBUF ? cnt : TC_GBUF;
-      if (cnt > TC_GBUF) p.need_fix[s0 + row] = 1;          // candidates were dropped: the sample is scored exactly
+      p.cand_cnt[(size_t)vslice * p.Bpad + s0 + row] = cnt < p.gbuf ? cnt : p.gbuf;
+      if (cnt > p.gbuf) p.need_fix[s0 + row] = 1;          // candidates were dropped: the sample is scored exactly
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -390,7 +392,7 @@ __device__ __forceinline__ uint32_t tc_select(uint32_t mine, int cap) {
 // the cap best fell to different threads); -infinity when the subset is smaller than that.  Any threshold gives the
 // same results: it only decides how many candidates the filter pass hands on.
 constexpr int TAU_THREADS = 256;
-__global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int cols, int cap, float* tau) {
+__global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int cols, int rank, float* tau) {
   const int s = blockIdx.x, tid = threadIdx.x;
   griddep_launch_dependents();
   griddep_wait();                    // the threshold pass has completed
@@ -399,7 +401,7 @@ __global__ void __launch_bounds__(TAU_THREADS) k_tc_tau(const float* dump, int c
     const uint32_t key = tc_key(__ldcg(dump + (size_t)s * cols + e));
     mine = key > mine ? key : mine;
   }
-  const uint32_t K = tc_select(mine, cap);
+  const uint32_t K = tc_select(mine, rank);
   if (tid == 0) {
     float t = tc_unkey(K);
     if (K == 0u || !(t == t)) t = -INFINITY;      // everything passes
@@ -465,15 +467,13 @@ __device__ void tc_exact_scan(float* fx_smem, int s, const float* W2, const RowH
 // threads' maxima (cap of them, or a few more) -> their exact fp32 logits -> the k best by (logit descending, id
 // ascending).  need_fix[s] = 1 when the filter cannot be shown to be exact.
 constexpr int RF_THREADS = FX_THREADS;
-constexpr int RF_MAXC = 4096;      // candidates per sample at most
 constexpr int RF_MAXV = 512;       // buffers per sample at most
 constexpr int RF_SLOTS = 64;       // candidates scored exactly at most
 __global__ void __launch_bounds__(RF_THREADS)
-k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, const float* tau, int Bpad,
+k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* cand, const int* cand_cnt, int gbuf, const float* tau, int Bpad,
             const unsigned int* norm2max, int B, int H, int N, int cap, int nvs, int k, int32_t* out_ids, float* out_scores,
             const int* need_fix) {
-  __shared__ uint32_t ck[RF_MAXC];
-  __shared__ int ci[RF_MAXC];
+  __shared__ float fx_space[1024];               // the exact scan's work space (H <= 256 activations + 2 x 8 x 8 list entries + 8)
   __shared__ int offs[RF_MAXV + 1];
   __shared__ float ez[RF_SLOTS], sz[RF_SLOTS];
   __shared__ int ei[RF_SLOTS], si[RF_SLOTS];
@@ -505,23 +505,41 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
   const int total = offs[RF_MAXV];
   int nc = 0;
   uint32_t K = 0u;
-  bool fix = total > RF_MAXC;                     // more candidates than this pass handles: the sample is scored exactly
-  if (!fix) {
-  // gather: entry e of the list lies in the buffer v with offs[v] <= e < offs[v + 1]; a thread keeps its largest key
-  uint32_t mine = 0u;
-  for (int e = tid; e < total; e += RF_THREADS) {
+  bool fix = false;
+  {
+  // Entry e of the sample's list lies in the buffer v with offs[v] <= e < offs[v + 1].  First walk: a thread keeps the
+  // largest key of its entries.  The candidates that reach the cap-th largest of these maxima go on (all of them when
+  // there are no more than cap): a second walk over the same entries (they are in L2) collects them.
+  auto entry = [&](int e) {
     int lo = 0, hi = RF_MAXV;                     // invariant: offs[lo] <= e < offs[hi]
     while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (offs[mid] <= e) lo = mid; else hi = mid; }
-    const int2 x = __ldcg(cand + ((size_t)lo * Bpad + s) * TC_GBUF + (e - offs[lo]));
-    const uint32_t key = tc_key(__int_as_float(x.x));
-    ck[e] = key;
-    ci[e] = x.y;
+    return __ldcg(cand + ((size_t)lo * Bpad + s) * gbuf + (e - offs[lo]));
+  };
+  constexpr int KEEP = 8;                         // entries per thread that stay in registers between the walks
+  int2 keep[KEEP];
+  uint32_t mine = 0u;
+#pragma unroll
+  for (int i = 0; i < KEEP; ++i) {
+    const int e = tid + i * RF_THREADS;
+    keep[i] = e < total ? entry(e) : make_int2(0, 0);
+    const uint32_t key = e < total ? tc_key(__int_as_float(keep[i].x)) : 0u;
     mine = key > mine ? key : mine;
   }
-  // the candidates that reach the cap-th largest of the threads' maxima go on (all of them when there are no more than cap)
+  for (int e = tid + KEEP * RF_THREADS; e < total; e += RF_THREADS) {
+    const uint32_t key = tc_key(__int_as_float(entry(e).x));
+    mine = key > mine ? key : mine;
+  }
   K = total > cap ? tc_select(mine, cap) : 0u;
-  for (int e = tid; e < total; e += RF_THREADS)
-    if (ck[e] >= K) { const int slot = atomicAdd(&sh_n, 1); if (slot < RF_SLOTS) ei[slot] = ci[e]; }
+#pragma unroll
+  for (int i = 0; i < KEEP; ++i)
+    if (tid + i * RF_THREADS < total && tc_key(__int_as_float(keep[i].x)) >= K) {
+      const int slot = atomicAdd(&sh_n, 1);
+      if (slot < RF_SLOTS) ei[slot] = keep[i].y;
+    }
+  for (int e = tid + KEEP * RF_THREADS; e < total; e += RF_THREADS) {
+    const int2 x = entry(e);
+    if (tc_key(__int_as_float(x.x)) >= K) { const int slot = atomicAdd(&sh_n, 1); if (slot < RF_SLOTS) ei[slot] = x.y; }
+  }
   __syncthreads();
   nc = sh_n;
   fix = nc > RF_SLOTS;                            // many equal scores at the cut: the sample is scored exactly
@@ -577,7 +595,7 @@ k_tc_refine(const float* W2, const RowHdr* hdr2, const float* h, const int2* can
   }
   }
   __syncthreads();
-  if (fix || sh_fix) tc_exact_scan(reinterpret_cast<float*>(ck), s, W2, hdr2, h, H, N, k, out_ids, out_scores);
+  if (fix || sh_fix) tc_exact_scan(fx_space, s, W2, hdr2, h, H, N, k, out_ids, out_scores);
 }
 
 // ---------------------------------------------------------------------------
@@ -637,7 +655,14 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
   const size_t off_fix = 256, off_tau = off_fix + up((size_t)Bpad * 4), off_cnt = off_tau + up((size_t)Bpad * 4);
   const size_t off_cand = off_cnt + up((size_t)nvs * Bpad * 4);
-  const size_t off_dump = off_cand + up((size_t)nvs * Bpad * TC_GBUF * sizeof(int2));
+  // The threshold is the rank-th best of the subset's maxima, the rank chosen so that about TC_TARGET x cap neurons
+  // reach it over all N whatever the subset's share; a buffer has room for four times its expected fill.
+  int rank = (cap * TC_TARGET + stride - 1) / stride;
+  if (rank > cap) rank = cap;
+  if (rank < 4) rank = 4;
+  int gbuf = TC_GBUF_MIN;
+  while (gbuf * nvs < 4 * rank * stride) gbuf <<= 1;
+  const size_t off_dump = off_cand + up((size_t)nvs * Bpad * gbuf * sizeof(int2));
   const size_t need = off_dump + (size_t)Bpad * dump_cols * 4;
   cudaError_t e;
   if (need > c->pd_cap) {
@@ -661,7 +686,7 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
 
   TcParams p;
   p.hdr2 = c->hdr2; p.h = c->h; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.norm2max = norm2; p.st = c->dstate;
-  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.dump_cols = dump_cols;
+  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.dump_cols = dump_cols; p.gbuf = gbuf;
   const size_t tile_bytes = (size_t)(c->H / TC_KB) * TC_SUB_BYTES;
   int stages = (int)(((size_t)200 << 10) / tile_bytes);
   if (stages > TC_STAGES) stages = TC_STAGES;
@@ -675,12 +700,12 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
     // each kernel of the call may be placed while the kernel before it drains (they wait for it before they read or
     // write anything); the first follows the hidden-layer kernel in the same way
     if ((e = launch_dependent(k_dense_tc<true>, dim3(nslices_sub, groups), dim3(TC_THREADS), smem, c->stream, tmW, p)) != cudaSuccess) return e;
-    if ((e = launch_dependent(k_tc_tau, dim3(Bpad), dim3(TAU_THREADS), 0, c->stream, (const float*)dump, dump_cols, cap, tau)) != cudaSuccess)
+    if ((e = launch_dependent(k_tc_tau, dim3(Bpad), dim3(TAU_THREADS), 0, c->stream, (const float*)dump, dump_cols, rank, tau)) != cudaSuccess)
       return e;
     p.nslices = nslices; p.ntiles = ntiles; p.tile_stride = 1;
     if ((e = launch_dependent(k_dense_tc<false>, dim3(nslices, groups), dim3(TC_THREADS), smem, c->stream, tmW, p)) != cudaSuccess) return e;
     if ((e = launch_dependent(k_tc_refine, dim3(batch), dim3(RF_THREADS), 0, c->stream, (const float*)c->W2, (const RowHdr*)c->hdr2,
-                              (const float*)c->h, (const int2*)cand, (const int*)cand_cnt, (const float*)tau, Bpad,
+                              (const float*)c->h, (const int2*)cand, (const int*)cand_cnt, gbuf, (const float*)tau, Bpad,
                               (const unsigned int*)norm2, batch, c->H, c->N, cap, nvs, k, out_ids, out_scores, (const int*)need_fix)) !=
         cudaSuccess)
       return e;

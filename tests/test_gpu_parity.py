@@ -325,35 +325,47 @@ def test_force_dense_matches_oracle_and_dense_softmax():
 def test_predict_topk(dense, k, H):
     pr = mid_pair(H=H)
     try:
-        pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.05)
-        pr.push_state()
-        wl = workloads.Workload(workloads.config("mid"), seed=7)
-        batch = wl.batch(0)
-        B = len(batch[0]) - 1
-        ids_o, sc_o = pr.o.predict_topk(batch[0], batch[1], batch[2], k, dense=bool(dense))
-        dev = to_dev(batch[:3])
-        ids_g = torch.empty(B * k, dtype=torch.int32, device="cuda")
-        sc_g = torch.empty(B * k, dtype=torch.float32, device="cuda")
-        ds.dslide_predict_topk(pr.ctx, B, *dev, k, dense, ids_g, sc_g)
-        ds.dslide_sync(pr.ctx)
-        ids_g = ids_g.cpu().numpy().reshape(B, k)
-        sc_g = sc_g.cpu().numpy().reshape(B, k)
-        for s in range(B):
-            valid = ids_o[s] >= 0
-            assert np.array_equal(ids_g[s] >= 0, valid)
-            assert max_rel_err(sc_g[s][valid], sc_o[s][valid], 1e-2) < ACT_TOL
-            assert np.all(np.isneginf(sc_g[s][~valid]))
-            # ids must agree wherever the scores are separated by more than the tolerance
-            for q in range(k):
-                if not valid[q]:
-                    continue
-                near = np.abs(sc_o[s][valid] - sc_o[s][q]) <= 2 * ACT_TOL * np.abs(sc_o[s][q])
-                if near.sum() == 1:
-                    assert ids_g[s][q] == ids_o[s][q]
-                else:
-                    assert ids_g[s][q] in ids_o[s][valid][near]
+        check_predict(pr, workloads.Workload(workloads.config("mid"), seed=7).batch(0), dense, k)
     finally:
         pr.close()
+
+
+def test_predict_topk_over_all_neurons_with_five_groups_of_samples():
+    """600 samples: five blocks of 128 samples share every tile of W2 (the last group ragged), fewer slices of the
+    neurons per group, larger candidate buffers."""
+    pr = mid_pair(max_batch=600)
+    try:
+        check_predict(pr, workloads.Workload(workloads.config("mid"), seed=8).batch(0, 600), 1, 5)
+    finally:
+        pr.close()
+
+
+def check_predict(pr, batch, dense, k):
+    pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.05)
+    pr.push_state()
+    B = len(batch[0]) - 1
+    ids_o, sc_o = pr.o.predict_topk(batch[0], batch[1], batch[2], k, dense=bool(dense))
+    dev = to_dev(batch[:3])
+    ids_g = torch.empty(B * k, dtype=torch.int32, device="cuda")
+    sc_g = torch.empty(B * k, dtype=torch.float32, device="cuda")
+    ds.dslide_predict_topk(pr.ctx, B, *dev, k, dense, ids_g, sc_g)
+    ds.dslide_sync(pr.ctx)
+    ids_g = ids_g.cpu().numpy().reshape(B, k)
+    sc_g = sc_g.cpu().numpy().reshape(B, k)
+    for s in range(B):
+        valid = ids_o[s] >= 0
+        assert np.array_equal(ids_g[s] >= 0, valid)
+        assert max_rel_err(sc_g[s][valid], sc_o[s][valid], 1e-2) < ACT_TOL
+        assert np.all(np.isneginf(sc_g[s][~valid]))
+        # ids must agree wherever the scores are separated by more than the tolerance
+        for q in range(k):
+            if not valid[q]:
+                continue
+            near = np.abs(sc_o[s][valid] - sc_o[s][q]) <= 2 * ACT_TOL * np.abs(sc_o[s][q])
+            if near.sum() == 1:
+                assert ids_g[s][q] == ids_o[s][q]
+            else:
+                assert ids_g[s][q] in ids_o[s][valid][near]
 
 
 # ------------------------------------------------------------------ error paths: status codes, never a fault
