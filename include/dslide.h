@@ -212,7 +212,11 @@ dslide_status dslide_host_result(dslide_ctx* ctx, float* loss_out, int32_t* have
  * (device, -inf there).  1 <= k <= 64.  The paper reports accuracy but not how it
  * evaluates; this is the reading taken.  With dense = 1 the first call (and any call
  * with a larger batch * k) allocates device work space for the partial lists after
- * waiting for the stream.  A predict call uses the per-sample work space of the training
+ * waiting for the stream.  With dense = 1, k <= 8 and a hidden width that is a multiple of
+ * 32 up to 256 the scores of all neurons are first taken on the tensor pipe in TF32 and
+ * used as a filter only: the candidates are re-scored in fp32, and a sample for which
+ * the filter cannot be shown to be exact (an error bound on the TF32 scores decides) is
+ * scored over all neurons in fp32, so the results are those of the fp32 path.  A predict call uses the per-sample work space of the training
  * step: afterwards the snapshot read by dslide_get_last (hidden activations with dense = 1;
  * active ids and logits with dense = 0, whose counts, codes and losses still belong to the
  * last training step) is no longer that of the last training step.  The next training step

@@ -1,22 +1,23 @@
 // Inference over all N neurons on the tensor pipe (dslide_predict_topk with dense = 1, k <= TC_K_MAX).
 //
 // The logits of a batch against every output neuron are one contraction, Z[B][N] = h[B][H] . W2[N][H]^T + b2
-// (Section 3.6: "layer sparsity is 1"), so this path runs it on the fifth-generation tensor cores: tiles of W2 and
-// the batch's hidden activations arrive in shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), a single
-// thread issues tcgen05.mma (kind::tf32, accumulators in tensor memory), and the read-back warps fetch the
-// accumulators (tcgen05.ld) and keep, per sample, the candidates of the block's slice of neurons; one more warp takes
-// the largest row norm of W2 from the tiles while they are in shared memory.  W2 is streamed once per 128 samples.
+// (Section 3.6: "layer sparsity is 1"), so this path runs it on the fifth-generation tensor cores: tiles of W2
+// arrive in shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), the 128 samples' hidden activations of a
+// block sit in tensor memory beside the accumulators, a single thread issues tcgen05.mma (kind::tf32), and the
+// read-back warps fetch the accumulators (tcgen05.ld) and keep, per sample, the candidates of the block's slice of
+// neurons; one more warp takes the largest row norm of W2 from the tiles while they are in shared memory.  W2 is
+// streamed once per 128 samples (the groups of samples walk the same tiles together, so HBM sees it once per call).
 //
 // TF32 rounds both operands to 10 mantissa bits, far from the 1e-4 the scores must meet.  The tensor pass is
 // therefore a FILTER, in two launches of the same kernel.  The first scores every TC_SUBSET-th tile of neurons and
-// writes the scores out; k_tc_tau takes, per sample, the cap-th best of them (cap = 2k + TC_EXTRA) as the sample's
-// threshold -- at least cap neurons reach it, and about cap * TC_SUBSET do over all N.  The second launch scores all
-// tiles and a thread appends the few scores of its sample that reach the threshold to the sample's candidate buffer.
-// k_tc_refine recomputes the cap best candidates exactly in fp32 and orders them (logit descending, id ascending).
-// The filter is exact when the k-th exact score clears every discarded neuron's approximate score by more than the
-// approximation's error bound, 2^-9 |h| |w|_max (plus accumulation); a sample for which that cannot be shown (or
-// whose buffers ran over) is flagged and its block then scores all N neurons for it in fp32.  Results are therefore
-// those of the exact path.
+// writes the scores out; k_tc_tau takes, per sample, about the cap-th best of them (cap = 2k + TC_EXTRA) as the
+// sample's threshold -- about cap * TC_SUBSET neurons reach it over all N.  The second launch scores all tiles and a
+// thread appends the few scores of its sample that reach the threshold to the sample's candidate buffer.
+// k_tc_refine recomputes the cap or so best candidates exactly in fp32 and orders them (logit descending, id
+// ascending).  The filter is exact when the k-th exact score clears every discarded neuron's approximate score by
+// more than the approximation's error bound, 2^-9 |h| |w|_max (plus accumulation); a sample for which that cannot
+// be shown (or whose buffers ran over) is flagged and its block then scores all N neurons for it in fp32.  Results
+// are therefore those of the exact path.  The kernels of a call follow one another by programmatic dependent launch.
 #include <cuda.h>
 
 #include "common.cuh"
