@@ -340,8 +340,22 @@ def test_predict_topk_over_all_neurons_with_five_groups_of_samples():
         pr.close()
 
 
-def check_predict(pr, batch, dense, k):
-    pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.05)
+def test_predict_topk_over_all_neurons_when_the_filter_cannot_decide():
+    """Every output neuron a copy of one of three rows and no bias: thousands of neurons tie at every cut, the candidate
+    buffers run over and the error bound cannot separate the k-th score from the rest, so every sample goes through
+    the exact fp32 scan inside the exact pass.  Ties are ordered by id (ascending), as the oracle's full sort does."""
+    pr = mid_pair()
+    try:
+        r = np.random.default_rng(3)
+        rows = (r.standard_normal((3, pr.H)) * 0.05).astype(np.float32)
+        pr.o.set("W2", rows[np.arange(pr.N) % 3].ravel())
+        check_predict(pr, workloads.Workload(workloads.config("mid"), seed=9).batch(0), 1, 5, b2=np.zeros(pr.N, dtype=np.float32), same_ids=True)
+    finally:
+        pr.close()
+
+
+def check_predict(pr, batch, dense, k, b2=None, same_ids=False):
+    pr.o.set("b2", np.random.default_rng(0).standard_normal(pr.N).astype(np.float32) * 0.05 if b2 is None else b2)
     pr.push_state()
     B = len(batch[0]) - 1
     ids_o, sc_o = pr.o.predict_topk(batch[0], batch[1], batch[2], k, dense=bool(dense))
@@ -352,6 +366,8 @@ def check_predict(pr, batch, dense, k):
     ds.dslide_sync(pr.ctx)
     ids_g = ids_g.cpu().numpy().reshape(B, k)
     sc_g = sc_g.cpu().numpy().reshape(B, k)
+    if same_ids:
+        assert np.array_equal(ids_g, ids_o)
     for s in range(B):
         valid = ids_o[s] >= 0
         assert np.array_equal(ids_g[s] >= 0, valid)
