@@ -51,7 +51,7 @@ struct TcParams {
   int* need_fix;                   // [B] set when a sample's buffer ran over
   unsigned int* norm2max;          // filter launch: largest squared norm of a row of W2, as the bits of a non-negative float
   DevState* st;
-  int B, Bpad, H, N, cap, nslices, ntiles;     // ntiles: tiles this launch walks
+  int B, Bpad, H, N, nslices, ntiles;          // ntiles: tiles this launch walks
   int tile_stride;                 // tile i of the launch is tile i * tile_stride of W2
   int stages;                      // tiles of W2 in flight, 1 .. TC_STAGES
   int dump_cols;
@@ -641,7 +641,7 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
   int nslices = c->num_sms / groups;
   if (nslices < 1) nslices = 1;
   if (nslices > ntiles) nslices = ntiles;
-  if (TC_SPLIT * nslices > 512) nslices = 512 / TC_SPLIT;       // k_tc_refine's table of buffer offsets
+  if (TC_SPLIT * nslices > RF_MAXV) nslices = RF_MAXV / TC_SPLIT;      // k_tc_refine's table of buffer offsets
   // threshold pass: every `stride`-th tile, at most TAU_MAX_TILES of them
   constexpr int TAU_MAX_TILES = 128;
   int stride = TC_SUBSET;
@@ -687,7 +687,7 @@ cudaError_t launch_dense_tc(Ctx* c, int batch, int k, int32_t* out_ids, float* o
 
   TcParams p;
   p.hdr2 = c->hdr2; p.h = c->h; p.cand = cand; p.cand_cnt = cand_cnt; p.dump = dump; p.tau = tau; p.need_fix = need_fix; p.norm2max = norm2; p.st = c->dstate;
-  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.cap = cap; p.dump_cols = dump_cols; p.gbuf = gbuf;
+  p.B = batch; p.Bpad = Bpad; p.H = c->H; p.N = c->N; p.dump_cols = dump_cols; p.gbuf = gbuf;
   const size_t tile_bytes = (size_t)(c->H / TC_KB) * TC_SUB_BYTES;
   int stages = (int)(((size_t)200 << 10) / tile_bytes);
   if (stages > TC_STAGES) stages = TC_STAGES;

@@ -84,6 +84,11 @@ __device__ __forceinline__ void axpy4(float4& a, float g, const float4 x) {
 // The pieces of one layer's update: the weight / moment arrays, the rows that multiply the
 // coefficients (h for W2, dh for W1), the per-row masks and the per-row records (touch count, slots and,
 // for W2, the bias with its moments).
+// Asks L2 for `bytes` (a multiple of 16, from a 16-byte boundary); nothing comes back to the multiprocessor.
+__device__ __forceinline__ void l2_fetch(const void* p, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 struct Side {
   float *W, *M, *V;
   const float* src;
@@ -551,6 +556,22 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
   int nxt = nwarps + cur;
   int fut = 0;
   if (lane == 0) fut = 2 * nwarps + (int)atomicAdd(ticket, 1u);
+  // The list entries of a warp's next ticket are read while it works on the current one, and the rows they name are
+  // asked into L2 (a ticket's time ahead of their use: the loads of the next ticket then wait for L2, not for DRAM).
+  int2 nrow = make_int2(0, 0);
+  int nidx = nrows, nfor = -1;         // the entries held are those of ticket nfor
+  auto entries_of = [&](int t, int2& row, int& idx) {
+    row = make_int2(0, 0);
+    idx = nrows;
+    const int k = t - n_hot_items - n_med;
+    if (t >= n_tickets || k < 0) return;
+    const int first = k < n_big ? k * UPD_TROWS : rows_big + (k - n_big) * G;
+    const int trows = k < n_big ? UPD_TROWS : G;
+    if (lane < trows && first + lane < nrows) {
+      idx = first + lane;
+      row = idx < n2 ? p.own2[idx] : p.own1[idx - n2];
+    }
+  };
   for (;; cur = nxt, nxt = __shfl_sync(FULL, fut, 0), fut = (lane == 0 && nxt < n_tickets) ? 2 * nwarps + (int)atomicAdd(ticket, 1u) : fut) {
     const int t = cur;
     if (t >= n_tickets) break;
@@ -558,15 +579,13 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
     if (t < n_hot_items + n_med) { medium_item<NCH, UMASK>(p, rowptr, t - n_hot_items, nwB, scratch[warp], H, H4, lane); continue; }
 
     // ---- ordinary rows: consecutive entries of the concatenated lists (rows of W2, then rows of W1) ----
-    const int k = t - n_hot_items - n_med;
-    const int first = k < n_big ? k * UPD_TROWS : rows_big + (k - n_big) * G;
-    const int trows = k < n_big ? UPD_TROWS : G;
-    int2 myrow = make_int2(0, 0);        // (row, the sample that touched it first = the sample of slot 0)
-    int myidx = nrows;
-    if (lane < trows) {
-      myidx = first + lane;
-      if (myidx < nrows) myrow = myidx < n2 ? p.own2[myidx] : p.own1[myidx - n2];
-      else myidx = nrows;
+    const int trows = t - n_hot_items - n_med < n_big ? UPD_TROWS : G;
+    int2 myrow = nrow;                   // (row, the sample that touched it first = the sample of slot 0)
+    int myidx = nidx;
+    if (NCH > 1 || nfor != t) entries_of(t, myrow, myidx);
+    if (NCH == 1) {                      // rows of up to 512 bytes; with longer rows the kernel is near the copy bandwidth
+      entries_of(nxt, nrow, nidx);       // and looking ahead only adds load.  Used after this ticket's own loads are issued
+      nfor = nxt;
     }
     for (int b0 = 0; b0 < trows; b0 += G) {
       int rr[G], tt[G];
@@ -590,6 +609,14 @@ __global__ void __launch_bounds__(UPD_THREADS, (NCH == 1 ? 2 : (NCH == 2 ? 2 : 1
           load_row<NCH>(sd.M, (size_t)rr[q], H, H4, lane, m[q]);
           load_row<NCH>(sd.V, (size_t)rr[q], H, H4, lane, v[q]);
         }
+      }
+      if (NCH == 1 && b0 == 0 && nidx < nrows) {
+        const Side sn = make_side(p, nidx < n2);
+        const uint32_t bytes = (uint32_t)H * 4u;
+        l2_fetch(sn.W + (size_t)nrow.x * H, bytes);
+        l2_fetch(sn.M + (size_t)nrow.x * H, bytes);
+        l2_fetch(sn.V + (size_t)nrow.x * H, bytes);
+        l2_fetch(sn.hdr + nrow.x, (uint32_t)sizeof(RowHdr));
       }
 #pragma unroll
       for (int q = 0; q < G; ++q)
