@@ -45,7 +45,7 @@ typedef enum {
   DSLIDE_ERR_BAD_INDEX = 5,  /* feature id outside [0,D) or label id outside [0,N), seen on the device */
   DSLIDE_ERR_STATE = 6,
   DSLIDE_ERR_TIMEOUT = 7     /* a bounded wait inside a kernel ran out.  The sample concerned is skipped: no loss, no
-                                gradient.  If the wait that ran out was for rows of W2, the sample's rows of W1 had
+                                gradient.  If the wait that ran out was for rows of W2, the sample's rows had
                                 been handed to the update already: they receive an Adam update with a zero
                                 gradient from this sample (their moments decay), unlike rows nobody touched.    */
 } dslide_status;

@@ -452,7 +452,9 @@ __device__ __forceinline__ void skip_sample(const FwdParams& p, int s, int code)
   if (tid == 0) set_status(p.st, code);
 }
 
-template <int MODE, int KPT>   // MODE 0 = training step, 1 = predict top-k; KPT = hidden units per thread (H <= KPT * FWD_THREADS)
+// MODE 0 = training step, 1 = predict top-k; KPT = hidden units per thread (H <= KPT * FWD_THREADS); BULK: active sets of
+// many chunks are expected (the host's estimate from the tables' shape) and their rows come by bulk copies
+template <int MODE, int KPT, bool BULK = false>
 __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   float* sh_h = reinterpret_cast<float*>(smem);
@@ -1015,17 +1017,33 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
   const int rp_r0 = tid / (H4 + 1), rp_c0 = tid - rp_r0 * (H4 + 1);
 #pragma unroll
   for (int u = 0; u < HO_PER; ++u) { jj0[u] = 0; nth0[u] = 0u; base0[u] = 0u; }
+  uint32_t w2phase = 0u;
+  bool timed_out = false;                          // block-uniform
+  const bool bulk = BULK && streaming && na >= 4 * stage_rows;      // many chunks: the batch's samples share most rows (see below)
   for (int c0 = 0; c0 < na; c0 += stage_rows) {
     const int nr = min(stage_rows, na - c0);
     __syncthreads();                               // earlier readers and writers of the staging space are done
-    // 16 bytes per thread and copy, all in flight at once: the H4 pieces of the row, and as piece H4 the head of the
-    // row's record (count, bias, bias moments), which lands in the row's padding
-    for (int r = rp_r0, c4 = rp_c0; r < nr;) {
-      const int j = dense ? c0 + r : idp[c0 + r];
-      const void* src = c4 < H4 ? static_cast<const void*>(p.W2 + (size_t)j * H + 4 * c4) : static_cast<const void*>(p.hdr2 + j);
-      cp_async16(stage + (size_t)r * ldr + 4 * c4, src);
-      c4 += rp_dc; r += rp_dr;
-      if (c4 > H4) { c4 -= H4 + 1; ++r; }
+    if (bulk) {
+      // A set streamed in many chunks re-reads rows that other samples of the batch have brought into L2; there the
+      // bulk-copy engine moves about twice what 16-byte copies do per multiprocessor: one copy per row and one for
+      // the head of its record (count, bias, bias moments), which lands in the row's padding; completion on an mbarrier
+      if (tid == 0) mbar_expect_tx(sh_bar, (uint32_t)nr * ((uint32_t)H * 4u + 16u));
+      fence_proxy_async();
+      for (int r = tid; r < nr; r += FWD_THREADS) {
+        const int j = dense ? c0 + r : idp[c0 + r];
+        bulk_g2s(stage + (size_t)r * ldr, p.W2 + (size_t)j * H, (uint32_t)H * 4u, sh_bar);
+        bulk_g2s(stage + (size_t)r * ldr + H, p.hdr2 + j, 16u, sh_bar);
+      }
+    } else {
+      // 16 bytes per thread and copy, all in flight at once: the H4 pieces of the row, and as piece H4 the head of
+      // the row's record, which lands in the row's padding
+      for (int r = rp_r0, c4 = rp_c0; r < nr;) {
+        const int j = dense ? c0 + r : idp[c0 + r];
+        const void* src = c4 < H4 ? static_cast<const void*>(p.W2 + (size_t)j * H + 4 * c4) : static_cast<const void*>(p.hdr2 + j);
+        cp_async16(stage + (size_t)r * ldr + 4 * c4, src);
+        c4 += rp_dc; r += rp_dr;
+        if (c4 > H4) { c4 -= H4 + 1; ++r; }
+      }
     }
     if (c0 == 0 && MODE == 0) {
       // the touch counters: this thread's nonzero of the sample, and its first HO_PER active rows
@@ -1049,8 +1067,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
         }
       }
     }
-    cp_async_wait_all();
-    __syncthreads();
+    if (bulk) {
+      const bool ok = mbar_wait(sh_bar, w2phase);
+      w2phase ^= 1u;
+      if (__syncthreads_or(ok ? 0 : 1)) { timed_out = true; break; }
+    } else {
+      cp_async_wait_all();
+      __syncthreads();
+    }
     // one thread per staged row
     for (int ab = 0; ab < nr; ab += FWD_THREADS) {
       const int a = ab + tid;
@@ -1151,6 +1175,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
       }
     }
   }
+  if (BULK && timed_out) {
+    // a copy did not complete in time: the copies in flight get one more bounded wait, then the sample is given up.
+    // Its touches are already counted, so the hand-off below still runs, with every coefficient zero.
+    mbar_wait(sh_bar, w2phase ^ 1u);
+    __syncthreads();
+    if (tid == 0) set_status(p.st, DSLIDE_ERR_TIMEOUT);
+  }
   if (MODE == 1) {
     // ---- merge the per-warp lists: k rounds over the list heads ----
     if (lane == 0) sh_misc[warp] = tk_cnt;
@@ -1209,7 +1240,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     const float logE = logf(E);
     for (int i = 0; i < nlab; ++i)
       if (sh_lab[i] >= 0) sum += zp[sh_lab[i]] - M - logE;
-    p.loss[s] = ny > 0 ? -sum / (float)ny : 0.f;
+    p.loss[s] = ny > 0 && !(BULK && timed_out) ? -sum / (float)ny : 0.f;
   }
   // the errors of a small set go to shared memory as well (beside the logits: no barrier before they are written)
   for (int a = tid; a < na; a += FWD_THREADS) {
@@ -1218,6 +1249,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     float ga = pa / fB;
     for (int i = 0; i < nlab; ++i)
       if (sh_lab[i] == a) ga = (pa - 1.f / (float)ny) / fB;
+    if (BULK && timed_out) ga = 0.f;
     g[a] = ga;
     if (small) sh_g[a] = ga;
   }
@@ -1264,7 +1296,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 2) k_forward(const FwdParams p) {
     for (int k = tid; k < H; k += FWD_THREADS) {
       float v = 0.f;
       for (int w = 0; w < nparts; ++w) v += sh_dh[(size_t)w * H + k];
-      p.dh[(size_t)s * H + k] = sh_h[k] > 0.f ? v : 0.f;
+      p.dh[(size_t)s * H + k] = sh_h[k] > 0.f && !(BULK && timed_out) ? v : 0.f;
     }
   }
 
@@ -1591,6 +1623,8 @@ cudaError_t setup_forward(Ctx* c) {
   c->fwd_smem = l.fixed_bytes + c->fwd_stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(k_forward<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<0, MAX_KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<0, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<0, MAX_KPT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_forward<1, MAX_KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   return e;
@@ -1635,9 +1669,19 @@ cudaError_t launch_forward_train(Ctx* c, int batch, const int32_t* row_ptr, cons
   {
     LaunchScope ls(c, KID_FORWARD);
     // hidden layers of up to FWD_THREADS units take the variant with one unit per thread (less code, fewer registers)
-    cudaError_t e = c->H <= FWD_THREADS
-                        ? launch_dependent(k_forward<0, 1>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p)
-                        : launch_dependent(k_forward<0, MAX_KPT>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p);
+    // Expected size of an active set from the tables' shape: L buckets of about N / 2^bits ids, cut at the cap (and at
+    // the sampling budget).  Sets of many chunks of the staging space take the variant that fetches rows by bulk copies.
+    const double per_bucket = (double)c->N / (double)(1ll << c->bits);
+    double expect = c->cfg.force_dense ? (double)c->N : (double)c->L * (per_bucket < c->cfg.bucket_cap ? per_bucket : (double)c->cfg.bucket_cap);
+    if (c->cfg.sample_budget > 0 && expect > c->cfg.sample_budget) expect = c->cfg.sample_budget;
+    const bool bulk = expect >= 4.0 * (double)(p.stage_bytes / ((c->H + 4) * 4 + 4));
+    cudaError_t e;
+    if (c->H <= FWD_THREADS)
+      e = bulk ? launch_dependent(k_forward<0, 1, true>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p)
+               : launch_dependent(k_forward<0, 1>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p);
+    else
+      e = bulk ? launch_dependent(k_forward<0, MAX_KPT, true>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p)
+               : launch_dependent(k_forward<0, MAX_KPT>, dim3(batch), dim3(FWD_THREADS), (size_t)c->fwd_smem, c->stream, p);
     if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
